@@ -1,0 +1,149 @@
+/*
+ * wersa.h -- C ABI of the B200 (sm_100a) implementation of the per-head WERSA attention
+ * operator (Wavelet-Enhanced Random Spectral Attention, arXiv 2507.08637).
+ *
+ * The operator, per (batch, head) slab, with Q, K, V in R^{n x d} (Sec. 3.1, problem
+ * statement) stored as (batch, heads, seq, head_dim) row-major (Algorithm 1, SplitHeads):
+ *
+ *   qbar = mean_t Q[t,:]                                   (Eq. 1)
+ *   u    = gate_w^T qbar + gate_b ;  f_i = sigmoid(u_i) * omega_i, i = 0..L   (Eqs. 2-3)
+ *   X_F  = IDWT_L( f (.) DWT_L(X) )  for X in {Q, K}, Haar wavelet along the sequence,
+ *          coefficient order [d_1, ..., d_L, a_L]          (Sec. 3.1 steps 3,5,6; Algorithm 2)
+ *   phi(x) = ReLU(x W / max(beta, bw_floor)) / sqrt(m)     (Eq. 6; Algorithm 1 scalings)
+ *   S = phi(K_F)^T V,  z = phi(K_F)^T 1                    (Eq. 7, key summary / normaliser)
+ *   O = phi(Q_F) S / (phi(Q_F) z + eps)                    (Eq. 7 / Sec. 3.1 step 8)
+ *
+ * Non-causal, unmasked.  One random matrix W (d x m) is shared by queries, keys and all
+ * heads.  Everything runs on one GPU in hand-written CUDA kernels; there is no CPU path:
+ * without a CUDA device every compute entry point returns WERSA_ERR_CUDA.
+ *
+ * Conventions
+ *   - All tensor pointers are DEVICE pointers, dense, row-major, 16-byte aligned.
+ *   - Q, K, V, O, dO, dQ, dK, dV: (batch, heads, seq_len, head_dim), head_dim contiguous.
+ *   - W: (head_dim, features).  beta: 1 float.  gate_w: (heads, head_dim, levels+1) float.
+ *     gate_b: (heads, levels+1) float.  omega: (levels+1) float; index i of the last axis
+ *     addresses the wavelet band: 0 = finest detail d_1, ..., L-1 = d_L, L = approximation a_L.
+ *   - The caller owns every tensor and the workspace; the library allocates no device memory.
+ *   - forward/backward enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL =
+ *     default stream) and return without synchronising.  A context is not thread-safe and
+ *     carries one forward/backward at a time.
+ *   - Errors are return codes; nothing is thrown, nothing aborts, no device trap is used.
+ */
+#ifndef WERSA_H_
+#define WERSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct wersa_ctx wersa_ctx; /* opaque, host memory, owned by the library */
+
+typedef enum {
+  WERSA_OK = 0,
+  WERSA_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, misaligned pointer      */
+  WERSA_ERR_UNSUPPORTED = 2, /* valid problem outside the compiled set of shapes / types */
+  WERSA_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small               */
+  WERSA_ERR_CUDA = 4,        /* a CUDA runtime call failed (no device, launch error)     */
+  WERSA_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired                       */
+  WERSA_ERR_STATE = 6        /* backward called without a preceding forward              */
+} wersa_status;
+
+typedef enum { WERSA_F32 = 0, WERSA_BF16 = 1 } wersa_dtype;
+
+/* Flags for wersa_config.flags. */
+enum {
+  WERSA_FLAG_SIMT_ONLY = 1,    /* bf16 storage but fp32 FFMA arithmetic everywhere (no tensor
+                                  cores); the fp32 dtype always computes this way        */
+  WERSA_FLAG_FORWARD_ONLY = 2  /* the context will never run wersa_backward: its workspace
+                                  omits the gradient scratch buffers                     */
+};
+
+typedef struct wersa_config {
+  int32_t batch;         /* B >= 1                                                      */
+  int32_t heads;         /* H >= 1                                                      */
+  int32_t seq_len;       /* n >= 2; 2^levels must not exceed the next power of two >= n */
+  int32_t head_dim;      /* d, must be 64                                               */
+  int32_t levels;        /* L, Haar levels, 1..8                                        */
+  int32_t features;      /* m, random features: 64, 128 or 256                          */
+  int32_t dtype;         /* wersa_dtype of Q, K, V, W, O, dO; accumulation is fp32      */
+  int32_t grad_dtype;    /* wersa_dtype of dQ, dK, dV                                   */
+  float eps;             /* denominator epsilon of Eq. 7 (paper: "small constant")      */
+  float bw_floor;        /* bw = max(beta, bw_floor) as in Algorithm 1                  */
+  int32_t gate_per_head; /* 1: u[b,h] = gate_w[h]^T qbar[b,h] + gate_b[h]  (Sec. 3.1)
+                            0: u[b] = sum_h gate_w[h]^T qbar[b,h] + gate_b[0], shared by
+                               all heads of a batch element (Algorithm 1, W_filter)     */
+  int32_t device;        /* CUDA device ordinal                                         */
+  int32_t flags;         /* WERSA_FLAG_*                                                */
+} wersa_config;
+
+/* Bytes of device workspace a context of this configuration needs (a multiple of 256);
+ * 0 if the configuration is invalid or unsupported.  Pure host arithmetic. */
+size_t wersa_workspace_bytes(const wersa_config* cfg);
+
+/* Validates cfg, records the plan (tiling, split-sequence chunking) and adopts `workspace`
+ * (device memory, 256-byte aligned, >= wersa_workspace_bytes(cfg); must outlive the context
+ * and must not be shared by contexts that run concurrently).  *out is set only on WERSA_OK.
+ * Launches no kernel. */
+wersa_status wersa_create(const wersa_config* cfg, void* workspace, size_t workspace_bytes,
+                          wersa_ctx** out);
+
+/* Forward pass of the operator defined at the top of this file (Sec. 3.1 steps 3-8, Eqs. 1-7).
+ * Argument order follows the problem statement: Q, K, V, then the random projection, the
+ * bandwidth and the scale-gating parameters.  gate_w may be NULL (treated as zeros).  O has the
+ * dtype of the inputs.  Also leaves f, qbar, S and z in the workspace for wersa_backward and
+ * wersa_saved.  Split-sequence partial sums are combined in a fixed order: results are
+ * bit-identical from run to run. */
+wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const void* V,
+                           const void* W, const float* beta, const float* gate_w,
+                           const float* gate_b, const float* omega, void* O,
+                           void* cuda_stream);
+
+/* Backward pass: gradients of sum(dO (.) O) with respect to Q, K, V (cfg.grad_dtype), beta
+ * (1 float), gate_w (heads, head_dim, levels+1), gate_b (heads, levels+1; rows >= 1 are zero
+ * when gate_per_head = 0) and omega (levels+1).  The paper does not write the backward pass;
+ * it is the chain rule through Eqs. 1-7 with dReLU(a)/da = 1[a > 0].  W is a fixed random
+ * matrix (Sec. 3.1 step 7) and gets no gradient.  Must follow a wersa_forward on the same
+ * context with the same inputs (it reuses f, qbar, S, z).  Any of the five parameter-gradient
+ * pointers may be NULL. */
+wersa_status wersa_backward(wersa_ctx* ctx, const void* Q, const void* K, const void* V,
+                            const void* W, const float* beta, const float* gate_w,
+                            const float* gate_b, const float* omega, const void* dO, void* dQ,
+                            void* dK, void* dV, float* dbeta, float* dgate_w, float* dgate_b,
+                            float* domega, void* cuda_stream);
+
+/* Stand-alone Haar filter (Sec. 3.1 steps 3, 5, 6; Algorithm 2): XF = IDWT_L(f (.) DWT_L(X))
+ * for every slab of X (batch, heads, seq_len, head_dim; cfg.dtype), with f a device array
+ * (batch*heads, levels+1) of floats.  XF has cfg.dtype.  Each element of X is read once. */
+wersa_status wersa_haar_filter(wersa_ctx* ctx, const void* X, const float* f, void* XF,
+                               void* cuda_stream);
+
+/* Device pointers into the workspace of quantities the last forward left there.
+ * which: 0 = f (batch*heads, levels+1); 1 = qbar (batch*heads, head_dim);
+ *        2 = S' (batch*heads, features, head_dim); 3 = z' (batch*heads, features),
+ * where S' = ReLU(K_F W)^T V and z' = ReLU(K_F W)^T 1 are the key summary and normaliser of
+ * Eq. 7 without the 1/(bw sqrt(m)) factor of the feature map (S = S' / (bw sqrt(m))).
+ * *count receives the number of floats. */
+wersa_status wersa_saved(wersa_ctx* ctx, int which, const float** device_ptr, size_t* count);
+
+/* Synchronises `cuda_stream`, then returns WERSA_ERR_TIMEOUT if a kernel of this context gave
+ * up on a bounded wait, WERSA_ERR_CUDA on a sticky CUDA error, else WERSA_OK.  Clears the
+ * device-side error word. */
+wersa_status wersa_query_status(wersa_ctx* ctx, void* cuda_stream);
+
+/* Releases the host-side context.  Does not touch the workspace.  NULL is accepted. */
+wersa_status wersa_destroy(wersa_ctx* ctx);
+
+/* Static, human-readable name of a status code. */
+const char* wersa_status_string(wersa_status status);
+
+/* Number of kernels the last forward (which = 0) or backward (which = 1) on this context
+ * launched; 0 before the first call. */
+int32_t wersa_launch_count(const wersa_ctx* ctx, int which);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WERSA_H_ */

@@ -1,0 +1,348 @@
+// C-ABI layer of the WERSA library: configuration checks, workspace planning and the launch
+// sequences of the forward and backward passes.  All arithmetic lives in the kernels.
+#include <new>
+
+#include "common.cuh"
+
+namespace wersa {
+
+bool tc_supported(const wersa_config& cfg);   // tc_fwd.cu
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+int ceil_div(int a, int b) { return (a + b - 1) / b; }
+int next_pow2(int n) {
+  int p = 1;
+  while (p < n) p <<= 1;
+  return p;
+}
+
+}  // namespace
+
+wersa_status make_plan(const wersa_config& c, Plan* p) {
+  if (c.batch < 1 || c.heads < 1 || c.seq_len < 2 || c.head_dim < 1 || c.levels < 1 || c.features < 1)
+    return WERSA_ERR_INVALID_ARG;
+  if (c.dtype != WERSA_F32 && c.dtype != WERSA_BF16) return WERSA_ERR_INVALID_ARG;
+  if (c.grad_dtype != WERSA_F32 && c.grad_dtype != WERSA_BF16) return WERSA_ERR_INVALID_ARG;
+  if (!(c.eps >= 0.f) || !(c.bw_floor > 0.f)) return WERSA_ERR_INVALID_ARG;
+  if (c.device < 0) return WERSA_ERR_INVALID_ARG;
+  if (c.levels <= 30 && (1LL << c.levels) > (long long)next_pow2(c.seq_len)) return WERSA_ERR_INVALID_ARG;
+  if (c.head_dim != kD) return WERSA_ERR_UNSUPPORTED;
+  if (c.levels > kMaxLevels) return WERSA_ERR_UNSUPPORTED;
+  if (c.features != 64 && c.features != 128 && c.features != 256) return WERSA_ERR_UNSUPPORTED;
+  if ((long long)c.batch * c.heads > 65535) return WERSA_ERR_UNSUPPORTED;   // gridDim.y
+
+  p->cfg = c;
+  p->slabs = c.batch * c.heads;
+  p->L1 = c.levels + 1;
+  p->bf16 = c.dtype == WERSA_BF16;
+  p->grad_bf16 = c.grad_dtype == WERSA_BF16;
+  p->with_backward = !(c.flags & WERSA_FLAG_FORWARD_ONLY);
+  p->use_tc = p->bf16 && !(c.flags & WERSA_FLAG_SIMT_ONLY) && tc_supported(c);
+  const int n = c.seq_len, m = c.features;
+
+  p->qchunks = ceil_div(592, p->slabs);
+  if (p->qchunks > ceil_div(n, 128)) p->qchunks = ceil_div(n, 128);
+  if (p->qchunks < 1) p->qchunks = 1;
+  p->qchunk_rows = ceil_div(ceil_div(n, p->qchunks), 32) * 32;
+  p->qchunks = ceil_div(n, p->qchunk_rows);
+
+  p->htiles = ceil_div(n, kHaarTile);
+
+  const int tiles32 = ceil_div(n, kSimtTile);
+  p->schunks = ceil_div(296, p->slabs);
+  if (p->schunks > tiles32) p->schunks = tiles32;
+  p->schunk_tiles = ceil_div(tiles32, p->schunks);
+  p->schunks = ceil_div(tiles32, p->schunk_tiles);
+
+  p->tchunks = 0;
+  p->tchunk_tiles = 0;
+  if (p->use_tc) {
+    const int tiles128 = ceil_div(n, 128);
+    p->tchunks = 148 / p->slabs;
+    if (p->tchunks < 1) p->tchunks = 1;
+    if (p->tchunks > tiles128) p->tchunks = tiles128;
+    p->tchunk_tiles = ceil_div(tiles128, p->tchunks);
+    if (c.levels == 8) p->tchunk_tiles = ceil_div(p->tchunk_tiles, 2) * 2;   // whole 256-token blocks
+    p->tchunks = ceil_div(tiles128, p->tchunk_tiles);
+  }
+  p->part_chunks = p->schunks > p->tchunks ? p->schunks : p->tchunks;
+
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  };
+  const size_t slabs = (size_t)p->slabs;
+  p->off_status = take(256);
+  p->off_qpart = take(sizeof(float) * slabs * p->qchunks * kD);
+  p->off_qbar = take(sizeof(float) * slabs * kD);
+  p->off_sg = take(sizeof(float) * slabs * p->L1);
+  p->off_f = take(sizeof(float) * slabs * p->L1);
+  p->off_spart = take(sizeof(float) * slabs * p->part_chunks * m * kD);
+  p->off_zpart = take(sizeof(float) * slabs * p->part_chunks * m);
+  p->off_S = take(sizeof(float) * slabs * m * kD);
+  p->off_z = take(sizeof(float) * slabs * m);
+  p->off_Sbf = take(sizeof(__nv_bfloat16) * slabs * m * kD);
+  p->off_Wt = take(sizeof(__nv_bfloat16) * (size_t)m * kD);
+  const size_t slab_elems = slabs * (size_t)n * kD;
+  const bool need_xf = !p->use_tc || p->with_backward;
+  p->off_QF = take(need_xf ? sizeof(float) * slab_elems : 0);
+  p->off_KF = take(need_xf ? sizeof(float) * slab_elems : 0);
+  if (p->with_backward) {
+    p->off_dS = take(sizeof(float) * slabs * m * kD);
+    p->off_dz = take(sizeof(float) * slabs * m);
+    p->off_sumdD = take(sizeof(float) * slabs * p->schunks);
+    p->off_bands = take(sizeof(float) * 2 * slabs * p->htiles * kBandVals);
+    p->off_dqbar = take(sizeof(float) * slabs * (kD + kBandVals));
+    p->off_dQF = take(sizeof(float) * slab_elems);
+    p->off_dKF = take(sizeof(float) * slab_elems);
+  } else {
+    p->off_dS = p->off_dz = p->off_sumdD = p->off_bands = p->off_dqbar = p->off_dQF = p->off_dKF = 0;
+  }
+  p->total = off;
+  return WERSA_OK;
+}
+
+Ws resolve(const Plan& p, void* workspace) {
+  char* b = static_cast<char*>(workspace);
+  Ws w;
+  w.status = reinterpret_cast<int*>(b + p.off_status);
+  w.qpart = reinterpret_cast<float*>(b + p.off_qpart);
+  w.qbar = reinterpret_cast<float*>(b + p.off_qbar);
+  w.sg = reinterpret_cast<float*>(b + p.off_sg);
+  w.f = reinterpret_cast<float*>(b + p.off_f);
+  w.spart = reinterpret_cast<float*>(b + p.off_spart);
+  w.zpart = reinterpret_cast<float*>(b + p.off_zpart);
+  w.S = reinterpret_cast<float*>(b + p.off_S);
+  w.z = reinterpret_cast<float*>(b + p.off_z);
+  w.Sbf = reinterpret_cast<__nv_bfloat16*>(b + p.off_Sbf);
+  w.Wt = reinterpret_cast<__nv_bfloat16*>(b + p.off_Wt);
+  w.QF = reinterpret_cast<float*>(b + p.off_QF);
+  w.KF = reinterpret_cast<float*>(b + p.off_KF);
+  w.dS = reinterpret_cast<float*>(b + p.off_dS);
+  w.dz = reinterpret_cast<float*>(b + p.off_dz);
+  w.sumdD = reinterpret_cast<float*>(b + p.off_sumdD);
+  w.bands = reinterpret_cast<float*>(b + p.off_bands);
+  w.dqbar = reinterpret_cast<float*>(b + p.off_dqbar);
+  w.dQF = reinterpret_cast<float*>(b + p.off_dQF);
+  w.dKF = reinterpret_cast<float*>(b + p.off_dKF);
+  return w;
+}
+
+}  // namespace wersa
+
+using namespace wersa;
+
+struct wersa_ctx {
+  Plan plan;
+  Ws ws;
+  void* workspace;
+  bool forward_done;
+  bool status_cleared;
+  int launches_fwd, launches_bwd;
+};
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Makes cfg.device current for the lifetime of the object and restores the caller's device.
+struct DeviceGuard {
+  int prev = -1;
+  cudaError_t err;
+  explicit DeviceGuard(int dev) {
+    err = cudaGetDevice(&prev);
+    if (err == cudaSuccess && prev != dev) err = cudaSetDevice(dev);
+    else if (err == cudaSuccess) prev = -1;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+#define WERSA_CUDA(call)                                   \
+  do {                                                     \
+    cudaError_t e_ = (call);                               \
+    if (e_ != cudaSuccess) return WERSA_ERR_CUDA;          \
+  } while (0)
+
+wersa_status clear_status_once(wersa_ctx* ctx, cudaStream_t st) {
+  if (!ctx->status_cleared) {
+    WERSA_CUDA(cudaMemsetAsync(ctx->ws.status, 0, 256, st));
+    ctx->status_cleared = true;
+  }
+  return WERSA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t wersa_workspace_bytes(const wersa_config* cfg) {
+  if (cfg == nullptr) return 0;
+  Plan p;
+  if (make_plan(*cfg, &p) != WERSA_OK) return 0;
+  return p.total;
+}
+
+wersa_status wersa_create(const wersa_config* cfg, void* workspace, size_t workspace_bytes, wersa_ctx** out) {
+  if (cfg == nullptr || out == nullptr) return WERSA_ERR_INVALID_ARG;
+  Plan p;
+  wersa_status s = make_plan(*cfg, &p);
+  if (s != WERSA_OK) return s;
+  if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || workspace_bytes < p.total)
+    return WERSA_ERR_WORKSPACE;
+  wersa_ctx* ctx = new (std::nothrow) wersa_ctx;
+  if (ctx == nullptr) return WERSA_ERR_INVALID_ARG;
+  ctx->plan = p;
+  ctx->workspace = workspace;
+  ctx->ws = resolve(p, workspace);
+  ctx->forward_done = false;
+  ctx->status_cleared = false;
+  ctx->launches_fwd = ctx->launches_bwd = 0;
+  *out = ctx;
+  return WERSA_OK;
+}
+
+wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const void* V, const void* W,
+                           const float* beta, const float* gate_w, const float* gate_b, const float* omega,
+                           void* O, void* cuda_stream) {
+  if (ctx == nullptr || Q == nullptr || K == nullptr || V == nullptr || W == nullptr || beta == nullptr ||
+      omega == nullptr || O == nullptr)
+    return WERSA_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(W) || !aligned16(O))
+    return WERSA_ERR_INVALID_ARG;
+  const Plan& p = ctx->plan;
+  const Ws& w = ctx->ws;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DeviceGuard guard(p.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  wersa_status s = clear_status_once(ctx, st);
+  if (s != WERSA_OK) return s;
+  int launches = 0;
+  const int kind = p.bf16 ? 1 : 0;
+  WERSA_CUDA(launch_qmean_gate(p, w, Q, gate_w, gate_b, omega, st, &launches));
+  if (p.use_tc) {
+    WERSA_CUDA(launch_tc_prepare_w(p, w, W, st, &launches));
+    WERSA_CUDA(launch_tc_kside(p, w, K, V, st, &launches));
+    WERSA_CUDA(launch_reduce_partials(p, w.spart, w.zpart, p.tchunks, w.S, w.z, w.Sbf, st, &launches));
+    WERSA_CUDA(launch_tc_qside(p, w, Q, beta, O, st, &launches));
+  } else {
+    WERSA_CUDA(launch_haar_filter(p, Q, kind, w.f, w.QF, 0, st, &launches));
+    WERSA_CUDA(launch_haar_filter(p, K, kind, w.f, w.KF, 0, st, &launches));
+    WERSA_CUDA(launch_simt_kside(p, w, V, W, st, &launches));
+    WERSA_CUDA(launch_reduce_partials(p, w.spart, w.zpart, p.schunks, w.S, w.z, nullptr, st, &launches));
+    WERSA_CUDA(launch_simt_qside(p, w, W, beta, O, st, &launches));
+  }
+  ctx->launches_fwd = launches;
+  ctx->forward_done = true;
+  return WERSA_OK;
+}
+
+wersa_status wersa_backward(wersa_ctx* ctx, const void* Q, const void* K, const void* V, const void* W,
+                            const float* beta, const float* gate_w, const float* gate_b, const float* omega,
+                            const void* dO, void* dQ, void* dK, void* dV, float* dbeta, float* dgate_w,
+                            float* dgate_b, float* domega, void* cuda_stream) {
+  (void)gate_b;
+  if (ctx == nullptr || Q == nullptr || K == nullptr || V == nullptr || W == nullptr || beta == nullptr ||
+      omega == nullptr || dO == nullptr || dQ == nullptr || dK == nullptr || dV == nullptr)
+    return WERSA_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(W) || !aligned16(dO) || !aligned16(dQ) ||
+      !aligned16(dK) || !aligned16(dV))
+    return WERSA_ERR_INVALID_ARG;
+  const Plan& p = ctx->plan;
+  if (!p.with_backward) return WERSA_ERR_UNSUPPORTED;
+  if (!ctx->forward_done) return WERSA_ERR_STATE;
+  const Ws& w = ctx->ws;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DeviceGuard guard(p.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  int launches = 0;
+  const int kind = p.bf16 ? 1 : 0, gkind = p.grad_bf16 ? 1 : 0;
+  if (p.use_tc) {   // the tensor-core forward keeps Q_F, K_F on chip: rebuild them
+    WERSA_CUDA(launch_haar_filter(p, Q, kind, w.f, w.QF, 0, st, &launches));
+    WERSA_CUDA(launch_haar_filter(p, K, kind, w.f, w.KF, 0, st, &launches));
+  }
+  WERSA_CUDA(launch_simt_bwd_qside(p, w, W, beta, dO, st, &launches));
+  WERSA_CUDA(launch_reduce_partials(p, w.spart, w.zpart, p.schunks, w.dS, w.dz, nullptr, st, &launches));
+  WERSA_CUDA(launch_simt_bwd_kside(p, w, V, W, dV, st, &launches));
+  WERSA_CUDA(launch_haar_backward(p, w, Q, kind, w.dQF, dQ, gkind, 0, st, &launches));
+  WERSA_CUDA(launch_haar_backward(p, w, K, kind, w.dKF, dK, gkind, 1, st, &launches));
+  WERSA_CUDA(launch_gate_backward(p, w, beta, gate_w, omega, dbeta, dgate_w, dgate_b, domega, st, &launches));
+  if (gate_w != nullptr) WERSA_CUDA(launch_add_rowvec(p, w, dQ, st, &launches));
+  ctx->launches_bwd = launches;
+  return WERSA_OK;
+}
+
+wersa_status wersa_haar_filter(wersa_ctx* ctx, const void* X, const float* f, void* XF, void* cuda_stream) {
+  if (ctx == nullptr || X == nullptr || f == nullptr || XF == nullptr) return WERSA_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(XF)) return WERSA_ERR_INVALID_ARG;
+  const Plan& p = ctx->plan;
+  DeviceGuard guard(p.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  int launches = 0;
+  const int kind = p.bf16 ? 1 : 0;
+  WERSA_CUDA(launch_haar_filter(p, X, kind, f, XF, kind, static_cast<cudaStream_t>(cuda_stream), &launches));
+  return WERSA_OK;
+}
+
+wersa_status wersa_saved(wersa_ctx* ctx, int which, const float** device_ptr, size_t* count) {
+  if (ctx == nullptr || device_ptr == nullptr || count == nullptr) return WERSA_ERR_INVALID_ARG;
+  if (!ctx->forward_done) return WERSA_ERR_STATE;
+  const Plan& p = ctx->plan;
+  const size_t slabs = (size_t)p.slabs;
+  switch (which) {
+    case 0: *device_ptr = ctx->ws.f; *count = slabs * p.L1; break;
+    case 1: *device_ptr = ctx->ws.qbar; *count = slabs * kD; break;
+    case 2: *device_ptr = ctx->ws.S; *count = slabs * p.cfg.features * kD; break;
+    case 3: *device_ptr = ctx->ws.z; *count = slabs * p.cfg.features; break;
+    default: return WERSA_ERR_INVALID_ARG;
+  }
+  return WERSA_OK;
+}
+
+wersa_status wersa_query_status(wersa_ctx* ctx, void* cuda_stream) {
+  if (ctx == nullptr) return WERSA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DeviceGuard guard(ctx->plan.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  WERSA_CUDA(cudaStreamSynchronize(st));
+  if (!ctx->status_cleared) return WERSA_OK;   // nothing has run yet
+  int word = 0;
+  WERSA_CUDA(cudaMemcpyAsync(&word, ctx->ws.status, sizeof(int), cudaMemcpyDeviceToHost, st));
+  WERSA_CUDA(cudaStreamSynchronize(st));
+  if (word != 0) {
+    WERSA_CUDA(cudaMemsetAsync(ctx->ws.status, 0, 256, st));
+    WERSA_CUDA(cudaStreamSynchronize(st));
+    return WERSA_ERR_TIMEOUT;
+  }
+  return WERSA_OK;
+}
+
+wersa_status wersa_destroy(wersa_ctx* ctx) {
+  delete ctx;
+  return WERSA_OK;
+}
+
+const char* wersa_status_string(wersa_status status) {
+  switch (status) {
+    case WERSA_OK: return "ok";
+    case WERSA_ERR_INVALID_ARG: return "invalid argument";
+    case WERSA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case WERSA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case WERSA_ERR_CUDA: return "CUDA runtime error";
+    case WERSA_ERR_TIMEOUT: return "bounded device wait expired";
+    case WERSA_ERR_STATE: return "backward or saved-tensor query without a preceding forward";
+  }
+  return "unknown status";
+}
+
+int32_t wersa_launch_count(const wersa_ctx* ctx, int which) {
+  if (ctx == nullptr) return 0;
+  return which == 0 ? ctx->launches_fwd : ctx->launches_bwd;
+}
+
+}  // extern "C"

@@ -1,0 +1,136 @@
+// Shared declarations of the WERSA CUDA library: the host-side plan, the workspace layout and
+// the launch functions each translation unit exports to the C-ABI layer (api.cu).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/wersa.h"
+
+namespace wersa {
+
+constexpr int kD = 64;           // head dim (fixed)
+constexpr int kMaxLevels = 8;    // Haar levels supported: block of 2^8 = 256 tokens
+constexpr int kHaarTile = 256;   // tokens per Haar tile (>= 2^kMaxLevels)
+constexpr int kSimtTile = 32;    // tokens per tile in the fp32 FFMA kernels
+constexpr int kBandVals = 16;    // per-tile band inner products kept by the Haar backward
+
+// Host-side plan: problem sizes, chunking and byte offsets into the caller's workspace.
+struct Plan {
+  wersa_config cfg;
+  int slabs;          // B*H
+  int L1;             // levels + 1
+  bool bf16;          // storage type of Q,K,V,W,O,dO
+  bool grad_bf16;     // storage type of dQ,dK,dV
+  bool use_tc;        // bf16 tcgen05 forward kernels
+  bool with_backward;
+  // mean pool
+  int qchunks, qchunk_rows;
+  // haar tiles
+  int htiles;
+  // fp32 FFMA key-side / backward query-side split of the sequence
+  int schunks, schunk_tiles;   // chunks per slab, 32-token tiles per chunk
+  // tcgen05 key-side split
+  int tchunks, tchunk_tiles;   // chunks per slab, 128-token tiles per chunk
+  // workspace offsets (bytes)
+  size_t off_status, off_qpart, off_qbar, off_sg, off_f, off_spart, off_zpart, off_S, off_z,
+      off_Sbf, off_Wt, off_dS, off_dz, off_sumdD, off_bands, off_dqbar, off_QF, off_KF, off_dQF,
+      off_dKF, total;
+  int part_chunks;    // max(schunks, tchunks): leading extent of the partial buffers
+};
+
+// Fills `p` from `cfg`; returns WERSA_OK, WERSA_ERR_INVALID_ARG or WERSA_ERR_UNSUPPORTED.
+wersa_status make_plan(const wersa_config& cfg, Plan* p);
+
+struct Ws {   // resolved workspace pointers
+  int* status;
+  float *qpart, *qbar, *sg, *f, *spart, *zpart, *S, *z, *dS, *dz, *sumdD, *bands, *dqbar;
+  __nv_bfloat16 *Sbf, *Wt;
+  float *QF, *KF, *dQF, *dKF;
+};
+Ws resolve(const Plan& p, void* workspace);
+
+// ---- gate.cu -------------------------------------------------------------------------------
+// Partial column sums of Q over row chunks, then qbar, sigmoid(u) and f per slab (Eqs. 1-3).
+cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const float* gate_w,
+                              const float* gate_b, const float* omega, cudaStream_t st, int* launches);
+// Gate backward: band inner products -> df -> domega, dgate_b, dgate_w, dqbar; dbeta.
+cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, const float* gate_w,
+                                 const float* omega, float* dbeta, float* dgate_w, float* dgate_b,
+                                 float* domega, cudaStream_t st, int* launches);
+// dQ[s,t,:] += dqbar[s,:] / n.
+cudaError_t launch_add_rowvec(const Plan& p, const Ws& w, void* dQ, cudaStream_t st, int* launches);
+
+// ---- haar.cu -------------------------------------------------------------------------------
+// XF = T_f(X).  in_kind/out_kind: 0 = float, 1 = bf16.
+cudaError_t launch_haar_filter(const Plan& p, const void* X, int in_kind, const float* f, void* XF,
+                               int out_kind, cudaStream_t st, int* launches);
+// dX = T_f(G) (G fp32) and per-tile band inner products of (G, X) into bands[which].
+cudaError_t launch_haar_backward(const Plan& p, const Ws& w, const void* X, int in_kind,
+                                 const float* G, void* dX, int out_kind, int which, cudaStream_t st,
+                                 int* launches);
+
+// ---- simt.cu -------------------------------------------------------------------------------
+cudaError_t launch_simt_kside(const Plan& p, const Ws& w, const void* V, const void* W,
+                              cudaStream_t st, int* launches);
+// S = sum_chunks spart, z = sum_chunks zpart in chunk order (also used for dS, dz).
+cudaError_t launch_reduce_partials(const Plan& p, const float* spart, const float* zpart, int chunks,
+                                   float* S, float* z, __nv_bfloat16* Sbf, cudaStream_t st,
+                                   int* launches);
+cudaError_t launch_simt_qside(const Plan& p, const Ws& w, const void* W, const float* beta, void* O,
+                              cudaStream_t st, int* launches);
+cudaError_t launch_simt_bwd_qside(const Plan& p, const Ws& w, const void* W, const float* beta,
+                                  const void* dO, cudaStream_t st, int* launches);
+cudaError_t launch_simt_bwd_kside(const Plan& p, const Ws& w, const void* V, const void* W, void* dV,
+                                  cudaStream_t st, int* launches);
+
+// ---- tc_fwd.cu -----------------------------------------------------------------------------
+cudaError_t launch_tc_prepare_w(const Plan& p, const Ws& w, const void* W, cudaStream_t st,
+                                int* launches);
+cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const void* V, cudaStream_t st,
+                            int* launches);
+cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const float* beta, void* O,
+                            cudaStream_t st, int* launches);
+
+// ---- device helpers ------------------------------------------------------------------------
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) {
+  return __float2bfloat16_rn(x);
+}
+
+// Loads 8 consecutive elements (16-byte aligned for bf16, 32-byte for float) as floats.
+__device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
+  float4 a = *reinterpret_cast<const float4*>(p);
+  float4 b = *reinterpret_cast<const float4*>(p + 4);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+  v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
+  uint4 raw = *reinterpret_cast<const uint4*>(p);
+  const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(u[i] << 16);
+    v[2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
+  }
+}
+__device__ __forceinline__ void store8(float* p, const float (&v)[8]) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+  *reinterpret_cast<float4*>(p + 4) = make_float4(v[4], v[5], v[6], v[7]);
+}
+__device__ __forceinline__ void store8(__nv_bfloat16* p, const float (&v)[8]) {
+  uint4 raw;
+  uint32_t* u = reinterpret_cast<uint32_t*>(&raw);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+    u[i] = *reinterpret_cast<uint32_t*>(&h);
+  }
+  *reinterpret_cast<uint4*>(p) = raw;
+}
+
+}  // namespace wersa

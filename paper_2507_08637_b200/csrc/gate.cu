@@ -1,0 +1,237 @@
+// Mean-pooled query, content-adaptive gate (Eqs. 1-3 of the WERSA paper) and its backward pass.
+#include "common.cuh"
+
+namespace wersa {
+namespace {
+
+// Partial column sums of one row chunk of one slab of Q.  grid (qchunks, slabs), block 256:
+// thread (cg = tid & 7, rl = tid >> 3) owns 8 consecutive columns and every 32nd row, loads
+// 16 bytes (bf16) / 32 bytes (fp32) per row, four rows in flight.
+template <typename T>
+__global__ void __launch_bounds__(256) k_qmean_partial(const T* __restrict__ Q, float* __restrict__ qpart,
+                                                       int n, int chunk_rows) {
+  const int chunk = blockIdx.x, slab = blockIdx.y;
+  const int cg = threadIdx.x & 7, rl = threadIdx.x >> 3;
+  const int r0 = chunk * chunk_rows;
+  const int r1 = min(n, r0 + chunk_rows);
+  const T* base = Q + (size_t)slab * n * kD + cg * 8;
+  float acc[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+  int r = r0 + rl;
+  for (; r + 96 < r1; r += 128) {
+    float v0[8], v1[8], v2[8], v3[8];
+    load8(base + (size_t)r * kD, v0);
+    load8(base + (size_t)(r + 32) * kD, v1);
+    load8(base + (size_t)(r + 64) * kD, v2);
+    load8(base + (size_t)(r + 96) * kD, v3);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] += (v0[j] + v1[j]) + (v2[j] + v3[j]);
+  }
+  for (; r < r1; r += 32) {
+    float v0[8];
+    load8(base + (size_t)r * kD, v0);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] += v0[j];
+  }
+  __shared__ float red[32][kD + 1];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) red[rl][cg * 8 + j] = acc[j];
+  __syncthreads();
+  if (threadIdx.x < kD) {
+    float s = 0.f;
+#pragma unroll 8
+    for (int i = 0; i < 32; ++i) s += red[i][threadIdx.x];   // fixed order
+    qpart[((size_t)slab * gridDim.x + chunk) * kD + threadIdx.x] = s;
+  }
+}
+
+// One CTA per batch element, 64 threads (one per column).  qbar = sum of partials / n (Eq. 1),
+// u = gate_w^T qbar + gate_b (Eq. 2), f = sigmoid(u) * omega (Eq. 3).
+__global__ void __launch_bounds__(kD) k_gate(const float* __restrict__ qpart, int qchunks, int H, int n,
+                                             int L1, int per_head, const float* __restrict__ gate_w,
+                                             const float* __restrict__ gate_b,
+                                             const float* __restrict__ omega, float* __restrict__ qbar,
+                                             float* __restrict__ sg, float* __restrict__ f) {
+  const int b = blockIdx.x, c = threadIdx.x;
+  __shared__ float qs[kD];
+  __shared__ float utot[kMaxLevels + 1];
+  if (c <= kMaxLevels) utot[c] = 0.f;
+  for (int h = 0; h < H; ++h) {
+    const int slab = b * H + h;
+    float s = 0.f;
+    for (int k = 0; k < qchunks; ++k) s += qpart[((size_t)slab * qchunks + k) * kD + c];
+    s = s / (float)n;
+    qbar[(size_t)slab * kD + c] = s;
+    __syncthreads();
+    qs[c] = s;
+    __syncthreads();
+    if (c < L1) {
+      float u = 0.f;
+      if (gate_w != nullptr)
+        for (int k = 0; k < kD; ++k) u += gate_w[((size_t)h * kD + k) * L1 + c] * qs[k];
+      if (per_head) {
+        if (gate_b != nullptr) u += gate_b[h * L1 + c];
+        float sgm = 1.f / (1.f + expf(-u));
+        sg[(size_t)slab * L1 + c] = sgm;
+        f[(size_t)slab * L1 + c] = sgm * omega[c];
+      } else {
+        utot[c] += u;
+      }
+    }
+  }
+  if (!per_head && c < L1) {
+    float u = utot[c] + (gate_b != nullptr ? gate_b[c] : 0.f);
+    float sgm = 1.f / (1.f + expf(-u));
+    for (int h = 0; h < H; ++h) {
+      sg[((size_t)b * H + h) * L1 + c] = sgm;
+      f[((size_t)b * H + h) * L1 + c] = sgm * omega[c];
+    }
+  }
+}
+
+// Sum the per-tile band inner products of both filtered tensors in tile order and turn them
+// into df[slab][i]: i < L takes the detail-band product of level i+1, i = L the approximation
+// product of level L.  One CTA per slab, 32 threads.
+__global__ void __launch_bounds__(32) k_band_reduce(const float* __restrict__ bands, int slabs, int htiles,
+                                                    int L, float* __restrict__ df) {
+  const int slab = blockIdx.x, j = threadIdx.x;
+  if (j >= kBandVals) return;
+  float s = 0.f;
+  for (int which = 0; which < 2; ++which) {
+    const float* src = bands + (((size_t)which * slabs + slab) * htiles) * kBandVals;
+    for (int t = 0; t < htiles; ++t) s += src[(size_t)t * kBandVals + j];
+  }
+  // slots 0..7: detail products of levels 1..8; slots 8..15: approximation products of levels 1..8
+  if (j < L) df[(size_t)slab * kBandVals + j] = s;
+  if (j == 8 + L - 1) df[(size_t)slab * kBandVals + L] = s;
+}
+
+// Single CTA, 64 threads (thread c = column).  Chain rule through f = sigmoid(u) * omega,
+// u = gate(qbar): domega, dgate_b, dgate_w, dqbar; and the bandwidth gradient
+// dbeta = 2 eps m bw * sum_t dDh_t (ReLU is positively homogeneous, so beta only acts through eps).
+__global__ void __launch_bounds__(kD) k_gate_backward(
+    const float* __restrict__ df, const float* __restrict__ sg, const float* __restrict__ qbar,
+    const float* __restrict__ gate_w, const float* __restrict__ omega, const float* __restrict__ sumdD,
+    int n_sumdD, const float* __restrict__ beta, float eps, float bw_floor, int m, int B, int H, int L1,
+    int per_head, float* __restrict__ dbeta, float* __restrict__ dgate_w, float* __restrict__ dgate_b,
+    float* __restrict__ domega, float* __restrict__ dqbar) {
+  const int c = threadIdx.x;
+  __shared__ float du[kMaxLevels + 1];
+  for (int h = 0; h < H; ++h) {
+    float gw_acc[kMaxLevels + 1], gb_acc = 0.f;
+#pragma unroll
+    for (int i = 0; i <= kMaxLevels; ++i) gw_acc[i] = 0.f;
+    for (int b = 0; b < B; ++b) {
+      const int slab = b * H + h;
+      __syncthreads();
+      if (c < L1) {
+        float dfi = 0.f;
+        if (per_head) {
+          dfi = df[(size_t)slab * kBandVals + c];
+        } else {
+          for (int hh = 0; hh < H; ++hh) dfi += df[((size_t)b * H + hh) * kBandVals + c];
+        }
+        float s = sg[(size_t)slab * L1 + c];
+        du[c] = dfi * omega[c] * s * (1.f - s);
+        if (per_head || h == 0) gb_acc += du[c];
+      }
+      __syncthreads();
+      float dq = 0.f;
+      const float qb = qbar[(size_t)slab * kD + c];
+#pragma unroll
+      for (int i = 0; i <= kMaxLevels; ++i)
+        if (i < L1) {
+          gw_acc[i] += qb * du[i];
+          if (gate_w != nullptr) dq += gate_w[((size_t)h * kD + c) * L1 + i] * du[i];
+        }
+      dqbar[(size_t)slab * kD + c] = dq;
+    }
+    if (dgate_w != nullptr) {
+#pragma unroll
+      for (int i = 0; i <= kMaxLevels; ++i)
+        if (i < L1) dgate_w[((size_t)h * kD + c) * L1 + i] = gw_acc[i];
+    }
+    if (dgate_b != nullptr && c < L1) dgate_b[h * L1 + c] = (per_head || h == 0) ? gb_acc : 0.f;
+  }
+  if (domega != nullptr && c < L1) {
+    float acc = 0.f;
+    for (int b = 0; b < B; ++b) {
+      if (per_head) {
+        for (int h = 0; h < H; ++h) {
+          const int slab = b * H + h;
+          acc += df[(size_t)slab * kBandVals + c] * sg[(size_t)slab * L1 + c];
+        }
+      } else {
+        float dfi = 0.f;
+        for (int h = 0; h < H; ++h) dfi += df[((size_t)b * H + h) * kBandVals + c];
+        acc += dfi * sg[((size_t)b * H) * L1 + c];
+      }
+    }
+    domega[c] = acc;
+  }
+  if (dbeta != nullptr && c == 0) {
+    float tot = 0.f;
+    for (int i = 0; i < n_sumdD; ++i) tot += sumdD[i];
+    const float bt = beta[0];
+    const float bw = fmaxf(bt, bw_floor);
+    dbeta[0] = bt > bw_floor ? 2.f * eps * (float)m * bw * tot : 0.f;
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) k_add_rowvec(T* __restrict__ dQ, const float* __restrict__ dqbar,
+                                                    int n, float inv_n) {
+  const int slab = blockIdx.y;
+  const size_t idx8 = (size_t)blockIdx.x * 256 + threadIdx.x;   // group of 8 elements in the slab
+  if (idx8 >= (size_t)n * (kD / 8)) return;
+  const int cg = (int)(idx8 & 7);
+  T* p = dQ + (size_t)slab * n * kD + idx8 * 8;
+  float v[8];
+  load8(p, v);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) v[j] += dqbar[(size_t)slab * kD + cg * 8 + j] * inv_n;
+  store8(p, v);
+}
+
+}  // namespace
+
+cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const float* gate_w,
+                              const float* gate_b, const float* omega, cudaStream_t st, int* launches) {
+  dim3 grid(p.qchunks, p.slabs);
+  if (p.bf16)
+    k_qmean_partial<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)Q, w.qpart, p.cfg.seq_len,
+                                                         p.qchunk_rows);
+  else
+    k_qmean_partial<float><<<grid, 256, 0, st>>>((const float*)Q, w.qpart, p.cfg.seq_len, p.qchunk_rows);
+  k_gate<<<p.cfg.batch, kD, 0, st>>>(w.qpart, p.qchunks, p.cfg.heads, p.cfg.seq_len, p.L1,
+                                     p.cfg.gate_per_head, gate_w, gate_b, omega, w.qbar, w.sg, w.f);
+  *launches += 2;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, const float* gate_w,
+                                 const float* omega, float* dbeta, float* dgate_w, float* dgate_b,
+                                 float* domega, cudaStream_t st, int* launches) {
+  float* df = w.dqbar + (size_t)p.slabs * kD;   // df lives behind dqbar in the same region
+  k_band_reduce<<<p.slabs, 32, 0, st>>>(w.bands, p.slabs, p.htiles, p.cfg.levels, df);
+  k_gate_backward<<<1, kD, 0, st>>>(df, w.sg, w.qbar, gate_w, omega, w.sumdD, p.slabs * p.schunks, beta,
+                                    p.cfg.eps, p.cfg.bw_floor, p.cfg.features, p.cfg.batch, p.cfg.heads,
+                                    p.L1, p.cfg.gate_per_head, dbeta, dgate_w, dgate_b, domega, w.dqbar);
+  *launches += 2;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_add_rowvec(const Plan& p, const Ws& w, void* dQ, cudaStream_t st, int* launches) {
+  const size_t groups = (size_t)p.cfg.seq_len * (kD / 8);
+  dim3 grid((unsigned)((groups + 255) / 256), p.slabs);
+  const float inv_n = 1.f / (float)p.cfg.seq_len;
+  if (p.grad_bf16)
+    k_add_rowvec<__nv_bfloat16><<<grid, 256, 0, st>>>((__nv_bfloat16*)dQ, w.dqbar, p.cfg.seq_len, inv_n);
+  else
+    k_add_rowvec<float><<<grid, 256, 0, st>>>((float*)dQ, w.dqbar, p.cfg.seq_len, inv_n);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
+}  // namespace wersa

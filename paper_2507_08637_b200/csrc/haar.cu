@@ -1,0 +1,257 @@
+// Multi-level Haar analysis -> per-scale gating -> synthesis along the sequence, as one on-chip
+// pass over tiles of 256 tokens (Sec. 3.1 steps 3, 5, 6 and Algorithm 2 of the WERSA paper).
+//
+// Because the Haar detail projector of level l equals blockmean_{2^(l-1)} - blockmean_{2^l} and
+// the approximation projector of level L equals blockmean_{2^L}, the filtered signal is
+//   T_f x = f_0 x + sum_{i=1..L} (f_i - f_{i-1}) * blockmean_{2^i}(x),
+// so one pass needs only the aligned block sums of 2, 4, ..., 2^L rows.  A thread holds 8
+// consecutive rows x 8 columns in registers (levels 1-3), partner lanes give levels 4-5 through
+// warp shuffles and the eight warps exchange their 32-row sums through shared memory (levels 6-8).
+// Rows past the end of the sequence read as zero, which is the zero padding of Algorithm 2.
+#include "common.cuh"
+
+namespace wersa {
+namespace {
+
+struct LevelCoef {
+  float f0;
+  float k[kMaxLevels + 1];   // k[i] = (f_i - f_{i-1}) / 2^i for 1 <= i <= L, else 0
+};
+
+__device__ __forceinline__ LevelCoef level_coef(const float* __restrict__ f, int L) {
+  LevelCoef c;
+  c.f0 = f[0];
+  float scale = 0.5f;
+#pragma unroll
+  for (int i = 1; i <= kMaxLevels; ++i) {
+    c.k[i] = (i <= L) ? (f[i] - f[i - 1]) * scale : 0.f;
+    scale *= 0.5f;
+  }
+  c.k[0] = 0.f;
+  return c;
+}
+
+// Block sums of the 8x8 register tile and of its partners.  s1[4], s2[2], s3..s8 per column.
+struct Sums {
+  float s1[4][8], s2[2][8], s3[8], s4[8], s5[8], s6[8], s7[8], s8[8];
+  float p3[8], p4[8], p5[8], p6[8], p7[8];   // the partner's half at levels 4..8 (for details)
+};
+
+__device__ __forceinline__ void block_sums(const float (&x)[8][8], Sums& s, float (*sh)[kD], int L) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, cg = threadIdx.x & 7;
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+#pragma unroll
+    for (int p = 0; p < 4; ++p) s.s1[p][c] = x[2 * p][c] + x[2 * p + 1][c];
+    s.s2[0][c] = s.s1[0][c] + s.s1[1][c];
+    s.s2[1][c] = s.s1[2][c] + s.s1[3][c];
+    s.s3[c] = s.s2[0][c] + s.s2[1][c];
+    s.p3[c] = __shfl_xor_sync(0xffffffffu, s.s3[c], 8);
+    s.s4[c] = s.s3[c] + s.p3[c];
+    s.p4[c] = __shfl_xor_sync(0xffffffffu, s.s4[c], 16);
+    s.s5[c] = s.s4[c] + s.p4[c];
+    s.s6[c] = s.s7[c] = s.s8[c] = 0.f;
+    s.p5[c] = s.p6[c] = s.p7[c] = 0.f;
+  }
+  if (L > 5) {   // uniform over the grid
+    __syncthreads();   // previous use of sh is over
+    if ((lane >> 3) == 0) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) sh[warp][cg * 8 + c] = s.s5[c];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const int col = cg * 8 + c;
+      s.p5[c] = sh[warp ^ 1][col];
+      s.s6[c] = s.s5[c] + s.p5[c];
+      s.p6[c] = sh[warp ^ 2][col] + sh[warp ^ 3][col];
+      s.s7[c] = s.s6[c] + s.p6[c];
+      s.p7[c] = (sh[warp ^ 4][col] + sh[warp ^ 5][col]) + (sh[warp ^ 6][col] + sh[warp ^ 7][col]);
+      s.s8[c] = s.s7[c] + s.p7[c];
+    }
+  }
+}
+
+__device__ __forceinline__ void apply_filter(float (&x)[8][8], const Sums& s, const LevelCoef& k) {
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    const float hi = k.k[3] * s.s3[c] + k.k[4] * s.s4[c] + k.k[5] * s.s5[c] + k.k[6] * s.s6[c] +
+                     k.k[7] * s.s7[c] + k.k[8] * s.s8[c];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      x[j][c] = k.f0 * x[j][c] + k.k[1] * s.s1[j >> 1][c] + k.k[2] * s.s2[j >> 2][c] + hi;
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ void load_tile(const T* __restrict__ X, int n, int row0, float (&x)[8][8]) {
+  const int cg = threadIdx.x & 7;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int r = row0 + j;
+    if (r < n) {
+      load8(X + (size_t)r * kD + cg * 8, x[j]);
+    } else {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) x[j][c] = 0.f;
+    }
+  }
+}
+
+// grid (htiles, slabs), block 256.
+template <typename Tin, typename Tout>
+__global__ void __launch_bounds__(256, 2) k_haar_filter(const Tin* __restrict__ X, const float* __restrict__ f,
+                                                     Tout* __restrict__ XF, int n, int L) {
+  __shared__ float sh[8][kD];
+  const int slab = blockIdx.y;
+  const int cg = threadIdx.x & 7, rg = threadIdx.x >> 3;
+  const int row0 = blockIdx.x * kHaarTile + rg * 8;
+  const LevelCoef k = level_coef(f + (size_t)slab * (L + 1), L);
+  float x[8][8];
+  load_tile(X + (size_t)slab * n * kD, n, row0, x);
+  Sums s;
+  block_sums(x, s, sh, L);
+  apply_filter(x, s, k);
+  Tout* dst = XF + (size_t)slab * n * kD + cg * 8;
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    if (row0 + j < n) store8(dst + (size_t)(row0 + j) * kD, x[j]);
+}
+
+// Backward of the filter for one tile: dX = T_f(G) (the operator is symmetric) and the band
+// inner products of (G, X) that give df:
+//   slot l-1 (l = 1..8): sum over blocks of Delta_l(G) * Delta_l(X) / 2^l, the product of the
+//                        level-l detail coefficients (Delta_l = left half sum - right half sum);
+//   slot 8+l-1:          sum over blocks of s_l(G) * s_l(X) / 2^l, the product of the level-l
+//                        approximation coefficients.
+template <typename Tin, typename Tout>
+__global__ void __launch_bounds__(256) k_haar_backward(const Tin* __restrict__ X, const float* __restrict__ G,
+                                                       const float* __restrict__ f, Tout* __restrict__ dX,
+                                                       float* __restrict__ bands, int n, int L) {
+  __shared__ float sh[8][kD];
+  __shared__ float red[8][kBandVals];
+  const int slab = blockIdx.y;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int cg = threadIdx.x & 7, rg = threadIdx.x >> 3;
+  const int row0 = blockIdx.x * kHaarTile + rg * 8;
+  const LevelCoef k = level_coef(f + (size_t)slab * (L + 1), L);
+  float acc[kBandVals];
+#pragma unroll
+  for (int i = 0; i < kBandVals; ++i) acc[i] = 0.f;
+  float g[8][8];
+  Sums sg;
+  load_tile(G + (size_t)slab * n * kD, n, row0, g);
+  block_sums(g, sg, sh, L);
+  {
+    Tout* dst = dX + (size_t)slab * n * kD + cg * 8;
+    // same expression as apply_filter, row by row, so that g survives for the band products
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      float y[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const float hi = k.k[3] * sg.s3[c] + k.k[4] * sg.s4[c] + k.k[5] * sg.s5[c] + k.k[6] * sg.s6[c] +
+                         k.k[7] * sg.s7[c] + k.k[8] * sg.s8[c];
+        y[c] = k.f0 * g[j][c] + k.k[1] * sg.s1[j >> 1][c] + k.k[2] * sg.s2[j >> 2][c] + hi;
+      }
+      if (row0 + j < n) store8(dst + (size_t)(row0 + j) * kD, y);
+    }
+  }
+  {
+    float x[8][8];
+    Sums sx;
+    load_tile(X + (size_t)slab * n * kD, n, row0, x);
+    block_sums(x, sx, sh, L);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+#pragma unroll
+      for (int p = 0; p < 4; ++p) {
+        acc[0] += (g[2 * p][c] - g[2 * p + 1][c]) * (x[2 * p][c] - x[2 * p + 1][c]);
+        acc[8] += sg.s1[p][c] * sx.s1[p][c];
+      }
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        acc[1] += (sg.s1[2 * q][c] - sg.s1[2 * q + 1][c]) * (sx.s1[2 * q][c] - sx.s1[2 * q + 1][c]);
+        acc[9] += sg.s2[q][c] * sx.s2[q][c];
+      }
+      acc[2] += (sg.s2[0][c] - sg.s2[1][c]) * (sx.s2[0][c] - sx.s2[1][c]);
+      acc[10] += sg.s3[c] * sx.s3[c];
+      // levels 4..8: every lane of a block holds the same block sum; the weights undo the
+      // replication (2, 4, 8, 16, 32 holders per column).
+      acc[3] += (sg.s3[c] - sg.p3[c]) * (sx.s3[c] - sx.p3[c]);
+      acc[11] += sg.s4[c] * sx.s4[c];
+      acc[4] += (sg.s4[c] - sg.p4[c]) * (sx.s4[c] - sx.p4[c]);
+      acc[12] += sg.s5[c] * sx.s5[c];
+      acc[5] += (sg.s5[c] - sg.p5[c]) * (sx.s5[c] - sx.p5[c]);
+      acc[13] += sg.s6[c] * sx.s6[c];
+      acc[6] += (sg.s6[c] - sg.p6[c]) * (sx.s6[c] - sx.p6[c]);
+      acc[14] += sg.s7[c] * sx.s7[c];
+      acc[7] += (sg.s7[c] - sg.p7[c]) * (sx.s7[c] - sx.p7[c]);
+      acc[15] += sg.s8[c] * sx.s8[c];
+    }
+  }
+  // 1/2^l normalisation times 1/replication.
+  const float wgt[8] = {0.5f, 0.25f, 0.125f, 0.0625f * 0.5f, 0.03125f * 0.25f, 0.015625f * 0.125f,
+                        0.0078125f * 0.0625f, 0.00390625f * 0.03125f};
+#pragma unroll
+  for (int l = 0; l < 8; ++l) {
+    acc[l] *= wgt[l];
+    acc[8 + l] *= wgt[l];
+  }
+#pragma unroll
+  for (int i = 0; i < kBandVals; ++i) {
+    float v = acc[i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (lane == 0) red[warp][i] = v;
+  }
+  __syncthreads();
+  if (threadIdx.x < kBandVals) {
+    float v = 0.f;
+#pragma unroll
+    for (int wi = 0; wi < 8; ++wi) v += red[wi][threadIdx.x];
+    bands[((size_t)slab * gridDim.x + blockIdx.x) * kBandVals + threadIdx.x] = v;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_haar_filter(const Plan& p, const void* X, int in_kind, const float* f, void* XF,
+                               int out_kind, cudaStream_t st, int* launches) {
+  dim3 grid(p.htiles, p.slabs);
+  const int n = p.cfg.seq_len, L = p.cfg.levels;
+  if (in_kind == 1 && out_kind == 1)
+    k_haar_filter<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, f,
+                                                                       (__nv_bfloat16*)XF, n, L);
+  else if (in_kind == 1 && out_kind == 0)
+    k_haar_filter<__nv_bfloat16, float><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, f, (float*)XF, n, L);
+  else if (in_kind == 0 && out_kind == 0)
+    k_haar_filter<float, float><<<grid, 256, 0, st>>>((const float*)X, f, (float*)XF, n, L);
+  else
+    k_haar_filter<float, __nv_bfloat16><<<grid, 256, 0, st>>>((const float*)X, f, (__nv_bfloat16*)XF, n, L);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_haar_backward(const Plan& p, const Ws& w, const void* X, int in_kind, const float* G,
+                                 void* dX, int out_kind, int which, cudaStream_t st, int* launches) {
+  dim3 grid(p.htiles, p.slabs);
+  const int n = p.cfg.seq_len, L = p.cfg.levels;
+  float* bands = w.bands + (size_t)which * p.slabs * p.htiles * kBandVals;
+  if (in_kind == 1 && out_kind == 1)
+    k_haar_backward<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
+        (const __nv_bfloat16*)X, G, w.f, (__nv_bfloat16*)dX, bands, n, L);
+  else if (in_kind == 1 && out_kind == 0)
+    k_haar_backward<__nv_bfloat16, float><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, G, w.f, (float*)dX,
+                                                               bands, n, L);
+  else if (in_kind == 0 && out_kind == 0)
+    k_haar_backward<float, float><<<grid, 256, 0, st>>>((const float*)X, G, w.f, (float*)dX, bands, n, L);
+  else
+    k_haar_backward<float, __nv_bfloat16><<<grid, 256, 0, st>>>((const float*)X, G, w.f, (__nv_bfloat16*)dX,
+                                                               bands, n, L);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
+}  // namespace wersa

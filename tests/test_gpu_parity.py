@@ -1,0 +1,295 @@
+"""GPU parity tests: the CUDA library, called through its C ABI (ctypes binding), against the
+float64 CPU oracle on the same seeded inputs.  Tolerances: fp32 storage max normalised error
+1e-4; bf16 storage max 2e-2 and mean 3e-3 (errors normalised by max(|ref|, slab rms))."""
+import numpy as np
+import pytest
+
+import wersa_inputs as wi
+from oracle import wersa_oracle as orc
+from tests.util import device_inputs, normalised_error, small_vector_error, to_device, to_numpy64
+
+pytestmark = pytest.mark.gpu
+
+F32_MAX = 1e-4
+BF16_MAX, BF16_MEAN = 2e-2, 3e-3
+
+
+def _ctx(cfg, **kw):
+    import paper_2507_08637_b200 as wersa
+    args = dict(dtype=cfg["dtype"], grad_dtype="f32", eps=cfg.get("eps", 1e-6),
+                gate_per_head=cfg.get("gate_per_head", 1))
+    args.update(kw)
+    return wersa.wersa_create(cfg["B"], cfg["H"], cfg["n"], cfg["d"], cfg["L"], cfg["m"], **args)
+
+
+def _oracle_forward(cfg, inp, **kw):
+    return orc.forward(inp["Q"], inp["K"], inp["V"], inp["W"], float(inp["beta"][0]), inp["gate_w"],
+                       inp["gate_b"], inp["omega"], cfg["L"], eps=cfg.get("eps", 1e-6),
+                       gate_per_head=cfg.get("gate_per_head", 1), **kw)
+
+
+def _check(got, ref, dtype, what=""):
+    err = normalised_error(got, ref)
+    if dtype == "f32":
+        assert err.max() <= F32_MAX, (what, err.max())
+    else:
+        assert err.max() <= BF16_MAX, (what, "max", err.max())
+        assert err.mean() <= BF16_MEAN, (what, "mean", err.mean())
+    return err
+
+
+# ---------------------------------------------------------------- Haar filter kernel
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("n,L", [(8, 3), (256, 8), (1024, 5), (2048, 8), (1000, 3), (300, 4), (77, 2)])
+def test_haar_filter_kernel(n, L, dtype):
+    import torch
+    B, H, d = 2, 3, 64
+    rng = np.random.default_rng(n * 10 + L)
+    X = (rng.standard_normal((B, H, n, d)) + 0.5).astype(np.float32)
+    # multi-scale structure so that every band carries energy
+    X += np.sin(np.arange(n)[None, None, :, None] * 2 * np.pi / 64.0).astype(np.float32)
+    if dtype == "bf16":
+        X = wi.round_to_bf16(X)
+    f = rng.uniform(0.2, 1.5, (B, H, L + 1)).astype(np.float32)
+    cfg = dict(B=B, H=H, n=n, d=d, L=L, m=64, dtype=dtype)
+    ctx = _ctx(cfg)
+    got = ctx.haar_filter(to_device(X, dtype), torch.from_numpy(f).cuda())
+    torch.cuda.synchronize()
+    got = to_numpy64(got)
+    for b in range(B):
+        for h in range(H):
+            ref = orc.haar_filter(X[b, h].astype(np.float64), f[b, h].astype(np.float64))
+            scale = np.abs(ref).max()
+            tol = 2e-6 if dtype == "f32" else 2.0 ** -8
+            assert np.max(np.abs(got[b, h] - ref)) <= tol * scale, (b, h)
+
+
+# ---------------------------------------------------------------- gate
+@pytest.mark.parametrize("per_head", [1, 0])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_gate_and_saved_tensors(dtype, per_head):
+    cfg = dict(B=2, H=3, n=1280, d=64, L=4, m=64, dtype=dtype, gate_per_head=per_head)
+    inp = wi.make_inputs(**cfg, seed=11, w_seed=12, gate_std=0.3, gate_seed=13, mean_shift=0.4)
+    ctx = _ctx(cfg)
+    dev = device_inputs(inp, dtype)
+    ctx.forward(dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    qbar, f = orc.gate(inp["Q"], inp["gate_w"], inp["gate_b"], inp["omega"], cfg["L"], gate_per_head=per_head)
+    assert np.max(np.abs(to_numpy64(ctx.saved("qbar")) - qbar)) < 2e-6
+    assert np.max(np.abs(to_numpy64(ctx.saved("f")) - f)) < 2e-6
+    # the gate must actually have moved away from sigmoid(0)
+    assert np.abs(f - 0.5).max() > 0.05
+
+
+# ---------------------------------------------------------------- forward, small shapes
+SMALL = [
+    dict(B=1, H=1, n=8, d=64, L=3, m=64),
+    dict(B=2, H=2, n=64, d=64, L=3, m=128),
+    dict(B=1, H=3, n=1024, d=64, L=5, m=256),
+    dict(B=2, H=1, n=1000, d=64, L=3, m=64),      # ragged: not a multiple of 32 nor of 2^L
+    dict(B=1, H=2, n=4100, d=64, L=8, m=128),     # several Haar tiles and a ragged tail
+    dict(B=3, H=2, n=512, d=64, L=8, m=256, gate_per_head=0),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("case", range(len(SMALL)))
+def test_forward_small_simt(case, dtype):
+    import paper_2507_08637_b200 as wersa
+    import torch
+    cfg = dict(SMALL[case], dtype=dtype)
+    inp = wi.make_inputs(**cfg, seed=100 + case, w_seed=200 + case, gate_std=0.3, gate_seed=300 + case,
+                         mean_shift=0.25, scale=0.7)
+    ctx = _ctx(cfg, flags=wersa.WERSA_FLAG_SIMT_ONLY)
+    dev = device_inputs(inp, dtype)
+    O = ctx.forward(dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"],
+                    dev["omega"])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    ref, aux = _oracle_forward(cfg, inp, want_aux=True)
+    _check(to_numpy64(O), ref, dtype, "O")
+    # key summary and normaliser (library keeps them without the 1/(bw sqrt(m)) factor)
+    c = 1.0 / (max(float(inp["beta"][0]), 1e-6) * np.sqrt(cfg["m"]))
+    errS = normalised_error(to_numpy64(ctx.saved("S")) * c, aux["S"])
+    errz = normalised_error(to_numpy64(ctx.saved("z")) * c, aux["z"])
+    assert errS.max() < 1e-4 and errz.max() < 1e-4
+    assert ctx.launch_count(0) >= 5
+
+
+def test_forward_is_bit_identical_run_to_run():
+    import paper_2507_08637_b200 as wersa
+    import torch
+    cfg = dict(B=2, H=2, n=4096, d=64, L=6, m=256, dtype="bf16")
+    inp = wi.make_inputs(**cfg, seed=5, w_seed=6, gate_std=0.1, gate_seed=7)
+    dev = device_inputs(inp, "bf16")
+    for flags in (wersa.WERSA_FLAG_SIMT_ONLY, 0):
+        ctx = _ctx(cfg, flags=flags)
+        a = ctx.forward(dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"],
+                        dev["omega"]).clone()
+        b = ctx.forward(dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"],
+                        dev["omega"])
+        torch.cuda.synchronize()
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+# ---------------------------------------------------------------- the five configurations
+def _run_config(name, flags=0, **overrides):
+    import torch
+    cfg, inp = wi.make_config(name, **overrides)
+    ctx = _ctx(cfg, flags=flags)
+    dev = device_inputs(inp, cfg["dtype"])
+    O = ctx.forward(dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"],
+                    dev["omega"])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    return cfg, inp, dev, ctx, O
+
+
+def test_config1_single_head_fp32():
+    cfg, inp, dev, ctx, O = _run_config("cfg1_single_head_fp32")
+    ref = _oracle_forward(cfg, inp)
+    err = _check(to_numpy64(O), ref, "f32", "cfg1")
+    # initial gate values: f = 0.5 everywhere
+    assert np.allclose(to_numpy64(ctx.saved("f")), 0.5, atol=1e-7)
+    print("cfg1 max err", err.max())
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+def test_config2_text_bf16(flags):
+    cfg, inp, dev, ctx, O = _run_config("cfg2_text_bf16", flags=flags)
+    # oracle on a sample of slabs (every slab is independent given its head's gate parameters)
+    got = to_numpy64(O)
+    for (b, h) in [(0, 0), (3, 5), (7, 7)]:
+        sub = {k: (v[b:b + 1, h:h + 1] if k in ("Q", "K", "V") else v) for k, v in inp.items()}
+        sub["gate_w"], sub["gate_b"] = inp["gate_w"][h:h + 1], inp["gate_b"][h:h + 1]
+        ref = _oracle_forward(dict(cfg, B=1, H=1), sub)
+        _check(got[b:b + 1, h:h + 1], ref, "bf16", f"cfg2 slab {b},{h}")
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+def test_config3_vision_bf16(flags):
+    cfg, inp, dev, ctx, O = _run_config("cfg3_vision_bf16", flags=flags)
+    got = to_numpy64(O)
+    for (b, h) in [(0, 0), (17, 3), (63, 11), (40, 8)]:
+        sub = {k: (v[b:b + 1, h:h + 1] if k in ("Q", "K", "V") else v) for k, v in inp.items()}
+        sub["gate_w"], sub["gate_b"] = inp["gate_w"][h:h + 1], inp["gate_b"][h:h + 1]
+        ref = _oracle_forward(dict(cfg, B=1, H=1), sub)
+        _check(got[b:b + 1, h:h + 1], ref, "bf16", f"cfg3 slab {b},{h}")
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+def test_config4_long_sequence_bf16(flags):
+    cfg, inp, dev, ctx, O = _run_config("cfg4_long_bf16", flags=flags)
+    got = to_numpy64(O)
+    n = cfg["n"]
+    rng = np.random.default_rng(0)
+    # whole 256-row Haar blocks at both ends and the middle plus scattered rows
+    rows = np.unique(np.concatenate([np.arange(0, 256), np.arange(n // 2 - 128, n // 2 + 128),
+                                     np.arange(n - 256, n), rng.integers(0, n, 1200)]))
+    for h in (0, 5):
+        sub = {k: (v[:, h:h + 1] if k in ("Q", "K", "V") else v) for k, v in inp.items()}
+        sub["gate_w"], sub["gate_b"] = inp["gate_w"][h:h + 1], inp["gate_b"][h:h + 1]
+        ref, aux = _oracle_forward(dict(cfg, H=1), sub, sample_rows=rows, want_aux=True)
+        # normalise by the rms of the sampled reference rows
+        err = normalised_error(got[:, h:h + 1, rows], ref[:, :, rows])
+        assert err.max() <= BF16_MAX and err.mean() <= BF16_MEAN, (h, err.max(), err.mean())
+        c = 1.0 / np.sqrt(cfg["m"])
+        S = to_numpy64(ctx.saved("S"))[:, h:h + 1] * c
+        assert normalised_error(S, aux["S"]).max() < 2e-2
+
+
+def _check_backward(cfg, inp, grads, sub_slabs=None):
+    ref = orc.backward(inp["Q"], inp["K"], inp["V"], inp["W"], float(inp["beta"][0]), inp["gate_w"],
+                       inp["gate_b"], inp["omega"], inp["dO"], cfg["L"], eps=cfg.get("eps", 1e-6),
+                       gate_per_head=cfg.get("gate_per_head", 1))
+    dtype = cfg["dtype"]
+    for key in ("dQ", "dK", "dV"):
+        _check(to_numpy64(grads[key]), ref[key], dtype, key)
+    tol = 1e-4 if dtype == "f32" else 2e-2
+    for key in ("dgate_w", "dgate_b", "domega"):
+        err = small_vector_error(to_numpy64(grads[key]), ref[key])
+        assert err.max() <= tol, (key, err.max())
+    db = float(grads["dbeta"].cpu()[0])
+    assert abs(db - ref["dbeta_closed"]) <= tol * max(abs(ref["dbeta_closed"]), 1e-30) * 5, (db, ref["dbeta_closed"])
+    return ref
+
+
+BWD_SMALL = [
+    dict(B=1, H=1, n=64, d=64, L=3, m=64),
+    dict(B=2, H=2, n=1024, d=64, L=5, m=128),
+    dict(B=1, H=2, n=1000, d=64, L=8, m=256),
+    dict(B=2, H=3, n=512, d=64, L=4, m=64, gate_per_head=0),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("case", range(len(BWD_SMALL)))
+def test_backward_small(case, dtype):
+    import torch
+    cfg = dict(BWD_SMALL[case], dtype=dtype, eps=1e-3)
+    inp = wi.make_inputs(**cfg, seed=400 + case, w_seed=500 + case, gate_std=0.3, gate_seed=600 + case,
+                         mean_shift=0.25, scale=0.7, backward=True)
+    ctx = _ctx(cfg)
+    dev = device_inputs(inp, dtype)
+    args = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    ctx.forward(*args)
+    grads = ctx.backward(*args, dev["dO"])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    _check_backward(cfg, inp, grads)
+
+
+def test_config5_training_step_bf16():
+    import torch
+    # full configuration on the GPU ...
+    cfg, inp, dev, ctx, O = _run_config("cfg5_train_bf16")
+    args = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    grads = ctx.backward(*args, dev["dO"])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    # ... oracle on two slabs (a slab depends only on its own rows and its head's gate)
+    b, hs = 1, slice(2, 4)
+    sub = {k: (v[b:b + 1, hs] if k in ("Q", "K", "V", "dO") else v) for k, v in inp.items()}
+    sub["gate_w"], sub["gate_b"] = inp["gate_w"][hs], inp["gate_b"][hs]
+    scfg = dict(cfg, B=1, H=2)
+    ref = orc.backward(sub["Q"], sub["K"], sub["V"], sub["W"], float(sub["beta"][0]), sub["gate_w"],
+                       sub["gate_b"], sub["omega"], sub["dO"], scfg["L"])
+    for key in ("dQ", "dK", "dV"):
+        _check(to_numpy64(grads[key])[b:b + 1, hs], ref[key], "bf16", key)
+    refO = _oracle_forward(scfg, sub)
+    _check(to_numpy64(O)[b:b + 1, hs], refO, "bf16", "O")
+    # parameter gradients sum over slabs: compare them on the two-slab problem run on its own
+    sctx = _ctx(scfg)
+    sdev = device_inputs(sub, "bf16")
+    sargs = (sdev["Q"], sdev["K"], sdev["V"], sdev["W"], sdev["beta"], sdev["gate_w"], sdev["gate_b"], sdev["omega"])
+    sctx.forward(*sargs)
+    sg = sctx.backward(*sargs, sdev["dO"])
+    torch.cuda.synchronize()
+    for key in ("dgate_w", "dgate_b", "domega"):
+        err = small_vector_error(to_numpy64(sg[key]), ref[key])
+        assert err.max() <= 2e-2, (key, err.max())
+    db = float(sg["dbeta"].cpu()[0])
+    assert abs(db - ref["dbeta_closed"]) <= 0.1 * abs(ref["dbeta_closed"]) + 1e-12
+
+
+# ---------------------------------------------------------------- error paths that need a device
+def test_error_paths_on_device():
+    import paper_2507_08637_b200 as wersa
+    import torch
+    cfg = dict(B=1, H=1, n=64, d=64, L=3, m=64, dtype="f32")
+    inp = wi.make_inputs(**cfg, backward=True)
+    dev = device_inputs(inp, "f32")
+    ctx = _ctx(cfg)
+    args = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    with pytest.raises(wersa.WersaError) as e:
+        ctx.backward(*args, dev["dO"])
+    assert e.value.status == 6
+    # misaligned Q
+    big = torch.zeros(dev["Q"].numel() + 1, device="cuda")
+    with pytest.raises(wersa.WersaError) as e:
+        ctx.forward(big[1:].view_as(dev["Q"]), *args[1:])
+    assert e.value.status == 1
+    fo = _ctx(cfg, flags=wersa.WERSA_FLAG_FORWARD_ONLY)
+    fo.forward(*args)
+    with pytest.raises(wersa.WersaError) as e:
+        fo.backward(*args, dev["dO"])
+    assert e.value.status == 2
