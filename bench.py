@@ -1,0 +1,346 @@
+#!/usr/bin/env python
+"""Benchmark of the WERSA attention forward on B200: tokens/s at n = 128k and fraction of roofline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One step = one whole forward pass of the operator (all kernels, all heads) on one batch of
+synthetic input.  With N > 1 (torchrun) every rank runs the same per-GPU workload on its own
+GPU (slabs are independent: no data-path collective, weak scaling); times are CUDA-event times,
+max over ranks.  Rank 0 prints ONE JSON line.
+
+--impl reference times the float64 CPU oracle (oracle/) on the host cores instead.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "WERSA attn tokens/sec on 1 B200 at n=128k (device-timed), % of roofline"
+DEFAULT_WORKLOAD = "cfg4_long_bf16"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# fp32 FFMA peak of the fp32 kernels: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (max SM clock)
+FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def workload_string(cfg):
+    return (f"{cfg['name']}: B={cfg['B']} H={cfg['H']} n={cfg['n']} d={cfg['d']} L={cfg['L']} "
+            f"m={cfg['m']} {cfg['dtype']}")
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples during the timed region."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, smax, reasons, power = [], [], set(), []
+        with open(self.path) as fh:
+            for line in fh:
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1]))
+                    smax.append(float(parts[2]))
+                    power.append(float(parts[3]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                      "sw_power_cap"), parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+def oracle_sample_rate(cfg, inp, budget_s):
+    """Times the float64 oracle, as it stands, on a bounded sample of the workload: the first
+    `heads` heads and the first `n_s` tokens of each (a multiple of 2^L), sized for ~budget_s.
+    Returns (tokens/s in whole-token units i.e. token-heads / H / s, description, threads, seconds)."""
+    from oracle import wersa_oracle as orc
+    threads = orc.threads()
+    H, n, L = cfg["H"], cfg["n"], cfg["L"]
+    heads = max(1, min(H, threads))
+    per_thread_rate = 2.0e4                 # token-heads / s / thread, order of magnitude at m=256
+    n_s = int(min(n, max(2 ** L, budget_s * per_thread_rate * (256.0 / cfg["m"]))))
+    n_s = max(2 ** L, (n_s // 2 ** L) * 2 ** L)
+    sl = (slice(0, cfg["B"]), slice(0, heads), slice(0, n_s))
+    Q, K, V = inp["Q"][sl], inp["K"][sl], inp["V"][sl]
+    gw, gb = inp["gate_w"][:heads], inp["gate_b"][:heads]
+    t0 = time.perf_counter()
+    orc.forward(Q, K, V, inp["W"], float(inp["beta"][0]), gw, gb, inp["omega"], L)
+    dt = time.perf_counter() - t0
+    token_heads = cfg["B"] * heads * n_s
+    used = min(threads, cfg["B"] * heads)
+    desc = (f"oracle forward on {cfg['B']}x{heads} of {cfg['B']}x{H} slabs, first {n_s} of {n} tokens "
+            f"each ({token_heads} token-heads), one run")
+    return token_heads / H / dt, desc, used, dt
+
+
+def run_reference(args, cfg, inp, rank):
+    """--impl reference: the CPU oracle on the host cores, rank 0 only."""
+    if rank != 0:
+        return
+    budget = max(0.5, min(20.0, 150.0 / (args.steps + args.warmup)))
+    rates, times = [], []
+    desc, used = "", 1
+    for i in range(args.warmup + args.steps):
+        rate, desc, used, dt = oracle_sample_rate(cfg, inp, budget)
+        if i >= args.warmup:
+            rates.append(rate)
+            times.append(dt)
+    value = sum(rates) / len(rates)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": workload_string(cfg)},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": used, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--simt", action="store_true", help="force the fp32 FFMA kernels")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    import wersa_inputs as wi
+    cfg = dict(wi.CONFIGS[args.workload], name=args.workload)
+
+    if args.impl == "reference":
+        if rank == 0:
+            _, inp = wi.make_config(args.workload)
+            run_reference(args, cfg, inp, rank)
+        return 0
+
+    import numpy as np
+    import torch
+
+    import paper_2507_08637_b200 as wersa
+    from tests.util import device_inputs
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local_rank))
+
+    # every rank draws its own batch of the same shape (different seed per rank)
+    cfg_r, inp = wi.make_config(args.workload, seed=wi.CONFIGS[args.workload]["seed"] + 1000 * rank)
+    dtype = cfg["dtype"]
+    flags = wersa.WERSA_FLAG_FORWARD_ONLY | (wersa.WERSA_FLAG_SIMT_ONLY if args.simt else 0)
+    ctx = wersa.wersa_create(cfg["B"], cfg["H"], cfg["n"], cfg["d"], cfg["L"], cfg["m"], dtype=dtype,
+                             grad_dtype="f32", device=local_rank, flags=flags)
+    dev = device_inputs(inp, dtype, device=f"cuda:{local_rank}")
+    fargs = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    O = torch.empty_like(dev["Q"])
+    stream = torch.cuda.current_stream()
+    tensor_cores = ctx.uses_tensor_cores()
+
+    def step():
+        wersa.wersa_forward(ctx, *fargs, out=O, stream=stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    if ctx.query_status() != 0:
+        raise SystemExit("device reported an expired wait during warm-up")
+
+    # ---- timed region: exactly K steps, device-timed on the launching stream -----------------
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    total_ms = e0.elapsed_time(e1)
+    launches = ctx.launch_count(0) * args.steps
+
+    # ---- per-kernel durations (second pass of K steps with an event behind every kernel) -----
+    ctx.set_step_timing(True)
+    per_kernel = {}
+    for _ in range(args.steps):
+        step()
+        for name, ms in ctx.step_times(0):
+            per_kernel.setdefault(name, []).append(ms)
+    ctx.set_step_timing(False)
+    clocks = sampler.stop()
+
+    if dist is not None:
+        t = torch.tensor([total_ms], device=f"cuda:{local_rank}", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    tokens_per_step = cfg["B"] * cfg["n"] * world
+    value = tokens_per_step / (ms_per_step * 1e-3)
+
+    # ---- end to end through the public API with HOST buffers ---------------------------------
+    host_in = [dev[k].cpu().pin_memory() for k in ("Q", "K", "V")]
+    host_out = torch.empty_like(host_in[0]).pin_memory()
+    dQ, dK, dV = (torch.empty_like(dev["Q"]) for _ in range(3))
+    h2d = sum(t.numel() * t.element_size() for t in host_in)
+    d2h = host_out.numel() * host_out.element_size()
+
+    def e2e_step():
+        dQ.copy_(host_in[0], non_blocking=True)
+        dK.copy_(host_in[1], non_blocking=True)
+        dV.copy_(host_in[2], non_blocking=True)
+        wersa.wersa_forward(ctx, dQ, dK, dV, *fargs[3:], out=O, stream=stream)
+        host_out.copy_(O, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0.record(stream)
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device=f"cuda:{local_rank}", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = tokens_per_step / (e2e_ms / args.e2e_steps * 1e-3)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- roofline of the dominant kernel -----------------------------------------------------
+    peaks, peak_kind = load_peaks()
+    TH = cfg["B"] * cfg["H"] * cfg["n"]
+    d, m = cfg["d"], cfg["m"]
+    s_bytes = 2 if dtype == "bf16" else 4
+    avg = {k: sum(v) / len(v) for k, v in per_kernel.items()}
+    tot = sum(avg.values())
+    dom = max(avg, key=avg.get)
+    # algorithmic work of each step per launch
+    flops = {"tc_kside": TH * (4 * d * m + 2 * m), "tc_qside": TH * (4 * d * m + 2 * m),
+             "simt_kside": TH * (4 * d * m + 2 * m), "simt_qside": TH * (4 * d * m + 2 * m)}
+    bytes_ = {"qmean_gate": TH * d * s_bytes, "haar_filter_q": TH * d * (s_bytes + 4),
+              "haar_filter_k": TH * d * (s_bytes + 4)}
+    if dom in flops:
+        if dom.startswith("tc_"):
+            bound, peak, unit = "tensor", float(peaks["bf16_tflops"]), "TFLOP/s"
+        else:
+            bound, peak, unit = "alu", FP32_ALU_TFLOPS, "TFLOP/s"
+        achieved = flops[dom] / (avg[dom] * 1e-3) / 1e12
+    else:
+        bound, peak, unit = "hbm", float(peaks["hbm_gbs"]), "GB/s"
+        achieved = bytes_.get(dom, 0) / (avg[dom] * 1e-3) / 1e9
+    roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
+                "frac": achieved / peak, "traffic": None,
+                "peak_source": f"{peak_kind} (burst)" if bound == "tensor" else
+                               (peak_kind if bound == "hbm" else "derived: 148 SM x 128 FFMA x 2 x 1.965 GHz"),
+                "kernel_ms": avg, "kernel_share": {k: v / tot for k, v in avg.items()},
+                "timing": "CUDA events behind every kernel, second pass of K steps"}
+    # whole-path roofline: slower of FLOPs at tensor peak and bytes at HBM bandwidth
+    path_flops = TH * (8 * d * m + 4 * m)
+    path_bytes = TH * 4 * d * s_bytes
+    t_roof = max(path_flops / (float(peaks["bf16_tflops"]) * 1e12), path_bytes / (float(peaks["hbm_gbs"]) * 1e9))
+    t_nom = max(path_flops / 2.25e15, path_bytes / 8.0e12)
+    path = {"roofline_us": t_roof * 1e6, "frac": t_roof / (ms_per_step * 1e-3), "peaks": peak_kind,
+            "roofline_us_nominal": t_nom * 1e6, "frac_nominal": t_nom / (ms_per_step * 1e-3),
+            "flops": path_flops, "bytes": path_bytes}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if tensor_cores else "f32",
+        "data": "synthetic",
+        "config": {"workload": workload_string(cfg), "per_gpu": True,
+                   "l2": "inputs+output 4 x %.0f MB per step exceed the 126 MB L2" % (TH * d * s_bytes / 1e6),
+                   "kernels": "tcgen05 bf16, fp32 accumulate" if tensor_cores else "fp32 FFMA", "storage": dtype},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": args.e2e_steps},
+        "gpu_launches": launches,
+        "roofline": roofline,
+        "path_roofline": path,
+    }
+    if not args.no_cpu_baseline:
+        rate, desc, used, _ = oracle_sample_rate(cfg, inp, 15.0)
+        line["cpu_baseline"] = {"value": rate, "unit": "tokens/s", "cores": used, "kind": "oracle",
+                                "sample": desc}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -143,6 +143,23 @@ const char* wersa_status_string(wersa_status status);
  * launched; 0 before the first call. */
 int32_t wersa_launch_count(const wersa_ctx* ctx, int which);
 
+/* 1 if this context's forward runs the bf16 tcgen05 tensor-core kernels, 0 if it runs the fp32
+ * FFMA kernels (fp32 storage, WERSA_FLAG_SIMT_ONLY, or a shape the tensor-core kernels do not
+ * cover). */
+int32_t wersa_uses_tensor_cores(const wersa_ctx* ctx);
+
+/* Step timing (a measurement aid; the paper has no counterpart).  When enabled, forward and
+ * backward record a CUDA event on `cuda_stream` before their first launch and after each step
+ * (a step is one kernel, or two for the gate).  Enabling creates the events, disabling destroys
+ * them; neither touches device memory. */
+wersa_status wersa_set_step_timing(wersa_ctx* ctx, int enable);
+
+/* Durations of the steps of the last forward (which = 0) or backward (which = 1), in
+ * milliseconds, after waiting for that pass to finish.  Writes min(*count, capacity) entries to
+ * `ms` and to `names` (static strings); either may be NULL.  WERSA_ERR_STATE if timing is off. */
+wersa_status wersa_step_times(wersa_ctx* ctx, int which, int capacity, float* ms,
+                              const char** names, int* count);
+
 #ifdef __cplusplus
 }
 #endif

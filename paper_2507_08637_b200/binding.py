@@ -68,6 +68,13 @@ def _lib():
     lib.wersa_status_string.argtypes = [ctypes.c_int]
     lib.wersa_launch_count.restype = ctypes.c_int32
     lib.wersa_launch_count.argtypes = [vp, ctypes.c_int]
+    lib.wersa_uses_tensor_cores.restype = ctypes.c_int32
+    lib.wersa_uses_tensor_cores.argtypes = [vp]
+    lib.wersa_set_step_timing.restype = ctypes.c_int
+    lib.wersa_set_step_timing.argtypes = [vp, ctypes.c_int]
+    lib.wersa_step_times.restype = ctypes.c_int
+    lib.wersa_step_times.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_float),
+                                     ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_int)]
     _LIB = lib
     return lib
 
@@ -194,6 +201,25 @@ class WersaContext:
 
     def query_status(self, stream=None):
         return int(_lib().wersa_query_status(self._h, _stream_ptr(stream)))
+
+    def set_step_timing(self, enable):
+        st = _lib().wersa_set_step_timing(self._h, int(bool(enable)))
+        if st != WERSA_OK:
+            raise WersaError(st, "wersa_set_step_timing")
+
+    def step_times(self, which=0):
+        """[(step name, milliseconds)] of the last forward (0) or backward (1); waits for it."""
+        cap = 16
+        ms = (ctypes.c_float * cap)()
+        names = (ctypes.c_char_p * cap)()
+        count = ctypes.c_int()
+        st = _lib().wersa_step_times(self._h, which, cap, ms, names, ctypes.byref(count))
+        if st != WERSA_OK:
+            raise WersaError(st, "wersa_step_times")
+        return [(names[i].decode(), float(ms[i])) for i in range(min(count.value, cap))]
+
+    def uses_tensor_cores(self):
+        return bool(_lib().wersa_uses_tensor_cores(self._h))
 
     def launch_count(self, which=0):
         return int(_lib().wersa_launch_count(self._h, which))

@@ -136,6 +136,16 @@ Ws resolve(const Plan& p, void* workspace) {
 
 using namespace wersa;
 
+constexpr int kMaxSteps = 16;
+
+// Optional per-step timing: an event before the first launch and one after every step.
+struct StepTimer {
+  bool enabled = false;
+  cudaEvent_t ev[2][kMaxSteps + 1];
+  const char* name[2][kMaxSteps];
+  int count[2] = {0, 0};
+};
+
 struct wersa_ctx {
   Plan plan;
   Ws ws;
@@ -143,6 +153,7 @@ struct wersa_ctx {
   bool forward_done;
   bool status_cleared;
   int launches_fwd, launches_bwd;
+  StepTimer timer;
 };
 
 namespace {
@@ -168,6 +179,25 @@ struct DeviceGuard {
     cudaError_t e_ = (call);                               \
     if (e_ != cudaSuccess) return WERSA_ERR_CUDA;          \
   } while (0)
+
+// Runs one step of a pass and, when step timing is on, records an event behind it.
+#define WERSA_STEP(which, label, call)                                             \
+  do {                                                                             \
+    WERSA_CUDA(call);                                                              \
+    StepTimer& t_ = ctx->timer;                                                    \
+    if (t_.enabled && t_.count[which] < kMaxSteps) {                               \
+      t_.name[which][t_.count[which]] = label;                                     \
+      WERSA_CUDA(cudaEventRecord(t_.ev[which][t_.count[which] + 1], st));          \
+      ++t_.count[which];                                                           \
+    }                                                                              \
+  } while (0)
+
+wersa_status begin_pass(wersa_ctx* ctx, int which, cudaStream_t st) {
+  StepTimer& t = ctx->timer;
+  t.count[which] = 0;
+  if (t.enabled) WERSA_CUDA(cudaEventRecord(t.ev[which][0], st));
+  return WERSA_OK;
+}
 
 wersa_status clear_status_once(wersa_ctx* ctx, cudaStream_t st) {
   if (!ctx->status_cleared) {
@@ -224,18 +254,21 @@ wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const v
   if (s != WERSA_OK) return s;
   int launches = 0;
   const int kind = p.bf16 ? 1 : 0;
-  WERSA_CUDA(launch_qmean_gate(p, w, Q, gate_w, gate_b, omega, st, &launches));
+  if ((s = begin_pass(ctx, 0, st)) != WERSA_OK) return s;
+  WERSA_STEP(0, "qmean_gate", launch_qmean_gate(p, w, Q, gate_w, gate_b, omega, st, &launches));
   if (p.use_tc) {
-    WERSA_CUDA(launch_tc_prepare_w(p, w, W, st, &launches));
-    WERSA_CUDA(launch_tc_kside(p, w, K, V, st, &launches));
-    WERSA_CUDA(launch_reduce_partials(p, w.spart, w.zpart, p.tchunks, w.S, w.z, w.Sbf, st, &launches));
-    WERSA_CUDA(launch_tc_qside(p, w, Q, beta, O, st, &launches));
+    WERSA_STEP(0, "tc_prepare_w", launch_tc_prepare_w(p, w, W, st, &launches));
+    WERSA_STEP(0, "tc_kside", launch_tc_kside(p, w, K, V, st, &launches));
+    WERSA_STEP(0, "reduce_partials",
+               launch_reduce_partials(p, w.spart, w.zpart, p.tchunks, w.S, w.z, w.Sbf, st, &launches));
+    WERSA_STEP(0, "tc_qside", launch_tc_qside(p, w, Q, beta, O, st, &launches));
   } else {
-    WERSA_CUDA(launch_haar_filter(p, Q, kind, w.f, w.QF, 0, st, &launches));
-    WERSA_CUDA(launch_haar_filter(p, K, kind, w.f, w.KF, 0, st, &launches));
-    WERSA_CUDA(launch_simt_kside(p, w, V, W, st, &launches));
-    WERSA_CUDA(launch_reduce_partials(p, w.spart, w.zpart, p.schunks, w.S, w.z, nullptr, st, &launches));
-    WERSA_CUDA(launch_simt_qside(p, w, W, beta, O, st, &launches));
+    WERSA_STEP(0, "haar_filter_q", launch_haar_filter(p, Q, kind, w.f, w.QF, 0, st, &launches));
+    WERSA_STEP(0, "haar_filter_k", launch_haar_filter(p, K, kind, w.f, w.KF, 0, st, &launches));
+    WERSA_STEP(0, "simt_kside", launch_simt_kside(p, w, V, W, st, &launches));
+    WERSA_STEP(0, "reduce_partials",
+               launch_reduce_partials(p, w.spart, w.zpart, p.schunks, w.S, w.z, nullptr, st, &launches));
+    WERSA_STEP(0, "simt_qside", launch_simt_qside(p, w, W, beta, O, st, &launches));
   }
   ctx->launches_fwd = launches;
   ctx->forward_done = true;
@@ -262,17 +295,21 @@ wersa_status wersa_backward(wersa_ctx* ctx, const void* Q, const void* K, const 
   if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
   int launches = 0;
   const int kind = p.bf16 ? 1 : 0, gkind = p.grad_bf16 ? 1 : 0;
+  wersa_status s = begin_pass(ctx, 1, st);
+  if (s != WERSA_OK) return s;
   if (p.use_tc) {   // the tensor-core forward keeps Q_F, K_F on chip: rebuild them
-    WERSA_CUDA(launch_haar_filter(p, Q, kind, w.f, w.QF, 0, st, &launches));
-    WERSA_CUDA(launch_haar_filter(p, K, kind, w.f, w.KF, 0, st, &launches));
+    WERSA_STEP(1, "haar_filter_q", launch_haar_filter(p, Q, kind, w.f, w.QF, 0, st, &launches));
+    WERSA_STEP(1, "haar_filter_k", launch_haar_filter(p, K, kind, w.f, w.KF, 0, st, &launches));
   }
-  WERSA_CUDA(launch_simt_bwd_qside(p, w, W, beta, dO, st, &launches));
-  WERSA_CUDA(launch_reduce_partials(p, w.spart, w.zpart, p.schunks, w.dS, w.dz, nullptr, st, &launches));
-  WERSA_CUDA(launch_simt_bwd_kside(p, w, V, W, dV, st, &launches));
-  WERSA_CUDA(launch_haar_backward(p, w, Q, kind, w.dQF, dQ, gkind, 0, st, &launches));
-  WERSA_CUDA(launch_haar_backward(p, w, K, kind, w.dKF, dK, gkind, 1, st, &launches));
-  WERSA_CUDA(launch_gate_backward(p, w, beta, gate_w, omega, dbeta, dgate_w, dgate_b, domega, st, &launches));
-  if (gate_w != nullptr) WERSA_CUDA(launch_add_rowvec(p, w, dQ, st, &launches));
+  WERSA_STEP(1, "simt_bwd_qside", launch_simt_bwd_qside(p, w, W, beta, dO, st, &launches));
+  WERSA_STEP(1, "reduce_partials",
+             launch_reduce_partials(p, w.spart, w.zpart, p.schunks, w.dS, w.dz, nullptr, st, &launches));
+  WERSA_STEP(1, "simt_bwd_kside", launch_simt_bwd_kside(p, w, V, W, dV, st, &launches));
+  WERSA_STEP(1, "haar_backward_q", launch_haar_backward(p, w, Q, kind, w.dQF, dQ, gkind, 0, st, &launches));
+  WERSA_STEP(1, "haar_backward_k", launch_haar_backward(p, w, K, kind, w.dKF, dK, gkind, 1, st, &launches));
+  WERSA_STEP(1, "gate_backward",
+             launch_gate_backward(p, w, beta, gate_w, omega, dbeta, dgate_w, dgate_b, domega, st, &launches));
+  if (gate_w != nullptr) WERSA_STEP(1, "add_rowvec", launch_add_rowvec(p, w, dQ, st, &launches));
   ctx->launches_bwd = launches;
   return WERSA_OK;
 }
@@ -322,7 +359,45 @@ wersa_status wersa_query_status(wersa_ctx* ctx, void* cuda_stream) {
   return WERSA_OK;
 }
 
+wersa_status wersa_set_step_timing(wersa_ctx* ctx, int enable) {
+  if (ctx == nullptr) return WERSA_ERR_INVALID_ARG;
+  StepTimer& t = ctx->timer;
+  if ((enable != 0) == t.enabled) return WERSA_OK;
+  DeviceGuard guard(ctx->plan.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  if (enable) {
+    for (int wch = 0; wch < 2; ++wch)
+      for (int i = 0; i <= kMaxSteps; ++i) WERSA_CUDA(cudaEventCreate(&t.ev[wch][i]));
+    t.count[0] = t.count[1] = 0;
+    t.enabled = true;
+  } else {
+    t.enabled = false;
+    for (int wch = 0; wch < 2; ++wch)
+      for (int i = 0; i <= kMaxSteps; ++i) cudaEventDestroy(t.ev[wch][i]);
+  }
+  return WERSA_OK;
+}
+
+wersa_status wersa_step_times(wersa_ctx* ctx, int which, int capacity, float* ms, const char** names,
+                              int* count) {
+  if (ctx == nullptr || count == nullptr || which < 0 || which > 1) return WERSA_ERR_INVALID_ARG;
+  StepTimer& t = ctx->timer;
+  if (!t.enabled) return WERSA_ERR_STATE;
+  DeviceGuard guard(ctx->plan.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  const int n = t.count[which];
+  *count = n;
+  if (n == 0) return WERSA_OK;
+  WERSA_CUDA(cudaEventSynchronize(t.ev[which][n]));
+  for (int i = 0; i < n && i < capacity; ++i) {
+    if (ms != nullptr) WERSA_CUDA(cudaEventElapsedTime(&ms[i], t.ev[which][i], t.ev[which][i + 1]));
+    if (names != nullptr) names[i] = t.name[which][i];
+  }
+  return WERSA_OK;
+}
+
 wersa_status wersa_destroy(wersa_ctx* ctx) {
+  if (ctx != nullptr && ctx->timer.enabled) wersa_set_step_timing(ctx, 0);
   delete ctx;
   return WERSA_OK;
 }
@@ -339,6 +414,8 @@ const char* wersa_status_string(wersa_status status) {
   }
   return "unknown status";
 }
+
+int32_t wersa_uses_tensor_cores(const wersa_ctx* ctx) { return ctx != nullptr && ctx->plan.use_tc ? 1 : 0; }
 
 int32_t wersa_launch_count(const wersa_ctx* ctx, int which) {
   if (ctx == nullptr) return 0;
