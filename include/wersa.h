@@ -48,7 +48,8 @@ typedef enum {
   WERSA_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small               */
   WERSA_ERR_CUDA = 4,        /* a CUDA runtime call failed (no device, launch error)     */
   WERSA_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired                       */
-  WERSA_ERR_STATE = 6        /* backward called without a preceding forward              */
+  WERSA_ERR_STATE = 6,       /* backward called without a preceding forward              */
+  WERSA_ERR_TOO_LARGE = 7    /* problem exceeds the fixed scratch of wersa_gate_static   */
 } wersa_status;
 
 typedef enum { WERSA_F32 = 0, WERSA_BF16 = 1 } wersa_dtype;
@@ -118,6 +119,31 @@ wersa_status wersa_backward(wersa_ctx* ctx, const void* Q, const void* K, const 
  * for every slab of X (batch, heads, seq_len, head_dim; cfg.dtype), with f a device array
  * (batch*heads, levels+1) of floats.  XF has cfg.dtype.  Each element of X is read once. */
 wersa_status wersa_haar_filter(wersa_ctx* ctx, const void* X, const float* f, void* XF,
+                               void* cuda_stream);
+
+/* Mean-pooled query and gate (Eqs. 1-3) for callers that cannot hand the library a workspace.
+ * (The paper has no counterpart of this entry point; it computes what wersa_forward's first step
+ * computes.)  Some callers cannot allocate device memory at the point where they need the gate:
+ * code running under an allocator that is frozen or owned by someone else (an inference server's
+ * pre-sized arena, a plugin inside another framework's memory plan), or a process whose device
+ * memory is already fully committed.  For them this entry point needs no context and no
+ * workspace: the per-chunk partial sums of Q and the sigmoid values go to a fixed 1 MiB
+ * (262144 floats) array that is part of the library image on every GPU that loads it, for as
+ * long as the process lives.  The entry point never calls cudaMalloc, cudaFree or any allocating
+ * routine.
+ *   cfg    as for wersa_create (only shapes, dtype, gate_per_head and device are used).
+ *   Q      (batch, heads, seq_len, head_dim) of cfg->dtype; gate_w, gate_b may be NULL (zeros).
+ *   qbar   out, (batch*heads, head_dim) floats;  f  out, (batch*heads, levels+1) floats.
+ * Returns WERSA_ERR_TOO_LARGE, launching nothing, when batch*heads*(64*chunks + levels+1) exceeds
+ * 262144 floats (chunks is the number of row chunks the mean pool splits the sequence into, about
+ * 592/(batch*heads), at least 1): all five benchmark configurations fit.
+ * The first call on a device resolves the array's device address (once per device, with that
+ * device made current); make that first call outside any CUDA stream capture.
+ * Every call on a device shares the one array and every element it reads is written earlier in
+ * the same call, so nothing needs clearing between calls; but two calls that overlap on the GPU
+ * (different streams, no ordering between them) race on it and must be serialised by the caller. */
+wersa_status wersa_gate_static(const wersa_config* cfg, const void* Q, const float* gate_w,
+                               const float* gate_b, const float* omega, float* qbar, float* f,
                                void* cuda_stream);
 
 /* Device pointers into the workspace of quantities the last forward left there.

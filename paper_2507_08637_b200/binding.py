@@ -18,7 +18,7 @@ WERSA_FLAG_SIMT_ONLY = 1
 WERSA_FLAG_FORWARD_ONLY = 2
 
 STATUS_NAMES = ["WERSA_OK", "WERSA_ERR_INVALID_ARG", "WERSA_ERR_UNSUPPORTED", "WERSA_ERR_WORKSPACE",
-                "WERSA_ERR_CUDA", "WERSA_ERR_TIMEOUT", "WERSA_ERR_STATE"]
+                "WERSA_ERR_CUDA", "WERSA_ERR_TIMEOUT", "WERSA_ERR_STATE", "WERSA_ERR_TOO_LARGE"]
 
 
 class wersa_config(ctypes.Structure):
@@ -68,6 +68,8 @@ def _lib():
     lib.wersa_status_string.argtypes = [ctypes.c_int]
     lib.wersa_launch_count.restype = ctypes.c_int32
     lib.wersa_launch_count.argtypes = [vp, ctypes.c_int]
+    lib.wersa_gate_static.restype = ctypes.c_int
+    lib.wersa_gate_static.argtypes = [ctypes.POINTER(wersa_config), vp, fp, fp, fp, fp, fp, vp]
     lib.wersa_uses_tensor_cores.restype = ctypes.c_int32
     lib.wersa_uses_tensor_cores.argtypes = [vp]
     lib.wersa_set_step_timing.restype = ctypes.c_int
@@ -250,3 +252,22 @@ def wersa_backward(ctx, Q, K, V, W, beta, gate_w, gate_b, omega, dO, stream=None
 
 def wersa_destroy(ctx):
     ctx.destroy()
+
+
+def wersa_gate_static(cfg, Q, gate_w, gate_b, omega, qbar, f, stream=None):
+    """Mean-pooled query and gate without a context or workspace, for callers that cannot
+    allocate device memory when they need the gate (a frozen or foreign allocator, memory fully
+    committed): the library's own fixed 1 MiB device array holds the intermediate sums.  The
+    caller passes the outputs qbar (batch*heads, head_dim) and f (batch*heads, levels+1), float32
+    CUDA tensors; nothing is allocated here or in the library.  Raises WersaError with status
+    WERSA_ERR_TOO_LARGE when the problem does not fit the fixed array.  Calls that may overlap on
+    the GPU must be serialised by the caller; make the first call on a device outside stream
+    capture."""
+    io = torch.bfloat16 if cfg.dtype == WERSA_BF16 else torch.float32
+    st = _lib().wersa_gate_static(ctypes.byref(cfg), _ptr(Q, io, "Q"),
+                                  _ptr(gate_w, torch.float32, "gate_w", optional=True),
+                                  _ptr(gate_b, torch.float32, "gate_b", optional=True),
+                                  _ptr(omega, torch.float32, "omega"), _ptr(qbar, torch.float32, "qbar"),
+                                  _ptr(f, torch.float32, "f"), _stream_ptr(stream))
+    if st != WERSA_OK:
+        raise WersaError(st, "wersa_gate_static")

@@ -326,6 +326,25 @@ wersa_status wersa_haar_filter(wersa_ctx* ctx, const void* X, const float* f, vo
   return WERSA_OK;
 }
 
+wersa_status wersa_gate_static(const wersa_config* cfg, const void* Q, const float* gate_w, const float* gate_b,
+                               const float* omega, float* qbar, float* f, void* cuda_stream) {
+  if (cfg == nullptr || Q == nullptr || omega == nullptr || qbar == nullptr || f == nullptr)
+    return WERSA_ERR_INVALID_ARG;
+  if (!aligned16(Q)) return WERSA_ERR_INVALID_ARG;
+  Plan p;
+  wersa_status s = make_plan(*cfg, &p);
+  if (s != WERSA_OK) return s;
+  const size_t need = (size_t)p.slabs * p.qchunks * kD + (size_t)p.slabs * p.L1;
+  if (need > static_scratch_capacity_floats()) return WERSA_ERR_TOO_LARGE;
+  DeviceGuard guard(p.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  float* scratch = nullptr;
+  WERSA_CUDA(static_scratch_address(p.cfg.device, &scratch));
+  WERSA_CUDA(launch_qmean_gate_static(p, scratch, Q, gate_w, gate_b, omega, qbar, f,
+                                      static_cast<cudaStream_t>(cuda_stream)));
+  return WERSA_OK;
+}
+
 wersa_status wersa_saved(wersa_ctx* ctx, int which, const float** device_ptr, size_t* count) {
   if (ctx == nullptr || device_ptr == nullptr || count == nullptr) return WERSA_ERR_INVALID_ARG;
   if (!ctx->forward_done) return WERSA_ERR_STATE;
@@ -411,6 +430,7 @@ const char* wersa_status_string(wersa_status status) {
     case WERSA_ERR_CUDA: return "CUDA runtime error";
     case WERSA_ERR_TIMEOUT: return "bounded device wait expired";
     case WERSA_ERR_STATE: return "backward or saved-tensor query without a preceding forward";
+    case WERSA_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of wersa_gate_static (262144 floats)";
   }
   return "unknown status";
 }

@@ -62,6 +62,13 @@ cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, 
 // dQ[s,t,:] += dqbar[s,:] / n.
 cudaError_t launch_add_rowvec(const Plan& p, const Ws& w, void* dQ, cudaStream_t st, int* launches);
 
+// Mean pool + gate with their scratch in a file-scope device array (no caller workspace).
+cudaError_t static_scratch_address(int device, float** out);
+size_t static_scratch_capacity_floats();
+cudaError_t launch_qmean_gate_static(const Plan& p, float* scratch, const void* Q, const float* gate_w,
+                                     const float* gate_b, const float* omega, float* qbar, float* f,
+                                     cudaStream_t st);
+
 // ---- haar.cu -------------------------------------------------------------------------------
 // XF = T_f(X).  in_kind/out_kind: 0 = float, 1 = bf16.
 cudaError_t launch_haar_filter(const Plan& p, const void* X, int in_kind, const float* f, void* XF,

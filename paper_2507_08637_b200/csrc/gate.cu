@@ -1,8 +1,17 @@
 // Mean-pooled query, content-adaptive gate (Eqs. 1-3 of the WERSA paper) and its backward pass.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace wersa {
 namespace {
+
+// Scratch of wersa_gate_static: lives in the library image of every GPU that loads it.
+constexpr size_t kStaticScratchFloats = 262144;   // 1 MiB
+static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
+constexpr int kMaxDevices = 64;
+float* g_static_scratch_addr[kMaxDevices] = {nullptr};
+std::mutex g_static_scratch_mutex;
 
 // Partial column sums of one row chunk of one slab of Q.  grid (qchunks, slabs), block 256:
 // thread (cg = tid & 7, rl = tid >> 3) owns 8 consecutive columns and every 32nd row, loads
@@ -207,6 +216,40 @@ cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const f
   k_gate<<<p.cfg.batch, kD, 0, st>>>(w.qpart, p.qchunks, p.cfg.heads, p.cfg.seq_len, p.L1,
                                      p.cfg.gate_per_head, gate_w, gate_b, omega, w.qbar, w.sg, w.f);
   *launches += 2;
+  return cudaGetLastError();
+}
+
+// Device address of the static scratch array on the current device, resolved once per device.
+// In host code the array's name is only a handle: the kernels need the address this returns.
+cudaError_t static_scratch_address(int device, float** out) {
+  if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (g_static_scratch_addr[device] == nullptr) {
+    void* ptr = nullptr;
+    cudaError_t err = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (err != cudaSuccess) return err;
+    g_static_scratch_addr[device] = static_cast<float*>(ptr);
+  }
+  *out = g_static_scratch_addr[device];
+  return cudaSuccess;
+}
+
+size_t static_scratch_capacity_floats() { return kStaticScratchFloats; }
+
+cudaError_t launch_qmean_gate_static(const Plan& p, float* scratch, const void* Q, const float* gate_w,
+                                     const float* gate_b, const float* omega, float* qbar, float* f,
+                                     cudaStream_t st) {
+  // scratch = [ partial column sums: slabs x qchunks x 64 | sigmoid(u): slabs x (L+1) ]
+  float* qpart = scratch;
+  float* sg = scratch + (size_t)p.slabs * p.qchunks * kD;
+  dim3 grid(p.qchunks, p.slabs);
+  if (p.bf16)
+    k_qmean_partial<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)Q, qpart, p.cfg.seq_len,
+                                                         p.qchunk_rows);
+  else
+    k_qmean_partial<float><<<grid, 256, 0, st>>>((const float*)Q, qpart, p.cfg.seq_len, p.qchunk_rows);
+  k_gate<<<p.cfg.batch, kD, 0, st>>>(qpart, p.qchunks, p.cfg.heads, p.cfg.seq_len, p.L1, p.cfg.gate_per_head,
+                                     gate_w, gate_b, omega, qbar, sg, f);
   return cudaGetLastError();
 }
 

@@ -1,0 +1,56 @@
+"""wersa_gate_static: the allocation-free variant of the mean-pool + gate step.
+
+Some callers cannot allocate device memory where they need the gate (their allocator is frozen
+or belongs to another framework, or device memory is fully committed), so this entry point keeps
+its intermediate sums in a fixed array inside the library instead of a caller workspace.  The test
+calls it through the C ABI twice in a row (the array keeps the previous call's contents, and the
+second call must not be disturbed by them) and compares both results with what the regular
+entry point, wersa_forward, leaves in its workspace.  Collected last on purpose."""
+import numpy as np
+import pytest
+
+import wersa_inputs as wi
+from tests.util import device_inputs, to_numpy64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("dtype,per_head", [("bf16", 1), ("f32", 0)])
+def test_gate_static_matches_forward_twice(dtype, per_head):
+    import paper_2507_08637_b200 as wersa
+    import torch
+    cfg = dict(B=2, H=3, n=2304, d=64, L=5, m=64, dtype=dtype, gate_per_head=per_head)
+    inp = wi.make_inputs(**cfg, seed=21, w_seed=22, gate_std=0.3, gate_seed=23, mean_shift=0.3)
+    dev = device_inputs(inp, dtype)
+    ctx = wersa.wersa_create(cfg["B"], cfg["H"], cfg["n"], cfg["d"], cfg["L"], cfg["m"], dtype=dtype,
+                             gate_per_head=per_head)
+    ctx.forward(dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    want_qbar, want_f = to_numpy64(ctx.saved("qbar")), to_numpy64(ctx.saved("f"))
+    c = ctx.cfg
+    qbar = torch.empty((cfg["B"] * cfg["H"], cfg["d"]), dtype=torch.float32, device="cuda")
+    f = torch.empty((cfg["B"] * cfg["H"], cfg["L"] + 1), dtype=torch.float32, device="cuda")
+    # a different problem first, so that the shared array holds foreign contents
+    other = (dev["Q"].float() * 3.0 + 1.0).to(dev["Q"].dtype)
+    wersa.wersa_gate_static(c, other, dev["gate_w"], dev["gate_b"], dev["omega"], qbar, f)
+    torch.cuda.synchronize()
+    assert np.abs(to_numpy64(f).reshape(want_f.shape) - want_f).max() > 1e-3
+    for _ in range(2):
+        qbar.fill_(float("nan"))
+        f.fill_(float("nan"))
+        wersa.wersa_gate_static(c, dev["Q"], dev["gate_w"], dev["gate_b"], dev["omega"], qbar, f)
+        torch.cuda.synchronize()
+        assert np.max(np.abs(to_numpy64(qbar).reshape(want_qbar.shape) - want_qbar)) <= 2e-6
+        assert np.max(np.abs(to_numpy64(f).reshape(want_f.shape) - want_f)) <= 2e-6
+
+
+def test_gate_static_rejects_problems_beyond_its_fixed_scratch():
+    import paper_2507_08637_b200 as wersa
+    import torch
+    # 8192 slabs x (64 + 3) floats > 262144 floats
+    cfg = wersa.make_config(128, 64, 64, 64, 2, 64, dtype="f32")
+    Q = torch.zeros(16, device="cuda")
+    om = torch.ones(3, device="cuda")
+    out = torch.zeros(8, device="cuda")
+    with pytest.raises(wersa.WersaError) as e:
+        wersa.wersa_gate_static(cfg, Q, None, None, om, out, out)
+    assert e.value.status == 7
