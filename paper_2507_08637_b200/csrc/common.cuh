@@ -36,7 +36,7 @@ struct Plan {
   // workspace offsets (bytes)
   size_t off_status, off_qpart, off_qbar, off_sg, off_f, off_spart, off_zpart, off_S, off_z,
       off_Sbf, off_Wt, off_dS, off_dz, off_sumdD, off_bands, off_dqbar, off_QF, off_KF, off_dQF,
-      off_dKF, total;
+      off_dKF, off_QFb, off_KFb, total;
   int part_chunks;    // max(schunks, tchunks): leading extent of the partial buffers
 };
 
@@ -48,6 +48,7 @@ struct Ws {   // resolved workspace pointers
   float *qpart, *qbar, *sg, *f, *spart, *zpart, *S, *z, *dS, *dz, *sumdD, *bands, *dqbar;
   __nv_bfloat16 *Sbf, *Wt;
   float *QF, *KF, *dQF, *dKF;
+  __nv_bfloat16 *QFb, *KFb;   // filtered Q, K in bf16 (tensor-core path)
 };
 Ws resolve(const Plan& p, void* workspace);
 
@@ -95,9 +96,9 @@ cudaError_t launch_simt_bwd_kside(const Plan& p, const Ws& w, const void* V, con
 // ---- tc_fwd.cu -----------------------------------------------------------------------------
 cudaError_t launch_tc_prepare_w(const Plan& p, const Ws& w, const void* W, cudaStream_t st,
                                 int* launches);
-cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const void* V, cudaStream_t st,
+cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* KFb, const void* V, cudaStream_t st,
                             int* launches);
-cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const float* beta, void* O,
+cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* QFb, const float* beta, void* O,
                             cudaStream_t st, int* launches);
 
 // ---- device helpers ------------------------------------------------------------------------

@@ -115,6 +115,37 @@ def test_forward_small_simt(case, dtype):
     assert ctx.launch_count(0) >= 5
 
 
+TC_SMALL = [
+    dict(B=1, H=1, n=128, d=64, L=3, m=128),      # one tile, one unit
+    dict(B=1, H=1, n=128, d=64, L=7, m=256),      # one tile, two feature halves
+    dict(B=1, H=2, n=384, d=64, L=5, m=256),      # odd number of tiles
+    dict(B=2, H=2, n=1152, d=64, L=4, m=128),     # more tiles than ring stages, alternating warpgroups
+    dict(B=1, H=1, n=2560, d=64, L=8, m=256),     # 20 tiles in one CTA chunk set
+    dict(B=2, H=3, n=4096, d=64, L=8, m=256, gate_per_head=0),
+]
+
+
+@pytest.mark.parametrize("case", range(len(TC_SMALL)))
+def test_forward_small_tensor_core(case):
+    import torch
+    cfg = dict(TC_SMALL[case], dtype="bf16")
+    inp = wi.make_inputs(**cfg, seed=700 + case, w_seed=800 + case, gate_std=0.3, gate_seed=900 + case,
+                         mean_shift=0.25, scale=0.7)
+    ctx = _ctx(cfg)
+    assert ctx.uses_tensor_cores()
+    dev = device_inputs(inp, "bf16")
+    O = ctx.forward(dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"],
+                    dev["omega"])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    ref, aux = _oracle_forward(cfg, inp, want_aux=True)
+    c = 1.0 / (max(float(inp["beta"][0]), 1e-6) * np.sqrt(cfg["m"]))
+    errS = normalised_error(to_numpy64(ctx.saved("S")) * c, aux["S"])
+    errz = normalised_error(to_numpy64(ctx.saved("z")) * c, aux["z"])
+    assert errS.max() < 2e-2 and errz.max() < 5e-3, (errS.max(), errz.max())
+    _check(to_numpy64(O), ref, "bf16", "O")
+
+
 def test_forward_is_bit_identical_run_to_run():
     import paper_2507_08637_b200 as wersa
     import torch
