@@ -57,14 +57,14 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   p->schunks = ceil_div(tiles32, p->schunk_tiles);
 
   p->tchunks = 0;
-  p->tchunk_tiles = 0;
+  p->tchunk_blocks = 0;
   if (p->use_tc) {
-    const int tiles128 = ceil_div(n, 128);
+    const int blocks = ceil_div(n, 256);
     p->tchunks = 148 / p->slabs;
     if (p->tchunks < 1) p->tchunks = 1;
-    if (p->tchunks > tiles128) p->tchunks = tiles128;
-    p->tchunk_tiles = ceil_div(tiles128, p->tchunks);
-    p->tchunks = ceil_div(tiles128, p->tchunk_tiles);
+    if (p->tchunks > blocks) p->tchunks = blocks;
+    p->tchunk_blocks = ceil_div(blocks, p->tchunks);
+    p->tchunks = ceil_div(blocks, p->tchunk_blocks);
   }
   p->part_chunks = p->schunks > p->tchunks ? p->schunks : p->tchunks;
 
@@ -90,8 +90,6 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   const bool need_xf = !p->use_tc || p->with_backward;
   p->off_QF = take(need_xf ? sizeof(float) * slab_elems : 0);
   p->off_KF = take(need_xf ? sizeof(float) * slab_elems : 0);
-  p->off_QFb = take(p->use_tc ? sizeof(__nv_bfloat16) * slab_elems : 0);
-  p->off_KFb = take(p->use_tc ? sizeof(__nv_bfloat16) * slab_elems : 0);
   if (p->with_backward) {
     p->off_dS = take(sizeof(float) * slabs * m * kD);
     p->off_dz = take(sizeof(float) * slabs * m);
@@ -130,8 +128,6 @@ Ws resolve(const Plan& p, void* workspace) {
   w.dqbar = reinterpret_cast<float*>(b + p.off_dqbar);
   w.dQF = reinterpret_cast<float*>(b + p.off_dQF);
   w.dKF = reinterpret_cast<float*>(b + p.off_dKF);
-  w.QFb = reinterpret_cast<__nv_bfloat16*>(b + p.off_QFb);
-  w.KFb = reinterpret_cast<__nv_bfloat16*>(b + p.off_KFb);
   return w;
 }
 
@@ -258,15 +254,13 @@ wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const v
   int launches = 0;
   const int kind = p.bf16 ? 1 : 0;
   if ((s = begin_pass(ctx, 0, st)) != WERSA_OK) return s;
-  WERSA_STEP(0, "qmean_gate", launch_qmean_gate(p, w, Q, gate_w, gate_b, omega, st, &launches));
+  WERSA_STEP(0, "qmean_gate",
+             launch_qmean_gate(p, w, Q, gate_w, gate_b, omega, p.use_tc ? W : nullptr, st, &launches));
   if (p.use_tc) {
-    WERSA_STEP(0, "tc_prepare_w", launch_tc_prepare_w(p, w, W, st, &launches));
-    WERSA_STEP(0, "haar_filter_q", launch_haar_filter(p, Q, 1, w.f, w.QFb, 1, st, &launches));
-    WERSA_STEP(0, "haar_filter_k", launch_haar_filter(p, K, 1, w.f, w.KFb, 1, st, &launches));
-    WERSA_STEP(0, "tc_kside", launch_tc_kside(p, w, w.KFb, V, st, &launches));
+    WERSA_STEP(0, "tc_kside", launch_tc_kside(p, w, K, V, st, &launches));
     WERSA_STEP(0, "reduce_partials",
                launch_reduce_partials(p, w.spart, w.zpart, p.tchunks, w.S, w.z, w.Sbf, st, &launches));
-    WERSA_STEP(0, "tc_qside", launch_tc_qside(p, w, w.QFb, beta, O, st, &launches));
+    WERSA_STEP(0, "tc_qside", launch_tc_qside(p, w, Q, beta, O, st, &launches));
   } else {
     WERSA_STEP(0, "haar_filter_q", launch_haar_filter(p, Q, kind, w.f, w.QF, 0, st, &launches));
     WERSA_STEP(0, "haar_filter_k", launch_haar_filter(p, K, kind, w.f, w.KF, 0, st, &launches));

@@ -32,11 +32,11 @@ struct Plan {
   // fp32 FFMA key-side / backward query-side split of the sequence
   int schunks, schunk_tiles;   // chunks per slab, 32-token tiles per chunk
   // tcgen05 key-side split
-  int tchunks, tchunk_tiles;   // chunks per slab, 128-token tiles per chunk
+  int tchunks, tchunk_blocks;  // chunks per slab, 256-token blocks per chunk
   // workspace offsets (bytes)
   size_t off_status, off_qpart, off_qbar, off_sg, off_f, off_spart, off_zpart, off_S, off_z,
       off_Sbf, off_Wt, off_dS, off_dz, off_sumdD, off_bands, off_dqbar, off_QF, off_KF, off_dQF,
-      off_dKF, off_QFb, off_KFb, total;
+      off_dKF, total;
   int part_chunks;    // max(schunks, tchunks): leading extent of the partial buffers
 };
 
@@ -48,14 +48,15 @@ struct Ws {   // resolved workspace pointers
   float *qpart, *qbar, *sg, *f, *spart, *zpart, *S, *z, *dS, *dz, *sumdD, *bands, *dqbar;
   __nv_bfloat16 *Sbf, *Wt;
   float *QF, *KF, *dQF, *dKF;
-  __nv_bfloat16 *QFb, *KFb;   // filtered Q, K in bf16 (tensor-core path)
 };
 Ws resolve(const Plan& p, void* workspace);
 
 // ---- gate.cu -------------------------------------------------------------------------------
 // Partial column sums of Q over row chunks, then qbar, sigmoid(u) and f per slab (Eqs. 1-3).
+// With W != nullptr the second launch also leaves the bf16 transpose of W (m x 64) in w.Wt.
 cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const float* gate_w,
-                              const float* gate_b, const float* omega, cudaStream_t st, int* launches);
+                              const float* gate_b, const float* omega, const void* W, cudaStream_t st,
+                              int* launches);
 // Gate backward: band inner products -> df -> domega, dgate_b, dgate_w, dqbar; dbeta.
 cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, const float* gate_w,
                                  const float* omega, float* dbeta, float* dgate_w, float* dgate_b,
@@ -94,11 +95,10 @@ cudaError_t launch_simt_bwd_kside(const Plan& p, const Ws& w, const void* V, con
                                   cudaStream_t st, int* launches);
 
 // ---- tc_fwd.cu -----------------------------------------------------------------------------
-cudaError_t launch_tc_prepare_w(const Plan& p, const Ws& w, const void* W, cudaStream_t st,
-                                int* launches);
-cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* KFb, const void* V, cudaStream_t st,
+// Both read the raw bf16 tensors and apply the Haar filter (coefficients from w.f) on chip.
+cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const void* V, cudaStream_t st,
                             int* launches);
-cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* QFb, const float* beta, void* O,
+cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const float* beta, void* O,
                             cudaStream_t st, int* launches);
 
 // ---- device helpers ------------------------------------------------------------------------

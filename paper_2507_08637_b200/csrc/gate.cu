@@ -55,47 +55,76 @@ __global__ void __launch_bounds__(256) k_qmean_partial(const T* __restrict__ Q, 
   }
 }
 
-// One CTA per batch element, 64 threads (one per column).  qbar = sum of partials / n (Eq. 1),
-// u = gate_w^T qbar + gate_b (Eq. 2), f = sigmoid(u) * omega (Eq. 3).
-__global__ void __launch_bounds__(kD) k_gate(const float* __restrict__ qpart, int qchunks, int H, int n,
-                                             int L1, int per_head, const float* __restrict__ gate_w,
-                                             const float* __restrict__ gate_b,
-                                             const float* __restrict__ omega, float* __restrict__ qbar,
-                                             float* __restrict__ sg, float* __restrict__ f) {
-  const int b = blockIdx.x, c = threadIdx.x;
+// grid (slabs + wt_blocks), block 256.
+// Blocks [0, slabs): qbar of one slab = sum of its chunk partials in a fixed order / n (Eq. 1), the
+// head's logits u = gate_w[h]^T qbar (Eq. 2) and, for the per-head gate, sigmoid(u + gate_b[h]) and
+// f = sigmoid * omega (Eq. 3).  For the batch-wide gate the bias-free logits are parked in f and
+// k_gate_shared finishes the job.
+// Blocks [slabs, ...): bf16 transpose Wt (m x 64) of W (64 x m) for the tensor-core kernels.
+__global__ void __launch_bounds__(256) k_qbar_gate(const float* __restrict__ qpart, int qchunks, int slabs, int H,
+                                                   int n, int L1, int per_head, const float* __restrict__ gate_w,
+                                                   const float* __restrict__ gate_b, const float* __restrict__ omega,
+                                                   float* __restrict__ qbar, float* __restrict__ sg,
+                                                   float* __restrict__ f, const __nv_bfloat16* __restrict__ W,
+                                                   __nv_bfloat16* __restrict__ Wt, int m) {
+  if ((int)blockIdx.x >= slabs) {
+    const int i = ((int)blockIdx.x - slabs) * 256 + threadIdx.x;
+    if (i < m * kD) {
+      const int r = i / kD, c = i - r * kD;
+      Wt[i] = W[(size_t)c * m + r];
+    }
+    return;
+  }
+  const int slab = blockIdx.x, h = slab % H;
+  const int c = threadIdx.x & (kD - 1), part = threadIdx.x >> 6;   // 4 interleaved partial sums per column
+  __shared__ float red[4][kD];
   __shared__ float qs[kD];
-  __shared__ float utot[kMaxLevels + 1];
-  if (c <= kMaxLevels) utot[c] = 0.f;
-  for (int h = 0; h < H; ++h) {
-    const int slab = b * H + h;
-    float s = 0.f;
-    for (int k = 0; k < qchunks; ++k) s += qpart[((size_t)slab * qchunks + k) * kD + c];
-    s = s / (float)n;
-    qbar[(size_t)slab * kD + c] = s;
-    __syncthreads();
-    qs[c] = s;
-    __syncthreads();
-    if (c < L1) {
-      float u = 0.f;
-      if (gate_w != nullptr)
-        for (int k = 0; k < kD; ++k) u += gate_w[((size_t)h * kD + k) * L1 + c] * qs[k];
-      if (per_head) {
-        if (gate_b != nullptr) u += gate_b[h * L1 + c];
-        float sgm = 1.f / (1.f + expf(-u));
-        sg[(size_t)slab * L1 + c] = sgm;
-        f[(size_t)slab * L1 + c] = sgm * omega[c];
-      } else {
-        utot[c] += u;
-      }
+  float s = 0.f;
+  const float* src = qpart + (size_t)slab * qchunks * kD + c;
+  int k = part;
+  for (; k + 12 < qchunks; k += 16) {
+    const float v0 = src[(size_t)k * kD], v1 = src[(size_t)(k + 4) * kD];
+    const float v2 = src[(size_t)(k + 8) * kD], v3 = src[(size_t)(k + 12) * kD];
+    s += (v0 + v1) + (v2 + v3);
+  }
+  for (; k < qchunks; k += 4) s += src[(size_t)k * kD];
+  red[part][c] = s;
+  __syncthreads();
+  if (threadIdx.x < kD) {
+    const float q = ((red[0][c] + red[1][c]) + (red[2][c] + red[3][c])) / (float)n;
+    qbar[(size_t)slab * kD + c] = q;
+    qs[c] = q;
+  }
+  __syncthreads();
+  if (threadIdx.x < L1) {
+    const int i = threadIdx.x;
+    float u = 0.f;
+    if (gate_w != nullptr)
+      for (int kk = 0; kk < kD; ++kk) u += gate_w[((size_t)h * kD + kk) * L1 + i] * qs[kk];
+    if (per_head) {
+      if (gate_b != nullptr) u += gate_b[h * L1 + i];
+      const float sgm = 1.f / (1.f + expf(-u));
+      sg[(size_t)slab * L1 + i] = sgm;
+      f[(size_t)slab * L1 + i] = sgm * omega[i];
+    } else {
+      f[(size_t)slab * L1 + i] = u;
     }
   }
-  if (!per_head && c < L1) {
-    float u = utot[c] + (gate_b != nullptr ? gate_b[c] : 0.f);
-    float sgm = 1.f / (1.f + expf(-u));
-    for (int h = 0; h < H; ++h) {
-      sg[((size_t)b * H + h) * L1 + c] = sgm;
-      f[((size_t)b * H + h) * L1 + c] = sgm * omega[c];
-    }
+}
+
+// Batch-wide gate (Algorithm 1, W_filter): u[b] = sum_h u[b,h] + gate_b[0], one sigmoid per batch
+// element shared by its heads.  grid (B), block 32; thread i owns band i of every head.
+__global__ void __launch_bounds__(32) k_gate_shared(int H, int L1, const float* __restrict__ gate_b,
+                                                    const float* __restrict__ omega, float* __restrict__ sg,
+                                                    float* __restrict__ f) {
+  const int b = blockIdx.x, i = threadIdx.x;
+  if (i >= L1) return;
+  float u = gate_b != nullptr ? gate_b[i] : 0.f;
+  for (int h = 0; h < H; ++h) u += f[((size_t)b * H + h) * L1 + i];
+  const float sgm = 1.f / (1.f + expf(-u));
+  for (int h = 0; h < H; ++h) {
+    sg[((size_t)b * H + h) * L1 + i] = sgm;
+    f[((size_t)b * H + h) * L1 + i] = sgm * omega[i];
   }
 }
 
@@ -205,18 +234,34 @@ __global__ void __launch_bounds__(256) k_add_rowvec(T* __restrict__ dQ, const fl
 
 }  // namespace
 
+// Second and third launch of the gate step, shared by the workspace and the static-scratch variants.
+static cudaError_t launch_gate_tail(const Plan& p, const float* qpart, const float* gate_w, const float* gate_b,
+                                    const float* omega, float* qbar, float* sg, float* f, const void* W,
+                                    __nv_bfloat16* Wt, cudaStream_t st, int* launches) {
+  const int m = p.cfg.features;
+  const int wt_blocks = W != nullptr ? (m * kD + 255) / 256 : 0;
+  k_qbar_gate<<<p.slabs + wt_blocks, 256, 0, st>>>(qpart, p.qchunks, p.slabs, p.cfg.heads, p.cfg.seq_len, p.L1,
+                                                   p.cfg.gate_per_head, gate_w, gate_b, omega, qbar, sg, f,
+                                                   (const __nv_bfloat16*)W, Wt, m);
+  *launches += 1;
+  if (!p.cfg.gate_per_head) {
+    k_gate_shared<<<p.cfg.batch, 32, 0, st>>>(p.cfg.heads, p.L1, gate_b, omega, sg, f);
+    *launches += 1;
+  }
+  return cudaGetLastError();
+}
+
 cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const float* gate_w,
-                              const float* gate_b, const float* omega, cudaStream_t st, int* launches) {
+                              const float* gate_b, const float* omega, const void* W, cudaStream_t st,
+                              int* launches) {
   dim3 grid(p.qchunks, p.slabs);
   if (p.bf16)
     k_qmean_partial<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)Q, w.qpart, p.cfg.seq_len,
                                                          p.qchunk_rows);
   else
     k_qmean_partial<float><<<grid, 256, 0, st>>>((const float*)Q, w.qpart, p.cfg.seq_len, p.qchunk_rows);
-  k_gate<<<p.cfg.batch, kD, 0, st>>>(w.qpart, p.qchunks, p.cfg.heads, p.cfg.seq_len, p.L1,
-                                     p.cfg.gate_per_head, gate_w, gate_b, omega, w.qbar, w.sg, w.f);
-  *launches += 2;
-  return cudaGetLastError();
+  *launches += 1;
+  return launch_gate_tail(p, w.qpart, gate_w, gate_b, omega, w.qbar, w.sg, w.f, W, w.Wt, st, launches);
 }
 
 // Device address of the static scratch array on the current device, resolved once per device.
@@ -248,9 +293,8 @@ cudaError_t launch_qmean_gate_static(const Plan& p, float* scratch, const void* 
                                                          p.qchunk_rows);
   else
     k_qmean_partial<float><<<grid, 256, 0, st>>>((const float*)Q, qpart, p.cfg.seq_len, p.qchunk_rows);
-  k_gate<<<p.cfg.batch, kD, 0, st>>>(qpart, p.qchunks, p.cfg.heads, p.cfg.seq_len, p.L1, p.cfg.gate_per_head,
-                                     gate_w, gate_b, omega, qbar, sg, f);
-  return cudaGetLastError();
+  int launches = 0;
+  return launch_gate_tail(p, qpart, gate_w, gate_b, omega, qbar, sg, f, nullptr, nullptr, st, &launches);
 }
 
 cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, const float* gate_w,

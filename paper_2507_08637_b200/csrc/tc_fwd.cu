@@ -1,4 +1,7 @@
 // bf16 tensor-core (tcgen05 + TMEM + TMA) forward kernels of the WERSA attention path, sm_100a.
+// Each kernel reads its raw bf16 operands once with TMA, applies the multi-level Haar filter
+// (Sec. 3.1 steps 3, 5, 6; Algorithm 2) to 256-token blocks in shared memory, and feeds the
+// filtered tiles straight to the tensor cores: the filtered tensors never reach global memory.
 //
 // Key side  (Eq. 7, key summary):  S' = ReLU(K_F W)^T V,  z' = ReLU(K_F W)^T 1  per sequence chunk.
 //   MMA1: D1[128 features x 128 tokens] = W^T (smem, K-major) * K_F^T (smem, K-major)   -> TMEM fp32
@@ -9,9 +12,14 @@
 //   ReLU warps as above, plus the row dot product with z' (denominator)
 //   MMA2: N'[128 tokens x 64] (+)= Phi (TMEM operand, K = features) * S' (smem bf16, N-major)
 //   epilogue warps: TMEM -> registers -> * 1/(D' + eps') -> bf16 -> swizzled smem -> TMA store
-// Warp roles: warp 0 TMA producer, warp 1 MMA issuer (one thread), two ReLU warpgroups that
-// alternate over the 128-column units, and (query side) one epilogue warpgroup.  All operand
-// tiles use the 128-byte swizzle; every wait on an mbarrier is bounded.
+//
+// Work unit of the MMA pipeline: one 128-token tile times one 128-feature half ("unit").  Three D1
+// accumulators rotate, so the ReLU pass of a unit overlaps four MMAs of its neighbours.
+// Warp roles: warp 0 TMA producer (K or Q), warp 1 MMA issuer (one thread), warp 2 TMA producer
+// (V, key side), warps 4-11 two ReLU warpgroups that alternate over the units, warps 12-19 Haar
+// filter, warps 20-23 (query side) epilogue.  All operand tiles use the 128-byte swizzle.
+// Every wait on an mbarrier is bounded; a role whose wait expires keeps its control flow (so that
+// group barriers stay balanced) but skips all further work, and the host sees the status word.
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -20,42 +28,57 @@ using namespace tc;
 
 namespace {
 
-constexpr int kTile = 128;                       // tokens per MMA tile
-constexpr int kStages = 4;                       // TMA ring depth
-constexpr uint32_t kTileBytes = kTile * kD * 2;  // one 128 x 64 bf16 tile
+constexpr int kTile = 128;                        // tokens per MMA tile
+constexpr int kBlk = 256;                         // tokens per Haar block = one pipeline stage
+constexpr uint32_t kTileBytes = kTile * kD * 2;   // 128 x 64 bf16
+constexpr uint32_t kBlkBytes = kBlk * kD * 2;     // 256 x 64 bf16
+constexpr int kNX = 3;                            // ring of K (or Q) blocks
+constexpr int kNV = 2;                            // ring of V blocks
+constexpr int kND1 = 3;                           // D1 accumulators in TMEM (columns 0, 128, 256)
 constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kAccCol = 384;                 // S' halves (key side) / N' of two tiles (query side)
 constexpr uint32_t kIdesc1 = make_idesc_bf16(128, 128, false, false);  // both operands K-major
 constexpr uint32_t kIdesc2 = make_idesc_bf16(128, 64, false, true);    // B = V or S', N-major
 
-enum { kErrProducer = 11, kErrMma = 12, kErrRelu = 13, kErrEpilogue = 14 };
+constexpr int kWarpTma = 0, kWarpMma = 1, kWarpTmaV = 2;
+constexpr int kReluWarp0 = 4, kHaarWarp0 = 12, kEpiWarp0 = 20;
+constexpr int kKsideThreads = 32 * kEpiWarp0;     // 640
+constexpr int kQsideThreads = 32 * (kEpiWarp0 + 4);   // 768
+
+enum { kErrProducer = 11, kErrMma = 12, kErrRelu = 13, kErrEpilogue = 14, kErrHaar = 15 };
 
 struct alignas(8) KsideBars {
-  uint64_t full[kStages], empty[kStages], d1_full[2], phi_ready[2], acc_done;
+  uint64_t x_full[kNX], xf_ready[kNX], x_empty[kNX], v_full[kNV], v_empty[kNV];
+  uint64_t d1_full[6], phi_ready[kND1], acc_done, xch[2];
   uint32_t tmem_base;
   int abort_flag;
 };
 struct alignas(8) QsideBars {
-  uint64_t full[kStages], empty[kStages], d1_full[2], phi_ready[2], d2_full[2], d2_free[2];
+  uint64_t x_full[kNX], xf_ready[kNX], x_empty[kNX];
+  uint64_t d1_full[6], phi_ready[kND1], d2_full[2], d2_free[2], den_ready[2], xch[2];
   uint32_t tmem_base;
   int abort_flag;
 };
 
 template <int NH> struct KsideSmem {
   static constexpr uint32_t wt = 0;
-  static constexpr uint32_t kf = wt + NH * kTileBytes;
-  static constexpr uint32_t v = kf + kStages * kTileBytes;
-  static constexpr uint32_t zx = v + kStages * kTileBytes;       // 128 floats
+  static constexpr uint32_t x = wt + NH * kTileBytes;
+  static constexpr uint32_t v = x + kNX * kBlkBytes;
+  static constexpr uint32_t xch = v + kNV * kBlkBytes;           // 2 x 8 x 64 floats
+  static constexpr uint32_t zx = xch + 4096;                     // 128 floats
   static constexpr uint32_t bars = zx + 512;
-  static constexpr uint32_t total = bars + 256 + 1024;           // + alignment slack
+  static constexpr uint32_t total = bars + 512 + 1024;           // + alignment slack
 };
 template <int NH> struct QsideSmem {
   static constexpr uint32_t wt = 0;
   static constexpr uint32_t simg = wt + NH * kTileBytes;
-  static constexpr uint32_t qf = simg + NH * kTileBytes;
-  static constexpr uint32_t ost = qf + kStages * kTileBytes;     // 2 output staging tiles
-  static constexpr uint32_t zs = ost + 2 * kTileBytes;           // NH*128 floats
-  static constexpr uint32_t bars = zs + NH * 512;
-  static constexpr uint32_t total = bars + 256 + 1024;
+  static constexpr uint32_t x = simg + NH * kTileBytes;
+  static constexpr uint32_t ost = x + kNX * kBlkBytes;           // 2 output staging tiles
+  static constexpr uint32_t xch = ost + 2 * kTileBytes;          // 2 x 8 x 64 floats
+  static constexpr uint32_t zs = xch + 4096;                     // NH*128 floats
+  static constexpr uint32_t den = zs + NH * 512;                 // 2 x NH x 128 floats
+  static constexpr uint32_t bars = den + 2 * NH * 512;
+  static constexpr uint32_t total = bars + 512 + 1024;
 };
 
 // (rows x 64) bf16 row-major in global memory -> 128B-swizzled rows of 128 bytes in shared memory.
@@ -67,80 +90,262 @@ __device__ __forceinline__ void load_rows_swizzled(uint8_t* dst, const __nv_bflo
   }
 }
 
-// ReLU pass over one 128-column unit of D1: fp32 TMEM -> bf16 pairs back into columns [0, 64) of
-// the unit.  `sum` adds up the ReLU values of the row; `dot` their dot product with zrow[0..127]
-// (nullptr: skipped).
-__device__ __forceinline__ void relu_unit(uint32_t taddr, const float* __restrict__ zrow, float& sum, float& dot) {
-#pragma unroll 1
-  for (int c = 0; c < 4; ++c) {
-    uint32_t r[32];
-    tmem_ld32(taddr + 32 * c, r);
-    tmem_ld_wait();
-    uint32_t p[16];
-    if (zrow != nullptr) {
+// Ties the 32 registers of an asynchronous TMEM load to the point behind its wait, so that no use
+// of them is scheduled ahead of the wait.
+__device__ __forceinline__ void reg_fence32(uint32_t (&r)[32]) {
+  asm volatile(""
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
+                 "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]),
+                 "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]),
+                 "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
+
+// ReLU of 32 fp32 accumulator columns -> 16 packed bf16 pairs.  kDot = false: the ReLU values are
+// added up into acc[0..3]; kDot = true: their products with zrow[0..31] are (denominator of Eq. 7).
+template <bool kDot>
+__device__ __forceinline__ void relu_chunk(const uint32_t (&r)[32], uint32_t (&p)[16], const float* __restrict__ zrow,
+                                           float (&acc)[4]) {
+  if (kDot) {
 #pragma unroll
-      for (int j4 = 0; j4 < 8; ++j4) {
-        const float4 zv = *reinterpret_cast<const float4*>(zrow + 32 * c + 4 * j4);
-        const float a0 = fmaxf(__uint_as_float(r[4 * j4]), 0.f), a1 = fmaxf(__uint_as_float(r[4 * j4 + 1]), 0.f);
-        const float a2 = fmaxf(__uint_as_float(r[4 * j4 + 2]), 0.f), a3 = fmaxf(__uint_as_float(r[4 * j4 + 3]), 0.f);
-        dot = fmaf(a0, zv.x, dot);
-        dot = fmaf(a1, zv.y, dot);
-        dot = fmaf(a2, zv.z, dot);
-        dot = fmaf(a3, zv.w, dot);
-        p[2 * j4] = pack_bf16x2(a0, a1);
-        p[2 * j4 + 1] = pack_bf16x2(a2, a3);
+    for (int j4 = 0; j4 < 8; ++j4) {
+      const float4 zv = *reinterpret_cast<const float4*>(zrow + 4 * j4);
+      const float a0 = fmaxf(__uint_as_float(r[4 * j4]), 0.f), a1 = fmaxf(__uint_as_float(r[4 * j4 + 1]), 0.f);
+      const float a2 = fmaxf(__uint_as_float(r[4 * j4 + 2]), 0.f), a3 = fmaxf(__uint_as_float(r[4 * j4 + 3]), 0.f);
+      acc[0] = fmaf(a0, zv.x, acc[0]);
+      acc[1] = fmaf(a1, zv.y, acc[1]);
+      acc[2] = fmaf(a2, zv.z, acc[2]);
+      acc[3] = fmaf(a3, zv.w, acc[3]);
+      p[2 * j4] = pack_bf16x2(a0, a1);
+      p[2 * j4 + 1] = pack_bf16x2(a2, a3);
+    }
+  } else {
+#pragma unroll
+    for (int j4 = 0; j4 < 8; ++j4) {
+      const float a0 = fmaxf(__uint_as_float(r[4 * j4]), 0.f), a1 = fmaxf(__uint_as_float(r[4 * j4 + 1]), 0.f);
+      const float a2 = fmaxf(__uint_as_float(r[4 * j4 + 2]), 0.f), a3 = fmaxf(__uint_as_float(r[4 * j4 + 3]), 0.f);
+      acc[0] += a0;
+      acc[1] += a1;
+      acc[2] += a2;
+      acc[3] += a3;
+      p[2 * j4] = pack_bf16x2(a0, a1);
+      p[2 * j4 + 1] = pack_bf16x2(a2, a3);
+    }
+  }
+}
+
+// ReLU pass over one 128-column D1 accumulator: fp32 TMEM -> bf16 pairs back into columns [0, 64)
+// of the same accumulator.  The next 32 columns are in flight while the current 32 are processed.
+// Returns the row sum of the ReLU values (kDot = false) or their dot product with zrow[0..127].
+template <bool kDot>
+__device__ __forceinline__ float relu_unit(uint32_t taddr, const float* __restrict__ zrow) {
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  uint32_t a[32], b[32], p[16];
+  tmem_ld32(taddr, a);
+  tmem_ld_wait();
+  reg_fence32(a);
+  tmem_ld32(taddr + 32, b);
+  relu_chunk<kDot>(a, p, zrow, acc);
+  tmem_st16(taddr, p);
+  tmem_ld_wait();
+  reg_fence32(b);
+  tmem_ld32(taddr + 64, a);
+  relu_chunk<kDot>(b, p, zrow + 32, acc);
+  tmem_st16(taddr + 16, p);
+  tmem_ld_wait();
+  reg_fence32(a);
+  tmem_ld32(taddr + 96, b);
+  relu_chunk<kDot>(a, p, zrow + 64, acc);
+  tmem_st16(taddr + 32, p);
+  tmem_ld_wait();
+  reg_fence32(b);
+  relu_chunk<kDot>(b, p, zrow + 96, acc);
+  tmem_st16(taddr + 48, p);
+  tmem_st_wait();
+  return (acc[0] + acc[1]) + (acc[2] + acc[3]);
+}
+
+// ---- Haar filter of one 256-token block in shared memory ------------------------------------------
+// T_f x = f_0 x + sum_{i=1..L} (f_i - f_{i-1}) * blockmean_{2^i}(x): the detail projector of level l
+// is blockmean_{2^(l-1)} - blockmean_{2^l} and the approximation projector of level L is
+// blockmean_{2^L}, so only aligned block sums of 2, 4, ..., 2^L rows are needed.
+struct HaarCoef {
+  float f0;
+  float k[kMaxLevels + 1];   // k[i] = (f_i - f_{i-1}) / 2^i for 1 <= i <= L, else 0
+};
+
+__device__ __forceinline__ HaarCoef haar_coef(const float* __restrict__ f, int L) {
+  HaarCoef c;
+  c.f0 = f[0];
+  c.k[0] = 0.f;
+  float scale = 0.5f;
+#pragma unroll
+  for (int i = 1; i <= kMaxLevels; ++i) {
+    c.k[i] = (i <= L) ? (f[i] - f[i - 1]) * scale : 0.f;
+    scale *= 0.5f;
+  }
+  return c;
+}
+
+// 256 threads (ht = 0..255) filter the block in place.  Thread (c = ht & 7, rg = ht >> 3) owns rows
+// 8 rg .. 8 rg + 7 of 16-byte chunk c: levels 1-3 in registers, levels 4-5 through warp shuffles
+// (a warp covers 32 consecutive rows), levels 6-8 through the 32-row sums the eight warps leave in
+// `xch` (8 x 64 floats) and announce on `xbar` (8 arrivals per block).  Returns false if the wait
+// on `xbar` gave up.  Rows >= valid_rows lie past the end of the sequence: they arrive as zeros (the
+// zero padding of Algorithm 2) and leave as zeros (the trim before the feature map).
+__device__ __forceinline__ bool haar_block_inplace(uint8_t* slot, const HaarCoef& hc, bool cross, float* xch,
+                                                   uint64_t* xbar, uint32_t xparity, int ht, int valid_rows,
+                                                   volatile int* abort_flag, int* status) {
+  const int c = ht & 7, rg = ht >> 3, lane = ht & 31, hw = ht >> 5;
+  uint8_t* base = slot + rg * 1024;
+  float x[8][8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {   // row 8 rg + j has swizzle phase j
+    const uint4 raw = *reinterpret_cast<const uint4*>(base + j * 128 + ((c ^ j) << 4));
+    const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      x[j][2 * i] = __uint_as_float(u[i] << 16);
+      x[j][2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
+    }
+  }
+  float hi[8], s5[8];
+#pragma unroll
+  for (int col = 0; col < 8; ++col) {
+    const float s3 = ((x[0][col] + x[1][col]) + (x[2][col] + x[3][col])) +
+                     ((x[4][col] + x[5][col]) + (x[6][col] + x[7][col]));
+    const float s4 = s3 + __shfl_xor_sync(0xffffffffu, s3, 8);
+    s5[col] = s4 + __shfl_xor_sync(0xffffffffu, s4, 16);
+    hi[col] = fmaf(hc.k[3], s3, fmaf(hc.k[4], s4, hc.k[5] * s5[col]));
+  }
+  bool ok = true;
+  if (cross) {   // uniform over the kernel: L > 5
+    if ((lane >> 3) == 0) {
+      float4* dst = reinterpret_cast<float4*>(xch + hw * kD + c * 8);
+      dst[0] = make_float4(s5[0], s5[1], s5[2], s5[3]);
+      dst[1] = make_float4(s5[4], s5[5], s5[6], s5[7]);
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(xbar);
+    ok = __all_sync(0xffffffffu, mbar_wait(xbar, xparity, abort_flag, status, kErrHaar));
+    if (ok) {
+      float w8[8][8];
+#pragma unroll
+      for (int w = 0; w < 8; ++w) {
+        const float4* src = reinterpret_cast<const float4*>(xch + w * kD + c * 8);
+        const float4 lo = src[0], hi4 = src[1];
+        w8[w][0] = lo.x; w8[w][1] = lo.y; w8[w][2] = lo.z; w8[w][3] = lo.w;
+        w8[w][4] = hi4.x; w8[w][5] = hi4.y; w8[w][6] = hi4.z; w8[w][7] = hi4.w;
       }
-    } else {
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const float a0 = fmaxf(__uint_as_float(r[2 * j]), 0.f), a1 = fmaxf(__uint_as_float(r[2 * j + 1]), 0.f);
-        sum += a0 + a1;
-        p[j] = pack_bf16x2(a0, a1);
+      for (int col = 0; col < 8; ++col) {
+        const float p0 = w8[0][col] + w8[1][col], p1 = w8[2][col] + w8[3][col];
+        const float p2 = w8[4][col] + w8[5][col], p3 = w8[6][col] + w8[7][col];
+        const float q0 = p0 + p1, q1 = p2 + p3;
+        const float s8 = q0 + q1;
+        const float s7 = (hw & 4) ? q1 : q0;
+        const float s6 = (hw & 4) ? ((hw & 2) ? p3 : p2) : ((hw & 2) ? p1 : p0);
+        hi[col] += fmaf(hc.k[6], s6, fmaf(hc.k[7], s7, hc.k[8] * s8));
       }
     }
-    tmem_st16(taddr + 16 * c, p);
   }
-  tmem_st_wait();
+  if (ok) {
+#pragma unroll
+    for (int col = 0; col < 8; ++col) {
+      const float a0 = x[0][col] + x[1][col], a1 = x[2][col] + x[3][col];
+      const float a2 = x[4][col] + x[5][col], a3 = x[6][col] + x[7][col];
+      const float c20 = fmaf(hc.k[2], a0 + a1, hi[col]), c21 = fmaf(hc.k[2], a2 + a3, hi[col]);
+      const float c10 = fmaf(hc.k[1], a0, c20), c11 = fmaf(hc.k[1], a1, c20);
+      const float c12 = fmaf(hc.k[1], a2, c21), c13 = fmaf(hc.k[1], a3, c21);
+      x[0][col] = fmaf(hc.f0, x[0][col], c10);
+      x[1][col] = fmaf(hc.f0, x[1][col], c10);
+      x[2][col] = fmaf(hc.f0, x[2][col], c11);
+      x[3][col] = fmaf(hc.f0, x[3][col], c11);
+      x[4][col] = fmaf(hc.f0, x[4][col], c12);
+      x[5][col] = fmaf(hc.f0, x[5][col], c12);
+      x[6][col] = fmaf(hc.f0, x[6][col], c13);
+      x[7][col] = fmaf(hc.f0, x[7][col], c13);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      uint4 out;
+      out.x = pack_bf16x2(x[j][0], x[j][1]);
+      out.y = pack_bf16x2(x[j][2], x[j][3]);
+      out.z = pack_bf16x2(x[j][4], x[j][5]);
+      out.w = pack_bf16x2(x[j][6], x[j][7]);
+      if (rg * 8 + j >= valid_rows) out = make_uint4(0u, 0u, 0u, 0u);
+      *reinterpret_cast<uint4*>(base + j * 128 + ((c ^ j) << 4)) = out;
+    }
+  }
+  return ok;
+}
+
+// Haar role shared by both kernels: for every block, wait for the raw tile, filter it in place and
+// hand it to the MMA issuer.
+template <typename Bars>
+__device__ __forceinline__ void haar_role(uint8_t* xring, Bars* bars, float* xch, const float* __restrict__ f, int L,
+                                          int nblk, int rows_left, volatile int* abort_flag, int* status) {
+  const int ht = threadIdx.x - 32 * kHaarWarp0;
+  const HaarCoef hc = haar_coef(f, L);
+  const bool cross = L > 5;
+  bool ok = true;
+  for (int b = 0; b < nblk; ++b) {
+    const int s = b % kNX;
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[s], (b / kNX) & 1, abort_flag, status, kErrHaar));
+    if (ok)
+      ok = haar_block_inplace(xring + s * kBlkBytes, hc, cross, xch + (b & 1) * 8 * kD, &bars->xch[b & 1],
+                              (b >> 1) & 1, ht, rows_left - b * kBlk, abort_flag, status);
+    if (ok) {
+      fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
+      mbar_arrive(&bars->xf_ready[s]);
+    }
+  }
 }
 
 // ---- key side -----------------------------------------------------------------------------------
-// grid (chunks, slabs), block 320: warp 0 producer, warp 1 MMA, warps 2-5 / 6-9 ReLU warpgroups.
+// grid (chunks, slabs), block 640.  TMEM: D1[3] at columns 0 / 128 / 256, S' half h at 384 + 64 h.
 template <int NH>
-__global__ void __launch_bounds__(320, 1)
-k_tc_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant__ CUtensorMap map_v,
-           const __nv_bfloat16* __restrict__ Wt, float* __restrict__ spart, float* __restrict__ zpart, int n,
-           int chunk_tiles, int* __restrict__ status) {
+__global__ void __launch_bounds__(kKsideThreads, 1)
+k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+           const __nv_bfloat16* __restrict__ Wt, const float* __restrict__ f, float* __restrict__ spart,
+           float* __restrict__ zpart, int n, int L, int chunk_blocks, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  using L = KsideSmem<NH>;
-  KsideBars* bars = reinterpret_cast<KsideBars*>(smem + L::bars);
-  float* zx = reinterpret_cast<float*>(smem + L::zx);
+  using SL = KsideSmem<NH>;
+  KsideBars* bars = reinterpret_cast<KsideBars*>(smem + SL::bars);
+  float* zx = reinterpret_cast<float*>(smem + SL::zx);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunk = blockIdx.x, slab = blockIdx.y;
-  const int tiles_total = n / kTile;
-  const int tile0 = chunk * chunk_tiles;
-  const int ntiles = min(chunk_tiles, tiles_total - tile0);
-  const int units = ntiles * NH;
+  const int blk0 = chunk * chunk_blocks;
+  const int nblk = min(chunk_blocks, (n + kBlk - 1) / kBlk - blk0);
+  const int units = nblk * 2 * NH;
   constexpr int m = NH * 128;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(&bars->full[s], 1);
-      mbar_init(&bars->empty[s], 1);
+    for (int s = 0; s < kNX; ++s) {
+      mbar_init(&bars->x_full[s], 1);
+      mbar_init(&bars->xf_ready[s], 256);
+      mbar_init(&bars->x_empty[s], 1);
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(&bars->d1_full[b], 1);
-      mbar_init(&bars->phi_ready[b], 128);
+    for (int s = 0; s < kNV; ++s) {
+      mbar_init(&bars->v_full[s], 1);
+      mbar_init(&bars->v_empty[s], 1);
     }
+    for (int b = 0; b < 6; ++b) mbar_init(&bars->d1_full[b], 1);
+    for (int b = 0; b < kND1; ++b) mbar_init(&bars->phi_ready[b], 128);
     mbar_init(&bars->acc_done, 1);
+    mbar_init(&bars->xch[0], 8);
+    mbar_init(&bars->xch[1], 8);
     bars->abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 1) {
+  if (warp == kWarpMma) {
     tmem_alloc(&bars->tmem_base, kTmemCols);
     tmem_relinquish();
   }
-  load_rows_swizzled(smem + L::wt, Wt, m);
+  load_rows_swizzled(smem + SL::wt, Wt, m);
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
@@ -148,154 +353,166 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant__ C
   const uint32_t tmem = bars->tmem_base;
   volatile int* abort_flag = &bars->abort_flag;
 
-  if (warp == 0) {
+  if (warp == kWarpTma || warp == kWarpTmaV) {
     if (lane == 0) {
+      const bool is_v = warp == kWarpTmaV;
+      const int depth = is_v ? kNV : kNX;
+      uint64_t* full = is_v ? bars->v_full : bars->x_full;
+      uint64_t* empty = is_v ? bars->v_empty : bars->x_empty;
+      uint8_t* ring = smem + (is_v ? SL::v : SL::x);
+      const CUtensorMap* map = is_v ? &map_v : &map_k;
       int issued = 0;
-      for (int t = 0; t < ntiles; ++t) {
-        const int s = t % kStages;
-        if (!mbar_wait(&bars->empty[s], ((t / kStages) & 1) ^ 1, abort_flag, status, kErrProducer)) break;
-        const int row = slab * n + (tile0 + t) * kTile;
-        mbar_arrive_expect_tx(&bars->full[s], 2 * kTileBytes);
-        tma_load_2d(smem + L::kf + s * kTileBytes, &map_kf, 0, row, &bars->full[s]);
-        tma_load_2d(smem + L::v + s * kTileBytes, &map_v, 0, row, &bars->full[s]);
-        issued = t + 1;
+      for (int b = 0; b < nblk; ++b) {
+        const int s = b % depth;
+        if (!mbar_wait(&empty[s], ((b / depth) & 1) ^ 1, abort_flag, status, kErrProducer)) break;
+        mbar_arrive_expect_tx(&full[s], kBlkBytes);
+        tma_load_3d(ring + s * kBlkBytes, map, 0, (blk0 + b) * kBlk, slab, &full[s]);
+        issued = b + 1;
       }
       if (*abort_flag != 0) {   // let copies in flight land before the CTA's shared memory goes away
-        for (int t = max(0, issued - kStages); t < issued; ++t)
-          mbar_wait_drain(&bars->full[t % kStages], (t / kStages) & 1);
+        for (int b = max(0, issued - depth); b < issued; ++b) mbar_wait_drain(&full[b % depth], (b / depth) & 1);
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == kWarpMma) {
     if (lane == 0) {
-      const uint32_t wt_addr = smem_u32(smem + L::wt);
-      const uint32_t kf_addr = smem_u32(smem + L::kf);
-      const uint32_t v_addr = smem_u32(smem + L::v);
+      const uint32_t wt_addr = smem_u32(smem + SL::wt);
+      const uint32_t x_addr = smem_u32(smem + SL::x);
+      const uint32_t v_addr = smem_u32(smem + SL::v);
       bool ok = true;
-      for (int u = 0; u <= units && ok; ++u) {
-        if (u < units) {
-          const int t = u / NH, h = u % NH, s = t % kStages;
-          if (h == 0) {
-            ok = mbar_wait(&bars->full[s], (t / kStages) & 1, abort_flag, status, kErrMma);
+      for (int i = 0; i < units + 2 && ok; ++i) {
+        if (i < units) {
+          const int t = i / NH, h = i % NH, b = t >> 1, s = b % kNX;
+          if ((t & 1) == 0 && h == 0) {
+            ok = mbar_wait(&bars->xf_ready[s], (b / kNX) & 1, abort_flag, status, kErrMma);
             if (!ok) break;
             tc_fence_after_sync();
           }
-          const uint32_t d1 = tmem + (u & 1) * 128;
+          const uint32_t d1 = tmem + (i % kND1) * 128;
+          const uint32_t b_addr = x_addr + s * kBlkBytes + (t & 1) * kTileBytes;
 #pragma unroll
           for (int k = 0; k < 4; ++k)
             mma_ss(d1, make_smem_desc(wt_addr + h * kTileBytes + k * 32, 16, 1024),
-                   make_smem_desc(kf_addr + s * kTileBytes + k * 32, 16, 1024), kIdesc1, k > 0);
-          mma_commit(&bars->d1_full[u & 1]);
+                   make_smem_desc(b_addr + k * 32, 16, 1024), kIdesc1, k > 0);
+          mma_commit(&bars->d1_full[i % 6]);
+          if ((t & 1) == 1 && h == NH - 1) mma_commit(&bars->x_empty[s]);
         }
-        if (u >= 1) {
-          const int v = u - 1;
-          const int t = v / NH, h = v % NH, s = t % kStages;
-          ok = mbar_wait(&bars->phi_ready[v & 1], (v >> 1) & 1, abort_flag, status, kErrMma);
+        if (i >= 2) {
+          const int v = i - 2;
+          const int t = v / NH, h = v % NH, b = t >> 1, s = b % kNV;
+          if ((t & 1) == 0 && h == 0) {
+            ok = mbar_wait(&bars->v_full[s], (b / kNV) & 1, abort_flag, status, kErrMma);
+            if (!ok) break;
+          }
+          ok = mbar_wait(&bars->phi_ready[v % kND1], (v / kND1) & 1, abort_flag, status, kErrMma);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t acc = tmem + 256 + h * 64;
+          const uint32_t acc = tmem + kAccCol + h * 64;
+          const uint32_t b_addr = v_addr + s * kBlkBytes + (t & 1) * kTileBytes;
 #pragma unroll
           for (int k = 0; k < 8; ++k)
-            mma_ts(acc, tmem + (v & 1) * 128 + k * 8, make_smem_desc(v_addr + s * kTileBytes + k * 2048, 1024, 1024),
-                   kIdesc2, (t > 0 || k > 0) ? 1u : 0u);
-          if (h == NH - 1) mma_commit(&bars->empty[s]);
+            mma_ts(acc, tmem + (v % kND1) * 128 + k * 8, make_smem_desc(b_addr + k * 2048, 1024, 1024), kIdesc2,
+                   (t > 0 || k > 0) ? 1u : 0u);
+          if ((t & 1) == 1 && h == NH - 1) mma_commit(&bars->v_empty[s]);
         }
       }
       mma_commit(&bars->acc_done);
     }
-  } else {
-    const int g = (warp - 2) >> 2;                 // ReLU warpgroup 0 / 1
+  } else if (warp >= kReluWarp0 && warp < kHaarWarp0) {
+    const int g = (warp - kReluWarp0) >> 2;         // ReLU warpgroup 0 / 1
     const uint32_t lane_base = 32u * (warp & 3);
-    const int row = lane_base + lane;              // feature within the half = TMEM lane
-    const uint32_t taddr = tmem + (lane_base << 16) + g * 128;
-    float zacc = 0.f, unused = 0.f;
-    int it = 0;
+    const int row = lane_base + lane;               // feature within the half = TMEM lane
+    float zacc = 0.f;
     bool ok = true;
-    for (int u = g; u < units; u += 2, ++it) {
-      ok = mbar_wait(&bars->d1_full[g], it & 1, abort_flag, status, kErrRelu);
-      if (!ok) break;
-      tc_fence_after_sync();
-      relu_unit(taddr, nullptr, zacc, unused);
-      tc_fence_before_sync();
-      mbar_arrive(&bars->phi_ready[g]);
-    }
-    if (ok) ok = mbar_wait(&bars->acc_done, 0, abort_flag, status, kErrRelu);
-    if (ok) {
-      tc_fence_after_sync();
-      const size_t pidx = (size_t)slab * gridDim.x + chunk;
-      if (NH == 1) {   // both warpgroups saw the same 128 features on alternating tiles
-        if (g == 1) zx[row] = zacc;
-        named_bar_sync(1, 256);
-        if (g == 0) zacc += zx[row];
+    for (int u = g; u < units; u += 2) {
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d1_full[u % 6], (u / 6) & 1, abort_flag, status, kErrRelu));
+      if (ok) {
+        tc_fence_after_sync();
+        zacc += relu_unit<false>(tmem + (lane_base << 16) + (u % kND1) * 128, nullptr);
+        tc_fence_before_sync();
+        mbar_arrive(&bars->phi_ready[u % kND1]);
       }
-      if (NH == 2 || g == 0) {
-        const int feat = (NH == 2 ? g * 128 : 0) + row;
-        float* dst = spart + (pidx * m + feat) * kD;
+    }
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->acc_done, 0, abort_flag, status, kErrRelu));
+    if (ok) tc_fence_after_sync();
+    const size_t pidx = (size_t)slab * gridDim.x + chunk;
+    if (NH == 1) {   // both warpgroups saw the same 128 features on alternating tiles
+      if (g == 1) zx[row] = zacc;
+      named_bar_sync(1, 256);
+      if (g == 0) zacc += zx[row];
+    }
+    if (ok && (NH == 2 || g == 0)) {
+      const int feat = (NH == 2 ? g * 128 : 0) + row;
+      float* dst = spart + (pidx * m + feat) * kD;
 #pragma unroll 1
-        for (int c = 0; c < 2; ++c) {
-          uint32_t r[32];
-          tmem_ld32(tmem + (lane_base << 16) + 256 + (NH == 2 ? g * 64 : 0) + 32 * c, r);
-          tmem_ld_wait();
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
+        tmem_ld32(tmem + (lane_base << 16) + kAccCol + (NH == 2 ? g * 64 : 0) + 32 * c, r);
+        tmem_ld_wait();
+        reg_fence32(r);
 #pragma unroll
-          for (int j = 0; j < 8; ++j)
-            *reinterpret_cast<uint4*>(dst + 32 * c + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
-        }
-        zpart[pidx * m + feat] = zacc;
+        for (int j = 0; j < 8; ++j)
+          *reinterpret_cast<uint4*>(dst + 32 * c + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
       }
-    } else if (NH == 1) {
-      named_bar_sync(1, 256);   // keep the barrier count balanced on the abort path
+      zpart[pidx * m + feat] = zacc;
     }
+  } else if (warp >= kHaarWarp0) {
+    haar_role(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), f + (size_t)slab * (L + 1), L, nblk,
+              n - blk0 * kBlk, abort_flag, status);
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == kWarpMma) {
     tc_fence_after_sync();
     tmem_dealloc(tmem, kTmemCols);
   }
 }
 
 // ---- query side ---------------------------------------------------------------------------------
-// grid (chunks, slabs), block 448: warp 0 producer, warp 1 MMA, warps 2-5 / 6-9 ReLU warpgroups,
-// warps 10-13 epilogue.  TMEM: D1[2] at columns 0/128, N' of tile parity p at 256 + 128 p (64
-// columns) followed by the NH partial denominators of the tile's rows.
+// grid (chunks, slabs), block 768.  TMEM: D1[3] at columns 0 / 128 / 256, N' of tile parity p at
+// 384 + 64 p.  The partial denominators of a tile travel through shared memory (den).
 template <int NH>
-__global__ void __launch_bounds__(448, 1)
-k_tc_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant__ CUtensorMap map_o,
+__global__ void __launch_bounds__(kQsideThreads, 1)
+k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
            const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ Sbf,
-           const float* __restrict__ zg, const float* __restrict__ beta, float eps, float bw_floor, int n,
-           int chunk_tiles, int* __restrict__ status) {
+           const float* __restrict__ zg, const float* __restrict__ f, const float* __restrict__ beta, float eps,
+           float bw_floor, int n, int L, int chunk_blocks, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  using L = QsideSmem<NH>;
-  QsideBars* bars = reinterpret_cast<QsideBars*>(smem + L::bars);
-  float* zs = reinterpret_cast<float*>(smem + L::zs);
+  using SL = QsideSmem<NH>;
+  QsideBars* bars = reinterpret_cast<QsideBars*>(smem + SL::bars);
+  float* zs = reinterpret_cast<float*>(smem + SL::zs);
+  float* den = reinterpret_cast<float*>(smem + SL::den);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunk = blockIdx.x, slab = blockIdx.y;
-  const int tiles_total = n / kTile;
-  const int tile0 = chunk * chunk_tiles;
-  const int ntiles = min(chunk_tiles, tiles_total - tile0);
+  const int blk0 = chunk * chunk_blocks;
+  const int nblk = min(chunk_blocks, (n + kBlk - 1) / kBlk - blk0);
+  const int ntiles = nblk * 2;
   const int units = ntiles * NH;
   constexpr int m = NH * 128;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(&bars->full[s], 1);
-      mbar_init(&bars->empty[s], 1);
+    for (int s = 0; s < kNX; ++s) {
+      mbar_init(&bars->x_full[s], 1);
+      mbar_init(&bars->xf_ready[s], 256);
+      mbar_init(&bars->x_empty[s], 1);
     }
+    for (int b = 0; b < 6; ++b) mbar_init(&bars->d1_full[b], 1);
+    for (int b = 0; b < kND1; ++b) mbar_init(&bars->phi_ready[b], 128);
     for (int b = 0; b < 2; ++b) {
-      mbar_init(&bars->d1_full[b], 1);
-      mbar_init(&bars->phi_ready[b], 128);
       mbar_init(&bars->d2_full[b], 1);
       mbar_init(&bars->d2_free[b], 128);
+      mbar_init(&bars->den_ready[b], 128 * NH);
+      mbar_init(&bars->xch[b], 8);
     }
     bars->abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 1) {
+  if (warp == kWarpMma) {
     tmem_alloc(&bars->tmem_base, kTmemCols);
     tmem_relinquish();
   }
-  load_rows_swizzled(smem + L::wt, Wt, m);
-  load_rows_swizzled(smem + L::simg, Sbf + (size_t)slab * m * kD, m);
+  load_rows_swizzled(smem + SL::wt, Wt, m);
+  load_rows_swizzled(smem + SL::simg, Sbf + (size_t)slab * m * kD, m);
   for (int i = threadIdx.x; i < m; i += blockDim.x) zs[i] = zg[(size_t)slab * m + i];
   fence_proxy_async_smem();
   tc_fence_before_sync();
@@ -304,135 +521,142 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant__ C
   const uint32_t tmem = bars->tmem_base;
   volatile int* abort_flag = &bars->abort_flag;
 
-  if (warp == 0) {
+  if (warp == kWarpTma) {
     if (lane == 0) {
       int issued = 0;
-      for (int t = 0; t < ntiles; ++t) {
-        const int s = t % kStages;
-        if (!mbar_wait(&bars->empty[s], ((t / kStages) & 1) ^ 1, abort_flag, status, kErrProducer)) break;
-        mbar_arrive_expect_tx(&bars->full[s], kTileBytes);
-        tma_load_2d(smem + L::qf + s * kTileBytes, &map_qf, 0, slab * n + (tile0 + t) * kTile, &bars->full[s]);
-        issued = t + 1;
+      for (int b = 0; b < nblk; ++b) {
+        const int s = b % kNX;
+        if (!mbar_wait(&bars->x_empty[s], ((b / kNX) & 1) ^ 1, abort_flag, status, kErrProducer)) break;
+        mbar_arrive_expect_tx(&bars->x_full[s], kBlkBytes);
+        tma_load_3d(smem + SL::x + s * kBlkBytes, &map_q, 0, (blk0 + b) * kBlk, slab, &bars->x_full[s]);
+        issued = b + 1;
       }
       if (*abort_flag != 0) {
-        for (int t = max(0, issued - kStages); t < issued; ++t)
-          mbar_wait_drain(&bars->full[t % kStages], (t / kStages) & 1);
+        for (int b = max(0, issued - kNX); b < issued; ++b) mbar_wait_drain(&bars->x_full[b % kNX], (b / kNX) & 1);
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == kWarpMma) {
     if (lane == 0) {
-      const uint32_t wt_addr = smem_u32(smem + L::wt);
-      const uint32_t s_addr = smem_u32(smem + L::simg);
-      const uint32_t qf_addr = smem_u32(smem + L::qf);
+      const uint32_t wt_addr = smem_u32(smem + SL::wt);
+      const uint32_t s_addr = smem_u32(smem + SL::simg);
+      const uint32_t x_addr = smem_u32(smem + SL::x);
       bool ok = true;
-      for (int u = 0; u <= units && ok; ++u) {
-        if (u < units) {
-          const int t = u / NH, h = u % NH, s = t % kStages;
-          if (h == 0) {
-            ok = mbar_wait(&bars->full[s], (t / kStages) & 1, abort_flag, status, kErrMma);
+      for (int i = 0; i < units + 2 && ok; ++i) {
+        if (i < units) {
+          const int t = i / NH, h = i % NH, b = t >> 1, s = b % kNX;
+          if ((t & 1) == 0 && h == 0) {
+            ok = mbar_wait(&bars->xf_ready[s], (b / kNX) & 1, abort_flag, status, kErrMma);
             if (!ok) break;
             tc_fence_after_sync();
           }
-          const uint32_t d1 = tmem + (u & 1) * 128;
+          const uint32_t d1 = tmem + (i % kND1) * 128;
+          const uint32_t a_addr = x_addr + s * kBlkBytes + (t & 1) * kTileBytes;
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            mma_ss(d1, make_smem_desc(qf_addr + s * kTileBytes + k * 32, 16, 1024),
+            mma_ss(d1, make_smem_desc(a_addr + k * 32, 16, 1024),
                    make_smem_desc(wt_addr + h * kTileBytes + k * 32, 16, 1024), kIdesc1, k > 0);
-          mma_commit(&bars->d1_full[u & 1]);
+          mma_commit(&bars->d1_full[i % 6]);
+          if ((t & 1) == 1 && h == NH - 1) mma_commit(&bars->x_empty[s]);
         }
-        if (u >= 1) {
-          const int v = u - 1;
-          const int t = v / NH, h = v % NH, s = t % kStages;
-          ok = mbar_wait(&bars->phi_ready[v & 1], (v >> 1) & 1, abort_flag, status, kErrMma);
+        if (i >= 2) {
+          const int v = i - 2;
+          const int t = v / NH, h = v % NH;
+          ok = mbar_wait(&bars->phi_ready[v % kND1], (v / kND1) & 1, abort_flag, status, kErrMma);
           if (!ok) break;
           if (h == 0 && t >= 2) {
             ok = mbar_wait(&bars->d2_free[t & 1], ((t >> 1) - 1) & 1, abort_flag, status, kErrMma);
             if (!ok) break;
           }
           tc_fence_after_sync();
-          const uint32_t d2 = tmem + 256 + (t & 1) * 128;
+          const uint32_t d2 = tmem + kAccCol + (t & 1) * 64;
 #pragma unroll
           for (int k = 0; k < 8; ++k)
-            mma_ts(d2, tmem + (v & 1) * 128 + k * 8, make_smem_desc(s_addr + h * kTileBytes + k * 2048, 1024, 1024),
+            mma_ts(d2, tmem + (v % kND1) * 128 + k * 8, make_smem_desc(s_addr + h * kTileBytes + k * 2048, 1024, 1024),
                    kIdesc2, (h > 0 || k > 0) ? 1u : 0u);
-          if (h == NH - 1) {
-            mma_commit(&bars->d2_full[t & 1]);
-            mma_commit(&bars->empty[s]);
-          }
+          if (h == NH - 1) mma_commit(&bars->d2_full[t & 1]);
         }
       }
     }
-  } else if (warp < 10) {
-    const int g = (warp - 2) >> 2;
+  } else if (warp >= kReluWarp0 && warp < kHaarWarp0) {
+    const int g = (warp - kReluWarp0) >> 2;
     const uint32_t lane_base = 32u * (warp & 3);
-    const uint32_t taddr = tmem + (lane_base << 16) + g * 128;
-    int it = 0;
-    for (int u = g; u < units; u += 2, ++it) {
+    const int row = lane_base + lane;               // token within the tile = TMEM lane
+    bool ok = true;
+    for (int u = g; u < units; u += 2) {
       const int t = u / NH, h = u % NH;
-      if (!mbar_wait(&bars->d1_full[g], it & 1, abort_flag, status, kErrRelu)) break;
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d1_full[u % 6], (u / 6) & 1, abort_flag, status, kErrRelu));
+      if (!ok) continue;
       tc_fence_after_sync();
-      float dot = 0.f, unused = 0.f;
-      relu_unit(taddr, zs + h * 128, unused, dot);
-      // the tile's N' columns (and the denominator slots behind them) must have been read by the
-      // epilogue of tile t-2 before they are written again
-      if (t >= 2) {
-        if (!mbar_wait(&bars->d2_free[t & 1], ((t >> 1) - 1) & 1, abort_flag, status, kErrRelu)) break;
-        tc_fence_after_sync();
-      }
-      tmem_st1(tmem + (lane_base << 16) + 256 + (t & 1) * 128 + 64 + h, __float_as_uint(dot));
-      tmem_st_wait();
+      const float dot = relu_unit<true>(tmem + (lane_base << 16) + (u % kND1) * 128, zs + h * 128);
       tc_fence_before_sync();
-      mbar_arrive(&bars->phi_ready[g]);
+      mbar_arrive(&bars->phi_ready[u % kND1]);
+      // the denominator slots of this tile parity must have been read by the epilogue of tile t-2
+      if (t >= 2)
+        ok = __all_sync(0xffffffffu,
+                        mbar_wait(&bars->d2_free[t & 1], ((t >> 1) - 1) & 1, abort_flag, status, kErrRelu));
+      if (!ok) continue;
+      den[((t & 1) * NH + h) * 128 + row] = dot;
+      mbar_arrive(&bars->den_ready[t & 1]);
     }
-  } else {
+  } else if (warp >= kHaarWarp0 && warp < kEpiWarp0) {
+    haar_role(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), f + (size_t)slab * (L + 1), L, nblk,
+              n - blk0 * kBlk, abort_flag, status);
+  } else if (warp >= kEpiWarp0) {
     const uint32_t lane_base = 32u * (warp & 3);
-    const int row = lane_base + lane;              // token within the tile = TMEM lane
-    const int et = threadIdx.x - 320;              // 0..127 inside the epilogue warpgroup
+    const int row = lane_base + lane;               // token within the tile = TMEM lane
+    const int et = threadIdx.x - 32 * kEpiWarp0;    // 0..127 inside the epilogue warpgroup
     const float bw = fmaxf(beta[0], bw_floor);
     const float epsp = eps * (float)m * bw * bw;
+    bool ok = true;
     for (int t = 0; t < ntiles; ++t) {
       const int p = t & 1;
-      if (!mbar_wait(&bars->d2_full[p], (t >> 1) & 1, abort_flag, status, kErrEpilogue)) break;
-      tc_fence_after_sync();
-      const uint32_t base = tmem + (lane_base << 16) + 256 + p * 128;
-      uint32_t r0[32], r1[32], dd[NH];
-      tmem_ld32(base, r0);
-      tmem_ld32(base + 32, r1);
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d2_full[p], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->den_ready[p], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
+      uint32_t r0[32], r1[32];
+      float inv = 0.f;
+      if (ok) {
+        tc_fence_after_sync();
+        const uint32_t base = tmem + (lane_base << 16) + kAccCol + p * 64;
+        tmem_ld32(base, r0);
+        tmem_ld32(base + 32, r1);
+        float dsum = epsp;
 #pragma unroll
-      for (int h = 0; h < NH; ++h) tmem_ld1(base + 64 + h, dd[h]);
-      tmem_ld_wait();
-      tc_fence_before_sync();
-      mbar_arrive(&bars->d2_free[p]);
-      float den = epsp;
-#pragma unroll
-      for (int h = 0; h < NH; ++h) den += __uint_as_float(dd[h]);
-      const float inv = 1.f / den;
+        for (int h = 0; h < NH; ++h) dsum += den[(p * NH + h) * 128 + row];
+        inv = 1.f / dsum;
+        tmem_ld_wait();
+        reg_fence32(r0);
+        reg_fence32(r1);
+        tc_fence_before_sync();
+        mbar_arrive(&bars->d2_free[p]);
+      }
       // staging buffer p was last used by tile t-2: its TMA store must have finished reading
       if (et == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
       named_bar_sync(2, 128);
-      uint8_t* ost = smem + L::ost + p * kTileBytes;
+      uint8_t* ost = smem + SL::ost + p * kTileBytes;
+      if (ok) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint4 v;
-        v.x = pack_bf16x2(__uint_as_float(r0[8 * c]) * inv, __uint_as_float(r0[8 * c + 1]) * inv);
-        v.y = pack_bf16x2(__uint_as_float(r0[8 * c + 2]) * inv, __uint_as_float(r0[8 * c + 3]) * inv);
-        v.z = pack_bf16x2(__uint_as_float(r0[8 * c + 4]) * inv, __uint_as_float(r0[8 * c + 5]) * inv);
-        v.w = pack_bf16x2(__uint_as_float(r0[8 * c + 6]) * inv, __uint_as_float(r0[8 * c + 7]) * inv);
-        *reinterpret_cast<uint4*>(ost + swz128(row, c)) = v;
-      }
+        for (int c = 0; c < 4; ++c) {
+          uint4 v;
+          v.x = pack_bf16x2(__uint_as_float(r0[8 * c]) * inv, __uint_as_float(r0[8 * c + 1]) * inv);
+          v.y = pack_bf16x2(__uint_as_float(r0[8 * c + 2]) * inv, __uint_as_float(r0[8 * c + 3]) * inv);
+          v.z = pack_bf16x2(__uint_as_float(r0[8 * c + 4]) * inv, __uint_as_float(r0[8 * c + 5]) * inv);
+          v.w = pack_bf16x2(__uint_as_float(r0[8 * c + 6]) * inv, __uint_as_float(r0[8 * c + 7]) * inv);
+          *reinterpret_cast<uint4*>(ost + swz128(row, c)) = v;
+        }
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint4 v;
-        v.x = pack_bf16x2(__uint_as_float(r1[8 * c]) * inv, __uint_as_float(r1[8 * c + 1]) * inv);
-        v.y = pack_bf16x2(__uint_as_float(r1[8 * c + 2]) * inv, __uint_as_float(r1[8 * c + 3]) * inv);
-        v.z = pack_bf16x2(__uint_as_float(r1[8 * c + 4]) * inv, __uint_as_float(r1[8 * c + 5]) * inv);
-        v.w = pack_bf16x2(__uint_as_float(r1[8 * c + 6]) * inv, __uint_as_float(r1[8 * c + 7]) * inv);
-        *reinterpret_cast<uint4*>(ost + swz128(row, 4 + c)) = v;
+        for (int c = 0; c < 4; ++c) {
+          uint4 v;
+          v.x = pack_bf16x2(__uint_as_float(r1[8 * c]) * inv, __uint_as_float(r1[8 * c + 1]) * inv);
+          v.y = pack_bf16x2(__uint_as_float(r1[8 * c + 2]) * inv, __uint_as_float(r1[8 * c + 3]) * inv);
+          v.z = pack_bf16x2(__uint_as_float(r1[8 * c + 4]) * inv, __uint_as_float(r1[8 * c + 5]) * inv);
+          v.w = pack_bf16x2(__uint_as_float(r1[8 * c + 6]) * inv, __uint_as_float(r1[8 * c + 7]) * inv);
+          *reinterpret_cast<uint4*>(ost + swz128(row, 4 + c)) = v;
+        }
+        fence_proxy_async_smem();
       }
-      fence_proxy_async_smem();
       named_bar_sync(2, 128);
-      if (et == 0) {
-        tma_store_2d(&map_o, ost, 0, slab * n + (tile0 + t) * kTile);
+      if (et == 0 && ok && blk0 * kBlk + t * kTile < n) {   // rows past n are clipped by the store
+        tma_store_3d(&map_o, ost, 0, blk0 * kBlk + t * kTile, slab);
         bulk_commit_group();
       }
     }
@@ -440,18 +664,9 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant__ C
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == kWarpMma) {
     tc_fence_after_sync();
     tmem_dealloc(tmem, kTmemCols);
-  }
-}
-
-// W (64 x m) -> Wt (m x 64), bf16.
-__global__ void k_transpose_w(const __nv_bfloat16* __restrict__ W, __nv_bfloat16* __restrict__ Wt, int m) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < m * kD) {
-    const int r = i / kD, c = i - r * kD;
-    Wt[i] = W[(size_t)c * m + r];
   }
 }
 
@@ -472,15 +687,16 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// (rows x 64) bf16 row-major tensor, boxes of 128 rows x 64 columns, 128-byte swizzle.
-cudaError_t make_tile_map(const void* base, size_t rows, CUtensorMap* out) {
+// (slabs x n x 64) bf16 row-major tensor, boxes of `box_rows` rows x 64 columns of one slab, 128-byte
+// swizzle.  Rows past the end of a slab read as zeros and are not written.
+cudaError_t make_tile_map(const void* base, int slabs, int n, int box_rows, CUtensorMap* out) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return cudaErrorNotSupported;
-  const cuuint64_t dims[2] = {kD, rows};
-  const cuuint64_t strides[1] = {kD * 2};
-  const cuuint32_t box[2] = {kD, kTile};
-  const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  const cuuint64_t dims[3] = {kD, (cuuint64_t)n, (cuuint64_t)slabs};
+  const cuuint64_t strides[2] = {kD * 2, (cuuint64_t)n * kD * 2};
+  const cuuint32_t box[3] = {kD, (cuuint32_t)box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
@@ -489,62 +705,54 @@ cudaError_t make_tile_map(const void* base, size_t rows, CUtensorMap* out) {
 }  // namespace
 
 bool tc_supported(const wersa_config& cfg) {
-  return cfg.dtype == WERSA_BF16 && (cfg.features == 128 || cfg.features == 256) && cfg.seq_len % kTile == 0 &&
-         cfg.head_dim == kD;
+  return cfg.dtype == WERSA_BF16 && (cfg.features == 128 || cfg.features == 256) && cfg.head_dim == kD;
 }
 
-cudaError_t launch_tc_prepare_w(const Plan& p, const Ws& w, const void* W, cudaStream_t st, int* launches) {
-  const int m = p.cfg.features;
-  k_transpose_w<<<(m * kD + 255) / 256, 256, 0, st>>>((const __nv_bfloat16*)W, w.Wt, m);
-  *launches += 1;
-  return cudaGetLastError();
-}
-
-cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* KFb, const void* V, cudaStream_t st,
+cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const void* V, cudaStream_t st,
                             int* launches) {
-  CUtensorMap map_kf, map_v;
-  const size_t rows = (size_t)p.slabs * p.cfg.seq_len;
+  CUtensorMap map_k, map_v;
   cudaError_t err;
-  if ((err = make_tile_map(KFb, rows, &map_kf)) != cudaSuccess) return err;
-  if ((err = make_tile_map(V, rows, &map_v)) != cudaSuccess) return err;
+  if ((err = make_tile_map(K, p.slabs, p.cfg.seq_len, kBlk, &map_k)) != cudaSuccess) return err;
+  if ((err = make_tile_map(V, p.slabs, p.cfg.seq_len, kBlk, &map_v)) != cudaSuccess) return err;
   dim3 grid(p.tchunks, p.slabs);
   if (p.cfg.features == 256) {
     auto k = k_tc_kside<2>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, KsideSmem<2>::total)) != cudaSuccess)
       return err;
-    k<<<grid, 320, KsideSmem<2>::total, st>>>(map_kf, map_v, w.Wt, w.spart, w.zpart, p.cfg.seq_len, p.tchunk_tiles,
-                                              w.status);
+    k<<<grid, kKsideThreads, KsideSmem<2>::total, st>>>(map_k, map_v, w.Wt, w.f, w.spart, w.zpart, p.cfg.seq_len,
+                                                         p.cfg.levels, p.tchunk_blocks, w.status);
   } else {
     auto k = k_tc_kside<1>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, KsideSmem<1>::total)) != cudaSuccess)
       return err;
-    k<<<grid, 320, KsideSmem<1>::total, st>>>(map_kf, map_v, w.Wt, w.spart, w.zpart, p.cfg.seq_len, p.tchunk_tiles,
-                                              w.status);
+    k<<<grid, kKsideThreads, KsideSmem<1>::total, st>>>(map_k, map_v, w.Wt, w.f, w.spart, w.zpart, p.cfg.seq_len,
+                                                         p.cfg.levels, p.tchunk_blocks, w.status);
   }
   *launches += 1;
   return cudaGetLastError();
 }
 
-cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* QFb, const float* beta, void* O, cudaStream_t st,
+cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const float* beta, void* O, cudaStream_t st,
                             int* launches) {
-  CUtensorMap map_qf, map_o;
-  const size_t rows = (size_t)p.slabs * p.cfg.seq_len;
+  CUtensorMap map_q, map_o;
   cudaError_t err;
-  if ((err = make_tile_map(QFb, rows, &map_qf)) != cudaSuccess) return err;
-  if ((err = make_tile_map(O, rows, &map_o)) != cudaSuccess) return err;
+  if ((err = make_tile_map(Q, p.slabs, p.cfg.seq_len, kBlk, &map_q)) != cudaSuccess) return err;
+  if ((err = make_tile_map(O, p.slabs, p.cfg.seq_len, kTile, &map_o)) != cudaSuccess) return err;
   dim3 grid(p.tchunks, p.slabs);
   if (p.cfg.features == 256) {
     auto k = k_tc_qside<2>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, QsideSmem<2>::total)) != cudaSuccess)
       return err;
-    k<<<grid, 448, QsideSmem<2>::total, st>>>(map_qf, map_o, w.Wt, w.Sbf, w.z, beta, p.cfg.eps, p.cfg.bw_floor,
-                                              p.cfg.seq_len, p.tchunk_tiles, w.status);
+    k<<<grid, kQsideThreads, QsideSmem<2>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
+                                                         p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks,
+                                                         w.status);
   } else {
     auto k = k_tc_qside<1>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, QsideSmem<1>::total)) != cudaSuccess)
       return err;
-    k<<<grid, 448, QsideSmem<1>::total, st>>>(map_qf, map_o, w.Wt, w.Sbf, w.z, beta, p.cfg.eps, p.cfg.bw_floor,
-                                              p.cfg.seq_len, p.tchunk_tiles, w.status);
+    k<<<grid, kQsideThreads, QsideSmem<1>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
+                                                         p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks,
+                                                         w.status);
   }
   *launches += 1;
   return cudaGetLastError();

@@ -122,6 +122,9 @@ TC_SMALL = [
     dict(B=2, H=2, n=1152, d=64, L=4, m=128),     # more tiles than ring stages, alternating warpgroups
     dict(B=1, H=1, n=2560, d=64, L=8, m=256),     # 20 tiles in one CTA chunk set
     dict(B=2, H=3, n=4096, d=64, L=8, m=256, gate_per_head=0),
+    dict(B=2, H=1, n=1000, d=64, L=3, m=128),     # ragged: last block is partly past the end
+    dict(B=1, H=2, n=4100, d=64, L=8, m=256),     # ragged tail of 4 rows in a 256-row Haar block
+    dict(B=1, H=1, n=77, d=64, L=2, m=128),       # shorter than one tile
 ]
 
 
