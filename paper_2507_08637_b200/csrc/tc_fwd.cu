@@ -11,13 +11,13 @@
 //   MMA1: D1[128 tokens x 128 features] = Q_F (smem, K-major) * W (as W^T, K-major)
 //   ReLU warps as above, plus the row dot product with z' (denominator)
 //   MMA2: N'[128 tokens x 64] (+)= Phi (TMEM operand, K = features) * S' (smem bf16, N-major)
-//   epilogue warps: TMEM -> registers -> * 1/(D' + eps') -> bf16 -> swizzled smem -> TMA store
+//   epilogue (aux warps): TMEM -> registers -> * 1/(D' + eps') -> bf16 -> swizzled smem -> TMA store
 //
 // Work unit of the MMA pipeline: one 128-token tile times one 128-feature half ("unit").  Three D1
 // accumulators rotate, so the ReLU pass of a unit overlaps four MMAs of its neighbours.
 // Warp roles: warp 0 TMA producer (K or Q), warp 1 MMA issuer (one thread), warp 2 TMA producer
-// (V, key side), warps 4-11 two ReLU warpgroups that alternate over the units, warps 12-19 Haar
-// filter, warps 20-23 (query side) epilogue.  All operand tiles use the 128-byte swizzle.
+// (V, key side), warps 4-11 two ReLU warpgroups that alternate over the units, warps 12-19 aux: Haar
+// filter and (query side) epilogue.  All operand tiles use the 128-byte swizzle.
 // Every wait on an mbarrier is bounded; a role whose wait expires keeps its control flow (so that
 // group barriers stay balanced) but skips all further work, and the host sees the status word.
 #include "common.cuh"
@@ -41,21 +41,23 @@ constexpr uint32_t kIdesc1 = make_idesc_bf16(128, 128, false, false);  // both o
 constexpr uint32_t kIdesc2 = make_idesc_bf16(128, 64, false, true);    // B = V or S', N-major
 
 constexpr int kWarpTma = 0, kWarpMma = 1, kWarpTmaV = 2;
-constexpr int kReluWarp0 = 4, kHaarWarp0 = 12, kEpiWarp0 = 20;
-constexpr int kKsideThreads = 32 * kEpiWarp0;     // 640
-constexpr int kQsideThreads = 32 * (kEpiWarp0 + 4);   // 768
+constexpr int kReluWarp0 = 4, kAuxWarp0 = 12;       // 8 ReLU warps, 8 aux warps (Haar filter, epilogue)
+constexpr int kThreads = 32 * (kAuxWarp0 + 8);      // 640
+// Registers per thread: 96 at launch (640 threads); the producer / MMA warpgroup gives most of its
+// share to the aux warps, whose Haar step holds a 256 x 64 block in registers.
+constexpr int kRegsCtl = 40, kRegsAux = 120;
 
 enum { kErrProducer = 11, kErrMma = 12, kErrRelu = 13, kErrEpilogue = 14, kErrHaar = 15 };
 
 struct alignas(8) KsideBars {
   uint64_t x_full[kNX], xf_ready[kNX], x_empty[kNX], v_full[kNV], v_empty[kNV];
-  uint64_t d1_full[6], phi_ready[kND1], acc_done, xch[2];
+  uint64_t d1_full[6], phi_ready[kND1], acc_done;
   uint32_t tmem_base;
   int abort_flag;
 };
 struct alignas(8) QsideBars {
   uint64_t x_full[kNX], xf_ready[kNX], x_empty[kNX];
-  uint64_t d1_full[6], phi_ready[kND1], d2_full[2], d2_free[2], den_ready[2], xch[2];
+  uint64_t d1_full[6], phi_ready[kND1], d2_full[2], d2_free[2], den_ready[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -65,7 +67,8 @@ template <int NH> struct KsideSmem {
   static constexpr uint32_t x = wt + NH * kTileBytes;
   static constexpr uint32_t v = x + kNX * kBlkBytes;
   static constexpr uint32_t xch = v + kNV * kBlkBytes;           // 2 x 8 x 64 floats
-  static constexpr uint32_t zx = xch + 4096;                     // 128 floats
+  static constexpr uint32_t hcoef = xch + 4096;                  // kHaarCoefPairs pairs
+  static constexpr uint32_t zx = hcoef + 1024;                   // 128 floats
   static constexpr uint32_t bars = zx + 512;
   static constexpr uint32_t total = bars + 512 + 1024;           // + alignment slack
 };
@@ -75,7 +78,8 @@ template <int NH> struct QsideSmem {
   static constexpr uint32_t x = simg + NH * kTileBytes;
   static constexpr uint32_t ost = x + kNX * kBlkBytes;           // 2 output staging tiles
   static constexpr uint32_t xch = ost + 2 * kTileBytes;          // 2 x 8 x 64 floats
-  static constexpr uint32_t zs = xch + 4096;                     // NH*128 floats
+  static constexpr uint32_t hcoef = xch + 4096;                  // kHaarCoefPairs pairs
+  static constexpr uint32_t zs = hcoef + 1024;                   // NH*128 floats
   static constexpr uint32_t den = zs + NH * 512;                 // 2 x NH x 128 floats
   static constexpr uint32_t bars = den + 2 * NH * 512;
   static constexpr uint32_t total = bars + 512 + 1024;
@@ -103,35 +107,62 @@ __device__ __forceinline__ void reg_fence32(uint32_t (&r)[32]) {
                : "memory");
 }
 
-// ReLU of 32 fp32 accumulator columns -> 16 packed bf16 pairs.  kDot = false: the ReLU values are
-// added up into acc[0..3]; kDot = true: their products with zrow[0..31] are (denominator of Eq. 7).
+// Register budget per role (all warps of a warpgroup execute the same one).
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
+// Two fp32 values in one 64-bit register: the packed add / multiply / fma of sm_100 issue one
+// instruction for both halves.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pk2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void upk2(f32x2 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint32_t pack2_bf16(f32x2 v) {
+  float lo, hi;
+  upk2(v, lo, hi);
+  return pack_bf16x2(lo, hi);
+}
+
+// ReLU of 32 fp32 accumulator columns -> 16 packed bf16 pairs (one fused relu + round + pack per
+// pair).  The side sums use 2 relu(a) = a + |a| (one full-rate add), accumulated as packed pairs:
+// kDot = false: acc += 2 relu(a);  kDot = true: acc += 2 relu(a) * zrow[.]; relu_unit halves the total.
 template <bool kDot>
 __device__ __forceinline__ void relu_chunk(const uint32_t (&r)[32], uint32_t (&p)[16], const float* __restrict__ zrow,
-                                           float (&acc)[4]) {
-  if (kDot) {
+                                           f32x2 (&acc)[2]) {
 #pragma unroll
-    for (int j4 = 0; j4 < 8; ++j4) {
+  for (int j4 = 0; j4 < 8; ++j4) {
+    const float a0 = __uint_as_float(r[4 * j4]), a1 = __uint_as_float(r[4 * j4 + 1]);
+    const float a2 = __uint_as_float(r[4 * j4 + 2]), a3 = __uint_as_float(r[4 * j4 + 3]);
+    p[2 * j4] = relu_pack_bf16x2(a0, a1);
+    p[2 * j4 + 1] = relu_pack_bf16x2(a2, a3);
+    const f32x2 r01 = pk2(a0 + fabsf(a0), a1 + fabsf(a1)), r23 = pk2(a2 + fabsf(a2), a3 + fabsf(a3));
+    if (kDot) {
       const float4 zv = *reinterpret_cast<const float4*>(zrow + 4 * j4);
-      const float a0 = fmaxf(__uint_as_float(r[4 * j4]), 0.f), a1 = fmaxf(__uint_as_float(r[4 * j4 + 1]), 0.f);
-      const float a2 = fmaxf(__uint_as_float(r[4 * j4 + 2]), 0.f), a3 = fmaxf(__uint_as_float(r[4 * j4 + 3]), 0.f);
-      acc[0] = fmaf(a0, zv.x, acc[0]);
-      acc[1] = fmaf(a1, zv.y, acc[1]);
-      acc[2] = fmaf(a2, zv.z, acc[2]);
-      acc[3] = fmaf(a3, zv.w, acc[3]);
-      p[2 * j4] = pack_bf16x2(a0, a1);
-      p[2 * j4 + 1] = pack_bf16x2(a2, a3);
-    }
-  } else {
-#pragma unroll
-    for (int j4 = 0; j4 < 8; ++j4) {
-      const float a0 = fmaxf(__uint_as_float(r[4 * j4]), 0.f), a1 = fmaxf(__uint_as_float(r[4 * j4 + 1]), 0.f);
-      const float a2 = fmaxf(__uint_as_float(r[4 * j4 + 2]), 0.f), a3 = fmaxf(__uint_as_float(r[4 * j4 + 3]), 0.f);
-      acc[0] += a0;
-      acc[1] += a1;
-      acc[2] += a2;
-      acc[3] += a3;
-      p[2 * j4] = pack_bf16x2(a0, a1);
-      p[2 * j4 + 1] = pack_bf16x2(a2, a3);
+      acc[0] = fma2(r01, pk2(zv.x, zv.y), acc[0]);
+      acc[1] = fma2(r23, pk2(zv.z, zv.w), acc[1]);
+    } else {
+      acc[0] = add2(acc[0], r01);
+      acc[1] = add2(acc[1], r23);
     }
   }
 }
@@ -141,7 +172,7 @@ __device__ __forceinline__ void relu_chunk(const uint32_t (&r)[32], uint32_t (&p
 // Returns the row sum of the ReLU values (kDot = false) or their dot product with zrow[0..127].
 template <bool kDot>
 __device__ __forceinline__ float relu_unit(uint32_t taddr, const float* __restrict__ zrow) {
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  f32x2 acc[2] = {0ull, 0ull};
   uint32_t a[32], b[32], p[16];
   tmem_ld32(taddr, a);
   tmem_ld_wait();
@@ -152,162 +183,160 @@ __device__ __forceinline__ float relu_unit(uint32_t taddr, const float* __restri
   tmem_ld_wait();
   reg_fence32(b);
   tmem_ld32(taddr + 64, a);
-  relu_chunk<kDot>(b, p, zrow + 32, acc);
+  relu_chunk<kDot>(b, p, kDot ? zrow + 32 : zrow, acc);
   tmem_st16(taddr + 16, p);
   tmem_ld_wait();
   reg_fence32(a);
   tmem_ld32(taddr + 96, b);
-  relu_chunk<kDot>(a, p, zrow + 64, acc);
+  relu_chunk<kDot>(a, p, kDot ? zrow + 64 : zrow, acc);
   tmem_st16(taddr + 32, p);
   tmem_ld_wait();
   reg_fence32(b);
-  relu_chunk<kDot>(b, p, zrow + 96, acc);
+  relu_chunk<kDot>(b, p, kDot ? zrow + 96 : zrow, acc);
   tmem_st16(taddr + 48, p);
   tmem_st_wait();
-  return (acc[0] + acc[1]) + (acc[2] + acc[3]);
+  float s0, s1, s2, s3;
+  upk2(acc[0], s0, s1);
+  upk2(acc[1], s2, s3);
+  return 0.5f * ((s0 + s1) + (s2 + s3));
 }
 
 // ---- Haar filter of one 256-token block in shared memory ------------------------------------------
 // T_f x = f_0 x + sum_{i=1..L} (f_i - f_{i-1}) * blockmean_{2^i}(x): the detail projector of level l
 // is blockmean_{2^(l-1)} - blockmean_{2^l} and the approximation projector of level L is
 // blockmean_{2^L}, so only aligned block sums of 2, 4, ..., 2^L rows are needed.
-struct HaarCoef {
-  float f0;
-  float k[kMaxLevels + 1];   // k[i] = (f_i - f_{i-1}) / 2^i for 1 <= i <= L, else 0
-};
+// Filter coefficients as (v, v) pairs in shared memory, written once per CTA by the aux warps:
+//   hcoef[0] = f_0, hcoef[i] = k_i = (f_i - f_{i-1}) / 2^i for i = 1..5 (0 beyond L),
+//   hcoef[8 + 8 hw + w] = weight of warp w's 32-row sum in warp hw's levels 6-8 term
+//                       = k_8 + [same 128-row group] k_7 + [same 64-row group] k_6.
+constexpr int kHaarCoefPairs = 8 + 64;
 
-__device__ __forceinline__ HaarCoef haar_coef(const float* __restrict__ f, int L) {
-  HaarCoef c;
-  c.f0 = f[0];
-  c.k[0] = 0.f;
+__device__ __forceinline__ void haar_coef_init(f32x2* hcoef, const float* __restrict__ f, int L, int ht) {
+  float k[kMaxLevels + 1];
+  k[0] = f[0];
   float scale = 0.5f;
 #pragma unroll
   for (int i = 1; i <= kMaxLevels; ++i) {
-    c.k[i] = (i <= L) ? (f[i] - f[i - 1]) * scale : 0.f;
+    k[i] = (i <= L) ? (f[i] - f[i - 1]) * scale : 0.f;
     scale *= 0.5f;
   }
-  return c;
+  if (ht < 6) {
+    float v = k[0];
+#pragma unroll
+    for (int i = 1; i < 6; ++i) v = (ht == i) ? k[i] : v;
+    hcoef[ht] = pk2(v, v);
+  }
+  if (ht < 64) {
+    const int hw = ht >> 3, w = ht & 7;
+    const float v = k[8] + ((w >> 2) == (hw >> 2) ? k[7] : 0.f) + ((w >> 1) == (hw >> 1) ? k[6] : 0.f);
+    hcoef[8 + ht] = pk2(v, v);
+  }
 }
 
 // 256 threads (ht = 0..255) filter the block in place.  Thread (c = ht & 7, rg = ht >> 3) owns rows
 // 8 rg .. 8 rg + 7 of 16-byte chunk c: levels 1-3 in registers, levels 4-5 through warp shuffles
 // (a warp covers 32 consecutive rows), levels 6-8 through the 32-row sums the eight warps leave in
-// `xch` (8 x 64 floats) and announce on `xbar` (8 arrivals per block).  Returns false if the wait
-// on `xbar` gave up.  Rows >= valid_rows lie past the end of the sequence: they arrive as zeros (the
-// zero padding of Algorithm 2) and leave as zeros (the trim before the feature map).
-__device__ __forceinline__ bool haar_block_inplace(uint8_t* slot, const HaarCoef& hc, bool cross, float* xch,
-                                                   uint64_t* xbar, uint32_t xparity, int ht, int valid_rows,
-                                                   volatile int* abort_flag, int* status) {
+// `xch` (8 x 64 floats, double-buffered by the caller) around one named barrier of the 256 threads.
+// The barrier is executed whether or not `ok` holds, so that a role that gave up on a wait keeps the
+// barrier balanced; with ok = false no memory is touched.  Rows >= valid_rows lie past the end of the
+// sequence: they arrive as zeros (the zero padding of Algorithm 2) and leave as zeros (the trim
+// before the feature map).
+__device__ __forceinline__ void haar_block_inplace(uint8_t* slot, const f32x2* hcoef, bool cross, float* xch, int ht,
+                                                   int valid_rows, bool ok) {
   const int c = ht & 7, rg = ht >> 3, lane = ht & 31, hw = ht >> 5;
   uint8_t* base = slot + rg * 1024;
-  float x[8][8];
+  f32x2 x[8][4];   // 8 rows x 4 column pairs
+  f32x2 hi[4], s5[4];
+  if (ok) {
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {   // row 8 rg + j has swizzle phase j
-    const uint4 raw = *reinterpret_cast<const uint4*>(base + j * 128 + ((c ^ j) << 4));
-    const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+    for (int j = 0; j < 8; ++j) {   // row 8 rg + j has swizzle phase j
+      const uint4 raw = *reinterpret_cast<const uint4*>(base + j * 128 + ((c ^ j) << 4));
+      const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      x[j][2 * i] = __uint_as_float(u[i] << 16);
-      x[j][2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
+      for (int i = 0; i < 4; ++i) x[j][i] = pk2(__uint_as_float(u[i] << 16), __uint_as_float(u[i] & 0xFFFF0000u));
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const f32x2 s3 = add2(add2(add2(x[0][q], x[1][q]), add2(x[2][q], x[3][q])),
+                            add2(add2(x[4][q], x[5][q]), add2(x[6][q], x[7][q])));
+      float lo, hi_;
+      upk2(s3, lo, hi_);
+      const f32x2 s4 = add2(s3, pk2(__shfl_xor_sync(0xffffffffu, lo, 8), __shfl_xor_sync(0xffffffffu, hi_, 8)));
+      upk2(s4, lo, hi_);
+      s5[q] = add2(s4, pk2(__shfl_xor_sync(0xffffffffu, lo, 16), __shfl_xor_sync(0xffffffffu, hi_, 16)));
+      hi[q] = fma2(hcoef[3], s3, fma2(hcoef[4], s4, mul2(hcoef[5], s5[q])));
     }
   }
-  float hi[8], s5[8];
-#pragma unroll
-  for (int col = 0; col < 8; ++col) {
-    const float s3 = ((x[0][col] + x[1][col]) + (x[2][col] + x[3][col])) +
-                     ((x[4][col] + x[5][col]) + (x[6][col] + x[7][col]));
-    const float s4 = s3 + __shfl_xor_sync(0xffffffffu, s3, 8);
-    s5[col] = s4 + __shfl_xor_sync(0xffffffffu, s4, 16);
-    hi[col] = fmaf(hc.k[3], s3, fmaf(hc.k[4], s4, hc.k[5] * s5[col]));
-  }
-  bool ok = true;
   if (cross) {   // uniform over the kernel: L > 5
-    if ((lane >> 3) == 0) {
-      float4* dst = reinterpret_cast<float4*>(xch + hw * kD + c * 8);
-      dst[0] = make_float4(s5[0], s5[1], s5[2], s5[3]);
-      dst[1] = make_float4(s5[4], s5[5], s5[6], s5[7]);
+    if (ok && (lane >> 3) == 0) {
+      ulonglong2* dst = reinterpret_cast<ulonglong2*>(xch + hw * kD + c * 8);
+      dst[0] = make_ulonglong2(s5[0], s5[1]);
+      dst[1] = make_ulonglong2(s5[2], s5[3]);
     }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(xbar);
-    ok = __all_sync(0xffffffffu, mbar_wait(xbar, xparity, abort_flag, status, kErrHaar));
+    named_bar_sync(4, 256);
     if (ok) {
-      float w8[8][8];
+      // lane (c, q = lane >> 3) combines the eight warps' sums of column pair q of chunk c, then the
+      // four lanes that share a chunk swap their pairs
+      const int qq = lane >> 3;
+      f32x2 acc = 0ull;
 #pragma unroll
-      for (int w = 0; w < 8; ++w) {
-        const float4* src = reinterpret_cast<const float4*>(xch + w * kD + c * 8);
-        const float4 lo = src[0], hi4 = src[1];
-        w8[w][0] = lo.x; w8[w][1] = lo.y; w8[w][2] = lo.z; w8[w][3] = lo.w;
-        w8[w][4] = hi4.x; w8[w][5] = hi4.y; w8[w][6] = hi4.z; w8[w][7] = hi4.w;
-      }
+      for (int w = 0; w < 8; ++w)
+        acc = fma2(hcoef[8 + 8 * hw + w], *reinterpret_cast<const f32x2*>(xch + w * kD + c * 8 + 2 * qq), acc);
+      float lo, hi_;
+      upk2(acc, lo, hi_);
 #pragma unroll
-      for (int col = 0; col < 8; ++col) {
-        const float p0 = w8[0][col] + w8[1][col], p1 = w8[2][col] + w8[3][col];
-        const float p2 = w8[4][col] + w8[5][col], p3 = w8[6][col] + w8[7][col];
-        const float q0 = p0 + p1, q1 = p2 + p3;
-        const float s8 = q0 + q1;
-        const float s7 = (hw & 4) ? q1 : q0;
-        const float s6 = (hw & 4) ? ((hw & 2) ? p3 : p2) : ((hw & 2) ? p1 : p0);
-        hi[col] += fmaf(hc.k[6], s6, fmaf(hc.k[7], s7, hc.k[8] * s8));
+      for (int q = 0; q < 4; ++q) {
+        const int src = (q << 3) | c;
+        hi[q] = add2(hi[q], pk2(__shfl_sync(0xffffffffu, lo, src), __shfl_sync(0xffffffffu, hi_, src)));
       }
     }
   }
   if (ok) {
+    const f32x2 f0 = hcoef[0], k1 = hcoef[1], k2 = hcoef[2];
 #pragma unroll
-    for (int col = 0; col < 8; ++col) {
-      const float a0 = x[0][col] + x[1][col], a1 = x[2][col] + x[3][col];
-      const float a2 = x[4][col] + x[5][col], a3 = x[6][col] + x[7][col];
-      const float c20 = fmaf(hc.k[2], a0 + a1, hi[col]), c21 = fmaf(hc.k[2], a2 + a3, hi[col]);
-      const float c10 = fmaf(hc.k[1], a0, c20), c11 = fmaf(hc.k[1], a1, c20);
-      const float c12 = fmaf(hc.k[1], a2, c21), c13 = fmaf(hc.k[1], a3, c21);
-      x[0][col] = fmaf(hc.f0, x[0][col], c10);
-      x[1][col] = fmaf(hc.f0, x[1][col], c10);
-      x[2][col] = fmaf(hc.f0, x[2][col], c11);
-      x[3][col] = fmaf(hc.f0, x[3][col], c11);
-      x[4][col] = fmaf(hc.f0, x[4][col], c12);
-      x[5][col] = fmaf(hc.f0, x[5][col], c12);
-      x[6][col] = fmaf(hc.f0, x[6][col], c13);
-      x[7][col] = fmaf(hc.f0, x[7][col], c13);
+    for (int q = 0; q < 4; ++q) {
+      const f32x2 a0 = add2(x[0][q], x[1][q]), a1 = add2(x[2][q], x[3][q]);
+      const f32x2 a2 = add2(x[4][q], x[5][q]), a3 = add2(x[6][q], x[7][q]);
+      const f32x2 c20 = fma2(k2, add2(a0, a1), hi[q]), c21 = fma2(k2, add2(a2, a3), hi[q]);
+      const f32x2 c10 = fma2(k1, a0, c20), c11 = fma2(k1, a1, c20);
+      const f32x2 c12 = fma2(k1, a2, c21), c13 = fma2(k1, a3, c21);
+      x[0][q] = fma2(f0, x[0][q], c10);
+      x[1][q] = fma2(f0, x[1][q], c10);
+      x[2][q] = fma2(f0, x[2][q], c11);
+      x[3][q] = fma2(f0, x[3][q], c11);
+      x[4][q] = fma2(f0, x[4][q], c12);
+      x[5][q] = fma2(f0, x[5][q], c12);
+      x[6][q] = fma2(f0, x[6][q], c13);
+      x[7][q] = fma2(f0, x[7][q], c13);
     }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      uint4 out;
-      out.x = pack_bf16x2(x[j][0], x[j][1]);
-      out.y = pack_bf16x2(x[j][2], x[j][3]);
-      out.z = pack_bf16x2(x[j][4], x[j][5]);
-      out.w = pack_bf16x2(x[j][6], x[j][7]);
+      uint4 out = make_uint4(pack2_bf16(x[j][0]), pack2_bf16(x[j][1]), pack2_bf16(x[j][2]), pack2_bf16(x[j][3]));
       if (rg * 8 + j >= valid_rows) out = make_uint4(0u, 0u, 0u, 0u);
       *reinterpret_cast<uint4*>(base + j * 128 + ((c ^ j) << 4)) = out;
     }
   }
-  return ok;
 }
 
-// Haar role shared by both kernels: for every block, wait for the raw tile, filter it in place and
-// hand it to the MMA issuer.
+// One Haar step of the aux role: wait for raw block b, filter it in place, hand it to the MMA issuer.
 template <typename Bars>
-__device__ __forceinline__ void haar_role(uint8_t* xring, Bars* bars, float* xch, const float* __restrict__ f, int L,
-                                          int nblk, int rows_left, volatile int* abort_flag, int* status) {
-  const int ht = threadIdx.x - 32 * kHaarWarp0;
-  const HaarCoef hc = haar_coef(f, L);
-  const bool cross = L > 5;
-  bool ok = true;
-  for (int b = 0; b < nblk; ++b) {
-    const int s = b % kNX;
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[s], (b / kNX) & 1, abort_flag, status, kErrHaar));
-    if (ok)
-      ok = haar_block_inplace(xring + s * kBlkBytes, hc, cross, xch + (b & 1) * 8 * kD, &bars->xch[b & 1],
-                              (b >> 1) & 1, ht, rows_left - b * kBlk, abort_flag, status);
-    if (ok) {
-      fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
-      mbar_arrive(&bars->xf_ready[s]);
-    }
+__device__ __forceinline__ bool haar_step(uint8_t* xring, Bars* bars, float* xch, const f32x2* hcoef, bool cross,
+                                          int b, int rows_left, int ht, bool ok, volatile int* abort_flag,
+                                          int* status) {
+  const int s = b % kNX;
+  if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[s], (b / kNX) & 1, abort_flag, status, kErrHaar));
+  haar_block_inplace(xring + s * kBlkBytes, hcoef, cross, xch + (b & 1) * 8 * kD, ht, rows_left - b * kBlk, ok);
+  if (ok) {
+    fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
+    mbar_arrive(&bars->xf_ready[s]);
   }
+  return ok;
 }
 
 // ---- key side -----------------------------------------------------------------------------------
 // grid (chunks, slabs), block 640.  TMEM: D1[3] at columns 0 / 128 / 256, S' half h at 384 + 64 h.
 template <int NH>
-__global__ void __launch_bounds__(kKsideThreads, 1)
+__global__ void __launch_bounds__(kThreads, 1)
 k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
            const __nv_bfloat16* __restrict__ Wt, const float* __restrict__ f, float* __restrict__ spart,
            float* __restrict__ zpart, int n, int L, int chunk_blocks, int* __restrict__ status) {
@@ -336,8 +365,6 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
     for (int b = 0; b < 6; ++b) mbar_init(&bars->d1_full[b], 1);
     for (int b = 0; b < kND1; ++b) mbar_init(&bars->phi_ready[b], 128);
     mbar_init(&bars->acc_done, 1);
-    mbar_init(&bars->xch[0], 8);
-    mbar_init(&bars->xch[1], 8);
     bars->abort_flag = 0;
     fence_mbar_init();
   }
@@ -353,8 +380,9 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
   const uint32_t tmem = bars->tmem_base;
   volatile int* abort_flag = &bars->abort_flag;
 
-  if (warp == kWarpTma || warp == kWarpTmaV) {
-    if (lane == 0) {
+  if (warp < kReluWarp0) {
+    reg_dec<kRegsCtl>();
+    if ((warp == kWarpTma || warp == kWarpTmaV) && lane == 0) {
       const bool is_v = warp == kWarpTmaV;
       const int depth = is_v ? kNV : kNX;
       uint64_t* full = is_v ? bars->v_full : bars->x_full;
@@ -372,52 +400,71 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       if (*abort_flag != 0) {   // let copies in flight land before the CTA's shared memory goes away
         for (int b = max(0, issued - depth); b < issued; ++b) mbar_wait_drain(&full[b % depth], (b / depth) & 1);
       }
-    }
-  } else if (warp == kWarpMma) {
-    if (lane == 0) {
-      const uint32_t wt_addr = smem_u32(smem + SL::wt);
-      const uint32_t x_addr = smem_u32(smem + SL::x);
-      const uint32_t v_addr = smem_u32(smem + SL::v);
+    } else if (warp == kWarpMma && lane == 0) {
+      // Issue order: MMA1 of unit u, then MMA2 of unit u - 2.  Everything that depends on the unit's
+      // position inside its block is resolved at compile time; ring slots, D1 buffers and barrier
+      // phases are running counters, and descriptors only add to their start-address word.
+      constexpr int UPB = 2 * NH;                       // units per 256-token block
+      constexpr uint32_t kTileStep = kTileBytes >> 4, kBlkStep = kBlkBytes >> 4;
+      const uint32_t hi = smem_desc_hi(1024);
+      const uint32_t wt_lo = smem_desc_lo(smem_u32(smem + SL::wt), 16);
+      const uint32_t x_lo = smem_desc_lo(smem_u32(smem + SL::x), 16);
+      const uint32_t v_lo = smem_desc_lo(smem_u32(smem + SL::v), 1024);
+      uint32_t xs = 0, xpar = 0, vs = 0, vpar = 0;     // ring slot and phase of the block MMA1 / MMA2 is in
+      uint32_t c3 = 0, c6 = 0;                          // MMA1: D1 buffer, d1_full barrier
+      uint32_t p3 = 0, ppar = 0;                        // MMA2: D1 buffer (= phi_ready barrier) and phase
       bool ok = true;
-      for (int i = 0; i < units + 2 && ok; ++i) {
-        if (i < units) {
-          const int t = i / NH, h = i % NH, b = t >> 1, s = b % kNX;
-          if ((t & 1) == 0 && h == 0) {
-            ok = mbar_wait(&bars->xf_ready[s], (b / kNX) & 1, abort_flag, status, kErrMma);
-            if (!ok) break;
-            tc_fence_after_sync();
-          }
-          const uint32_t d1 = tmem + (i % kND1) * 128;
-          const uint32_t b_addr = x_addr + s * kBlkBytes + (t & 1) * kTileBytes;
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            mma_ss(d1, make_smem_desc(wt_addr + h * kTileBytes + k * 32, 16, 1024),
-                   make_smem_desc(b_addr + k * 32, 16, 1024), kIdesc1, k > 0);
-          mma_commit(&bars->d1_full[i % 6]);
-          if ((t & 1) == 1 && h == NH - 1) mma_commit(&bars->x_empty[s]);
-        }
-        if (i >= 2) {
-          const int v = i - 2;
-          const int t = v / NH, h = v % NH, b = t >> 1, s = b % kNV;
-          if ((t & 1) == 0 && h == 0) {
-            ok = mbar_wait(&bars->v_full[s], (b / kNV) & 1, abort_flag, status, kErrMma);
-            if (!ok) break;
-          }
-          ok = mbar_wait(&bars->phi_ready[v % kND1], (v / kND1) & 1, abort_flag, status, kErrMma);
+      for (int b = 0; b <= nblk && ok; ++b) {
+        if (b < nblk) {
+          ok = mbar_wait(&bars->xf_ready[xs], xpar, abort_flag, status, kErrMma);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t acc = tmem + kAccCol + h * 64;
-          const uint32_t b_addr = v_addr + s * kBlkBytes + (t & 1) * kTileBytes;
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            mma_ts(acc, tmem + (v % kND1) * 128 + k * 8, make_smem_desc(b_addr + k * 2048, 1024, 1024), kIdesc2,
-                   (t > 0 || k > 0) ? 1u : 0u);
-          if ((t & 1) == 1 && h == NH - 1) mma_commit(&bars->v_empty[s]);
         }
+#pragma unroll
+        for (int j = 0; j < UPB; ++j) {
+          if (b < nblk) {
+            const int tt = j / NH, h = j % NH;
+            const uint32_t a_lo = wt_lo + h * kTileStep, b_lo = x_lo + xs * kBlkStep + tt * kTileStep;
+            const uint32_t d1 = tmem + c3 * 128;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              mma_ss(d1, smem_desc_join(a_lo + 2 * k, hi), smem_desc_join(b_lo + 2 * k, hi), kIdesc1, k > 0);
+            mma_commit(&bars->d1_full[c6]);
+            if (j == UPB - 1) mma_commit(&bars->x_empty[xs]);
+            c3 = c3 == kND1 - 1 ? 0 : c3 + 1;
+            c6 = c6 == 5 ? 0 : c6 + 1;
+          }
+          const int lj = j >= 2 ? j - 2 : j - 2 + UPB;   // unit u - 2: in this block, or late in the previous one
+          const int bb = j >= 2 ? b : b - 1;
+          if (bb >= 0 && bb < nblk) {
+            const int tt = lj / NH, h = lj % NH;
+            if (lj == 0) {
+              ok = mbar_wait(&bars->v_full[vs], vpar, abort_flag, status, kErrMma);
+              if (!ok) break;
+            }
+            ok = mbar_wait(&bars->phi_ready[p3], ppar, abort_flag, status, kErrMma);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t acc = tmem + kAccCol + h * 64, a_tm = tmem + p3 * 128;
+            const uint32_t b_lo = v_lo + vs * kBlkStep + tt * kTileStep;
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              mma_ts(acc, a_tm + k * 8, smem_desc_join(b_lo + 128 * k, hi), kIdesc2, (bb > 0 || tt > 0 || k > 0) ? 1u : 0u);
+            if (lj == UPB - 1) {
+              mma_commit(&bars->v_empty[vs]);
+              vs = vs == kNV - 1 ? 0 : vs + 1;
+              vpar ^= (vs == 0);
+            }
+            p3 = p3 == kND1 - 1 ? 0 : p3 + 1;
+            ppar ^= (p3 == 0);
+          }
+        }
+        xs = xs == kNX - 1 ? 0 : xs + 1;
+        xpar ^= (xs == 0);
       }
       mma_commit(&bars->acc_done);
     }
-  } else if (warp >= kReluWarp0 && warp < kHaarWarp0) {
+  } else if (warp >= kReluWarp0 && warp < kAuxWarp0) {
     const int g = (warp - kReluWarp0) >> 2;         // ReLU warpgroup 0 / 1
     const uint32_t lane_base = 32u * (warp & 3);
     const int row = lane_base + lane;               // feature within the half = TMEM lane
@@ -455,9 +502,16 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       }
       zpart[pidx * m + feat] = zacc;
     }
-  } else if (warp >= kHaarWarp0) {
-    haar_role(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), f + (size_t)slab * (L + 1), L, nblk,
-              n - blk0 * kBlk, abort_flag, status);
+  } else {
+    reg_inc<kRegsAux>();
+    const int ht = threadIdx.x - 32 * kAuxWarp0;
+    f32x2* hcoef = reinterpret_cast<f32x2*>(smem + SL::hcoef);
+    haar_coef_init(hcoef, f + (size_t)slab * (L + 1), L, ht);
+    named_bar_sync(3, 256);
+    bool ok = true;
+    for (int b = 0; b < nblk; ++b)
+      ok = haar_step(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
+                     ht, ok, abort_flag, status);
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -468,10 +522,11 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
 }
 
 // ---- query side ---------------------------------------------------------------------------------
-// grid (chunks, slabs), block 768.  TMEM: D1[3] at columns 0 / 128 / 256, N' of tile parity p at
-// 384 + 64 p.  The partial denominators of a tile travel through shared memory (den).
+// grid (chunks, slabs), block 640.  TMEM: D1[3] at columns 0 / 128 / 256, N' of tile parity p at
+// 384 + 64 p.  The partial denominators of a tile travel through shared memory (den).  The aux warps
+// filter block b, then write out the two tiles of block b - 1.
 template <int NH>
-__global__ void __launch_bounds__(kQsideThreads, 1)
+__global__ void __launch_bounds__(kThreads, 1)
 k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
            const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ Sbf,
            const float* __restrict__ zg, const float* __restrict__ f, const float* __restrict__ beta, float eps,
@@ -500,9 +555,8 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     for (int b = 0; b < kND1; ++b) mbar_init(&bars->phi_ready[b], 128);
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bars->d2_full[b], 1);
-      mbar_init(&bars->d2_free[b], 128);
+      mbar_init(&bars->d2_free[b], 256);
       mbar_init(&bars->den_ready[b], 128 * NH);
-      mbar_init(&bars->xch[b], 8);
     }
     bars->abort_flag = 0;
     fence_mbar_init();
@@ -521,8 +575,9 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
   const uint32_t tmem = bars->tmem_base;
   volatile int* abort_flag = &bars->abort_flag;
 
-  if (warp == kWarpTma) {
-    if (lane == 0) {
+  if (warp < kReluWarp0) {
+    reg_dec<kRegsCtl>();
+    if (warp == kWarpTma && lane == 0) {
       int issued = 0;
       for (int b = 0; b < nblk; ++b) {
         const int s = b % kNX;
@@ -534,50 +589,64 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       if (*abort_flag != 0) {
         for (int b = max(0, issued - kNX); b < issued; ++b) mbar_wait_drain(&bars->x_full[b % kNX], (b / kNX) & 1);
       }
-    }
-  } else if (warp == kWarpMma) {
-    if (lane == 0) {
-      const uint32_t wt_addr = smem_u32(smem + SL::wt);
-      const uint32_t s_addr = smem_u32(smem + SL::simg);
-      const uint32_t x_addr = smem_u32(smem + SL::x);
+    } else if (warp == kWarpMma && lane == 0) {
+      // Same issue scheme as the key side (MMA1 of unit u, then MMA2 of unit u - 2).
+      constexpr int UPB = 2 * NH;
+      constexpr uint32_t kTileStep = kTileBytes >> 4, kBlkStep = kBlkBytes >> 4;
+      const uint32_t hi = smem_desc_hi(1024);
+      const uint32_t wt_lo = smem_desc_lo(smem_u32(smem + SL::wt), 16);
+      const uint32_t x_lo = smem_desc_lo(smem_u32(smem + SL::x), 16);
+      const uint32_t s_lo = smem_desc_lo(smem_u32(smem + SL::simg), 1024);
+      uint32_t xs = 0, xpar = 0;
+      uint32_t c3 = 0, c6 = 0;
+      uint32_t p3 = 0, ppar = 0;
       bool ok = true;
-      for (int i = 0; i < units + 2 && ok; ++i) {
-        if (i < units) {
-          const int t = i / NH, h = i % NH, b = t >> 1, s = b % kNX;
-          if ((t & 1) == 0 && h == 0) {
-            ok = mbar_wait(&bars->xf_ready[s], (b / kNX) & 1, abort_flag, status, kErrMma);
-            if (!ok) break;
-            tc_fence_after_sync();
-          }
-          const uint32_t d1 = tmem + (i % kND1) * 128;
-          const uint32_t a_addr = x_addr + s * kBlkBytes + (t & 1) * kTileBytes;
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            mma_ss(d1, make_smem_desc(a_addr + k * 32, 16, 1024),
-                   make_smem_desc(wt_addr + h * kTileBytes + k * 32, 16, 1024), kIdesc1, k > 0);
-          mma_commit(&bars->d1_full[i % 6]);
-          if ((t & 1) == 1 && h == NH - 1) mma_commit(&bars->x_empty[s]);
-        }
-        if (i >= 2) {
-          const int v = i - 2;
-          const int t = v / NH, h = v % NH;
-          ok = mbar_wait(&bars->phi_ready[v % kND1], (v / kND1) & 1, abort_flag, status, kErrMma);
+      for (int b = 0; b <= nblk && ok; ++b) {
+        if (b < nblk) {
+          ok = mbar_wait(&bars->xf_ready[xs], xpar, abort_flag, status, kErrMma);
           if (!ok) break;
-          if (h == 0 && t >= 2) {
-            ok = mbar_wait(&bars->d2_free[t & 1], ((t >> 1) - 1) & 1, abort_flag, status, kErrMma);
-            if (!ok) break;
-          }
           tc_fence_after_sync();
-          const uint32_t d2 = tmem + kAccCol + (t & 1) * 64;
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            mma_ts(d2, tmem + (v % kND1) * 128 + k * 8, make_smem_desc(s_addr + h * kTileBytes + k * 2048, 1024, 1024),
-                   kIdesc2, (h > 0 || k > 0) ? 1u : 0u);
-          if (h == NH - 1) mma_commit(&bars->d2_full[t & 1]);
         }
+#pragma unroll
+        for (int j = 0; j < UPB; ++j) {
+          if (b < nblk) {
+            const int tt = j / NH, h = j % NH;
+            const uint32_t a_lo = x_lo + xs * kBlkStep + tt * kTileStep, b_lo = wt_lo + h * kTileStep;
+            const uint32_t d1 = tmem + c3 * 128;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              mma_ss(d1, smem_desc_join(a_lo + 2 * k, hi), smem_desc_join(b_lo + 2 * k, hi), kIdesc1, k > 0);
+            mma_commit(&bars->d1_full[c6]);
+            if (j == UPB - 1) mma_commit(&bars->x_empty[xs]);
+            c3 = c3 == kND1 - 1 ? 0 : c3 + 1;
+            c6 = c6 == 5 ? 0 : c6 + 1;
+          }
+          const int lj = j >= 2 ? j - 2 : j - 2 + UPB;
+          const int bb = j >= 2 ? b : b - 1;
+          if (bb >= 0 && bb < nblk) {
+            const int tt = lj / NH, h = lj % NH;      // tile 2 bb + tt has parity tt
+            ok = mbar_wait(&bars->phi_ready[p3], ppar, abort_flag, status, kErrMma);
+            if (!ok) break;
+            if (h == 0 && bb >= 1) {                  // N' of tile parity tt must have been drained (tile t - 2)
+              ok = mbar_wait(&bars->d2_free[tt], (bb - 1) & 1, abort_flag, status, kErrMma);
+              if (!ok) break;
+            }
+            tc_fence_after_sync();
+            const uint32_t d2 = tmem + kAccCol + tt * 64, a_tm = tmem + p3 * 128;
+            const uint32_t b_lo = s_lo + h * kTileStep;
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              mma_ts(d2, a_tm + k * 8, smem_desc_join(b_lo + 128 * k, hi), kIdesc2, (h > 0 || k > 0) ? 1u : 0u);
+            if (h == NH - 1) mma_commit(&bars->d2_full[tt]);
+            p3 = p3 == kND1 - 1 ? 0 : p3 + 1;
+            ppar ^= (p3 == 0);
+          }
+        }
+        xs = xs == kNX - 1 ? 0 : xs + 1;
+        xpar ^= (xs == 0);
       }
     }
-  } else if (warp >= kReluWarp0 && warp < kHaarWarp0) {
+  } else if (warp >= kReluWarp0 && warp < kAuxWarp0) {
     const int g = (warp - kReluWarp0) >> 2;
     const uint32_t lane_base = 32u * (warp & 3);
     const int row = lane_base + lane;               // token within the tile = TMEM lane
@@ -598,69 +667,66 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       den[((t & 1) * NH + h) * 128 + row] = dot;
       mbar_arrive(&bars->den_ready[t & 1]);
     }
-  } else if (warp >= kHaarWarp0 && warp < kEpiWarp0) {
-    haar_role(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), f + (size_t)slab * (L + 1), L, nblk,
-              n - blk0 * kBlk, abort_flag, status);
-  } else if (warp >= kEpiWarp0) {
+  } else {
+    reg_inc<kRegsAux>();
+    const int ht = threadIdx.x - 32 * kAuxWarp0;
+    f32x2* hcoef = reinterpret_cast<f32x2*>(smem + SL::hcoef);
+    haar_coef_init(hcoef, f + (size_t)slab * (L + 1), L, ht);
+    named_bar_sync(3, 256);
     const uint32_t lane_base = 32u * (warp & 3);
     const int row = lane_base + lane;               // token within the tile = TMEM lane
-    const int et = threadIdx.x - 32 * kEpiWarp0;    // 0..127 inside the epilogue warpgroup
+    const int ch = (warp - kAuxWarp0) >> 2;         // which 32 of the tile's 64 output columns
     const float bw = fmaxf(beta[0], bw_floor);
     const float epsp = eps * (float)m * bw * bw;
     bool ok = true;
-    for (int t = 0; t < ntiles; ++t) {
-      const int p = t & 1;
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d2_full[p], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->den_ready[p], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
-      uint32_t r0[32], r1[32];
-      float inv = 0.f;
-      if (ok) {
-        tc_fence_after_sync();
-        const uint32_t base = tmem + (lane_base << 16) + kAccCol + p * 64;
-        tmem_ld32(base, r0);
-        tmem_ld32(base + 32, r1);
-        float dsum = epsp;
+    for (int b = 0; b <= nblk; ++b) {
+      if (b < nblk)
+        ok = haar_step(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b,
+                       n - blk0 * kBlk, ht, ok, abort_flag, status);
+      if (b == 0) continue;
+      for (int t = 2 * b - 2; t < 2 * b; ++t) {     // epilogue of the two tiles of block b - 1
+        const int p = t & 1;
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d2_full[p], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->den_ready[p], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
+        uint32_t r[32];
+        f32x2 inv2 = 0ull;
+        if (ok) {
+          tc_fence_after_sync();
+          tmem_ld32(tmem + (lane_base << 16) + kAccCol + p * 64 + 32 * ch, r);
+          float dsum = epsp;
 #pragma unroll
-        for (int h = 0; h < NH; ++h) dsum += den[(p * NH + h) * 128 + row];
-        inv = 1.f / dsum;
-        tmem_ld_wait();
-        reg_fence32(r0);
-        reg_fence32(r1);
-        tc_fence_before_sync();
-        mbar_arrive(&bars->d2_free[p]);
-      }
-      // staging buffer p was last used by tile t-2: its TMA store must have finished reading
-      if (et == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-      named_bar_sync(2, 128);
-      uint8_t* ost = smem + SL::ost + p * kTileBytes;
-      if (ok) {
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint4 v;
-          v.x = pack_bf16x2(__uint_as_float(r0[8 * c]) * inv, __uint_as_float(r0[8 * c + 1]) * inv);
-          v.y = pack_bf16x2(__uint_as_float(r0[8 * c + 2]) * inv, __uint_as_float(r0[8 * c + 3]) * inv);
-          v.z = pack_bf16x2(__uint_as_float(r0[8 * c + 4]) * inv, __uint_as_float(r0[8 * c + 5]) * inv);
-          v.w = pack_bf16x2(__uint_as_float(r0[8 * c + 6]) * inv, __uint_as_float(r0[8 * c + 7]) * inv);
-          *reinterpret_cast<uint4*>(ost + swz128(row, c)) = v;
+          for (int h = 0; h < NH; ++h) dsum += den[(p * NH + h) * 128 + row];
+          const float inv = 1.f / dsum;
+          inv2 = pk2(inv, inv);
+          tmem_ld_wait();
+          reg_fence32(r);
+          tc_fence_before_sync();
+          mbar_arrive(&bars->d2_free[p]);
         }
+        // staging buffer p was last used by tile t-2: its TMA store must have finished reading
+        if (ht == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        named_bar_sync(2, 256);
+        uint8_t* ost = smem + SL::ost + p * kTileBytes;
+        if (ok) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint4 v;
-          v.x = pack_bf16x2(__uint_as_float(r1[8 * c]) * inv, __uint_as_float(r1[8 * c + 1]) * inv);
-          v.y = pack_bf16x2(__uint_as_float(r1[8 * c + 2]) * inv, __uint_as_float(r1[8 * c + 3]) * inv);
-          v.z = pack_bf16x2(__uint_as_float(r1[8 * c + 4]) * inv, __uint_as_float(r1[8 * c + 5]) * inv);
-          v.w = pack_bf16x2(__uint_as_float(r1[8 * c + 6]) * inv, __uint_as_float(r1[8 * c + 7]) * inv);
-          *reinterpret_cast<uint4*>(ost + swz128(row, 4 + c)) = v;
+          for (int c = 0; c < 4; ++c) {
+            uint4 v;
+            v.x = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c]), __uint_as_float(r[8 * c + 1])), inv2));
+            v.y = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c + 2]), __uint_as_float(r[8 * c + 3])), inv2));
+            v.z = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c + 4]), __uint_as_float(r[8 * c + 5])), inv2));
+            v.w = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c + 6]), __uint_as_float(r[8 * c + 7])), inv2));
+            *reinterpret_cast<uint4*>(ost + swz128(row, 4 * ch + c)) = v;
+          }
+          fence_proxy_async_smem();
         }
-        fence_proxy_async_smem();
-      }
-      named_bar_sync(2, 128);
-      if (et == 0 && ok && blk0 * kBlk + t * kTile < n) {   // rows past n are clipped by the store
-        tma_store_3d(&map_o, ost, 0, blk0 * kBlk + t * kTile, slab);
-        bulk_commit_group();
+        named_bar_sync(2, 256);
+        if (ht == 0 && ok && blk0 * kBlk + t * kTile < n) {   // rows past n are clipped by the store
+          tma_store_3d(&map_o, ost, 0, blk0 * kBlk + t * kTile, slab);
+          bulk_commit_group();
+        }
       }
     }
-    if (et == 0) bulk_wait_group0();
+    if (ht == 0) bulk_wait_group0();
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -719,13 +785,13 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
     auto k = k_tc_kside<2>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, KsideSmem<2>::total)) != cudaSuccess)
       return err;
-    k<<<grid, kKsideThreads, KsideSmem<2>::total, st>>>(map_k, map_v, w.Wt, w.f, w.spart, w.zpart, p.cfg.seq_len,
+    k<<<grid, kThreads, KsideSmem<2>::total, st>>>(map_k, map_v, w.Wt, w.f, w.spart, w.zpart, p.cfg.seq_len,
                                                          p.cfg.levels, p.tchunk_blocks, w.status);
   } else {
     auto k = k_tc_kside<1>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, KsideSmem<1>::total)) != cudaSuccess)
       return err;
-    k<<<grid, kKsideThreads, KsideSmem<1>::total, st>>>(map_k, map_v, w.Wt, w.f, w.spart, w.zpart, p.cfg.seq_len,
+    k<<<grid, kThreads, KsideSmem<1>::total, st>>>(map_k, map_v, w.Wt, w.f, w.spart, w.zpart, p.cfg.seq_len,
                                                          p.cfg.levels, p.tchunk_blocks, w.status);
   }
   *launches += 1;
@@ -743,14 +809,14 @@ cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const flo
     auto k = k_tc_qside<2>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, QsideSmem<2>::total)) != cudaSuccess)
       return err;
-    k<<<grid, kQsideThreads, QsideSmem<2>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
+    k<<<grid, kThreads, QsideSmem<2>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
                                                          p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks,
                                                          w.status);
   } else {
     auto k = k_tc_qside<1>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, QsideSmem<1>::total)) != cudaSuccess)
       return err;
-    k<<<grid, kQsideThreads, QsideSmem<1>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
+    k<<<grid, kThreads, QsideSmem<1>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
                                                          p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks,
                                                          w.status);
   }
