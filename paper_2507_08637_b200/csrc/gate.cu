@@ -96,11 +96,19 @@ __global__ void __launch_bounds__(256) k_qbar_gate(const float* __restrict__ qpa
     qs[c] = q;
   }
   __syncthreads();
-  if (threadIdx.x < L1) {
-    const int i = threadIdx.x;
-    float u = 0.f;
-    if (gate_w != nullptr)
-      for (int kk = 0; kk < kD; ++kk) u += gate_w[((size_t)h * kD + kk) * L1 + i] * qs[kk];
+  // logits: 16 lanes per band, four of the 64 terms each, then a fixed-order butterfly
+  const int i = threadIdx.x >> 4, seg = threadIdx.x & 15;
+  float u = 0.f;
+  if (gate_w != nullptr && i < L1) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int kk = seg * 4 + j;
+      u += gate_w[((size_t)h * kD + kk) * L1 + i] * qs[kk];
+    }
+  }
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) u += __shfl_xor_sync(0xffffffffu, u, o);
+  if (i < L1 && seg == 0) {
     if (per_head) {
       if (gate_b != nullptr) u += gate_b[h * L1 + i];
       const float sgm = 1.f / (1.f + expf(-u));

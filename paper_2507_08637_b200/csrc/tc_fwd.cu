@@ -1,7 +1,8 @@
 // bf16 tensor-core (tcgen05 + TMEM + TMA) forward kernels of the WERSA attention path, sm_100a.
-// Each kernel reads its raw bf16 operands once with TMA, applies the multi-level Haar filter
-// (Sec. 3.1 steps 3, 5, 6; Algorithm 2) to 256-token blocks in shared memory, and feeds the
-// filtered tiles straight to the tensor cores: the filtered tensors never reach global memory.
+// Each kernel reads its raw bf16 operands once with TMA (rings of 128-token tiles), applies the
+// multi-level Haar filter (Sec. 3.1 steps 3, 5, 6; Algorithm 2) in shared memory to 256-token blocks
+// (two ring tiles, not necessarily adjacent), and feeds the filtered tiles straight to the tensor
+// cores: the filtered tensors never reach global memory.  A ring slot is released tile by tile.
 //
 // Key side  (Eq. 7, key summary):  S' = ReLU(K_F W)^T V,  z' = ReLU(K_F W)^T 1  per sequence chunk.
 //   MMA1: D1[128 features x 128 tokens] = W^T (smem, K-major) * K_F^T (smem, K-major)   -> TMEM fp32
@@ -31,9 +32,9 @@ namespace {
 constexpr int kTile = 128;                        // tokens per MMA tile
 constexpr int kBlk = 256;                         // tokens per Haar block = one pipeline stage
 constexpr uint32_t kTileBytes = kTile * kD * 2;   // 128 x 64 bf16
-constexpr uint32_t kBlkBytes = kBlk * kD * 2;     // 256 x 64 bf16
-constexpr int kNX = 3;                            // ring of K (or Q) blocks
-constexpr int kNV = 2;                            // ring of V blocks
+constexpr int kNXK = 6, kNV = 5;                  // key side: ring of K tiles, ring of V tiles
+constexpr int kNXQ = 7;                           // query side: ring of Q tiles
+constexpr int kNF = 4;                            // "block filtered" barriers (block b uses b % 4)
 constexpr int kND1 = 3;                           // D1 accumulators in TMEM (columns 0, 128, 256)
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kAccCol = 384;                 // S' halves (key side) / N' of two tiles (query side)
@@ -51,13 +52,13 @@ constexpr int kRegsCtl = 40, kRegsAux = 120, kRegsReluQ = 64, kRegsEpi = 64;
 enum { kErrProducer = 11, kErrMma = 12, kErrRelu = 13, kErrEpilogue = 14, kErrHaar = 15 };
 
 struct alignas(8) KsideBars {
-  uint64_t x_full[kNX], xf_ready[kNX], x_empty[kNX], v_full[kNV], v_empty[kNV];
+  uint64_t x_full[kNXK], x_empty[kNXK], xf_ready[kNF], v_full[kNV], v_empty[kNV];
   uint64_t d1_full[6], phi_ready[kND1], acc_done;
   uint32_t tmem_base;
   int abort_flag;
 };
 struct alignas(8) QsideBars {
-  uint64_t x_full[kNX], xf_ready[kNX], x_empty[kNX];
+  uint64_t x_full[kNXQ], x_empty[kNXQ], xf_ready[kNF];
   uint64_t d1_full[6], phi_ready[kND1], d2_full[2], d2_free[2], den_ready[2];
   uint32_t tmem_base;
   int abort_flag;
@@ -66,8 +67,8 @@ struct alignas(8) QsideBars {
 template <int NH> struct KsideSmem {
   static constexpr uint32_t wt = 0;
   static constexpr uint32_t x = wt + NH * kTileBytes;
-  static constexpr uint32_t v = x + kNX * kBlkBytes;
-  static constexpr uint32_t xch = v + kNV * kBlkBytes;           // 2 x 8 x 64 floats
+  static constexpr uint32_t v = x + kNXK * kTileBytes;
+  static constexpr uint32_t xch = v + kNV * kTileBytes;           // 2 x 8 x 64 floats
   static constexpr uint32_t hcoef = xch + 4096;                  // kHaarCoefPairs pairs
   static constexpr uint32_t zx = hcoef + 1024;                   // 128 floats
   static constexpr uint32_t bars = zx + 512;
@@ -77,7 +78,7 @@ template <int NH> struct QsideSmem {
   static constexpr uint32_t wt = 0;
   static constexpr uint32_t simg = wt + NH * kTileBytes;
   static constexpr uint32_t x = simg + NH * kTileBytes;
-  static constexpr uint32_t ost = x + kNX * kBlkBytes;           // 2 output staging tiles
+  static constexpr uint32_t ost = x + kNXQ * kTileBytes;           // 2 output staging tiles
   static constexpr uint32_t xch = ost + 2 * kTileBytes;          // 2 x 8 x 64 floats
   static constexpr uint32_t hcoef = xch + 4096;                  // kHaarCoefPairs pairs
   static constexpr uint32_t zs = hcoef + 1024;                   // NH*128 floats
@@ -258,6 +259,7 @@ __device__ __forceinline__ float relu_dot_unit16(uint32_t taddr, const float* __
 //   hcoef[8 + 8 hw + w] = weight of warp w's 32-row sum in warp hw's levels 6-8 term
 //                       = k_8 + [same 128-row group] k_7 + [same 64-row group] k_6.
 constexpr int kHaarCoefPairs = 8 + 64;
+static_assert(kHaarCoefPairs * 8 <= 1024, "coefficient table must fit its shared-memory slot");
 
 __device__ __forceinline__ void haar_coef_init(f32x2* hcoef, const float* __restrict__ f, int L, int ht) {
   float k[kMaxLevels + 1];
@@ -281,7 +283,7 @@ __device__ __forceinline__ void haar_coef_init(f32x2* hcoef, const float* __rest
   }
 }
 
-// 256 threads (ht = 0..255) filter the block in place.  Thread (c = ht & 7, rg = ht >> 3) owns rows
+// 256 threads (ht = 0..255) filter the block (two 128-row tiles) in place.  Thread (c = ht & 7, rg = ht >> 3) owns rows
 // 8 rg .. 8 rg + 7 of 16-byte chunk c: levels 1-3 in registers, levels 4-5 through warp shuffles
 // (a warp covers 32 consecutive rows), levels 6-8 through the 32-row sums the eight warps leave in
 // `xch` (8 x 64 floats, double-buffered by the caller) around one named barrier of the 256 threads.
@@ -289,10 +291,10 @@ __device__ __forceinline__ void haar_coef_init(f32x2* hcoef, const float* __rest
 // barrier balanced; with ok = false no memory is touched.  Rows >= valid_rows lie past the end of the
 // sequence: they arrive as zeros (the zero padding of Algorithm 2) and leave as zeros (the trim
 // before the feature map).
-__device__ __forceinline__ void haar_block_inplace(uint8_t* slot, const f32x2* hcoef, bool cross, float* xch, int ht,
-                                                   int valid_rows, bool ok) {
+__device__ __forceinline__ void haar_block_inplace(uint8_t* tile0, uint8_t* tile1, const f32x2* hcoef, bool cross,
+                                                   float* xch, int ht, int valid_rows, bool ok) {
   const int c = ht & 7, rg = ht >> 3, lane = ht & 31, hw = ht >> 5;
-  uint8_t* base = slot + rg * 1024;
+  uint8_t* base = (rg < 16 ? tile0 : tile1) + (rg & 15) * 1024;   // rows 0-127 / 128-255 of the block
   f32x2 x[8][4];   // 8 rows x 4 column pairs
   f32x2 hi[4], s5[4];
   if (ok) {
@@ -366,17 +368,21 @@ __device__ __forceinline__ void haar_block_inplace(uint8_t* slot, const f32x2* h
   }
 }
 
-// One Haar step of the aux role: wait for raw block b, filter it in place, hand it to the MMA issuer.
-template <typename Bars>
+// One Haar step: wait for the two raw tiles of block b, filter them in place, hand the block to the
+// MMA issuer.  NX = number of tile slots in the ring.
+template <int NX, typename Bars>
 __device__ __forceinline__ bool haar_step(uint8_t* xring, Bars* bars, float* xch, const f32x2* hcoef, bool cross,
                                           int b, int rows_left, int ht, bool ok, volatile int* abort_flag,
                                           int* status) {
-  const int s = b % kNX;
-  if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[s], (b / kNX) & 1, abort_flag, status, kErrHaar));
-  haar_block_inplace(xring + s * kBlkBytes, hcoef, cross, xch + (b & 1) * 8 * kD, ht, rows_left - b * kBlk, ok);
+  const int t0 = 2 * b, t1 = 2 * b + 1;
+  const int s0 = t0 % NX, s1 = t1 % NX;
+  if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[s0], (t0 / NX) & 1, abort_flag, status, kErrHaar));
+  if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[s1], (t1 / NX) & 1, abort_flag, status, kErrHaar));
+  haar_block_inplace(xring + s0 * kTileBytes, xring + s1 * kTileBytes, hcoef, cross, xch + (b & 1) * 8 * kD, ht,
+                     rows_left - b * kBlk, ok);
   if (ok) {
     fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
-    mbar_arrive(&bars->xf_ready[s]);
+    mbar_arrive(&bars->xf_ready[b & (kNF - 1)]);
   }
   return ok;
 }
@@ -401,11 +407,11 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
   constexpr int m = NH * 128;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kNX; ++s) {
+    for (int s = 0; s < kNXK; ++s) {
       mbar_init(&bars->x_full[s], 1);
-      mbar_init(&bars->xf_ready[s], 256);
       mbar_init(&bars->x_empty[s], 1);
     }
+    for (int s = 0; s < kNF; ++s) mbar_init(&bars->xf_ready[s], 256);
     for (int s = 0; s < kNV; ++s) {
       mbar_init(&bars->v_full[s], 1);
       mbar_init(&bars->v_empty[s], 1);
@@ -432,17 +438,17 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
     reg_dec<kRegsCtl>();
     if ((warp == kWarpTma || warp == kWarpTmaV) && lane == 0) {
       const bool is_v = warp == kWarpTmaV;
-      const int depth = is_v ? kNV : kNX;
+      const int depth = is_v ? kNV : kNXK;
       uint64_t* full = is_v ? bars->v_full : bars->x_full;
       uint64_t* empty = is_v ? bars->v_empty : bars->x_empty;
       uint8_t* ring = smem + (is_v ? SL::v : SL::x);
       const CUtensorMap* map = is_v ? &map_v : &map_k;
       int issued = 0;
-      for (int b = 0; b < nblk; ++b) {
+      for (int b = 0; b < 2 * nblk; ++b) {   // b counts 128-token tiles here
         const int s = b % depth;
         if (!mbar_wait(&empty[s], ((b / depth) & 1) ^ 1, abort_flag, status, kErrProducer)) break;
-        mbar_arrive_expect_tx(&full[s], kBlkBytes);
-        tma_load_3d(ring + s * kBlkBytes, map, 0, (blk0 + b) * kBlk, slab, &full[s]);
+        mbar_arrive_expect_tx(&full[s], kTileBytes);
+        tma_load_3d(ring + s * kTileBytes, map, 0, blk0 * kBlk + b * kTile, slab, &full[s]);
         issued = b + 1;
       }
       if (*abort_flag != 0) {   // let copies in flight land before the CTA's shared memory goes away
@@ -453,32 +459,36 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       // position inside its block is resolved at compile time; ring slots, D1 buffers and barrier
       // phases are running counters, and descriptors only add to their start-address word.
       constexpr int UPB = 2 * NH;                       // units per 256-token block
-      constexpr uint32_t kTileStep = kTileBytes >> 4, kBlkStep = kBlkBytes >> 4;
+      constexpr uint32_t kTileStep = kTileBytes >> 4;
       const uint32_t hi = smem_desc_hi(1024);
       const uint32_t wt_lo = smem_desc_lo(smem_u32(smem + SL::wt), 16);
       const uint32_t x_lo = smem_desc_lo(smem_u32(smem + SL::x), 16);
       const uint32_t v_lo = smem_desc_lo(smem_u32(smem + SL::v), 1024);
-      uint32_t xs = 0, xpar = 0, vs = 0, vpar = 0;     // ring slot and phase of the block MMA1 / MMA2 is in
+      uint32_t xs = 0, vs = 0, vpar = 0;               // ring slot of the tile MMA1 / MMA2 is in, V phase
+      uint32_t fs = 0, fpar = 0;                        // "block filtered" barrier and phase
       uint32_t c3 = 0, c6 = 0;                          // MMA1: D1 buffer, d1_full barrier
       uint32_t p3 = 0, ppar = 0;                        // MMA2: D1 buffer (= phi_ready barrier) and phase
       bool ok = true;
       for (int b = 0; b <= nblk && ok; ++b) {
         if (b < nblk) {
-          ok = mbar_wait(&bars->xf_ready[xs], xpar, abort_flag, status, kErrMma);
+          ok = mbar_wait(&bars->xf_ready[fs], fpar, abort_flag, status, kErrMma);
           if (!ok) break;
           tc_fence_after_sync();
         }
 #pragma unroll
         for (int j = 0; j < UPB; ++j) {
           if (b < nblk) {
-            const int tt = j / NH, h = j % NH;
-            const uint32_t a_lo = wt_lo + h * kTileStep, b_lo = x_lo + xs * kBlkStep + tt * kTileStep;
+            const int h = j % NH;
+            const uint32_t a_lo = wt_lo + h * kTileStep, b_lo = x_lo + xs * kTileStep;
             const uint32_t d1 = tmem + c3 * 128;
 #pragma unroll
             for (int k = 0; k < 4; ++k)
               mma_ss(d1, smem_desc_join(a_lo + 2 * k, hi), smem_desc_join(b_lo + 2 * k, hi), kIdesc1, k > 0);
             mma_commit(&bars->d1_full[c6]);
-            if (j == UPB - 1) mma_commit(&bars->x_empty[xs]);
+            if (h == NH - 1) {   // last MMA1 that reads this tile
+              mma_commit(&bars->x_empty[xs]);
+              xs = xs == kNXK - 1 ? 0 : xs + 1;
+            }
             c3 = c3 == kND1 - 1 ? 0 : c3 + 1;
             c6 = c6 == 5 ? 0 : c6 + 1;
           }
@@ -486,7 +496,7 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
           const int bb = j >= 2 ? b : b - 1;
           if (bb >= 0 && bb < nblk) {
             const int tt = lj / NH, h = lj % NH;
-            if (lj == 0) {
+            if (h == 0) {
               ok = mbar_wait(&bars->v_full[vs], vpar, abort_flag, status, kErrMma);
               if (!ok) break;
             }
@@ -494,11 +504,11 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
             if (!ok) break;
             tc_fence_after_sync();
             const uint32_t acc = tmem + kAccCol + h * 64, a_tm = tmem + p3 * 128;
-            const uint32_t b_lo = v_lo + vs * kBlkStep + tt * kTileStep;
+            const uint32_t b_lo = v_lo + vs * kTileStep;
 #pragma unroll
             for (int k = 0; k < 8; ++k)
               mma_ts(acc, a_tm + k * 8, smem_desc_join(b_lo + 128 * k, hi), kIdesc2, (bb > 0 || tt > 0 || k > 0) ? 1u : 0u);
-            if (lj == UPB - 1) {
+            if (h == NH - 1) {
               mma_commit(&bars->v_empty[vs]);
               vs = vs == kNV - 1 ? 0 : vs + 1;
               vpar ^= (vs == 0);
@@ -507,8 +517,8 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
             ppar ^= (p3 == 0);
           }
         }
-        xs = xs == kNX - 1 ? 0 : xs + 1;
-        xpar ^= (xs == 0);
+        fs = (fs + 1) & (kNF - 1);
+        fpar ^= (fs == 0);
       }
       mma_commit(&bars->acc_done);
     }
@@ -558,7 +568,7 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
     named_bar_sync(3, 256);
     bool ok = true;
     for (int b = 0; b < nblk; ++b)
-      ok = haar_step(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
+      ok = haar_step<kNXK>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
                      ht, ok, abort_flag, status);
   }
   tc_fence_before_sync();
@@ -593,11 +603,11 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
   constexpr int m = NH * 128;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kNX; ++s) {
+    for (int s = 0; s < kNXQ; ++s) {
       mbar_init(&bars->x_full[s], 1);
-      mbar_init(&bars->xf_ready[s], 256);
       mbar_init(&bars->x_empty[s], 1);
     }
+    for (int s = 0; s < kNF; ++s) mbar_init(&bars->xf_ready[s], 256);
     for (int b = 0; b < 6; ++b) mbar_init(&bars->d1_full[b], 1);
     for (int b = 0; b < kND1; ++b) mbar_init(&bars->phi_ready[b], 128);
     for (int b = 0; b < 2; ++b) {
@@ -626,45 +636,48 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     reg_dec<kRegsCtl>();
     if (warp == kWarpTma && lane == 0) {
       int issued = 0;
-      for (int b = 0; b < nblk; ++b) {
-        const int s = b % kNX;
-        if (!mbar_wait(&bars->x_empty[s], ((b / kNX) & 1) ^ 1, abort_flag, status, kErrProducer)) break;
-        mbar_arrive_expect_tx(&bars->x_full[s], kBlkBytes);
-        tma_load_3d(smem + SL::x + s * kBlkBytes, &map_q, 0, (blk0 + b) * kBlk, slab, &bars->x_full[s]);
+      for (int b = 0; b < ntiles; ++b) {   // b counts 128-token tiles here
+        const int s = b % kNXQ;
+        if (!mbar_wait(&bars->x_empty[s], ((b / kNXQ) & 1) ^ 1, abort_flag, status, kErrProducer)) break;
+        mbar_arrive_expect_tx(&bars->x_full[s], kTileBytes);
+        tma_load_3d(smem + SL::x + s * kTileBytes, &map_q, 0, blk0 * kBlk + b * kTile, slab, &bars->x_full[s]);
         issued = b + 1;
       }
       if (*abort_flag != 0) {
-        for (int b = max(0, issued - kNX); b < issued; ++b) mbar_wait_drain(&bars->x_full[b % kNX], (b / kNX) & 1);
+        for (int b = max(0, issued - kNXQ); b < issued; ++b) mbar_wait_drain(&bars->x_full[b % kNXQ], (b / kNXQ) & 1);
       }
     } else if (warp == kWarpMma && lane == 0) {
       // Same issue scheme as the key side (MMA1 of unit u, then MMA2 of unit u - 2).
       constexpr int UPB = 2 * NH;
-      constexpr uint32_t kTileStep = kTileBytes >> 4, kBlkStep = kBlkBytes >> 4;
+      constexpr uint32_t kTileStep = kTileBytes >> 4;
       const uint32_t hi = smem_desc_hi(1024);
       const uint32_t wt_lo = smem_desc_lo(smem_u32(smem + SL::wt), 16);
       const uint32_t x_lo = smem_desc_lo(smem_u32(smem + SL::x), 16);
       const uint32_t s_lo = smem_desc_lo(smem_u32(smem + SL::simg), 1024);
-      uint32_t xs = 0, xpar = 0;
+      uint32_t xs = 0, fs = 0, fpar = 0;
       uint32_t c3 = 0, c6 = 0;
       uint32_t p3 = 0, ppar = 0;
       bool ok = true;
       for (int b = 0; b <= nblk && ok; ++b) {
         if (b < nblk) {
-          ok = mbar_wait(&bars->xf_ready[xs], xpar, abort_flag, status, kErrMma);
+          ok = mbar_wait(&bars->xf_ready[fs], fpar, abort_flag, status, kErrMma);
           if (!ok) break;
           tc_fence_after_sync();
         }
 #pragma unroll
         for (int j = 0; j < UPB; ++j) {
           if (b < nblk) {
-            const int tt = j / NH, h = j % NH;
-            const uint32_t a_lo = x_lo + xs * kBlkStep + tt * kTileStep, b_lo = wt_lo + h * kTileStep;
+            const int h = j % NH;
+            const uint32_t a_lo = x_lo + xs * kTileStep, b_lo = wt_lo + h * kTileStep;
             const uint32_t d1 = tmem + c3 * 128;
 #pragma unroll
             for (int k = 0; k < 4; ++k)
               mma_ss(d1, smem_desc_join(a_lo + 2 * k, hi), smem_desc_join(b_lo + 2 * k, hi), kIdesc1, k > 0);
             mma_commit(&bars->d1_full[c6]);
-            if (j == UPB - 1) mma_commit(&bars->x_empty[xs]);
+            if (h == NH - 1) {   // last MMA1 that reads this tile
+              mma_commit(&bars->x_empty[xs]);
+              xs = xs == kNXQ - 1 ? 0 : xs + 1;
+            }
             c3 = c3 == kND1 - 1 ? 0 : c3 + 1;
             c6 = c6 == 5 ? 0 : c6 + 1;
           }
@@ -689,8 +702,8 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
             ppar ^= (p3 == 0);
           }
         }
-        xs = xs == kNX - 1 ? 0 : xs + 1;
-        xpar ^= (xs == 0);
+        fs = (fs + 1) & (kNF - 1);
+        fpar ^= (fs == 0);
       }
     }
   } else if (warp >= kReluWarp0 && warp < kAuxWarp0) {
@@ -723,7 +736,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     named_bar_sync(3, 256);
     bool ok = true;
     for (int b = 0; b < nblk; ++b)
-      ok = haar_step(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
+      ok = haar_step<kNXQ>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
                      ht, ok, abort_flag, status);
   } else {
     reg_dec<kRegsEpi>();
@@ -829,8 +842,8 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
                             int* launches) {
   CUtensorMap map_k, map_v;
   cudaError_t err;
-  if ((err = make_tile_map(K, p.slabs, p.cfg.seq_len, kBlk, &map_k)) != cudaSuccess) return err;
-  if ((err = make_tile_map(V, p.slabs, p.cfg.seq_len, kBlk, &map_v)) != cudaSuccess) return err;
+  if ((err = make_tile_map(K, p.slabs, p.cfg.seq_len, kTile, &map_k)) != cudaSuccess) return err;
+  if ((err = make_tile_map(V, p.slabs, p.cfg.seq_len, kTile, &map_v)) != cudaSuccess) return err;
   dim3 grid(p.tchunks, p.slabs);
   if (p.cfg.features == 256) {
     auto k = k_tc_kside<2>;
@@ -853,7 +866,7 @@ cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const flo
                             int* launches) {
   CUtensorMap map_q, map_o;
   cudaError_t err;
-  if ((err = make_tile_map(Q, p.slabs, p.cfg.seq_len, kBlk, &map_q)) != cudaSuccess) return err;
+  if ((err = make_tile_map(Q, p.slabs, p.cfg.seq_len, kTile, &map_q)) != cudaSuccess) return err;
   if ((err = make_tile_map(O, p.slabs, p.cfg.seq_len, kTile, &map_o)) != cudaSuccess) return err;
   dim3 grid(p.tchunks, p.slabs);
   if (p.cfg.features == 256) {
