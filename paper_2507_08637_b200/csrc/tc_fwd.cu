@@ -109,6 +109,13 @@ __device__ __forceinline__ void reg_fence32(uint32_t (&r)[32]) {
                : "memory");
 }
 
+// One arrival per warp: every lane has finished (and fenced) its part, the warp converges, lane 0
+// arrives.  The barriers that collect these arrivals count warps, not threads.
+__device__ __forceinline__ void warp_arrive(uint64_t* bar) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+}
+
 // Register budget per role (all warps of a warpgroup execute the same one).
 template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
@@ -382,7 +389,7 @@ __device__ __forceinline__ bool haar_step(uint8_t* xring, Bars* bars, float* xch
                      rows_left - b * kBlk, ok);
   if (ok) {
     fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
-    mbar_arrive(&bars->xf_ready[b & (kNF - 1)]);
+    warp_arrive(&bars->xf_ready[b & (kNF - 1)]);
   }
   return ok;
 }
@@ -411,13 +418,13 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       mbar_init(&bars->x_full[s], 1);
       mbar_init(&bars->x_empty[s], 1);
     }
-    for (int s = 0; s < kNF; ++s) mbar_init(&bars->xf_ready[s], 256);
+    for (int s = 0; s < kNF; ++s) mbar_init(&bars->xf_ready[s], 8);
     for (int s = 0; s < kNV; ++s) {
       mbar_init(&bars->v_full[s], 1);
       mbar_init(&bars->v_empty[s], 1);
     }
     for (int b = 0; b < 6; ++b) mbar_init(&bars->d1_full[b], 1);
-    for (int b = 0; b < kND1; ++b) mbar_init(&bars->phi_ready[b], 128);
+    for (int b = 0; b < kND1; ++b) mbar_init(&bars->phi_ready[b], 4);
     mbar_init(&bars->acc_done, 1);
     bars->abort_flag = 0;
     fence_mbar_init();
@@ -534,7 +541,7 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
         tc_fence_after_sync();
         zacc += relu_unit<false>(tmem + (lane_base << 16) + (u % kND1) * 128, nullptr);
         tc_fence_before_sync();
-        mbar_arrive(&bars->phi_ready[u % kND1]);
+        warp_arrive(&bars->phi_ready[u % kND1]);
       }
     }
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->acc_done, 0, abort_flag, status, kErrRelu));
@@ -607,13 +614,13 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       mbar_init(&bars->x_full[s], 1);
       mbar_init(&bars->x_empty[s], 1);
     }
-    for (int s = 0; s < kNF; ++s) mbar_init(&bars->xf_ready[s], 256);
+    for (int s = 0; s < kNF; ++s) mbar_init(&bars->xf_ready[s], 8);
     for (int b = 0; b < 6; ++b) mbar_init(&bars->d1_full[b], 1);
-    for (int b = 0; b < kND1; ++b) mbar_init(&bars->phi_ready[b], 128);
+    for (int b = 0; b < kND1; ++b) mbar_init(&bars->phi_ready[b], 4);
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bars->d2_full[b], 1);
-      mbar_init(&bars->d2_free[b], 128);
-      mbar_init(&bars->den_ready[b], 128 * NH);
+      mbar_init(&bars->d2_free[b], 4);
+      mbar_init(&bars->den_ready[b], 4 * NH);
     }
     bars->abort_flag = 0;
     fence_mbar_init();
@@ -719,14 +726,14 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       tc_fence_after_sync();
       const float dot = relu_dot_unit16(tmem + (lane_base << 16) + (u % kND1) * 128, zs + h * 128);
       tc_fence_before_sync();
-      mbar_arrive(&bars->phi_ready[u % kND1]);
+      warp_arrive(&bars->phi_ready[u % kND1]);
       // the denominator slots of this tile parity must have been read by the epilogue of tile t-2
       if (t >= 2)
         ok = __all_sync(0xffffffffu,
                         mbar_wait(&bars->d2_free[t & 1], ((t >> 1) - 1) & 1, abort_flag, status, kErrRelu));
       if (!ok) continue;
       den[((t & 1) * NH + h) * 128 + row] = dot;
-      mbar_arrive(&bars->den_ready[t & 1]);
+      warp_arrive(&bars->den_ready[t & 1]);
     }
   } else if (warp < kEpiWarp0) {
     reg_inc<kRegsAux>();
@@ -770,7 +777,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
           reg_fence32(r);
           if (half == 1) {   // N' and the denominators of this tile parity are free again
             tc_fence_before_sync();
-            mbar_arrive(&bars->d2_free[p]);
+            warp_arrive(&bars->d2_free[p]);
           }
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
