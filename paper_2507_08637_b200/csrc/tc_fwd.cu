@@ -12,13 +12,14 @@
 //   MMA1: D1[128 tokens x 128 features] = Q_F (smem, K-major) * W (as W^T, K-major)
 //   ReLU warps as above, plus the row dot product with z' (denominator)
 //   MMA2: N'[128 tokens x 64] (+)= Phi (TMEM operand, K = features) * S' (smem bf16, N-major)
-//   epilogue warps: TMEM -> registers -> * 1/(D' + eps') -> bf16 -> swizzled smem -> TMA store
+//   epilogue (ReLU warpgroup t & 1 for tile t): TMEM -> registers -> * 1/(D' + eps') -> bf16 ->
+//   swizzled smem -> TMA store
 //
 // Work unit of the MMA pipeline: one 128-token tile times one 128-feature half ("unit").  Three D1
 // accumulators rotate, so the ReLU pass of a unit overlaps four MMAs of its neighbours.
 // Warp roles: warp 0 TMA producer (K or Q), warp 1 MMA issuer (one thread), warp 2 TMA producer
-// (V, key side), warps 4-11 two ReLU warpgroups that alternate over the units, warps 12-19 Haar
-// filter, warps 20-23 (query side) epilogue.  All operand tiles use the 128-byte swizzle.
+// (V, key side), warps 4-11 two ReLU warpgroups that alternate over the units (query side: they also
+// write out the finished tiles), warps 12-19 Haar filter.  All operand tiles use the 128-byte swizzle.
 // Every wait on an mbarrier is bounded; a role whose wait expires keeps its control flow (so that
 // group barriers stay balanced) but skips all further work, and the host sees the status word.
 #include "common.cuh"
@@ -42,13 +43,14 @@ constexpr uint32_t kIdesc1 = make_idesc_bf16(128, 128, false, false);  // both o
 constexpr uint32_t kIdesc2 = make_idesc_bf16(128, 64, false, true);    // B = V or S', N-major
 
 constexpr int kWarpTma = 0, kWarpMma = 1, kWarpTmaV = 2;
-constexpr int kReluWarp0 = 4, kAuxWarp0 = 12, kEpiWarp0 = 20;   // 8 ReLU warps, 8 Haar warps, 4 epilogue warps
-constexpr int kThreadsK = 32 * kEpiWarp0;           // key side: 640 threads, 96 registers each at launch
-constexpr int kThreadsQ = 32 * (kEpiWarp0 + 4);     // query side: 768 threads, 80 registers each at launch
+constexpr int kReluWarp0 = 4, kAuxWarp0 = 12;       // 8 ReLU warps, 8 Haar warps
+constexpr int kThreads = 32 * (kAuxWarp0 + 8);      // 640 threads, 96 registers each at launch
 // Registers per thread after the roles have traded: the Haar step holds a 256 x 64 block in registers
-// and gets what the producer / MMA warpgroup (and, query side, the ReLU and epilogue warps) give up.
-constexpr int kRegsCtl = 40, kRegsAux = 120, kRegsReluQ = 64, kRegsEpi = 64;
+// and gets what the producer / MMA warpgroup gives up.
+constexpr int kRegsCtl = 40, kRegsAux = 120;
 
+// Named barriers (id 0 is __syncthreads).
+enum { kBarZsum = 1, kBarCoef = 3, kBarHaar = 4, kBarOut0 = 5 /* and 6: one per ReLU warpgroup */ };
 enum { kErrProducer = 11, kErrMma = 12, kErrRelu = 13, kErrEpilogue = 14, kErrHaar = 15 };
 
 struct alignas(8) KsideBars {
@@ -210,53 +212,6 @@ __device__ __forceinline__ float relu_unit(uint32_t taddr, const float* __restri
   return 0.5f * ((s0 + s1) + (s2 + s3));
 }
 
-// The same pass in 16-column steps (fewer live registers; the query side's ReLU warps run on 64).
-__device__ __forceinline__ void reg_fence16(uint32_t (&r)[16]) {
-  asm volatile(""
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
-                 "+r"(r[15])
-               :
-               : "memory");
-}
-__device__ __forceinline__ void relu_dot_chunk16(const uint32_t (&r)[16], uint32_t (&p)[8], const float* __restrict__ zrow,
-                                                 f32x2 (&acc)[2]) {
-#pragma unroll
-  for (int j4 = 0; j4 < 4; ++j4) {
-    const float a0 = __uint_as_float(r[4 * j4]), a1 = __uint_as_float(r[4 * j4 + 1]);
-    const float a2 = __uint_as_float(r[4 * j4 + 2]), a3 = __uint_as_float(r[4 * j4 + 3]);
-    p[2 * j4] = relu_pack_bf16x2(a0, a1);
-    p[2 * j4 + 1] = relu_pack_bf16x2(a2, a3);
-    const float4 zv = *reinterpret_cast<const float4*>(zrow + 4 * j4);
-    acc[0] = fma2(pk2(a0 + fabsf(a0), a1 + fabsf(a1)), pk2(zv.x, zv.y), acc[0]);
-    acc[1] = fma2(pk2(a2 + fabsf(a2), a3 + fabsf(a3)), pk2(zv.z, zv.w), acc[1]);
-  }
-}
-// 128 columns at taddr, dot product of the ReLU values with zrow[0..127] (denominator of Eq. 7).
-__device__ __forceinline__ float relu_dot_unit16(uint32_t taddr, const float* __restrict__ zrow) {
-  f32x2 acc[2] = {0ull, 0ull};
-  uint32_t a[16], b[16], p[8];
-  tmem_ld16(taddr, a);
-#pragma unroll
-  for (int c = 0; c < 8; c += 2) {
-    tmem_ld_wait();
-    reg_fence16(a);
-    tmem_ld16(taddr + 16 * (c + 1), b);
-    relu_dot_chunk16(a, p, zrow + 16 * c, acc);
-    tmem_st8(taddr + 8 * c, p);
-    tmem_ld_wait();
-    reg_fence16(b);
-    if (c + 2 < 8) tmem_ld16(taddr + 16 * (c + 2), a);
-    relu_dot_chunk16(b, p, zrow + 16 * (c + 1), acc);
-    tmem_st8(taddr + 8 * (c + 1), p);
-  }
-  tmem_st_wait();
-  float s0, s1, s2, s3;
-  upk2(acc[0], s0, s1);
-  upk2(acc[1], s2, s3);
-  return 0.5f * ((s0 + s1) + (s2 + s3));
-}
-
 // ---- Haar filter of one 256-token block in shared memory ------------------------------------------
 // T_f x = f_0 x + sum_{i=1..L} (f_i - f_{i-1}) * blockmean_{2^i}(x): the detail projector of level l
 // is blockmean_{2^(l-1)} - blockmean_{2^l} and the approximation projector of level L is
@@ -330,7 +285,7 @@ __device__ __forceinline__ void haar_block_inplace(uint8_t* tile0, uint8_t* tile
       dst[0] = make_ulonglong2(s5[0], s5[1]);
       dst[1] = make_ulonglong2(s5[2], s5[3]);
     }
-    named_bar_sync(4, 256);
+    named_bar_sync(kBarHaar, 256);
     if (ok) {
       // lane (c, q = lane >> 3) combines the eight warps' sums of column pair q of chunk c, then the
       // four lanes that share a chunk swap their pairs
@@ -397,7 +352,7 @@ __device__ __forceinline__ bool haar_step(uint8_t* xring, Bars* bars, float* xch
 // ---- key side -----------------------------------------------------------------------------------
 // grid (chunks, slabs), block 640.  TMEM: D1[3] at columns 0 / 128 / 256, S' half h at 384 + 64 h.
 template <int NH>
-__global__ void __launch_bounds__(kThreadsK, 1)
+__global__ void __launch_bounds__(kThreads, 1)
 k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
            const __nv_bfloat16* __restrict__ Wt, const float* __restrict__ f, float* __restrict__ spart,
            float* __restrict__ zpart, int n, int L, int chunk_blocks, int* __restrict__ status) {
@@ -549,7 +504,7 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
     const size_t pidx = (size_t)slab * gridDim.x + chunk;
     if (NH == 1) {   // both warpgroups saw the same 128 features on alternating tiles
       if (g == 1) zx[row] = zacc;
-      named_bar_sync(1, 256);
+      named_bar_sync(kBarZsum, 256);
       if (g == 0) zacc += zx[row];
     }
     if (ok && (NH == 2 || g == 0)) {
@@ -572,7 +527,7 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
     const int ht = threadIdx.x - 32 * kAuxWarp0;
     f32x2* hcoef = reinterpret_cast<f32x2*>(smem + SL::hcoef);
     haar_coef_init(hcoef, f + (size_t)slab * (L + 1), L, ht);
-    named_bar_sync(3, 256);
+    named_bar_sync(kBarCoef, 256);
     bool ok = true;
     for (int b = 0; b < nblk; ++b)
       ok = haar_step<kNXK>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
@@ -587,10 +542,65 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
 }
 
 // ---- query side ---------------------------------------------------------------------------------
-// grid (chunks, slabs), block 768.  TMEM: D1[3] at columns 0 / 128 / 256, N' of tile parity p at
+// Epilogue of tile t by the ReLU warpgroup g = t & 1 (128 threads, thread = token row): waits for N'
+// and the denominators, scales, rounds to bf16 into the warpgroup's own staging tile and stores it
+// with TMA.  The group barrier is executed whether or not `ok` holds.
+template <int NH, typename SL>
+__device__ __forceinline__ bool qside_write_tile(QsideBars* bars, uint8_t* smem, const float* den,
+                                                 const CUtensorMap* map_o, uint32_t tmem, float epsp, int t, int row0,
+                                                 int n, int slab, int g, int gt, bool ok, volatile int* abort_flag,
+                                                 int* status) {
+  const uint32_t lane_base = 32u * ((gt >> 5) & 3);
+  const int row = gt;                               // token within the tile = TMEM lane
+  const int p = t & 1;                              // == g
+  if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d2_full[p], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
+  if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->den_ready[p], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
+  // the staging tile was last used by tile t-2: its TMA store must have finished reading
+  if (gt == 0) bulk_wait_group_read0();
+  named_bar_sync(kBarOut0 + g, 128);
+  uint8_t* ost = smem + SL::ost + p * kTileBytes;
+  if (ok) {
+    tc_fence_after_sync();
+    const uint32_t base = tmem + (lane_base << 16) + kAccCol + p * 64;
+    float dsum = epsp;
+#pragma unroll
+    for (int h = 0; h < NH; ++h) dsum += den[(p * NH + h) * 128 + row];
+    const float inv = 1.f / dsum;
+    const f32x2 inv2 = pk2(inv, inv);
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      uint32_t r[32];
+      tmem_ld32(base + 32 * half, r);
+      tmem_ld_wait();
+      reg_fence32(r);
+      if (half == 1) {   // N' and the denominators of this tile parity are free again
+        tc_fence_before_sync();
+        warp_arrive(&bars->d2_free[p]);
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint4 v;
+        v.x = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c]), __uint_as_float(r[8 * c + 1])), inv2));
+        v.y = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c + 2]), __uint_as_float(r[8 * c + 3])), inv2));
+        v.z = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c + 4]), __uint_as_float(r[8 * c + 5])), inv2));
+        v.w = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c + 6]), __uint_as_float(r[8 * c + 7])), inv2));
+        *reinterpret_cast<uint4*>(ost + swz128(row, 4 * half + c)) = v;
+      }
+    }
+    fence_proxy_async_smem();
+  }
+  named_bar_sync(kBarOut0 + g, 128);
+  if (gt == 0 && ok && row0 < n) {   // rows past n are clipped by the store
+    tma_store_3d(map_o, ost, 0, row0, slab);
+    bulk_commit_group();
+  }
+  return ok;
+}
+
+// grid (chunks, slabs), block 640.  TMEM: D1[3] at columns 0 / 128 / 256, N' of tile parity p at
 // 384 + 64 p.  The partial denominators of a tile travel through shared memory (den).
 template <int NH>
-__global__ void __launch_bounds__(kThreadsQ, 1)
+__global__ void __launch_bounds__(kThreads, 1)
 k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
            const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ Sbf,
            const float* __restrict__ zg, const float* __restrict__ f, const float* __restrict__ beta, float eps,
@@ -714,90 +724,53 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       }
     }
   } else if (warp >= kReluWarp0 && warp < kAuxWarp0) {
-    reg_dec<kRegsReluQ>();
     const int g = (warp - kReluWarp0) >> 2;
+    const int gt = threadIdx.x - 32 * kReluWarp0 - 128 * g;   // 0..127 inside the warpgroup
     const uint32_t lane_base = 32u * (warp & 3);
-    const int row = lane_base + lane;               // token within the tile = TMEM lane
+    const int row = lane_base + lane;               // token within the tile = TMEM lane (== gt)
+    const float bw = fmaxf(beta[0], bw_floor);
+    const float epsp = eps * (float)m * bw * bw;
+    int next_out = g;                               // next tile this warpgroup writes out (tiles of parity g)
     bool ok = true;
     for (int u = g; u < units; u += 2) {
       const int t = u / NH, h = u % NH;
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d1_full[u % 6], (u / 6) & 1, abort_flag, status, kErrRelu));
-      if (!ok) continue;
-      tc_fence_after_sync();
-      const float dot = relu_dot_unit16(tmem + (lane_base << 16) + (u % kND1) * 128, zs + h * 128);
-      tc_fence_before_sync();
-      warp_arrive(&bars->phi_ready[u % kND1]);
+      float dot = 0.f;
+      if (ok) {
+        tc_fence_after_sync();
+        dot = relu_unit<true>(tmem + (lane_base << 16) + (u % kND1) * 128, zs + h * 128);
+        tc_fence_before_sync();
+        warp_arrive(&bars->phi_ready[u % kND1]);
+      }
+      // write out this warpgroup's earlier tiles (all their units were handed to the MMA issuer before
+      // this one); this is also what frees the denominator slots waited for below.  Not conditional on
+      // `ok`: the group barriers inside must see all 128 threads.
+      for (; next_out < t; next_out += 2)
+        ok = qside_write_tile<NH, SL>(bars, smem, den, &map_o, tmem, epsp, next_out, blk0 * kBlk + next_out * kTile, n,
+                                      slab, g, gt, ok, abort_flag, status);
       // the denominator slots of this tile parity must have been read by the epilogue of tile t-2
-      if (t >= 2)
+      if (ok && t >= 2)
         ok = __all_sync(0xffffffffu,
                         mbar_wait(&bars->d2_free[t & 1], ((t >> 1) - 1) & 1, abort_flag, status, kErrRelu));
-      if (!ok) continue;
-      den[((t & 1) * NH + h) * 128 + row] = dot;
-      warp_arrive(&bars->den_ready[t & 1]);
+      if (ok) {
+        den[((t & 1) * NH + h) * 128 + row] = dot;
+        warp_arrive(&bars->den_ready[t & 1]);
+      }
     }
-  } else if (warp < kEpiWarp0) {
+    for (; next_out < ntiles; next_out += 2)
+      ok = qside_write_tile<NH, SL>(bars, smem, den, &map_o, tmem, epsp, next_out, blk0 * kBlk + next_out * kTile, n, slab,
+                                    g, gt, ok, abort_flag, status);
+    if (gt == 0) bulk_wait_group0();
+  } else {
     reg_inc<kRegsAux>();
     const int ht = threadIdx.x - 32 * kAuxWarp0;
     f32x2* hcoef = reinterpret_cast<f32x2*>(smem + SL::hcoef);
     haar_coef_init(hcoef, f + (size_t)slab * (L + 1), L, ht);
-    named_bar_sync(3, 256);
+    named_bar_sync(kBarCoef, 256);
     bool ok = true;
     for (int b = 0; b < nblk; ++b)
       ok = haar_step<kNXQ>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
                      ht, ok, abort_flag, status);
-  } else {
-    reg_dec<kRegsEpi>();
-    const uint32_t lane_base = 32u * (warp & 3);
-    const int row = lane_base + lane;               // token within the tile = TMEM lane
-    const int et = threadIdx.x - 32 * kEpiWarp0;    // 0..127 inside the epilogue warpgroup
-    const float bw = fmaxf(beta[0], bw_floor);
-    const float epsp = eps * (float)m * bw * bw;
-    bool ok = true;
-    for (int t = 0; t < ntiles; ++t) {
-      const int p = t & 1;
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d2_full[p], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->den_ready[p], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
-      // staging buffer p was last used by tile t-2: its TMA store must have finished reading
-      if (et == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-      named_bar_sync(2, 128);
-      uint8_t* ost = smem + SL::ost + p * kTileBytes;
-      if (ok) {
-        tc_fence_after_sync();
-        const uint32_t base = tmem + (lane_base << 16) + kAccCol + p * 64;
-        float dsum = epsp;
-#pragma unroll
-        for (int h = 0; h < NH; ++h) dsum += den[(p * NH + h) * 128 + row];
-        const float inv = 1.f / dsum;
-        const f32x2 inv2 = pk2(inv, inv);
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          uint32_t r[32];
-          tmem_ld32(base + 32 * half, r);
-          tmem_ld_wait();
-          reg_fence32(r);
-          if (half == 1) {   // N' and the denominators of this tile parity are free again
-            tc_fence_before_sync();
-            warp_arrive(&bars->d2_free[p]);
-          }
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint4 v;
-            v.x = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c]), __uint_as_float(r[8 * c + 1])), inv2));
-            v.y = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c + 2]), __uint_as_float(r[8 * c + 3])), inv2));
-            v.z = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c + 4]), __uint_as_float(r[8 * c + 5])), inv2));
-            v.w = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c + 6]), __uint_as_float(r[8 * c + 7])), inv2));
-            *reinterpret_cast<uint4*>(ost + swz128(row, 4 * half + c)) = v;
-          }
-        }
-        fence_proxy_async_smem();
-      }
-      named_bar_sync(2, 128);
-      if (et == 0 && ok && blk0 * kBlk + t * kTile < n) {   // rows past n are clipped by the store
-        tma_store_3d(&map_o, ost, 0, blk0 * kBlk + t * kTile, slab);
-        bulk_commit_group();
-      }
-    }
-    if (et == 0) bulk_wait_group0();
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -856,13 +829,13 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
     auto k = k_tc_kside<2>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, KsideSmem<2>::total)) != cudaSuccess)
       return err;
-    k<<<grid, kThreadsK, KsideSmem<2>::total, st>>>(map_k, map_v, w.Wt, w.f, w.spart, w.zpart, p.cfg.seq_len,
+    k<<<grid, kThreads, KsideSmem<2>::total, st>>>(map_k, map_v, w.Wt, w.f, w.spart, w.zpart, p.cfg.seq_len,
                                                          p.cfg.levels, p.tchunk_blocks, w.status);
   } else {
     auto k = k_tc_kside<1>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, KsideSmem<1>::total)) != cudaSuccess)
       return err;
-    k<<<grid, kThreadsK, KsideSmem<1>::total, st>>>(map_k, map_v, w.Wt, w.f, w.spart, w.zpart, p.cfg.seq_len,
+    k<<<grid, kThreads, KsideSmem<1>::total, st>>>(map_k, map_v, w.Wt, w.f, w.spart, w.zpart, p.cfg.seq_len,
                                                          p.cfg.levels, p.tchunk_blocks, w.status);
   }
   *launches += 1;
@@ -880,14 +853,14 @@ cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const flo
     auto k = k_tc_qside<2>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, QsideSmem<2>::total)) != cudaSuccess)
       return err;
-    k<<<grid, kThreadsQ, QsideSmem<2>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
+    k<<<grid, kThreads, QsideSmem<2>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
                                                          p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks,
                                                          w.status);
   } else {
     auto k = k_tc_qside<1>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, QsideSmem<1>::total)) != cudaSuccess)
       return err;
-    k<<<grid, kThreadsQ, QsideSmem<1>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
+    k<<<grid, kThreads, QsideSmem<1>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
                                                          p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks,
                                                          w.status);
   }
