@@ -17,7 +17,8 @@
 //
 // Work unit of the MMA pipeline: one 128-token tile times one 128-feature half ("unit").  Three D1
 // accumulators rotate, so the ReLU pass of a unit overlaps four MMAs of its neighbours.
-// Warp roles: warp 0 TMA producer (K or Q), warp 1 MMA issuer (one thread), warp 2 TMA producer
+// Warp roles: warp 0 TMA producer (K or Q), warps 1 and 3 MMA issuers (one thread each: warp 1 issues
+// every MMA1 and runs up to three units ahead, warp 3 every MMA2), warp 2 TMA producer
 // (V, key side), warps 4-11 two ReLU warpgroups that alternate over the units (query side: they also
 // write out the finished tiles), warps 12-19 Haar filter.  All operand tiles use the 128-byte swizzle.
 // Every wait on an mbarrier is bounded; a role whose wait expires keeps its control flow (so that
@@ -42,7 +43,7 @@ constexpr uint32_t kAccCol = 384;                 // S' halves (key side) / N' o
 constexpr uint32_t kIdesc1 = make_idesc_bf16(128, 128, false, false);  // both operands K-major
 constexpr uint32_t kIdesc2 = make_idesc_bf16(128, 64, false, true);    // B = V or S', N-major
 
-constexpr int kWarpTma = 0, kWarpMma = 1, kWarpTmaV = 2;
+constexpr int kWarpTma = 0, kWarpMma = 1, kWarpTmaV = 2, kWarpMma2 = 3;
 constexpr int kReluWarp0 = 4, kAuxWarp0 = 12;       // 8 ReLU warps, 8 Haar warps
 constexpr int kThreads = 32 * (kAuxWarp0 + 8);      // 640 threads, 96 registers each at launch
 // Registers per thread after the roles have traded: the Haar step holds a 256 x 64 block in registers
@@ -55,13 +56,13 @@ enum { kErrProducer = 11, kErrMma = 12, kErrRelu = 13, kErrEpilogue = 14, kErrHa
 
 struct alignas(8) KsideBars {
   uint64_t x_full[kNXK], x_empty[kNXK], xf_ready[kNF], v_full[kNV], v_empty[kNV];
-  uint64_t d1_full[6], phi_ready[kND1], acc_done;
+  uint64_t d1_full[6], phi_ready[kND1], d1_free[kND1], acc_done;
   uint32_t tmem_base;
   int abort_flag;
 };
 struct alignas(8) QsideBars {
   uint64_t x_full[kNXQ], x_empty[kNXQ], xf_ready[kNF];
-  uint64_t d1_full[6], phi_ready[kND1], d2_full[2], d2_free[2], den_ready[2];
+  uint64_t d1_full[6], phi_ready[kND1], d1_free[kND1], d2_full[2], d2_free[2], den_ready[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -379,7 +380,10 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       mbar_init(&bars->v_empty[s], 1);
     }
     for (int b = 0; b < 6; ++b) mbar_init(&bars->d1_full[b], 1);
-    for (int b = 0; b < kND1; ++b) mbar_init(&bars->phi_ready[b], 4);
+    for (int b = 0; b < kND1; ++b) {
+      mbar_init(&bars->phi_ready[b], 4);
+      mbar_init(&bars->d1_free[b], 1);
+    }
     mbar_init(&bars->acc_done, 1);
     bars->abort_flag = 0;
     fence_mbar_init();
@@ -417,70 +421,71 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
         for (int b = max(0, issued - depth); b < issued; ++b) mbar_wait_drain(&full[b % depth], (b / depth) & 1);
       }
     } else if (warp == kWarpMma && lane == 0) {
-      // Issue order: MMA1 of unit u, then MMA2 of unit u - 2.  Everything that depends on the unit's
-      // position inside its block is resolved at compile time; ring slots, D1 buffers and barrier
-      // phases are running counters, and descriptors only add to their start-address word.
-      constexpr int UPB = 2 * NH;                       // units per 256-token block
+      // MMA1 of every unit.  Ring slots, D1 buffers and barrier phases are running counters, and the
+      // descriptors only add to their start-address word.
       constexpr uint32_t kTileStep = kTileBytes >> 4;
       const uint32_t hi = smem_desc_hi(1024);
       const uint32_t wt_lo = smem_desc_lo(smem_u32(smem + SL::wt), 16);
       const uint32_t x_lo = smem_desc_lo(smem_u32(smem + SL::x), 16);
-      const uint32_t v_lo = smem_desc_lo(smem_u32(smem + SL::v), 1024);
-      uint32_t xs = 0, vs = 0, vpar = 0;               // ring slot of the tile MMA1 / MMA2 is in, V phase
-      uint32_t fs = 0, fpar = 0;                        // "block filtered" barrier and phase
-      uint32_t c3 = 0, c6 = 0;                          // MMA1: D1 buffer, d1_full barrier
-      uint32_t p3 = 0, ppar = 0;                        // MMA2: D1 buffer (= phi_ready barrier) and phase
+      uint32_t xs = 0, fs = 0, fpar = 0;               // K ring slot; "block filtered" barrier and phase
+      uint32_t c3 = 0, c6 = 0, round = 0;              // D1 buffer, d1_full barrier, uses of buffer 0 so far
       bool ok = true;
-      for (int b = 0; b <= nblk && ok; ++b) {
-        if (b < nblk) {
-          ok = mbar_wait(&bars->xf_ready[fs], fpar, abort_flag, status, kErrMma);
-          if (!ok) break;
-          tc_fence_after_sync();
-        }
+      for (int b = 0; b < nblk && ok; ++b) {
+        ok = mbar_wait(&bars->xf_ready[fs], fpar, abort_flag, status, kErrMma);
+        if (!ok) break;
+        tc_fence_after_sync();
 #pragma unroll
-        for (int j = 0; j < UPB; ++j) {
-          if (b < nblk) {
-            const int h = j % NH;
-            const uint32_t a_lo = wt_lo + h * kTileStep, b_lo = x_lo + xs * kTileStep;
-            const uint32_t d1 = tmem + c3 * 128;
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              mma_ss(d1, smem_desc_join(a_lo + 2 * k, hi), smem_desc_join(b_lo + 2 * k, hi), kIdesc1, k > 0);
-            mma_commit(&bars->d1_full[c6]);
-            if (h == NH - 1) {   // last MMA1 that reads this tile
-              mma_commit(&bars->x_empty[xs]);
-              xs = xs == kNXK - 1 ? 0 : xs + 1;
-            }
-            c3 = c3 == kND1 - 1 ? 0 : c3 + 1;
-            c6 = c6 == 5 ? 0 : c6 + 1;
-          }
-          const int lj = j >= 2 ? j - 2 : j - 2 + UPB;   // unit u - 2: in this block, or late in the previous one
-          const int bb = j >= 2 ? b : b - 1;
-          if (bb >= 0 && bb < nblk) {
-            const int tt = lj / NH, h = lj % NH;
-            if (h == 0) {
-              ok = mbar_wait(&bars->v_full[vs], vpar, abort_flag, status, kErrMma);
-              if (!ok) break;
-            }
-            ok = mbar_wait(&bars->phi_ready[p3], ppar, abort_flag, status, kErrMma);
+        for (int j = 0; j < 2 * NH; ++j) {
+          const int h = j % NH;
+          if (round > 0) {   // the MMA2 that read this D1 buffer three units ago must have completed
+            ok = mbar_wait(&bars->d1_free[c3], (round - 1) & 1, abort_flag, status, kErrMma);
             if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t acc = tmem + kAccCol + h * 64, a_tm = tmem + p3 * 128;
-            const uint32_t b_lo = v_lo + vs * kTileStep;
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-              mma_ts(acc, a_tm + k * 8, smem_desc_join(b_lo + 128 * k, hi), kIdesc2, (bb > 0 || tt > 0 || k > 0) ? 1u : 0u);
-            if (h == NH - 1) {
-              mma_commit(&bars->v_empty[vs]);
-              vs = vs == kNV - 1 ? 0 : vs + 1;
-              vpar ^= (vs == 0);
-            }
-            p3 = p3 == kND1 - 1 ? 0 : p3 + 1;
-            ppar ^= (p3 == 0);
           }
+          const uint32_t a_lo = wt_lo + h * kTileStep, b_lo = x_lo + xs * kTileStep;
+          const uint32_t d1 = tmem + c3 * 128;
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            mma_ss(d1, smem_desc_join(a_lo + 2 * k, hi), smem_desc_join(b_lo + 2 * k, hi), kIdesc1, k > 0);
+          mma_commit(&bars->d1_full[c6]);
+          if (h == NH - 1) {   // last MMA1 that reads this tile
+            mma_commit(&bars->x_empty[xs]);
+            xs = xs == kNXK - 1 ? 0 : xs + 1;
+          }
+          c3 = c3 == kND1 - 1 ? 0 : c3 + 1;
+          round += (c3 == 0);
+          c6 = c6 == 5 ? 0 : c6 + 1;
         }
         fs = (fs + 1) & (kNF - 1);
         fpar ^= (fs == 0);
+      }
+    } else if (warp == kWarpMma2 && lane == 0) {
+      // MMA2 of every unit: S'[half h] += Phi^T (the unit's D1 buffer, bf16 pairs) * V tile.
+      constexpr uint32_t kTileStep = kTileBytes >> 4;
+      const uint32_t hi = smem_desc_hi(1024);
+      const uint32_t v_lo = smem_desc_lo(smem_u32(smem + SL::v), 1024);
+      uint32_t vs = 0, vpar = 0, p3 = 0, ppar = 0;     // V ring slot / phase, D1 buffer / phi_ready phase
+      bool ok = true;
+      for (int t = 0; t < 2 * nblk && ok; ++t) {
+        ok = mbar_wait(&bars->v_full[vs], vpar, abort_flag, status, kErrMma);
+        if (!ok) break;
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+          ok = mbar_wait(&bars->phi_ready[p3], ppar, abort_flag, status, kErrMma);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t acc = tmem + kAccCol + h * 64, a_tm = tmem + p3 * 128;
+          const uint32_t b_lo = v_lo + vs * kTileStep;
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            mma_ts(acc, a_tm + k * 8, smem_desc_join(b_lo + 128 * k, hi), kIdesc2, (t > 0 || k > 0) ? 1u : 0u);
+          mma_commit(&bars->d1_free[p3]);
+          p3 = p3 == kND1 - 1 ? 0 : p3 + 1;
+          ppar ^= (p3 == 0);
+        }
+        mma_commit(&bars->v_empty[vs]);
+        vs = vs == kNV - 1 ? 0 : vs + 1;
+        vpar ^= (vs == 0);
       }
       mma_commit(&bars->acc_done);
     }
@@ -626,7 +631,10 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     }
     for (int s = 0; s < kNF; ++s) mbar_init(&bars->xf_ready[s], 8);
     for (int b = 0; b < 6; ++b) mbar_init(&bars->d1_full[b], 1);
-    for (int b = 0; b < kND1; ++b) mbar_init(&bars->phi_ready[b], 4);
+    for (int b = 0; b < kND1; ++b) {
+      mbar_init(&bars->phi_ready[b], 4);
+      mbar_init(&bars->d1_free[b], 1);
+    }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bars->d2_full[b], 1);
       mbar_init(&bars->d2_free[b], 4);
@@ -664,63 +672,70 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
         for (int b = max(0, issued - kNXQ); b < issued; ++b) mbar_wait_drain(&bars->x_full[b % kNXQ], (b / kNXQ) & 1);
       }
     } else if (warp == kWarpMma && lane == 0) {
-      // Same issue scheme as the key side (MMA1 of unit u, then MMA2 of unit u - 2).
-      constexpr int UPB = 2 * NH;
+      // MMA1 of every unit (see the key side).
       constexpr uint32_t kTileStep = kTileBytes >> 4;
       const uint32_t hi = smem_desc_hi(1024);
       const uint32_t wt_lo = smem_desc_lo(smem_u32(smem + SL::wt), 16);
       const uint32_t x_lo = smem_desc_lo(smem_u32(smem + SL::x), 16);
-      const uint32_t s_lo = smem_desc_lo(smem_u32(smem + SL::simg), 1024);
       uint32_t xs = 0, fs = 0, fpar = 0;
-      uint32_t c3 = 0, c6 = 0;
-      uint32_t p3 = 0, ppar = 0;
+      uint32_t c3 = 0, c6 = 0, round = 0;
       bool ok = true;
-      for (int b = 0; b <= nblk && ok; ++b) {
-        if (b < nblk) {
-          ok = mbar_wait(&bars->xf_ready[fs], fpar, abort_flag, status, kErrMma);
-          if (!ok) break;
-          tc_fence_after_sync();
-        }
+      for (int b = 0; b < nblk && ok; ++b) {
+        ok = mbar_wait(&bars->xf_ready[fs], fpar, abort_flag, status, kErrMma);
+        if (!ok) break;
+        tc_fence_after_sync();
 #pragma unroll
-        for (int j = 0; j < UPB; ++j) {
-          if (b < nblk) {
-            const int h = j % NH;
-            const uint32_t a_lo = x_lo + xs * kTileStep, b_lo = wt_lo + h * kTileStep;
-            const uint32_t d1 = tmem + c3 * 128;
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              mma_ss(d1, smem_desc_join(a_lo + 2 * k, hi), smem_desc_join(b_lo + 2 * k, hi), kIdesc1, k > 0);
-            mma_commit(&bars->d1_full[c6]);
-            if (h == NH - 1) {   // last MMA1 that reads this tile
-              mma_commit(&bars->x_empty[xs]);
-              xs = xs == kNXQ - 1 ? 0 : xs + 1;
-            }
-            c3 = c3 == kND1 - 1 ? 0 : c3 + 1;
-            c6 = c6 == 5 ? 0 : c6 + 1;
-          }
-          const int lj = j >= 2 ? j - 2 : j - 2 + UPB;
-          const int bb = j >= 2 ? b : b - 1;
-          if (bb >= 0 && bb < nblk) {
-            const int tt = lj / NH, h = lj % NH;      // tile 2 bb + tt has parity tt
-            ok = mbar_wait(&bars->phi_ready[p3], ppar, abort_flag, status, kErrMma);
+        for (int j = 0; j < 2 * NH; ++j) {
+          const int h = j % NH;
+          if (round > 0) {
+            ok = mbar_wait(&bars->d1_free[c3], (round - 1) & 1, abort_flag, status, kErrMma);
             if (!ok) break;
-            if (h == 0 && bb >= 1) {                  // N' of tile parity tt must have been drained (tile t - 2)
-              ok = mbar_wait(&bars->d2_free[tt], (bb - 1) & 1, abort_flag, status, kErrMma);
-              if (!ok) break;
-            }
             tc_fence_after_sync();
-            const uint32_t d2 = tmem + kAccCol + tt * 64, a_tm = tmem + p3 * 128;
-            const uint32_t b_lo = s_lo + h * kTileStep;
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-              mma_ts(d2, a_tm + k * 8, smem_desc_join(b_lo + 128 * k, hi), kIdesc2, (h > 0 || k > 0) ? 1u : 0u);
-            if (h == NH - 1) mma_commit(&bars->d2_full[tt]);
-            p3 = p3 == kND1 - 1 ? 0 : p3 + 1;
-            ppar ^= (p3 == 0);
           }
+          const uint32_t a_lo = x_lo + xs * kTileStep, b_lo = wt_lo + h * kTileStep;
+          const uint32_t d1 = tmem + c3 * 128;
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            mma_ss(d1, smem_desc_join(a_lo + 2 * k, hi), smem_desc_join(b_lo + 2 * k, hi), kIdesc1, k > 0);
+          mma_commit(&bars->d1_full[c6]);
+          if (h == NH - 1) {   // last MMA1 that reads this tile
+            mma_commit(&bars->x_empty[xs]);
+            xs = xs == kNXQ - 1 ? 0 : xs + 1;
+          }
+          c3 = c3 == kND1 - 1 ? 0 : c3 + 1;
+          round += (c3 == 0);
+          c6 = c6 == 5 ? 0 : c6 + 1;
         }
         fs = (fs + 1) & (kNF - 1);
         fpar ^= (fs == 0);
+      }
+    } else if (warp == kWarpMma2 && lane == 0) {
+      // MMA2 of every unit: N'[tile parity] (+)= Phi (the unit's D1 buffer, bf16 pairs) * S' half h.
+      constexpr uint32_t kTileStep = kTileBytes >> 4;
+      const uint32_t hi = smem_desc_hi(1024);
+      const uint32_t s_lo = smem_desc_lo(smem_u32(smem + SL::simg), 1024);
+      uint32_t p3 = 0, ppar = 0;
+      bool ok = true;
+      for (int t = 0; t < ntiles && ok; ++t) {
+        if (t >= 2) {   // N' of this tile parity must have been drained (tile t - 2)
+          ok = mbar_wait(&bars->d2_free[t & 1], ((t >> 1) - 1) & 1, abort_flag, status, kErrMma);
+          if (!ok) break;
+        }
+        const uint32_t d2 = tmem + kAccCol + (t & 1) * 64;
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+          ok = mbar_wait(&bars->phi_ready[p3], ppar, abort_flag, status, kErrMma);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t a_tm = tmem + p3 * 128, b_lo = s_lo + h * kTileStep;
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            mma_ts(d2, a_tm + k * 8, smem_desc_join(b_lo + 128 * k, hi), kIdesc2, (h > 0 || k > 0) ? 1u : 0u);
+          mma_commit(&bars->d1_free[p3]);
+          p3 = p3 == kND1 - 1 ? 0 : p3 + 1;
+          ppar ^= (p3 == 0);
+        }
+        if (ok) mma_commit(&bars->d2_full[t & 1]);
       }
     }
   } else if (warp >= kReluWarp0 && warp < kAuxWarp0) {
