@@ -287,10 +287,16 @@ def main():
     tot = sum(avg.values())
     dom = max(avg, key=avg.get)
     # algorithmic work of each step per launch
-    flops = {"tc_kside": TH * (4 * d * m + 2 * m), "tc_qside": TH * (4 * d * m + 2 * m),
-             "simt_kside": TH * (4 * d * m + 2 * m), "simt_qside": TH * (4 * d * m + 2 * m)}
+    unit_flops = TH * (4 * d * m + 2 * m)            # one projection + one (m x d) contraction per token-head
+    flops = {"tc_kside": unit_flops, "tc_qside": unit_flops, "simt_kside": unit_flops, "simt_qside": unit_flops}
     bytes_ = {"qmean_gate": TH * d * s_bytes, "haar_filter_q": TH * d * (s_bytes + 4),
-              "haar_filter_k": TH * d * (s_bytes + 4)}
+              "haar_filter_k": TH * d * (s_bytes + 4),
+              "tc_kside": 2 * TH * d * s_bytes,      # K and V read once
+              "tc_qside": 2 * TH * d * s_bytes}      # Q read once, O written once
+    # DRAM bytes per token-head of one launch, from the ncu capture summarised in
+    # profiles/forward_cfg5_ncu_full_set.md (dram__bytes_read.sum + dram__bytes_write.sum on the cfg5
+    # forward, 524288 token-heads; traffic grows in proportion to the token-heads of a launch)
+    ncu_bytes_per_th = {"qmean_gate": 129.5, "tc_kside": 264.1, "tc_qside": 166.3}
     if dom in flops:
         if dom.startswith("tc_"):
             bound, peak, unit = "tensor", float(peaks["bf16_tflops"]), "TFLOP/s"
@@ -300,12 +306,16 @@ def main():
     else:
         bound, peak, unit = "hbm", float(peaks["hbm_gbs"]), "GB/s"
         achieved = bytes_.get(dom, 0) / (avg[dom] * 1e-3) / 1e9
+    traffic = ncu_bytes_per_th[dom] * TH if (tensor_cores and dtype == "bf16" and dom in ncu_bytes_per_th) else None
     roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
-                "frac": achieved / peak, "traffic": None,
+                "frac": achieved / peak, "traffic": traffic,
                 "peak_source": f"{peak_kind} (burst)" if bound == "tensor" else
                                (peak_kind if bound == "hbm" else "derived: 148 SM x 128 FFMA x 2 x 1.965 GHz"),
                 "kernel_ms": avg, "kernel_share": {k: v / tot for k, v in avg.items()},
                 "timing": "CUDA events behind every kernel, second pass of K steps"}
+    if dom in flops and dom in bytes_:   # the tensor-core kernels sit on the ridge: report the HBM side too
+        roofline["hbm_gbs_achieved"] = bytes_[dom] / (avg[dom] * 1e-3) / 1e9
+        roofline["hbm_frac"] = roofline["hbm_gbs_achieved"] / float(peaks["hbm_gbs"])
     # whole-path roofline: slower of FLOPs at tensor peak and bytes at HBM bandwidth
     path_flops = TH * (8 * d * m + 4 * m)
     path_bytes = TH * 4 * d * s_bytes
