@@ -75,7 +75,11 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
     return o;
   };
   const size_t slabs = (size_t)p->slabs;
-  p->off_status = take(256);
+  // status word (256 bytes) followed by the arrival counters; cleared together before the first launch
+  p->off_status = off;
+  p->off_counters = off + 256;
+  p->status_bytes = align_up(256 + sizeof(int) * (2 * slabs + (size_t)c.batch), 256);
+  take(p->status_bytes);
   p->off_qpart = take(sizeof(float) * slabs * p->qchunks * kD);
   p->off_qbar = take(sizeof(float) * slabs * kD);
   p->off_sg = take(sizeof(float) * slabs * p->L1);
@@ -109,6 +113,7 @@ Ws resolve(const Plan& p, void* workspace) {
   char* b = static_cast<char*>(workspace);
   Ws w;
   w.status = reinterpret_cast<int*>(b + p.off_status);
+  w.counters = reinterpret_cast<int*>(b + p.off_counters);
   w.qpart = reinterpret_cast<float*>(b + p.off_qpart);
   w.qbar = reinterpret_cast<float*>(b + p.off_qbar);
   w.sg = reinterpret_cast<float*>(b + p.off_sg);
@@ -200,7 +205,7 @@ wersa_status begin_pass(wersa_ctx* ctx, int which, cudaStream_t st) {
 
 wersa_status clear_status_once(wersa_ctx* ctx, cudaStream_t st) {
   if (!ctx->status_cleared) {
-    WERSA_CUDA(cudaMemsetAsync(ctx->ws.status, 0, 256, st));
+    WERSA_CUDA(cudaMemsetAsync(ctx->ws.status, 0, ctx->plan.status_bytes, st));
     ctx->status_cleared = true;
   }
   return WERSA_OK;
@@ -333,8 +338,7 @@ wersa_status wersa_gate_static(const wersa_config* cfg, const void* Q, const flo
   Plan p;
   wersa_status s = make_plan(*cfg, &p);
   if (s != WERSA_OK) return s;
-  const size_t need = (size_t)p.slabs * p.qchunks * kD + (size_t)p.slabs * p.L1;
-  if (need > static_scratch_capacity_floats()) return WERSA_ERR_TOO_LARGE;
+  if (static_scratch_floats_needed(p) > static_scratch_capacity_floats()) return WERSA_ERR_TOO_LARGE;
   DeviceGuard guard(p.cfg.device);
   if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
   float* scratch = nullptr;

@@ -34,7 +34,7 @@ struct Plan {
   // tcgen05 key-side split
   int tchunks, tchunk_blocks;  // chunks per slab, 256-token blocks per chunk
   // workspace offsets (bytes)
-  size_t off_status, off_qpart, off_qbar, off_sg, off_f, off_spart, off_zpart, off_S, off_z,
+  size_t off_status, off_counters, status_bytes, off_qpart, off_qbar, off_sg, off_f, off_spart, off_zpart, off_S, off_z,
       off_Sbf, off_Wt, off_dS, off_dz, off_sumdD, off_bands, off_dqbar, off_QF, off_KF, off_dQF,
       off_dKF, total;
   int part_chunks;    // max(schunks, tchunks): leading extent of the partial buffers
@@ -45,6 +45,7 @@ wersa_status make_plan(const wersa_config& cfg, Plan* p);
 
 struct Ws {   // resolved workspace pointers
   int* status;
+  int* counters;   // arrival counters (slabs + batch + slabs ints), zero between launches
   float *qpart, *qbar, *sg, *f, *spart, *zpart, *S, *z, *dS, *dz, *sumdD, *bands, *dqbar;
   __nv_bfloat16 *Sbf, *Wt;
   float *QF, *KF, *dQF, *dKF;
@@ -67,6 +68,7 @@ cudaError_t launch_add_rowvec(const Plan& p, const Ws& w, void* dQ, cudaStream_t
 // Mean pool + gate with their scratch in a file-scope device array (no caller workspace).
 cudaError_t static_scratch_address(int device, float** out);
 size_t static_scratch_capacity_floats();
+size_t static_scratch_floats_needed(const Plan& p);
 cudaError_t launch_qmean_gate_static(const Plan& p, float* scratch, const void* Q, const float* gate_w,
                                      const float* gate_b, const float* omega, float* qbar, float* f,
                                      cudaStream_t st);

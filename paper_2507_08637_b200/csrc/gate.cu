@@ -13,81 +13,26 @@ constexpr int kMaxDevices = 64;
 float* g_static_scratch_addr[kMaxDevices] = {nullptr};
 std::mutex g_static_scratch_mutex;
 
-// Partial column sums of one row chunk of one slab of Q.  grid (qchunks, slabs), block 256:
-// thread (cg = tid & 7, rl = tid >> 3) owns 8 consecutive columns and every 32nd row, loads
-// 16 bytes (bf16) / 32 bytes (fp32) per row, four rows in flight.
-template <typename T>
-__global__ void __launch_bounds__(256) k_qmean_partial(const T* __restrict__ Q, float* __restrict__ qpart,
-                                                       int n, int chunk_rows) {
-  const int chunk = blockIdx.x, slab = blockIdx.y;
-  const int cg = threadIdx.x & 7, rl = threadIdx.x >> 3;
-  const int r0 = chunk * chunk_rows;
-  const int r1 = min(n, r0 + chunk_rows);
-  const T* base = Q + (size_t)slab * n * kD + cg * 8;
-  float acc[8];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-  int r = r0 + rl;
-  for (; r + 96 < r1; r += 128) {
-    float v0[8], v1[8], v2[8], v3[8];
-    load8(base + (size_t)r * kD, v0);
-    load8(base + (size_t)(r + 32) * kD, v1);
-    load8(base + (size_t)(r + 64) * kD, v2);
-    load8(base + (size_t)(r + 96) * kD, v3);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] += (v0[j] + v1[j]) + (v2[j] + v3[j]);
-  }
-  for (; r < r1; r += 32) {
-    float v0[8];
-    load8(base + (size_t)r * kD, v0);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] += v0[j];
-  }
-  __shared__ float red[32][kD + 1];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) red[rl][cg * 8 + j] = acc[j];
-  __syncthreads();
-  if (threadIdx.x < kD) {
-    float s = 0.f;
-#pragma unroll 8
-    for (int i = 0; i < 32; ++i) s += red[i][threadIdx.x];   // fixed order
-    qpart[((size_t)slab * gridDim.x + chunk) * kD + threadIdx.x] = s;
-  }
-}
-
-// grid (slabs + wt_blocks), block 256.
-// Blocks [0, slabs): qbar of one slab = sum of its chunk partials in a fixed order / n (Eq. 1), the
-// head's logits u = gate_w[h]^T qbar (Eq. 2) and, for the per-head gate, sigmoid(u + gate_b[h]) and
-// f = sigmoid * omega (Eq. 3).  For the batch-wide gate the bias-free logits are parked in f and
-// k_gate_shared finishes the job.
-// Blocks [slabs, ...): bf16 transpose Wt (m x 64) of W (64 x m) for the tensor-core kernels.
-__global__ void __launch_bounds__(256) k_qbar_gate(const float* __restrict__ qpart, int qchunks, int slabs, int H,
-                                                   int n, int L1, int per_head, const float* __restrict__ gate_w,
-                                                   const float* __restrict__ gate_b, const float* __restrict__ omega,
-                                                   float* __restrict__ qbar, float* __restrict__ sg,
-                                                   float* __restrict__ f, const __nv_bfloat16* __restrict__ W,
-                                                   __nv_bfloat16* __restrict__ Wt, int m) {
-  if ((int)blockIdx.x >= slabs) {
-    const int i = ((int)blockIdx.x - slabs) * 256 + threadIdx.x;
-    if (i < m * kD) {
-      const int r = i / kD, c = i - r * kD;
-      Wt[i] = W[(size_t)c * m + r];
-    }
-    return;
-  }
-  const int slab = blockIdx.x, h = slab % H;
+// Finish of one slab by the last CTA of that slab to arrive (256 threads): qbar = sum of the chunk
+// partials in chunk order / n (Eq. 1), the head's logits u = gate_w[h]^T qbar (Eq. 2) and, for the
+// per-head gate, sigmoid(u + gate_b[h]) and f = sigmoid * omega (Eq. 3).  For the batch-wide gate the
+// bias-free logits are parked in f for batch_gate.
+__device__ __forceinline__ void slab_gate(const float* __restrict__ qpart, int qchunks, int slab, int H, int n, int L1,
+                                          int per_head, const float* __restrict__ gate_w,
+                                          const float* __restrict__ gate_b, const float* __restrict__ omega,
+                                          float* __restrict__ qbar, float* __restrict__ sg, float* __restrict__ f,
+                                          float (*red)[kD], float* qs) {
+  const int h = slab % H;
   const int c = threadIdx.x & (kD - 1), part = threadIdx.x >> 6;   // 4 interleaved partial sums per column
-  __shared__ float red[4][kD];
-  __shared__ float qs[kD];
   float s = 0.f;
   const float* src = qpart + (size_t)slab * qchunks * kD + c;
   int k = part;
   for (; k + 12 < qchunks; k += 16) {
-    const float v0 = src[(size_t)k * kD], v1 = src[(size_t)(k + 4) * kD];
-    const float v2 = src[(size_t)(k + 8) * kD], v3 = src[(size_t)(k + 12) * kD];
+    const float v0 = __ldcg(src + (size_t)k * kD), v1 = __ldcg(src + (size_t)(k + 4) * kD);
+    const float v2 = __ldcg(src + (size_t)(k + 8) * kD), v3 = __ldcg(src + (size_t)(k + 12) * kD);
     s += (v0 + v1) + (v2 + v3);
   }
-  for (; k < qchunks; k += 4) s += src[(size_t)k * kD];
+  for (; k < qchunks; k += 4) s += __ldcg(src + (size_t)k * kD);
   red[part][c] = s;
   __syncthreads();
   if (threadIdx.x < kD) {
@@ -120,20 +65,102 @@ __global__ void __launch_bounds__(256) k_qbar_gate(const float* __restrict__ qpa
   }
 }
 
-// Batch-wide gate (Algorithm 1, W_filter): u[b] = sum_h u[b,h] + gate_b[0], one sigmoid per batch
-// element shared by its heads.  grid (B), block 32; thread i owns band i of every head.
-__global__ void __launch_bounds__(32) k_gate_shared(int H, int L1, const float* __restrict__ gate_b,
-                                                    const float* __restrict__ omega, float* __restrict__ sg,
-                                                    float* __restrict__ f) {
-  const int b = blockIdx.x, i = threadIdx.x;
+// Batch-wide gate (Algorithm 1, W_filter), by the last slab of a batch element to finish:
+// u[b] = sum_h u[b,h] + gate_b[0], one sigmoid per batch element shared by its heads.
+__device__ __forceinline__ void batch_gate(int b, int H, int L1, const float* __restrict__ gate_b,
+                                           const float* __restrict__ omega, float* __restrict__ sg,
+                                           float* __restrict__ f) {
+  const int i = threadIdx.x;
   if (i >= L1) return;
   float u = gate_b != nullptr ? gate_b[i] : 0.f;
-  for (int h = 0; h < H; ++h) u += f[((size_t)b * H + h) * L1 + i];
+  for (int h = 0; h < H; ++h) u += __ldcg(f + ((size_t)b * H + h) * L1 + i);
   const float sgm = 1.f / (1.f + expf(-u));
   for (int h = 0; h < H; ++h) {
     sg[((size_t)b * H + h) * L1 + i] = sgm;
     f[((size_t)b * H + h) * L1 + i] = sgm * omega[i];
   }
+}
+
+// Mean pool and gate in one launch.  grid (qchunks, slabs [+ 1]), block 256.
+// Rows y < slabs: partial column sums of one row chunk of one slab of Q -- thread (cg = tid & 7,
+// rl = tid >> 3) owns 8 consecutive columns and every 32nd row, loads 16 bytes (bf16) / 32 bytes
+// (fp32) per row, four rows in flight.  The CTA that finds it is the last of its slab to finish
+// (a counter per slab) then runs slab_gate, and for the batch-wide gate the last slab of a batch
+// element (a counter per batch element) runs batch_gate; sums are taken in a fixed order, so the
+// result does not depend on which CTA comes last.  The counters start at zero and are left at zero.
+// Row y == slabs (only with W != nullptr): bf16 transpose Wt (m x 64) of W (64 x m) for the
+// tensor-core kernels.
+template <typename T>
+__global__ void __launch_bounds__(256) k_qmean_gate(const T* __restrict__ Q, float* __restrict__ qpart, int n,
+                                                    int chunk_rows, int slabs, int H, int L1, int per_head,
+                                                    const float* __restrict__ gate_w, const float* __restrict__ gate_b,
+                                                    const float* __restrict__ omega, float* __restrict__ qbar,
+                                                    float* __restrict__ sg, float* __restrict__ f,
+                                                    int* __restrict__ slab_count, int* __restrict__ batch_count,
+                                                    const __nv_bfloat16* __restrict__ W, __nv_bfloat16* __restrict__ Wt,
+                                                    int m) {
+  if ((int)blockIdx.y == slabs) {
+    for (int i = blockIdx.x * 256 + threadIdx.x; i < m * kD; i += gridDim.x * 256) {
+      const int r = i / kD, c = i - r * kD;
+      Wt[i] = W[(size_t)c * m + r];
+    }
+    return;
+  }
+  const int chunk = blockIdx.x, slab = blockIdx.y;
+  const int cg = threadIdx.x & 7, rl = threadIdx.x >> 3;
+  const int r0 = chunk * chunk_rows;
+  const int r1 = min(n, r0 + chunk_rows);
+  const T* base = Q + (size_t)slab * n * kD + cg * 8;
+  float acc[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+  int r = r0 + rl;
+  for (; r + 96 < r1; r += 128) {
+    float v0[8], v1[8], v2[8], v3[8];
+    load8(base + (size_t)r * kD, v0);
+    load8(base + (size_t)(r + 32) * kD, v1);
+    load8(base + (size_t)(r + 64) * kD, v2);
+    load8(base + (size_t)(r + 96) * kD, v3);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] += (v0[j] + v1[j]) + (v2[j] + v3[j]);
+  }
+  for (; r < r1; r += 32) {
+    float v0[8];
+    load8(base + (size_t)r * kD, v0);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] += v0[j];
+  }
+  __shared__ float red[32][kD + 1];
+  __shared__ float red4[4][kD];
+  __shared__ float qs[kD];
+  __shared__ int s_last;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) red[rl][cg * 8 + j] = acc[j];
+  __syncthreads();
+  if (threadIdx.x < kD) {
+    float s = 0.f;
+#pragma unroll 8
+    for (int i = 0; i < 32; ++i) s += red[i][threadIdx.x];   // fixed order
+    qpart[((size_t)slab * gridDim.x + chunk) * kD + threadIdx.x] = s;
+    __threadfence();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(&slab_count[slab], 1) == (int)gridDim.x - 1;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  slab_gate(qpart, gridDim.x, slab, H, n, L1, per_head, gate_w, gate_b, omega, qbar, sg, f, red4, qs);
+  if (threadIdx.x == 0) slab_count[slab] = 0;
+  if (per_head) return;
+  __threadfence();
+  __syncthreads();
+  const int b = slab / H;
+  if (threadIdx.x == 0) s_last = atomicAdd(&batch_count[b], 1) == H - 1;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  batch_gate(b, H, L1, gate_b, omega, sg, f);
+  if (threadIdx.x == 0) batch_count[b] = 0;
 }
 
 // Sum the per-tile band inner products of both filtered tensors in tile order and turn them
@@ -242,34 +269,29 @@ __global__ void __launch_bounds__(256) k_add_rowvec(T* __restrict__ dQ, const fl
 
 }  // namespace
 
-// Second and third launch of the gate step, shared by the workspace and the static-scratch variants.
-static cudaError_t launch_gate_tail(const Plan& p, const float* qpart, const float* gate_w, const float* gate_b,
-                                    const float* omega, float* qbar, float* sg, float* f, const void* W,
-                                    __nv_bfloat16* Wt, cudaStream_t st, int* launches) {
-  const int m = p.cfg.features;
-  const int wt_blocks = W != nullptr ? (m * kD + 255) / 256 : 0;
-  k_qbar_gate<<<p.slabs + wt_blocks, 256, 0, st>>>(qpart, p.qchunks, p.slabs, p.cfg.heads, p.cfg.seq_len, p.L1,
-                                                   p.cfg.gate_per_head, gate_w, gate_b, omega, qbar, sg, f,
-                                                   (const __nv_bfloat16*)W, Wt, m);
-  *launches += 1;
-  if (!p.cfg.gate_per_head) {
-    k_gate_shared<<<p.cfg.batch, 32, 0, st>>>(p.cfg.heads, p.L1, gate_b, omega, sg, f);
-    *launches += 1;
-  }
+// The launch shared by the workspace and the static-scratch variants.
+static cudaError_t launch_qmean_gate_impl(const Plan& p, const void* Q, float* qpart, const float* gate_w,
+                                          const float* gate_b, const float* omega, float* qbar, float* sg, float* f,
+                                          int* counters, const void* W, __nv_bfloat16* Wt, cudaStream_t st) {
+  dim3 grid(p.qchunks, p.slabs + (W != nullptr ? 1 : 0));
+  int* slab_count = counters;
+  int* batch_count = counters + p.slabs;
+  if (p.bf16)
+    k_qmean_gate<__nv_bfloat16><<<grid, 256, 0, st>>>(
+        (const __nv_bfloat16*)Q, qpart, p.cfg.seq_len, p.qchunk_rows, p.slabs, p.cfg.heads, p.L1, p.cfg.gate_per_head,
+        gate_w, gate_b, omega, qbar, sg, f, slab_count, batch_count, (const __nv_bfloat16*)W, Wt, p.cfg.features);
+  else
+    k_qmean_gate<float><<<grid, 256, 0, st>>>((const float*)Q, qpart, p.cfg.seq_len, p.qchunk_rows, p.slabs,
+                                              p.cfg.heads, p.L1, p.cfg.gate_per_head, gate_w, gate_b, omega, qbar, sg,
+                                              f, slab_count, batch_count, (const __nv_bfloat16*)W, Wt, p.cfg.features);
   return cudaGetLastError();
 }
 
 cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const float* gate_w,
                               const float* gate_b, const float* omega, const void* W, cudaStream_t st,
                               int* launches) {
-  dim3 grid(p.qchunks, p.slabs);
-  if (p.bf16)
-    k_qmean_partial<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)Q, w.qpart, p.cfg.seq_len,
-                                                         p.qchunk_rows);
-  else
-    k_qmean_partial<float><<<grid, 256, 0, st>>>((const float*)Q, w.qpart, p.cfg.seq_len, p.qchunk_rows);
   *launches += 1;
-  return launch_gate_tail(p, w.qpart, gate_w, gate_b, omega, w.qbar, w.sg, w.f, W, w.Wt, st, launches);
+  return launch_qmean_gate_impl(p, Q, w.qpart, gate_w, gate_b, omega, w.qbar, w.sg, w.f, w.counters, W, w.Wt, st);
 }
 
 // Device address of the static scratch array on the current device, resolved once per device.
@@ -292,17 +314,16 @@ size_t static_scratch_capacity_floats() { return kStaticScratchFloats; }
 cudaError_t launch_qmean_gate_static(const Plan& p, float* scratch, const void* Q, const float* gate_w,
                                      const float* gate_b, const float* omega, float* qbar, float* f,
                                      cudaStream_t st) {
-  // scratch = [ partial column sums: slabs x qchunks x 64 | sigmoid(u): slabs x (L+1) ]
+  // scratch = [ partial column sums: slabs x qchunks x 64 | sigmoid(u): slabs x (L+1) | arrival counters:
+  //             slabs + batch ints, zero when the library is loaded and left at zero by every call ]
   float* qpart = scratch;
   float* sg = scratch + (size_t)p.slabs * p.qchunks * kD;
-  dim3 grid(p.qchunks, p.slabs);
-  if (p.bf16)
-    k_qmean_partial<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)Q, qpart, p.cfg.seq_len,
-                                                         p.qchunk_rows);
-  else
-    k_qmean_partial<float><<<grid, 256, 0, st>>>((const float*)Q, qpart, p.cfg.seq_len, p.qchunk_rows);
-  int launches = 0;
-  return launch_gate_tail(p, qpart, gate_w, gate_b, omega, qbar, sg, f, nullptr, nullptr, st, &launches);
+  int* counters = reinterpret_cast<int*>(sg + (size_t)p.slabs * p.L1);
+  return launch_qmean_gate_impl(p, Q, qpart, gate_w, gate_b, omega, qbar, sg, f, counters, nullptr, nullptr, st);
+}
+
+size_t static_scratch_floats_needed(const Plan& p) {
+  return (size_t)p.slabs * p.qchunks * kD + (size_t)p.slabs * p.L1 + (size_t)p.slabs + (size_t)p.cfg.batch;
 }
 
 cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, const float* gate_w,
