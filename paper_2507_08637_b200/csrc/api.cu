@@ -66,6 +66,13 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
     p->tchunk_blocks = ceil_div(blocks, p->tchunks);
     p->tchunks = ceil_div(blocks, p->tchunk_blocks);
   }
+  {
+    const int tiles128 = ceil_div(n, 128);
+    p->bchunks = ceil_div(148, p->slabs);
+    if (p->bchunks > tiles128) p->bchunks = tiles128;
+    p->bchunk_tiles = ceil_div(tiles128, p->bchunks);
+    p->bchunks = ceil_div(tiles128, p->bchunk_tiles);
+  }
   p->part_chunks = p->schunks > p->tchunks ? p->schunks : p->tchunks;
 
   size_t off = 0;
@@ -102,8 +109,10 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
     p->off_dqbar = take(sizeof(float) * slabs * (kD + kBandVals));
     p->off_dQF = take(sizeof(float) * slab_elems);
     p->off_dKF = take(sizeof(float) * slab_elems);
+    p->off_dSbf = take(sizeof(__nv_bfloat16) * slabs * m * kD);
+    p->off_KF3 = take(p->use_tc ? 3 * sizeof(__nv_bfloat16) * slab_elems : 0);
   } else {
-    p->off_dS = p->off_dz = p->off_sumdD = p->off_bands = p->off_dqbar = p->off_dQF = p->off_dKF = 0;
+    p->off_dS = p->off_dz = p->off_sumdD = p->off_bands = p->off_dqbar = p->off_dQF = p->off_dKF = p->off_dSbf = p->off_KF3 = 0;
   }
   p->total = off;
   return WERSA_OK;
@@ -133,6 +142,8 @@ Ws resolve(const Plan& p, void* workspace) {
   w.dqbar = reinterpret_cast<float*>(b + p.off_dqbar);
   w.dQF = reinterpret_cast<float*>(b + p.off_dQF);
   w.dKF = reinterpret_cast<float*>(b + p.off_dKF);
+  w.dSbf = reinterpret_cast<__nv_bfloat16*>(b + p.off_dSbf);
+  w.KF3 = reinterpret_cast<__nv_bfloat16*>(b + p.off_KF3);
   return w;
 }
 
@@ -301,14 +312,18 @@ wersa_status wersa_backward(wersa_ctx* ctx, const void* Q, const void* K, const 
   const int kind = p.bf16 ? 1 : 0, gkind = p.grad_bf16 ? 1 : 0;
   wersa_status s = begin_pass(ctx, 1, st);
   if (s != WERSA_OK) return s;
-  if (p.use_tc) {   // the tensor-core forward keeps Q_F, K_F on chip: rebuild them
+  if (p.use_tc) {   // the tensor-core forward keeps Q_F, K_F on chip: rebuild them (K_F as three bf16 planes)
     WERSA_STEP(1, "haar_filter_q", launch_haar_filter(p, Q, kind, w.f, w.QF, 0, st, &launches));
-    WERSA_STEP(1, "haar_filter_k", launch_haar_filter(p, K, kind, w.f, w.KF, 0, st, &launches));
+    WERSA_STEP(1, "haar_filter_k", launch_haar_filter_split3(p, K, kind, w.f, w.KF3, st, &launches));
   }
   WERSA_STEP(1, "simt_bwd_qside", launch_simt_bwd_qside(p, w, W, beta, dO, st, &launches));
   WERSA_STEP(1, "reduce_partials",
-             launch_reduce_partials(p, w.spart, w.zpart, p.schunks, w.dS, w.dz, nullptr, st, &launches));
-  WERSA_STEP(1, "simt_bwd_kside", launch_simt_bwd_kside(p, w, V, W, dV, st, &launches));
+             launch_reduce_partials(p, w.spart, w.zpart, p.schunks, w.dS, w.dz, p.use_tc ? w.dSbf : nullptr, st,
+                                    &launches));
+  if (p.use_tc)
+    WERSA_STEP(1, "tc_bwd_kside", launch_tc_bwd_kside(p, w, w.KF3, V, dV, st, &launches));
+  else
+    WERSA_STEP(1, "simt_bwd_kside", launch_simt_bwd_kside(p, w, V, W, dV, st, &launches));
   WERSA_STEP(1, "haar_backward_q", launch_haar_backward(p, w, Q, kind, w.dQF, dQ, gkind, 0, st, &launches));
   WERSA_STEP(1, "haar_backward_k", launch_haar_backward(p, w, K, kind, w.dKF, dK, gkind, 1, st, &launches));
   WERSA_STEP(1, "gate_backward",

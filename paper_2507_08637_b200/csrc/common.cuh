@@ -33,10 +33,12 @@ struct Plan {
   int schunks, schunk_tiles;   // chunks per slab, 32-token tiles per chunk
   // tcgen05 key-side split
   int tchunks, tchunk_blocks;  // chunks per slab, 256-token blocks per chunk
+  // tcgen05 backward: chunks per slab, 128-token tiles per chunk
+  int bchunks, bchunk_tiles;
   // workspace offsets (bytes)
   size_t off_status, off_counters, status_bytes, off_qpart, off_qbar, off_sg, off_f, off_spart, off_zpart, off_S, off_z,
       off_Sbf, off_Wt, off_dS, off_dz, off_sumdD, off_bands, off_dqbar, off_QF, off_KF, off_dQF,
-      off_dKF, total;
+      off_dKF, off_dSbf, off_KF3, total;
   int part_chunks;    // max(schunks, tchunks): leading extent of the partial buffers
 };
 
@@ -47,7 +49,7 @@ struct Ws {   // resolved workspace pointers
   int* status;
   int* counters;   // arrival counters (slabs + batch + slabs ints), zero between launches
   float *qpart, *qbar, *sg, *f, *spart, *zpart, *S, *z, *dS, *dz, *sumdD, *bands, *dqbar;
-  __nv_bfloat16 *Sbf, *Wt;
+  __nv_bfloat16 *Sbf, *Wt, *dSbf, *KF3;
   float *QF, *KF, *dQF, *dKF;
 };
 Ws resolve(const Plan& p, void* workspace);
@@ -77,6 +79,9 @@ cudaError_t launch_qmean_gate_static(const Plan& p, float* scratch, const void* 
 // XF = T_f(X).  in_kind/out_kind: 0 = float, 1 = bf16.
 cudaError_t launch_haar_filter(const Plan& p, const void* X, int in_kind, const float* f, void* XF,
                                int out_kind, cudaStream_t st, int* launches);
+// XF3 = T_f(X) as three bf16 planes hi, mid, lo (each slabs x n x 64) whose sum is the fp32 result.
+cudaError_t launch_haar_filter_split3(const Plan& p, const void* X, int in_kind, const float* f,
+                                      __nv_bfloat16* XF3, cudaStream_t st, int* launches);
 // dX = T_f(G) (G fp32) and per-tile band inner products of (G, X) into bands[which].
 cudaError_t launch_haar_backward(const Plan& p, const Ws& w, const void* X, int in_kind,
                                  const float* G, void* dX, int out_kind, int which, cudaStream_t st,
@@ -102,6 +107,12 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
                             int* launches);
 cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const float* beta, void* O,
                             cudaStream_t st, int* launches);
+
+// ---- tc_bwd.cu -----------------------------------------------------------------------------
+// Key-side backward on the tensor cores: dV and dK_F from K_F as three bf16 planes, V, the bf16 dS' image
+// (w.dSbf), dz' (w.dz) and the bf16 W^T image (w.Wt).
+cudaError_t launch_tc_bwd_kside(const Plan& p, const Ws& w, const void* KF3, const void* V, void* dV,
+                                cudaStream_t st, int* launches);
 
 // ---- device helpers ------------------------------------------------------------------------
 __device__ __forceinline__ float to_f32(float x) { return x; }

@@ -119,6 +119,43 @@ __global__ void __launch_bounds__(256, 2) k_haar_filter(const Tin* __restrict__ 
     if (row0 + j < n) store8(dst + (size_t)(row0 + j) * kD, x[j]);
 }
 
+// The same filter with the result written as three bf16 planes hi + mid + lo (each slabs x n x 64):
+// hi = bf16(x), mid = bf16(x - hi), lo = bf16(x - hi - mid), so that their sum carries the fp32
+// value (24 mantissa bits) into bf16 tensor-core products.  The backward kernels need that: the
+// ReLU mask 1[a > 0] of a = X_F W must not flip through the rounding of X_F.
+template <typename Tin>
+__global__ void __launch_bounds__(256, 2) k_haar_filter_split3(const Tin* __restrict__ X, const float* __restrict__ f,
+                                                            __nv_bfloat16* __restrict__ XF3, size_t plane, int n,
+                                                            int L) {
+  __shared__ float sh[8][kD];
+  const int slab = blockIdx.y;
+  const int cg = threadIdx.x & 7, rg = threadIdx.x >> 3;
+  const int row0 = blockIdx.x * kHaarTile + rg * 8;
+  const LevelCoef k = level_coef(f + (size_t)slab * (L + 1), L);
+  float x[8][8];
+  load_tile(X + (size_t)slab * n * kD, n, row0, x);
+  Sums s;
+  block_sums(x, s, sh, L);
+  apply_filter(x, s, k);
+  __nv_bfloat16* dst = XF3 + (size_t)slab * n * kD + cg * 8;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    if (row0 + j >= n) continue;
+    float hi[8], mid[8], lo[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      hi[c] = __bfloat162float(__float2bfloat16_rn(x[j][c]));
+      const float r1 = x[j][c] - hi[c];
+      mid[c] = __bfloat162float(__float2bfloat16_rn(r1));
+      lo[c] = r1 - mid[c];
+    }
+    __nv_bfloat16* row = dst + (size_t)(row0 + j) * kD;
+    store8(row, hi);
+    store8(row + plane, mid);
+    store8(row + 2 * plane, lo);
+  }
+}
+
 // Backward of the filter for one tile: dX = T_f(G) (the operator is symmetric) and the band
 // inner products of (G, X) that give df:
 //   slot l-1 (l = 1..8): sum over blocks of Delta_l(G) * Delta_l(X) / 2^l, the product of the
@@ -230,6 +267,19 @@ cudaError_t launch_haar_filter(const Plan& p, const void* X, int in_kind, const 
     k_haar_filter<float, float><<<grid, 256, 0, st>>>((const float*)X, f, (float*)XF, n, L);
   else
     k_haar_filter<float, __nv_bfloat16><<<grid, 256, 0, st>>>((const float*)X, f, (__nv_bfloat16*)XF, n, L);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_haar_filter_split3(const Plan& p, const void* X, int in_kind, const float* f,
+                                      __nv_bfloat16* XF3, cudaStream_t st, int* launches) {
+  dim3 grid(p.htiles, p.slabs);
+  const int n = p.cfg.seq_len, L = p.cfg.levels;
+  const size_t plane = (size_t)p.slabs * n * kD;
+  if (in_kind == 1)
+    k_haar_filter_split3<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, f, XF3, plane, n, L);
+  else
+    k_haar_filter_split3<float><<<grid, 256, 0, st>>>((const float*)X, f, XF3, plane, n, L);
   *launches += 1;
   return cudaGetLastError();
 }

@@ -1,0 +1,370 @@
+// bf16 tensor-core (tcgen05 + TMEM + TMA) backward kernels of the WERSA attention path, sm_100a.
+// The paper does not write the backward pass; these are the chain rule through Eq. 6 / Eq. 7 with
+// dReLU(a)/da = 1[a > 0], on the same unscaled quantities the forward kernels use.
+//
+// Key side, per 128-token tile (token = TMEM lane, one thread per token):
+//   MMA1: B_h = K_F (smem, K-major; three bf16 planes hi + mid + lo that add up to the fp32 K_F, so
+//         that the mask below does not flip through rounding) * W_h (as W^T, K-major) -> TMEM fp32
+//   threads: mask = 1[B_h > 0] (bits in registers), Phi_h = ReLU(B_h) -> bf16 pairs in place
+//   MMA2: dV = sum_h Phi_h (TMEM operand) * dS'_h (smem bf16, N-major) -> TMEM fp32 -> global
+//   MMA3: G_h = V (smem, K-major) * dS'_h^T (same image, K-major)      -> TMEM fp32
+//   threads: dB_h = (G_h + dz'_h) (.) mask                              -> bf16 pairs in place
+//   MMA4: dK_F = sum_h dB_h (TMEM operand) * W_h^T (W^T image, N-major) -> TMEM fp32 -> global
+// One CTA of 128 threads per SM walks a chunk of tiles one step at a time (thread 0 issues the copies
+// and the MMAs, everybody waits on one mbarrier); the copies of the next tile are in flight meanwhile.
+// TMEM per CTA: 128 columns per feature half; the two 64-column results (dV, dK_F) reuse the upper
+// half of the first accumulator.  Every mbarrier wait is bounded; after an expired wait the CTA
+// leaves its loop (the decision is taken CTA-wide, so barriers stay balanced) and the host sees the
+// status word.
+#include "common.cuh"
+#include "tc_common.cuh"
+
+namespace wersa {
+using namespace tc;
+
+namespace {
+
+constexpr int kTile = 128;
+constexpr uint32_t kTileBytes = kTile * kD * 2;   // 128 x 64 bf16
+constexpr uint32_t kIdescP = make_idesc_bf16(128, 128, false, false);  // projections: both operands K-major
+constexpr uint32_t kIdescC = make_idesc_bf16(128, 64, false, true);    // contractions over features: B N-major
+enum { kErrBwdCopy = 21, kErrBwdMma = 22 };
+
+struct alignas(8) BwdBars {
+  uint64_t full[2], mma;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <int NH> struct BwdKSmem {
+  static constexpr uint32_t wt = 0;                          // W^T image, NH x (128 x 64) bf16
+  static constexpr uint32_t ds = wt + NH * kTileBytes;       // dS' image, same shape
+  static constexpr uint32_t stage = ds + NH * kTileBytes;    // 2 stages x (3 K_F planes + V) tiles
+  static constexpr uint32_t stage_bytes = 4 * kTileBytes;
+  static constexpr uint32_t dz = stage + 2 * stage_bytes;    // NH x 128 floats
+  static constexpr uint32_t bars = dz + NH * 512;
+  static constexpr uint32_t total = bars + 64 + 1024;        // + alignment slack
+};
+
+__device__ __forceinline__ void load_rows_swizzled(uint8_t* dst, const __nv_bfloat16* src, int rows) {
+  for (int i = threadIdx.x; i < rows * 8; i += blockDim.x) {
+    const int r = i >> 3, c = i & 7;
+    const uint4 val = *reinterpret_cast<const uint4*>(src + (size_t)r * kD + c * 8);
+    *reinterpret_cast<uint4*>(dst + swz128(r, c)) = val;
+  }
+}
+
+__device__ __forceinline__ void reg_fence32(uint32_t (&r)[32]) {
+  asm volatile(""
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
+                 "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]),
+                 "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]),
+                 "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
+
+// CTA-wide wait: every thread waits (bounded) on the barrier; the outcome is made uniform.
+__device__ __forceinline__ bool cta_wait(uint64_t* bar, uint32_t parity, BwdBars* bars, int* status, int code) {
+  const bool ok = mbar_wait(bar, parity, &bars->abort_flag, status, code);
+  return __syncthreads_and(ok) != 0;
+}
+
+template <typename TG> __device__ __forceinline__ void store_row32(TG* dst, const uint32_t (&r)[32]);
+template <> __device__ __forceinline__ void store_row32<float>(float* dst, const uint32_t (&r)[32]) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    *reinterpret_cast<uint4*>(dst + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+}
+template <> __device__ __forceinline__ void store_row32<__nv_bfloat16>(__nv_bfloat16* dst, const uint32_t (&r)[32]) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    uint4 v;
+    v.x = pack_bf16x2(__uint_as_float(r[8 * j]), __uint_as_float(r[8 * j + 1]));
+    v.y = pack_bf16x2(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
+    v.z = pack_bf16x2(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
+    v.w = pack_bf16x2(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
+    *reinterpret_cast<uint4*>(dst + 8 * j) = v;
+  }
+}
+
+// ---- key side -----------------------------------------------------------------------------------
+// grid (chunks, slabs), block 128.
+template <int NH, typename TG>
+__global__ void __launch_bounds__(128, 1)
+k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant__ CUtensorMap map_v,
+               const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ dSbf,
+               const float* __restrict__ dzg, TG* __restrict__ dV, float* __restrict__ dKF, int n, int chunk_tiles,
+               int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  using SL = BwdKSmem<NH>;
+  BwdBars* bars = reinterpret_cast<BwdBars*>(smem + SL::bars);
+  float* dzs = reinterpret_cast<float*>(smem + SL::dz);
+  const int warp = threadIdx.x >> 5;
+  const int chunk = blockIdx.x, slab = blockIdx.y;
+  const int tiles_total = (n + kTile - 1) / kTile;
+  const int tile0 = chunk * chunk_tiles;
+  const int ntiles = min(chunk_tiles, tiles_total - tile0);
+  constexpr int m = NH * 128;
+  constexpr uint32_t kCols = NH * 128;            // TMEM columns (a power of two: 128 or 256)
+
+  if (threadIdx.x == 0) {
+    mbar_init(&bars->full[0], 1);
+    mbar_init(&bars->full[1], 1);
+    mbar_init(&bars->mma, 1);
+    bars->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(&bars->tmem_base, kCols);
+    tmem_relinquish();
+  }
+  load_rows_swizzled(smem + SL::wt, Wt, m);
+  load_rows_swizzled(smem + SL::ds, dSbf + (size_t)slab * m * kD, m);
+  for (int i = threadIdx.x; i < m; i += blockDim.x) dzs[i] = dzg[(size_t)slab * m + i];
+  fence_proxy_async_smem();
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = bars->tmem_base;
+  const uint32_t trow = tmem + ((32u * warp) << 16);     // this warp's lane quarter
+  const uint32_t acc = 64;                               // dV / dK_F live in columns 64..127 of accumulator 0
+
+  const uint32_t hi = smem_desc_hi(1024);
+  const uint32_t wt_k = smem_desc_lo(smem_u32(smem + SL::wt), 16), wt_n = smem_desc_lo(smem_u32(smem + SL::wt), 1024);
+  const uint32_t ds_k = smem_desc_lo(smem_u32(smem + SL::ds), 16), ds_n = smem_desc_lo(smem_u32(smem + SL::ds), 1024);
+  const uint32_t stage_k = smem_desc_lo(smem_u32(smem + SL::stage), 16);
+  constexpr uint32_t kTileStep = kTileBytes >> 4, kStageStep = SL::stage_bytes >> 4;
+  const int slabs = gridDim.y;
+  uint32_t mma_par = 0;
+  int issued = 0;
+  bool ok = true;
+
+  // copies of tile t into stage t & 1: the three K_F planes (plane p of slab s is slab p * slabs + s of
+  // the stacked tensor) and V
+  auto issue_copies = [&](int t) {
+    uint8_t* dst = smem + SL::stage + (t & 1) * SL::stage_bytes;
+    uint64_t* bar = &bars->full[t & 1];
+    const int r0 = (tile0 + t) * kTile;
+    mbar_arrive_expect_tx(bar, 4 * kTileBytes);
+#pragma unroll
+    for (int pl = 0; pl < 3; ++pl) tma_load_3d(dst + pl * kTileBytes, &map_kf, 0, r0, pl * slabs + slab, bar);
+    tma_load_3d(dst + 3 * kTileBytes, &map_v, 0, r0, slab, bar);
+  };
+  if (threadIdx.x == 0 && ntiles > 0) {
+    issue_copies(0);
+    issued = 1;
+  }
+
+  for (int ti = 0; ti < ntiles && ok; ++ti) {
+    const int row0 = (tile0 + ti) * kTile;
+    const int row = row0 + (int)threadIdx.x;
+    const uint32_t x_k = stage_k + (ti & 1) * kStageStep, v_k = x_k + 3 * kTileStep;
+    // ---- copies of the next tile (its stage was released by the barrier that ended tile ti - 1), MMA1
+    if (threadIdx.x == 0 && ti + 1 < ntiles) {
+      issue_copies(ti + 1);
+      issued = ti + 2;
+    }
+    ok = cta_wait(&bars->full[ti & 1], (ti >> 1) & 1, bars, status, kErrBwdCopy);
+    if (!ok) break;
+    if (threadIdx.x == 0) {
+      tc_fence_after_sync();
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+#pragma unroll
+        for (int pl = 0; pl < 3; ++pl)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            mma_ss(tmem + h * 128, smem_desc_join(x_k + pl * kTileStep + 2 * k, hi),
+                   smem_desc_join(wt_k + h * kTileStep + 2 * k, hi), kIdescP, (pl > 0 || k > 0) ? 1u : 0u);
+      mma_commit(&bars->mma);
+    }
+    ok = cta_wait(&bars->mma, mma_par, bars, status, kErrBwdMma);
+    mma_par ^= 1;
+    if (!ok) break;
+    tc_fence_after_sync();
+    // ---- mask and Phi
+    uint32_t mask[NH][4];
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32], p[16];
+        tmem_ld32(trow + h * 128 + 32 * c, r);
+        tmem_ld_wait();
+        reg_fence32(r);
+        uint32_t bits = 0;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) bits |= (__uint_as_float(r[j]) > 0.f ? 1u : 0u) << j;
+        mask[h][c] = bits;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) p[j] = relu_pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+        tmem_st16(trow + h * 128 + 16 * c, p);
+      }
+    }
+    tmem_st_wait();
+    tc_fence_before_sync();
+    __syncthreads();
+    // ---- MMA2: dV
+    if (threadIdx.x == 0) {
+      tc_fence_after_sync();
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          mma_ts(tmem + acc, tmem + h * 128 + k * 8, smem_desc_join(ds_n + h * kTileStep + 128 * k, hi), kIdescC,
+                 (h > 0 || k > 0) ? 1u : 0u);
+      mma_commit(&bars->mma);
+    }
+    ok = cta_wait(&bars->mma, mma_par, bars, status, kErrBwdMma);
+    mma_par ^= 1;
+    if (!ok) break;
+    tc_fence_after_sync();
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      uint32_t r[32];
+      tmem_ld32(trow + acc + 32 * c, r);
+      tmem_ld_wait();
+      reg_fence32(r);
+      if (row < n) store_row32<TG>(dV + ((size_t)slab * n + row) * kD + 32 * c, r);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    // ---- MMA3: G_h = V dS'_h^T
+    if (threadIdx.x == 0) {
+      tc_fence_after_sync();
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          mma_ss(tmem + h * 128, smem_desc_join(v_k + 2 * k, hi), smem_desc_join(ds_k + h * kTileStep + 2 * k, hi),
+                 kIdescP, k > 0);
+      mma_commit(&bars->mma);
+    }
+    ok = cta_wait(&bars->mma, mma_par, bars, status, kErrBwdMma);
+    mma_par ^= 1;
+    if (!ok) break;
+    tc_fence_after_sync();
+    // ---- dB_h = (G_h + dz'_h) (.) mask
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32], p[16];
+        tmem_ld32(trow + h * 128 + 32 * c, r);
+        tmem_ld_wait();
+        reg_fence32(r);
+        const uint32_t bits = mask[h][c];
+        const float* dzr = dzs + h * 128 + 32 * c;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float g0 = ((bits >> (2 * j)) & 1u) ? __uint_as_float(r[2 * j]) + dzr[2 * j] : 0.f;
+          const float g1 = ((bits >> (2 * j + 1)) & 1u) ? __uint_as_float(r[2 * j + 1]) + dzr[2 * j + 1] : 0.f;
+          p[j] = pack_bf16x2(g0, g1);
+        }
+        tmem_st16(trow + h * 128 + 16 * c, p);
+      }
+    }
+    tmem_st_wait();
+    tc_fence_before_sync();
+    __syncthreads();
+    // ---- MMA4: dK_F
+    if (threadIdx.x == 0) {
+      tc_fence_after_sync();
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          mma_ts(tmem + acc, tmem + h * 128 + k * 8, smem_desc_join(wt_n + h * kTileStep + 128 * k, hi), kIdescC,
+                 (h > 0 || k > 0) ? 1u : 0u);
+      mma_commit(&bars->mma);
+    }
+    ok = cta_wait(&bars->mma, mma_par, bars, status, kErrBwdMma);
+    mma_par ^= 1;
+    if (!ok) break;
+    tc_fence_after_sync();
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      uint32_t r[32];
+      tmem_ld32(trow + acc + 32 * c, r);
+      tmem_ld_wait();
+      reg_fence32(r);
+      if (row < n) store_row32<float>(dKF + ((size_t)slab * n + row) * kD + 32 * c, r);
+    }
+    tc_fence_before_sync();
+    __syncthreads();   // the next tile's copies and MMA1 overwrite what this tile read
+  }
+  if (!ok && threadIdx.x == 0) {   // copies may still be in flight
+    for (int t = max(0, issued - 2); t < issued; ++t) mbar_wait_drain(&bars->full[t & 1], (t >> 1) & 1);
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem, kCols);
+  }
+}
+
+// ---- host side ----------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// (slabs x n x 64) bf16 tensor, boxes of 128 rows x 64 columns of one slab, 128-byte swizzle; rows past
+// the end of a slab read as zeros.
+cudaError_t make_tile_map(const void* base, int slabs, int n, CUtensorMap* out) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return cudaErrorNotSupported;
+  const cuuint64_t dims[3] = {kD, (cuuint64_t)n, (cuuint64_t)slabs};
+  const cuuint64_t strides[2] = {kD * 2, (cuuint64_t)n * kD * 2};
+  const cuuint32_t box[3] = {kD, kTile, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+template <int NH, typename TG>
+cudaError_t launch_kside(const Plan& p, const Ws& w, const CUtensorMap& map_kf, const CUtensorMap& map_v, void* dV,
+                         cudaStream_t st) {
+  auto k = k_tc_bwd_kside<NH, TG>;
+  cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdKSmem<NH>::total);
+  if (err != cudaSuccess) return err;
+  dim3 grid(p.bchunks, p.slabs);
+  k<<<grid, 128, BwdKSmem<NH>::total, st>>>(map_kf, map_v, w.Wt, w.dSbf, w.dz, static_cast<TG*>(dV), w.dKF,
+                                            p.cfg.seq_len, p.bchunk_tiles, w.status);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_tc_bwd_kside(const Plan& p, const Ws& w, const void* KF3, const void* V, void* dV, cudaStream_t st,
+                                int* launches) {
+  CUtensorMap map_kf, map_v;
+  cudaError_t err;
+  if ((err = make_tile_map(KF3, 3 * p.slabs, p.cfg.seq_len, &map_kf)) != cudaSuccess) return err;
+  if ((err = make_tile_map(V, p.slabs, p.cfg.seq_len, &map_v)) != cudaSuccess) return err;
+  *launches += 1;
+  if (p.cfg.features == 256)
+    return p.grad_bf16 ? launch_kside<2, __nv_bfloat16>(p, w, map_kf, map_v, dV, st)
+                       : launch_kside<2, float>(p, w, map_kf, map_v, dV, st);
+  return p.grad_bf16 ? launch_kside<1, __nv_bfloat16>(p, w, map_kf, map_v, dV, st)
+                     : launch_kside<1, float>(p, w, map_kf, map_v, dV, st);
+}
+
+}  // namespace wersa
