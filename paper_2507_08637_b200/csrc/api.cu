@@ -68,7 +68,8 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   }
   {
     const int tiles128 = ceil_div(n, 128);
-    p->bchunks = ceil_div(148, p->slabs);
+    p->bchunks = 148 / p->slabs;   // one CTA per SM, a single wave
+    if (p->bchunks < 1) p->bchunks = 1;
     if (p->bchunks > tiles128) p->bchunks = tiles128;
     p->bchunk_tiles = ceil_div(tiles128, p->bchunks);
     p->bchunks = ceil_div(tiles128, p->bchunk_tiles);
@@ -111,8 +112,9 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
     p->off_dKF = take(sizeof(float) * slab_elems);
     p->off_dSbf = take(sizeof(__nv_bfloat16) * slabs * m * kD);
     p->off_KF3 = take(p->use_tc ? 3 * sizeof(__nv_bfloat16) * slab_elems : 0);
+    p->off_QF3 = take(p->use_tc ? 3 * sizeof(__nv_bfloat16) * slab_elems : 0);
   } else {
-    p->off_dS = p->off_dz = p->off_sumdD = p->off_bands = p->off_dqbar = p->off_dQF = p->off_dKF = p->off_dSbf = p->off_KF3 = 0;
+    p->off_dS = p->off_dz = p->off_sumdD = p->off_bands = p->off_dqbar = p->off_dQF = p->off_dKF = p->off_dSbf = p->off_KF3 = p->off_QF3 = 0;
   }
   p->total = off;
   return WERSA_OK;
@@ -144,6 +146,7 @@ Ws resolve(const Plan& p, void* workspace) {
   w.dKF = reinterpret_cast<float*>(b + p.off_dKF);
   w.dSbf = reinterpret_cast<__nv_bfloat16*>(b + p.off_dSbf);
   w.KF3 = reinterpret_cast<__nv_bfloat16*>(b + p.off_KF3);
+  w.QF3 = reinterpret_cast<__nv_bfloat16*>(b + p.off_QF3);
   return w;
 }
 
@@ -312,13 +315,17 @@ wersa_status wersa_backward(wersa_ctx* ctx, const void* Q, const void* K, const 
   const int kind = p.bf16 ? 1 : 0, gkind = p.grad_bf16 ? 1 : 0;
   wersa_status s = begin_pass(ctx, 1, st);
   if (s != WERSA_OK) return s;
-  if (p.use_tc) {   // the tensor-core forward keeps Q_F, K_F on chip: rebuild them (K_F as three bf16 planes)
-    WERSA_STEP(1, "haar_filter_q", launch_haar_filter(p, Q, kind, w.f, w.QF, 0, st, &launches));
+  const int bwd_chunks = p.use_tc ? p.bchunks : p.schunks;   // chunks per slab of the dS', dz', sum dD' partials
+  if (p.use_tc) {
+    // the tensor-core forward keeps Q_F, K_F on chip: rebuild them, as three bf16 planes each
+    WERSA_STEP(1, "haar_filter_q", launch_haar_filter_split3(p, Q, kind, w.f, w.QF3, st, &launches));
     WERSA_STEP(1, "haar_filter_k", launch_haar_filter_split3(p, K, kind, w.f, w.KF3, st, &launches));
+    WERSA_STEP(1, "tc_bwd_qside", launch_tc_bwd_qside(p, w, w.QF3, beta, dO, st, &launches));
+  } else {
+    WERSA_STEP(1, "simt_bwd_qside", launch_simt_bwd_qside(p, w, W, beta, dO, st, &launches));
   }
-  WERSA_STEP(1, "simt_bwd_qside", launch_simt_bwd_qside(p, w, W, beta, dO, st, &launches));
   WERSA_STEP(1, "reduce_partials",
-             launch_reduce_partials(p, w.spart, w.zpart, p.schunks, w.dS, w.dz, p.use_tc ? w.dSbf : nullptr, st,
+             launch_reduce_partials(p, w.spart, w.zpart, bwd_chunks, w.dS, w.dz, p.use_tc ? w.dSbf : nullptr, st,
                                     &launches));
   if (p.use_tc)
     WERSA_STEP(1, "tc_bwd_kside", launch_tc_bwd_kside(p, w, w.KF3, V, dV, st, &launches));
@@ -327,7 +334,8 @@ wersa_status wersa_backward(wersa_ctx* ctx, const void* Q, const void* K, const 
   WERSA_STEP(1, "haar_backward_q", launch_haar_backward(p, w, Q, kind, w.dQF, dQ, gkind, 0, st, &launches));
   WERSA_STEP(1, "haar_backward_k", launch_haar_backward(p, w, K, kind, w.dKF, dK, gkind, 1, st, &launches));
   WERSA_STEP(1, "gate_backward",
-             launch_gate_backward(p, w, beta, gate_w, omega, dbeta, dgate_w, dgate_b, domega, st, &launches));
+             launch_gate_backward(p, w, beta, gate_w, omega, p.slabs * bwd_chunks, dbeta, dgate_w, dgate_b, domega, st,
+                                  &launches));
   if (gate_w != nullptr) WERSA_STEP(1, "add_rowvec", launch_add_rowvec(p, w, dQ, st, &launches));
   ctx->launches_bwd = launches;
   return WERSA_OK;

@@ -38,7 +38,7 @@ struct Plan {
   // workspace offsets (bytes)
   size_t off_status, off_counters, status_bytes, off_qpart, off_qbar, off_sg, off_f, off_spart, off_zpart, off_S, off_z,
       off_Sbf, off_Wt, off_dS, off_dz, off_sumdD, off_bands, off_dqbar, off_QF, off_KF, off_dQF,
-      off_dKF, off_dSbf, off_KF3, total;
+      off_dKF, off_dSbf, off_KF3, off_QF3, total;
   int part_chunks;    // max(schunks, tchunks): leading extent of the partial buffers
 };
 
@@ -49,7 +49,7 @@ struct Ws {   // resolved workspace pointers
   int* status;
   int* counters;   // arrival counters (slabs + batch + slabs ints), zero between launches
   float *qpart, *qbar, *sg, *f, *spart, *zpart, *S, *z, *dS, *dz, *sumdD, *bands, *dqbar;
-  __nv_bfloat16 *Sbf, *Wt, *dSbf, *KF3;
+  __nv_bfloat16 *Sbf, *Wt, *dSbf, *KF3, *QF3;
   float *QF, *KF, *dQF, *dKF;
 };
 Ws resolve(const Plan& p, void* workspace);
@@ -62,7 +62,7 @@ cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const f
                               int* launches);
 // Gate backward: band inner products -> df -> domega, dgate_b, dgate_w, dqbar; dbeta.
 cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, const float* gate_w,
-                                 const float* omega, float* dbeta, float* dgate_w, float* dgate_b,
+                                 const float* omega, int n_sumdD, float* dbeta, float* dgate_w, float* dgate_b,
                                  float* domega, cudaStream_t st, int* launches);
 // dQ[s,t,:] += dqbar[s,:] / n.
 cudaError_t launch_add_rowvec(const Plan& p, const Ws& w, void* dQ, cudaStream_t st, int* launches);
@@ -111,6 +111,11 @@ cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const flo
 // ---- tc_bwd.cu -----------------------------------------------------------------------------
 // Key-side backward on the tensor cores: dV and dK_F from K_F as three bf16 planes, V, the bf16 dS' image
 // (w.dSbf), dz' (w.dz) and the bf16 W^T image (w.Wt).
+// Query-side backward on the tensor cores: dQ_F, and the split-sequence partials of dS', dz' and
+// sum dD' (w.spart, w.zpart, w.sumdD; p.bchunks chunks per slab), from Q_F as three bf16 planes, dO,
+// the bf16 S' image (w.Sbf), z' (w.z) and the bf16 W^T image.
+cudaError_t launch_tc_bwd_qside(const Plan& p, const Ws& w, const void* QF3, const float* beta, const void* dO,
+                                cudaStream_t st, int* launches);
 cudaError_t launch_tc_bwd_kside(const Plan& p, const Ws& w, const void* KF3, const void* V, void* dV,
                                 cudaStream_t st, int* launches);
 

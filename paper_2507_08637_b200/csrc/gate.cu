@@ -327,11 +327,11 @@ size_t static_scratch_floats_needed(const Plan& p) {
 }
 
 cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, const float* gate_w,
-                                 const float* omega, float* dbeta, float* dgate_w, float* dgate_b,
+                                 const float* omega, int n_sumdD, float* dbeta, float* dgate_w, float* dgate_b,
                                  float* domega, cudaStream_t st, int* launches) {
   float* df = w.dqbar + (size_t)p.slabs * kD;   // df lives behind dqbar in the same region
   k_band_reduce<<<p.slabs, 32, 0, st>>>(w.bands, p.slabs, p.htiles, p.cfg.levels, df);
-  k_gate_backward<<<1, kD, 0, st>>>(df, w.sg, w.qbar, gate_w, omega, w.sumdD, p.slabs * p.schunks, beta,
+  k_gate_backward<<<1, kD, 0, st>>>(df, w.sg, w.qbar, gate_w, omega, w.sumdD, n_sumdD, beta,
                                     p.cfg.eps, p.cfg.bw_floor, p.cfg.features, p.cfg.batch, p.cfg.heads,
                                     p.L1, p.cfg.gate_per_head, dbeta, dgate_w, dgate_b, domega, w.dqbar);
   *launches += 2;

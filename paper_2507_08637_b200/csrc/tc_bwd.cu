@@ -10,6 +10,18 @@
 //   MMA3: G_h = V (smem, K-major) * dS'_h^T (same image, K-major)      -> TMEM fp32
 //   threads: dB_h = (G_h + dz'_h) (.) mask                              -> bf16 pairs in place
 //   MMA4: dK_F = sum_h dB_h (TMEM operand) * W_h^T (W^T image, N-major) -> TMEM fp32 -> global
+// Query side, per 128-token tile:
+//   MMA1: A_h = Q_F (three planes) * W_h                                -> TMEM fp32 (token = lane)
+//   threads: mask, Phi_h -> bf16 in place, D' = sum_h Phi_h . z'_h + eps'
+//   MMA2: N' = sum_h Phi_h * S'_h (smem bf16 image, N-major)            -> TMEM fp32
+//   threads: O = N'/D', dN' = dO/D' -> bf16 tile in smem, dD' = -sum_c dO O / D' -> smem
+//   MMA1t: A_h^T = W_h^T * Q_F^T (hi plane)                             -> TMEM fp32 (feature = lane)
+//   threads: Phi_h^T -> bf16 in place, dz'_h += Phi_h^T dD'
+//   MMA5: dS'_h += Phi_h^T (TMEM operand) * dN' (smem tile, N-major)    -> TMEM fp32, kept for the chunk
+//   MMA3: G_h = dN' (smem, K-major) * S'_h^T (same image, K-major)      -> TMEM fp32 (token = lane)
+//   threads: dA_h = (G_h + dD' z'_h) (.) mask                           -> bf16 in place
+//   MMA4: dQ_F = sum_h dA_h * W_h^T (W^T image, N-major)                -> TMEM fp32 -> global
+// and at the end of the chunk the partial dS', dz' and sum of dD' go to the split-sequence buffers.
 // One CTA of 128 threads per SM walks a chunk of tiles one step at a time (thread 0 issues the copies
 // and the MMAs, everybody waits on one mbarrier); the copies of the next tile are in flight meanwhile.
 // TMEM per CTA: 128 columns per feature half; the two 64-column results (dV, dK_F) reuse the upper
@@ -89,6 +101,41 @@ template <> __device__ __forceinline__ void store_row32<__nv_bfloat16>(__nv_bflo
   }
 }
 
+// bf16 hi + lo split of a pair of fp32 values: hi = bf16(x), lo = bf16(x - hi).  Feeding both to the
+// tensor core keeps 16 mantissa bits of an operand that would otherwise be rounded to 8.
+__device__ __forceinline__ void split_pack(float g0, float g1, uint32_t& p_hi, uint32_t& p_lo) {
+  p_hi = pack_bf16x2(g0, g1);
+  p_lo = pack_bf16x2(g0 - __uint_as_float(p_hi << 16), g1 - __uint_as_float(p_hi & 0xFFFF0000u));
+}
+
+// Gradient through the ReLU of one 128-column accumulator (token = lane): x_j = (G_j + s * zr_j) where
+// mask bit j is set, else 0; written back as bf16 hi pairs in columns [0, 64) and lo pairs in columns
+// [64, 128) of the same accumulator (all 128 columns are read before the first one is overwritten).
+__device__ __forceinline__ void relu_grad_split(uint32_t taddr, const uint32_t (&mask)[4], float s,
+                                                const float* __restrict__ zr) {
+  uint32_t r[4][32];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) tmem_ld32(taddr + 32 * c, r[c]);
+  tmem_ld_wait();
+#pragma unroll
+  for (int c = 0; c < 4; ++c) reg_fence32(r[c]);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint32_t ph[16], pl[16];
+    const uint32_t bits = mask[c];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const float g0 = ((bits >> (2 * j)) & 1u) ? fmaf(s, zr[32 * c + 2 * j], __uint_as_float(r[c][2 * j])) : 0.f;
+      const float g1 =
+          ((bits >> (2 * j + 1)) & 1u) ? fmaf(s, zr[32 * c + 2 * j + 1], __uint_as_float(r[c][2 * j + 1])) : 0.f;
+      split_pack(g0, g1, ph[j], pl[j]);
+    }
+    tmem_st16(taddr + 16 * c, ph);
+    tmem_st16(taddr + 64 + 16 * c, pl);
+  }
+  tmem_st_wait();
+}
+
 // ---- key side -----------------------------------------------------------------------------------
 // grid (chunks, slabs), block 128.
 template <int NH, typename TG>
@@ -108,7 +155,7 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
   const int tile0 = chunk * chunk_tiles;
   const int ntiles = min(chunk_tiles, tiles_total - tile0);
   constexpr int m = NH * 128;
-  constexpr uint32_t kCols = NH * 128;            // TMEM columns (a power of two: 128 or 256)
+  constexpr uint32_t kCols = NH * 256;            // TMEM columns: NH accumulators of 128, then dV / dK_F (64)
 
   if (threadIdx.x == 0) {
     mbar_init(&bars->full[0], 1);
@@ -130,7 +177,7 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
   tc_fence_after_sync();
   const uint32_t tmem = bars->tmem_base;
   const uint32_t trow = tmem + ((32u * warp) << 16);     // this warp's lane quarter
-  const uint32_t acc = 64;                               // dV / dK_F live in columns 64..127 of accumulator 0
+  const uint32_t acc = NH * 128;                         // dV / dK_F
 
   const uint32_t hi = smem_desc_hi(1024);
   const uint32_t wt_k = smem_desc_lo(smem_u32(smem + SL::wt), 16), wt_n = smem_desc_lo(smem_u32(smem + SL::wt), 1024);
@@ -247,27 +294,9 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
     mma_par ^= 1;
     if (!ok) break;
     tc_fence_after_sync();
-    // ---- dB_h = (G_h + dz'_h) (.) mask
+    // ---- dB_h = (G_h + dz'_h) (.) mask, as bf16 hi + lo
 #pragma unroll
-    for (int h = 0; h < NH; ++h) {
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32], p[16];
-        tmem_ld32(trow + h * 128 + 32 * c, r);
-        tmem_ld_wait();
-        reg_fence32(r);
-        const uint32_t bits = mask[h][c];
-        const float* dzr = dzs + h * 128 + 32 * c;
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float g0 = ((bits >> (2 * j)) & 1u) ? __uint_as_float(r[2 * j]) + dzr[2 * j] : 0.f;
-          const float g1 = ((bits >> (2 * j + 1)) & 1u) ? __uint_as_float(r[2 * j + 1]) + dzr[2 * j + 1] : 0.f;
-          p[j] = pack_bf16x2(g0, g1);
-        }
-        tmem_st16(trow + h * 128 + 16 * c, p);
-      }
-    }
-    tmem_st_wait();
+    for (int h = 0; h < NH; ++h) relu_grad_split(trow + h * 128, mask[h], 1.f, dzs + h * 128);
     tc_fence_before_sync();
     __syncthreads();
     // ---- MMA4: dK_F
@@ -277,8 +306,10 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
       for (int h = 0; h < NH; ++h)
 #pragma unroll
         for (int k = 0; k < 8; ++k)
-          mma_ts(tmem + acc, tmem + h * 128 + k * 8, smem_desc_join(wt_n + h * kTileStep + 128 * k, hi), kIdescC,
-                 (h > 0 || k > 0) ? 1u : 0u);
+#pragma unroll
+          for (int part = 0; part < 2; ++part)   // hi pairs at columns 0..63, lo pairs at 64..127
+            mma_ts(tmem + acc, tmem + h * 128 + 64 * part + k * 8, smem_desc_join(wt_n + h * kTileStep + 128 * k, hi),
+                   kIdescC, (h > 0 || k > 0 || part > 0) ? 1u : 0u);
       mma_commit(&bars->mma);
     }
     ok = cta_wait(&bars->mma, mma_par, bars, status, kErrBwdMma);
@@ -297,6 +328,326 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
     __syncthreads();   // the next tile's copies and MMA1 overwrite what this tile read
   }
   if (!ok && threadIdx.x == 0) {   // copies may still be in flight
+    for (int t = max(0, issued - 2); t < issued; ++t) mbar_wait_drain(&bars->full[t & 1], (t >> 1) & 1);
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem, kCols);
+  }
+}
+
+// ---- query side ---------------------------------------------------------------------------------
+template <int NH> struct BwdQSmem {
+  static constexpr uint32_t wt = 0;                          // W^T image
+  static constexpr uint32_t simg = wt + NH * kTileBytes;     // S' image
+  static constexpr uint32_t stage = simg + NH * kTileBytes;  // 2 stages x (3 Q_F planes + dO) tiles
+  static constexpr uint32_t stage_bytes = 4 * kTileBytes;
+  static constexpr uint32_t dn = stage + 2 * stage_bytes;    // dN' tiles, bf16 hi and lo
+  static constexpr uint32_t zs = dn + 2 * kTileBytes;        // NH x 128 floats
+  static constexpr uint32_t dd = zs + NH * 512;              // 128 floats
+  static constexpr uint32_t red = dd + 512;                  // 4 floats
+  static constexpr uint32_t bars = red + 64;
+  static constexpr uint32_t total = bars + 64 + 1024;
+};
+
+// grid (chunks, slabs), block 128.  TMEM: accumulator h at columns 128 h (A_h, A_h^T, G_h in turn; the
+// 64-column results N' and dQ_F sit at 384), dS'_h at 256 + 64 h.
+template <int NH>
+__global__ void __launch_bounds__(128, 1)
+k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant__ CUtensorMap map_do,
+               const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ Sbf,
+               const float* __restrict__ zg, const float* __restrict__ beta, float eps, float bw_floor,
+               float* __restrict__ dQF, float* __restrict__ dspart, float* __restrict__ dzpart,
+               float* __restrict__ sumdD, int n, int chunk_tiles, int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  using SL = BwdQSmem<NH>;
+  BwdBars* bars = reinterpret_cast<BwdBars*>(smem + SL::bars);
+  float* zs = reinterpret_cast<float*>(smem + SL::zs);
+  float* dds = reinterpret_cast<float*>(smem + SL::dd);
+  float* red = reinterpret_cast<float*>(smem + SL::red);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunk = blockIdx.x, slab = blockIdx.y;
+  const int tiles_total = (n + kTile - 1) / kTile;
+  const int tile0 = chunk * chunk_tiles;
+  const int ntiles = min(chunk_tiles, tiles_total - tile0);
+  constexpr int m = NH * 128;
+  constexpr uint32_t kCols = 512;
+  constexpr uint32_t kAccS = 256;                 // dS'_h accumulators
+
+  if (threadIdx.x == 0) {
+    mbar_init(&bars->full[0], 1);
+    mbar_init(&bars->full[1], 1);
+    mbar_init(&bars->mma, 1);
+    bars->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(&bars->tmem_base, kCols);
+    tmem_relinquish();
+  }
+  load_rows_swizzled(smem + SL::wt, Wt, m);
+  load_rows_swizzled(smem + SL::simg, Sbf + (size_t)slab * m * kD, m);
+  for (int i = threadIdx.x; i < m; i += blockDim.x) zs[i] = zg[(size_t)slab * m + i];
+  fence_proxy_async_smem();
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = bars->tmem_base;
+  const uint32_t trow = tmem + ((32u * warp) << 16);
+  const uint32_t acc = 384;
+  const float bw = fmaxf(beta[0], bw_floor);
+  const float epsp = eps * (float)m * bw * bw;
+
+  const uint32_t hi = smem_desc_hi(1024);
+  const uint32_t wt_k = smem_desc_lo(smem_u32(smem + SL::wt), 16), wt_n = smem_desc_lo(smem_u32(smem + SL::wt), 1024);
+  const uint32_t s_k = smem_desc_lo(smem_u32(smem + SL::simg), 16), s_n = smem_desc_lo(smem_u32(smem + SL::simg), 1024);
+  const uint32_t dn_k = smem_desc_lo(smem_u32(smem + SL::dn), 16), dn_n = smem_desc_lo(smem_u32(smem + SL::dn), 1024);
+  const uint32_t stage_k = smem_desc_lo(smem_u32(smem + SL::stage), 16);
+  constexpr uint32_t kTileStep = kTileBytes >> 4, kStageStep = SL::stage_bytes >> 4;
+  const int slabs = gridDim.y;
+  uint32_t mma_par = 0;
+  int issued = 0;
+  bool ok = true;
+  float dzacc[NH];                                // feature = thread: dz'_h partial of this chunk
+#pragma unroll
+  for (int h = 0; h < NH; ++h) dzacc[h] = 0.f;
+  float sum_dd = 0.f;                             // token = thread: sum of dD' over this thread's tokens
+
+  auto issue_copies = [&](int t) {
+    uint8_t* dst = smem + SL::stage + (t & 1) * SL::stage_bytes;
+    uint64_t* bar = &bars->full[t & 1];
+    const int r0 = (tile0 + t) * kTile;
+    mbar_arrive_expect_tx(bar, 4 * kTileBytes);
+#pragma unroll
+    for (int pl = 0; pl < 3; ++pl) tma_load_3d(dst + pl * kTileBytes, &map_qf, 0, r0, pl * slabs + slab, bar);
+    tma_load_3d(dst + 3 * kTileBytes, &map_do, 0, r0, slab, bar);
+  };
+  auto wait_mma = [&]() {
+    const bool r = cta_wait(&bars->mma, mma_par, bars, status, kErrBwdMma);
+    mma_par ^= 1;
+    if (r) tc_fence_after_sync();
+    return r;
+  };
+  if (threadIdx.x == 0 && ntiles > 0) {
+    issue_copies(0);
+    issued = 1;
+  }
+
+  for (int ti = 0; ti < ntiles && ok; ++ti) {
+    const int row0 = (tile0 + ti) * kTile;
+    const int row = row0 + (int)threadIdx.x;
+    const uint32_t x_k = stage_k + (ti & 1) * kStageStep;
+    const uint8_t* do_tile = smem + SL::stage + (ti & 1) * SL::stage_bytes + 3 * kTileBytes;
+    if (threadIdx.x == 0 && ti + 1 < ntiles) {
+      issue_copies(ti + 1);
+      issued = ti + 2;
+    }
+    ok = cta_wait(&bars->full[ti & 1], (ti >> 1) & 1, bars, status, kErrBwdCopy);
+    if (!ok) break;
+    // ---- MMA1: A_h (three planes)
+    if (threadIdx.x == 0) {
+      tc_fence_after_sync();
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+#pragma unroll
+        for (int pl = 0; pl < 3; ++pl)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            mma_ss(tmem + h * 128, smem_desc_join(x_k + pl * kTileStep + 2 * k, hi),
+                   smem_desc_join(wt_k + h * kTileStep + 2 * k, hi), kIdescP, (pl > 0 || k > 0) ? 1u : 0u);
+      mma_commit(&bars->mma);
+    }
+    if (!(ok = wait_mma())) break;
+    // ---- mask, Phi, denominator
+    uint32_t mask[NH][4];
+    float den = epsp;
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32], p[16];
+        tmem_ld32(trow + h * 128 + 32 * c, r);
+        tmem_ld_wait();
+        reg_fence32(r);
+        uint32_t bits = 0;
+        const float* zr = zs + h * 128 + 32 * c;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float a = __uint_as_float(r[j]);
+          bits |= (a > 0.f ? 1u : 0u) << j;
+          den = fmaf(fmaxf(a, 0.f), zr[j], den);
+        }
+        mask[h][c] = bits;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) p[j] = relu_pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+        tmem_st16(trow + h * 128 + 16 * c, p);
+      }
+    }
+    tmem_st_wait();
+    tc_fence_before_sync();
+    __syncthreads();
+    // ---- MMA2: N'
+    if (threadIdx.x == 0) {
+      tc_fence_after_sync();
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          mma_ts(tmem + acc, tmem + h * 128 + k * 8, smem_desc_join(s_n + h * kTileStep + 128 * k, hi), kIdescC,
+                 (h > 0 || k > 0) ? 1u : 0u);
+      mma_commit(&bars->mma);
+    }
+    if (!(ok = wait_mma())) break;
+    // ---- O, dN' (-> smem tile, bf16), dD'
+    const float inv = row < n ? 1.f / den : 0.f;   // rows past the end contribute nothing
+    float dd = 0.f;
+    {
+      uint8_t* dn_tile = smem + SL::dn;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
+        tmem_ld32(trow + acc + 32 * c, r);
+        tmem_ld_wait();
+        reg_fence32(r);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {   // 16-byte chunk 4 c + q of this token's row: 8 columns
+          const uint4 raw = *reinterpret_cast<const uint4*>(do_tile + swz128(threadIdx.x, 4 * c + q));
+          const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+          uint32_t oh[4], ol[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float g0 = __uint_as_float(u[i] << 16), g1 = __uint_as_float(u[i] & 0xFFFF0000u);
+            const float o0 = __uint_as_float(r[8 * q + 2 * i]) * inv, o1 = __uint_as_float(r[8 * q + 2 * i + 1]) * inv;
+            dd = fmaf(g0, o0, dd);
+            dd = fmaf(g1, o1, dd);
+            split_pack(g0 * inv, g1 * inv, oh[i], ol[i]);
+          }
+          *reinterpret_cast<uint4*>(dn_tile + swz128(threadIdx.x, 4 * c + q)) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+          *reinterpret_cast<uint4*>(dn_tile + kTileBytes + swz128(threadIdx.x, 4 * c + q)) =
+              make_uint4(ol[0], ol[1], ol[2], ol[3]);
+        }
+      }
+    }
+    dd = -dd * inv;
+    dds[threadIdx.x] = dd;
+    sum_dd += dd;
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    // ---- MMA1t: A_h^T (feature = lane), hi plane only
+    if (threadIdx.x == 0) {
+      tc_fence_after_sync();
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          mma_ss(tmem + h * 128, smem_desc_join(wt_k + h * kTileStep + 2 * k, hi), smem_desc_join(x_k + 2 * k, hi),
+                 kIdescP, k > 0);
+      mma_commit(&bars->mma);
+    }
+    if (!(ok = wait_mma())) break;
+    // ---- Phi^T, dz' partial
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32], p[16];
+        tmem_ld32(trow + h * 128 + 32 * c, r);
+        tmem_ld_wait();
+        reg_fence32(r);
+        const float* ddr = dds + 32 * c;
+        float part = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) part = fmaf(fmaxf(__uint_as_float(r[j]), 0.f), ddr[j], part);
+        dzacc[h] += part;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) p[j] = relu_pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+        tmem_st16(trow + h * 128 + 16 * c, p);
+      }
+    }
+    tmem_st_wait();
+    tc_fence_before_sync();
+    __syncthreads();
+    // ---- MMA5: dS'_h += Phi_h^T dN'   and   MMA3: G_h = dN' S'_h^T (after MMA5 has read Phi_h^T)
+    if (threadIdx.x == 0) {
+      tc_fence_after_sync();
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+#pragma unroll
+          for (int part = 0; part < 2; ++part)   // dN' hi tile, then lo tile
+            mma_ts(tmem + kAccS + h * 64, tmem + h * 128 + k * 8, smem_desc_join(dn_n + part * kTileStep + 128 * k, hi),
+                   kIdescC, (ti > 0 || k > 0 || part > 0) ? 1u : 0u);
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+#pragma unroll
+        for (int part = 0; part < 2; ++part)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            mma_ss(tmem + h * 128, smem_desc_join(dn_k + part * kTileStep + 2 * k, hi),
+                   smem_desc_join(s_k + h * kTileStep + 2 * k, hi), kIdescP, (part > 0 || k > 0) ? 1u : 0u);
+      mma_commit(&bars->mma);
+    }
+    if (!(ok = wait_mma())) break;
+    // ---- dA_h = (G_h + dD' z'_h) (.) mask, as bf16 hi + lo
+#pragma unroll
+    for (int h = 0; h < NH; ++h) relu_grad_split(trow + h * 128, mask[h], dd, zs + h * 128);
+    tc_fence_before_sync();
+    __syncthreads();
+    // ---- MMA4: dQ_F
+    if (threadIdx.x == 0) {
+      tc_fence_after_sync();
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+#pragma unroll
+          for (int part = 0; part < 2; ++part)
+            mma_ts(tmem + acc, tmem + h * 128 + 64 * part + k * 8, smem_desc_join(wt_n + h * kTileStep + 128 * k, hi),
+                   kIdescC, (h > 0 || k > 0 || part > 0) ? 1u : 0u);
+      mma_commit(&bars->mma);
+    }
+    if (!(ok = wait_mma())) break;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      uint32_t r[32];
+      tmem_ld32(trow + acc + 32 * c, r);
+      tmem_ld_wait();
+      reg_fence32(r);
+      if (row < n) store_row32<float>(dQF + ((size_t)slab * n + row) * kD + 32 * c, r);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+  }
+  // ---- partial dS', dz', sum dD' of this chunk (zeros if the chunk gave up)
+  const size_t pidx = (size_t)slab * gridDim.x + chunk;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum_dd += __shfl_xor_sync(0xffffffffu, sum_dd, o);
+  if (lane == 0) red[warp] = sum_dd;
+  __syncthreads();
+  if (threadIdx.x == 0) sumdD[pidx] = ok ? (red[0] + red[1]) + (red[2] + red[3]) : 0.f;
+  if (ok && ntiles > 0) {
+    tc_fence_after_sync();
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+      const int feat = h * 128 + threadIdx.x;
+      float* dst = dspart + (pidx * m + feat) * kD;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
+        tmem_ld32(trow + kAccS + h * 64 + 32 * c, r);
+        tmem_ld_wait();
+        reg_fence32(r);
+        store_row32<float>(dst + 32 * c, r);
+      }
+      dzpart[pidx * m + feat] = dzacc[h];
+    }
+  }
+  if (!ok && threadIdx.x == 0) {
     for (int t = max(0, issued - 2); t < issued; ++t) mbar_wait_drain(&bars->full[t & 1], (t >> 1) & 1);
   }
   tc_fence_before_sync();
@@ -351,7 +702,30 @@ cudaError_t launch_kside(const Plan& p, const Ws& w, const CUtensorMap& map_kf, 
   return cudaGetLastError();
 }
 
+template <int NH>
+cudaError_t launch_qside(const Plan& p, const Ws& w, const CUtensorMap& map_qf, const CUtensorMap& map_do,
+                         const float* beta, cudaStream_t st) {
+  auto k = k_tc_bwd_qside<NH>;
+  cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdQSmem<NH>::total);
+  if (err != cudaSuccess) return err;
+  dim3 grid(p.bchunks, p.slabs);
+  k<<<grid, 128, BwdQSmem<NH>::total, st>>>(map_qf, map_do, w.Wt, w.Sbf, w.z, beta, p.cfg.eps, p.cfg.bw_floor, w.dQF,
+                                            w.spart, w.zpart, w.sumdD, p.cfg.seq_len, p.bchunk_tiles, w.status);
+  return cudaGetLastError();
+}
+
 }  // namespace
+
+cudaError_t launch_tc_bwd_qside(const Plan& p, const Ws& w, const void* QF3, const float* beta, const void* dO,
+                                cudaStream_t st, int* launches) {
+  CUtensorMap map_qf, map_do;
+  cudaError_t err;
+  if ((err = make_tile_map(QF3, 3 * p.slabs, p.cfg.seq_len, &map_qf)) != cudaSuccess) return err;
+  if ((err = make_tile_map(dO, p.slabs, p.cfg.seq_len, &map_do)) != cudaSuccess) return err;
+  *launches += 1;
+  return p.cfg.features == 256 ? launch_qside<2>(p, w, map_qf, map_do, beta, st)
+                               : launch_qside<1>(p, w, map_qf, map_do, beta, st);
+}
 
 cudaError_t launch_tc_bwd_kside(const Plan& p, const Ws& w, const void* KF3, const void* V, void* dV, cudaStream_t st,
                                 int* launches) {
