@@ -296,7 +296,7 @@ def main():
     # DRAM bytes per token-head of one launch, from the ncu capture summarised in
     # profiles/forward_cfg5_ncu_full_set.md (dram__bytes_read.sum + dram__bytes_write.sum on the cfg5
     # forward, 524288 token-heads; traffic grows in proportion to the token-heads of a launch)
-    ncu_bytes_per_th = {"qmean_gate": 129.5, "tc_kside": 264.1, "tc_qside": 166.3}
+    ncu_bytes_per_th = {"qmean_gate": 128.7, "tc_kside": 264.0, "tc_qside": 165.4}
     if dom in flops:
         if dom.startswith("tc_"):
             bound, peak, unit = "tensor", float(peaks["bf16_tflops"]), "TFLOP/s"
@@ -340,6 +340,24 @@ def main():
         "roofline": roofline,
         "path_roofline": path,
     }
+    if cfg.get("backward"):   # training-shaped workload: also time forward + backward (device events)
+        ctx_t = wersa.wersa_create(cfg["B"], cfg["H"], cfg["n"], cfg["d"], cfg["L"], cfg["m"], dtype=dtype,
+                                   grad_dtype="f32", device=local_rank,
+                                   flags=wersa.WERSA_FLAG_SIMT_ONLY if args.simt else 0)
+        for _ in range(3):
+            wersa.wersa_forward(ctx_t, *fargs, out=O, stream=stream)
+            wersa.wersa_backward(ctx_t, *fargs, dev["dO"], stream=stream)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(20):
+            wersa.wersa_forward(ctx_t, *fargs, out=O, stream=stream)
+            wersa.wersa_backward(ctx_t, *fargs, dev["dO"], stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        tms = e0.elapsed_time(e1) / 20
+        line["training_step"] = {"ms_per_step": tms, "tokens_per_s": cfg["B"] * cfg["n"] / (tms * 1e-3),
+                                 "what": "forward + backward, device-timed, 20 steps",
+                                 "launches": ctx_t.launch_count(0) + ctx_t.launch_count(1)}
     if not args.no_cpu_baseline:
         rate, desc, used, _ = oracle_sample_rate(cfg, inp, 15.0)
         line["cpu_baseline"] = {"value": rate, "unit": "tokens/s", "cores": used, "kind": "oracle",

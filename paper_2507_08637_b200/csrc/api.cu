@@ -99,7 +99,7 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   p->off_Sbf = take(sizeof(__nv_bfloat16) * slabs * m * kD);
   p->off_Wt = take(sizeof(__nv_bfloat16) * (size_t)m * kD);
   const size_t slab_elems = slabs * (size_t)n * kD;
-  const bool need_xf = !p->use_tc || p->with_backward;
+  const bool need_xf = !p->use_tc;   // the tensor-core kernels filter on chip (forward) or read bf16 planes (backward)
   p->off_QF = take(need_xf ? sizeof(float) * slab_elems : 0);
   p->off_KF = take(need_xf ? sizeof(float) * slab_elems : 0);
   if (p->with_backward) {
