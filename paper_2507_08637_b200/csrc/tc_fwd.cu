@@ -41,7 +41,9 @@ constexpr int kND1 = 3;                           // D1 accumulators in TMEM (co
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kAccCol = 384;                 // S' halves (key side) / N' of two tiles (query side)
 constexpr uint32_t kIdesc1 = make_idesc_bf16(128, 128, false, false);  // both operands K-major
-constexpr uint32_t kIdesc2 = make_idesc_bf16(128, 64, false, true);    // B = V or S', N-major
+constexpr uint32_t kIdesc2 = make_idesc_bf16(128, 64, false, true);    // key side: B = V, N-major
+constexpr uint32_t kIdesc2Q = make_idesc_bf16(128, 80, false, false);  // query side: B = [S' | z' | 0]^T, K-major
+constexpr uint32_t kSztBlockBytes = 80 * 128;      // one 64-feature K block of that operand: 80 rows of 128 bytes
 
 constexpr int kWarpTma = 0, kWarpMma = 1, kWarpTmaV = 2, kWarpMma2 = 3;
 constexpr int kReluWarp0 = 4, kAuxWarp0 = 12;       // 8 ReLU warps, 8 Haar warps
@@ -49,6 +51,17 @@ constexpr int kThreads = 32 * (kAuxWarp0 + 8);      // 640 threads, 96 registers
 // Registers per thread after the roles have traded: the Haar step holds a 256 x 64 block in registers
 // and gets what the producer / MMA warpgroup gives up.
 constexpr int kRegsCtl = 40, kRegsAux = 120;
+// Query side: four more warps (12-15) form the epilogue, the Haar warps follow (16-23).  768 threads
+// start with kRegsLaunchQ registers each; the roles re-split exactly that pool (an increase waits
+// until other warps of the CTA have released enough, so the split must never exceed it).
+constexpr int kEpiWarp0Q = 12, kAuxWarp0Q = 16;
+constexpr int kThreadsQ = 32 * (kAuxWarp0Q + 8);
+constexpr int kRegsLaunchQ = 80;   // 65536 / 768 rounded down to a multiple of 8
+constexpr int kRegsCtlQ = 40, kRegsReluQ = 56, kRegsEpiQ = 88;
+static_assert(4 * kRegsCtlQ + 8 * kRegsReluQ + 4 * kRegsEpiQ + 8 * kRegsAux <= (kThreadsQ / 32) * kRegsLaunchQ,
+              "roles may not claim more registers than the CTA was launched with");
+// Key side: 640 threads start with 96 registers each.
+static_assert(4 * kRegsCtl + 8 * 96 + 8 * kRegsAux <= (kThreads / 32) * 96, "key-side register split");
 
 // Named barriers (id 0 is __syncthreads).
 enum { kBarZsum = 1, kBarCoef = 3, kBarHaar = 4, kBarOut0 = 5 /* and 6: one per ReLU warpgroup */ };
@@ -62,7 +75,7 @@ struct alignas(8) KsideBars {
 };
 struct alignas(8) QsideBars {
   uint64_t x_full[kNXQ], x_empty[kNXQ], xf_ready[kNF];
-  uint64_t d1_full[6], phi_ready[kND1], d1_free[kND1], d2_full[2], d2_free[2], den_ready[2];
+  uint64_t d1_full[6], phi_ready[kND1], d1_free[kND1], d2_full, d2_free;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -79,14 +92,12 @@ template <int NH> struct KsideSmem {
 };
 template <int NH> struct QsideSmem {
   static constexpr uint32_t wt = 0;
-  static constexpr uint32_t simg = wt + NH * kTileBytes;
-  static constexpr uint32_t x = simg + NH * kTileBytes;
+  static constexpr uint32_t simg = wt + NH * kTileBytes;          // 2 NH K blocks of [S' | z' | 0]^T
+  static constexpr uint32_t x = simg + 2 * NH * kSztBlockBytes;
   static constexpr uint32_t ost = x + kNXQ * kTileBytes;           // 2 output staging tiles
   static constexpr uint32_t xch = ost + 2 * kTileBytes;          // 2 x 8 x 64 floats
   static constexpr uint32_t hcoef = xch + 4096;                  // kHaarCoefPairs pairs
-  static constexpr uint32_t zs = hcoef + 1024;                   // NH*128 floats
-  static constexpr uint32_t den = zs + NH * 512;                 // 2 x NH x 128 floats
-  static constexpr uint32_t bars = den + 2 * NH * 512;
+  static constexpr uint32_t bars = hcoef + 1024;
   static constexpr uint32_t total = bars + 512 + 1024;
 };
 
@@ -547,65 +558,69 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
 }
 
 // ---- query side ---------------------------------------------------------------------------------
-// Epilogue of tile t by the ReLU warpgroup g = t & 1 (128 threads, thread = token row): waits for N'
-// and the denominators, scales, rounds to bf16 into the warpgroup's own staging tile and stores it
-// with TMA.  The group barrier is executed whether or not `ok` holds.
-template <int NH, typename SL>
-__device__ __forceinline__ bool qside_write_tile(QsideBars* bars, uint8_t* smem, const float* den,
-                                                 const CUtensorMap* map_o, uint32_t tmem, float epsp, int t, int row0,
-                                                 int n, int slab, int g, int gt, bool ok, volatile int* abort_flag,
-                                                 int* status) {
-  const uint32_t lane_base = 32u * ((gt >> 5) & 3);
-  const int row = gt;                               // token within the tile = TMEM lane
-  const int p = t & 1;                              // == g
-  if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d2_full[p], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
-  if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->den_ready[p], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
-  // the staging tile was last used by tile t-2: its TMA store must have finished reading
-  if (gt == 0) bulk_wait_group_read0();
-  named_bar_sync(kBarOut0 + g, 128);
-  uint8_t* ost = smem + SL::ost + p * kTileBytes;
-  if (ok) {
-    tc_fence_after_sync();
-    const uint32_t base = tmem + (lane_base << 16) + kAccCol + p * 64;
-    float dsum = epsp;
-#pragma unroll
-    for (int h = 0; h < NH; ++h) dsum += den[(p * NH + h) * 128 + row];
-    const float inv = 1.f / dsum;
-    const f32x2 inv2 = pk2(inv, inv);
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      uint32_t r[32];
-      tmem_ld32(base + 32 * half, r);
-      tmem_ld_wait();
-      reg_fence32(r);
-      if (half == 1) {   // N' and the denominators of this tile parity are free again
-        tc_fence_before_sync();
-        warp_arrive(&bars->d2_free[p]);
-      }
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint4 v;
-        v.x = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c]), __uint_as_float(r[8 * c + 1])), inv2));
-        v.y = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c + 2]), __uint_as_float(r[8 * c + 3])), inv2));
-        v.z = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c + 4]), __uint_as_float(r[8 * c + 5])), inv2));
-        v.w = pack2_bf16(mul2(pk2(__uint_as_float(r[8 * c + 6]), __uint_as_float(r[8 * c + 7])), inv2));
-        *reinterpret_cast<uint4*>(ost + swz128(row, 4 * half + c)) = v;
-      }
-    }
-    fence_proxy_async_smem();
+// The denominator rides on the tensor core: the B operand of MMA2 is the K-major image of
+// [S' | z' | 0]^T (80 rows of m features), so that column 64 of the accumulator is D' = Phi z'.
+//
+// Builds that image in shared memory from the bf16 S' (m x 64, row-major) and the fp32 z' of the slab:
+// 64-feature K blocks of 80 rows x 128 bytes (rows 0-63 = columns of S', row 64 = z', rows 65-79 = 0),
+// 128-byte swizzle.
+__device__ __forceinline__ void load_szt_image(uint8_t* dst, const __nv_bfloat16* __restrict__ Sbf,
+                                               const float* __restrict__ z, int m) {
+  for (int i = threadIdx.x; i < m * (kD / 2); i += blockDim.x) {   // two adjacent columns of one feature
+    const int f = i / (kD / 2), c = 2 * (i % (kD / 2));
+    const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(Sbf + (size_t)f * kD + c);
+    uint8_t* blk = dst + (f >> 6) * kSztBlockBytes + (f & 7) * 2;
+    *reinterpret_cast<__nv_bfloat16*>(blk + swz128(c, (f & 63) >> 3)) = v.x;
+    *reinterpret_cast<__nv_bfloat16*>(blk + swz128(c + 1, (f & 63) >> 3)) = v.y;
   }
-  named_bar_sync(kBarOut0 + g, 128);
-  if (gt == 0 && ok && row0 < n) {   // rows past n are clipped by the store
-    tma_store_3d(map_o, ost, 0, row0, slab);
-    bulk_commit_group();
+  for (int f = threadIdx.x; f < m; f += blockDim.x)
+    *reinterpret_cast<__nv_bfloat16*>(dst + (f >> 6) * kSztBlockBytes + swz128(64, (f & 63) >> 3) + (f & 7) * 2) =
+        __float2bfloat16_rn(z[f]);
+  for (int i = threadIdx.x; i < (m >> 6) * 15 * 8; i += blockDim.x) {   // 16-byte chunks of rows 65-79
+    const int kb = i / 120, r = 65 + (i % 120) / 8, c = i & 7;
+    *reinterpret_cast<uint4*>(dst + kb * kSztBlockBytes + r * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
   }
-  return ok;
 }
 
-// grid (chunks, slabs), block 640.  TMEM: D1[3] at columns 0 / 128 / 256, N' of tile parity p at
-// 384 + 64 p.  The partial denominators of a tile travel through shared memory (den).
+// ReLU pass over one 128-column D1 accumulator in 16-column steps (a smaller register footprint than
+// relu_unit): fp32 TMEM -> bf16 pairs back into columns [0, 64) of the same accumulator.
+__device__ __forceinline__ void reg_fence16(uint32_t (&r)[16]) {
+  asm volatile(""
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
+                 "+r"(r[15])
+               :
+               : "memory");
+}
+__device__ __forceinline__ void relu_pack16(const uint32_t (&r)[16], uint32_t (&p)[8]) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) p[j] = relu_pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+}
+__device__ __forceinline__ void relu_unit_plain(uint32_t taddr) {
+  uint32_t a[16], b[16], p[8];
+  tmem_ld16(taddr, a);
+#pragma unroll
+  for (int c = 0; c < 8; c += 2) {
+    tmem_ld_wait();
+    reg_fence16(a);
+    tmem_ld16(taddr + 16 * (c + 1), b);
+    relu_pack16(a, p);
+    tmem_st8(taddr + 8 * c, p);
+    tmem_ld_wait();
+    reg_fence16(b);
+    if (c + 2 < 8) tmem_ld16(taddr + 16 * (c + 2), a);
+    relu_pack16(b, p);
+    tmem_st8(taddr + 8 * (c + 1), p);
+  }
+  tmem_st_wait();
+}
+
+// grid (chunks, slabs), block 768.  TMEM: D1[3] at columns 0 / 128 / 256, [N' | D'] of the current tile
+// at 384 .. 463.  Warps 12-15 are the epilogue: they drain the accumulator of a tile as soon as its
+// last MMA2 has completed (which frees it for the next tile), scale by 1 / (D' + eps'), round to bf16
+// into one of two staging tiles and store it with TMA.
 template <int NH>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsQ, 1)
 k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
            const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ Sbf,
            const float* __restrict__ zg, const float* __restrict__ f, const float* __restrict__ beta, float eps,
@@ -614,8 +629,6 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   using SL = QsideSmem<NH>;
   QsideBars* bars = reinterpret_cast<QsideBars*>(smem + SL::bars);
-  float* zs = reinterpret_cast<float*>(smem + SL::zs);
-  float* den = reinterpret_cast<float*>(smem + SL::den);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunk = blockIdx.x, slab = blockIdx.y;
   const int blk0 = chunk * chunk_blocks;
@@ -635,11 +648,8 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       mbar_init(&bars->phi_ready[b], 4);
       mbar_init(&bars->d1_free[b], 1);
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(&bars->d2_full[b], 1);
-      mbar_init(&bars->d2_free[b], 4);
-      mbar_init(&bars->den_ready[b], 4 * NH);
-    }
+    mbar_init(&bars->d2_full, 1);
+    mbar_init(&bars->d2_free, 4);
     bars->abort_flag = 0;
     fence_mbar_init();
   }
@@ -648,8 +658,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     tmem_relinquish();
   }
   load_rows_swizzled(smem + SL::wt, Wt, m);
-  load_rows_swizzled(smem + SL::simg, Sbf + (size_t)slab * m * kD, m);
-  for (int i = threadIdx.x; i < m; i += blockDim.x) zs[i] = zg[(size_t)slab * m + i];
+  load_szt_image(smem + SL::simg, Sbf + (size_t)slab * m * kD, zg + (size_t)slab * m, m);
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
@@ -658,7 +667,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
   volatile int* abort_flag = &bars->abort_flag;
 
   if (warp < kReluWarp0) {
-    reg_dec<kRegsCtl>();
+    reg_dec<kRegsCtlQ>();
     if (warp == kWarpTma && lane == 0) {
       int issued = 0;
       for (int b = 0; b < ntiles; ++b) {   // b counts 128-token tiles here
@@ -710,75 +719,110 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
         fpar ^= (fs == 0);
       }
     } else if (warp == kWarpMma2 && lane == 0) {
-      // MMA2 of every unit: N'[tile parity] (+)= Phi (the unit's D1 buffer, bf16 pairs) * S' half h.
-      constexpr uint32_t kTileStep = kTileBytes >> 4;
+      // MMA2 of every unit: [N' | D'] (+)= Phi (the unit's D1 buffer, bf16 pairs) * [S' | z' | 0] half h.
       const uint32_t hi = smem_desc_hi(1024);
-      const uint32_t s_lo = smem_desc_lo(smem_u32(smem + SL::simg), 1024);
+      const uint32_t s_lo = smem_desc_lo(smem_u32(smem + SL::simg), 16);
+      const uint32_t d2 = tmem + kAccCol;
       uint32_t p3 = 0, ppar = 0;
       bool ok = true;
       for (int t = 0; t < ntiles && ok; ++t) {
-        if (t >= 2) {   // N' of this tile parity must have been drained (tile t - 2)
-          ok = mbar_wait(&bars->d2_free[t & 1], ((t >> 1) - 1) & 1, abort_flag, status, kErrMma);
+        if (t >= 1) {   // the accumulator of tile t - 1 must have been drained
+          ok = mbar_wait(&bars->d2_free, (t - 1) & 1, abort_flag, status, kErrMma);
           if (!ok) break;
+          tc_fence_after_sync();
         }
-        const uint32_t d2 = tmem + kAccCol + (t & 1) * 64;
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
           ok = mbar_wait(&bars->phi_ready[p3], ppar, abort_flag, status, kErrMma);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t a_tm = tmem + p3 * 128, b_lo = s_lo + h * kTileStep;
+          const uint32_t a_tm = tmem + p3 * 128;
 #pragma unroll
-          for (int k = 0; k < 8; ++k)
-            mma_ts(d2, a_tm + k * 8, smem_desc_join(b_lo + 128 * k, hi), kIdesc2, (h > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < 8; ++k) {   // K block 2 h + k / 4, 32 bytes per step of 16 features inside it
+            const uint32_t b_lo = s_lo + (2 * h + (k >> 2)) * (kSztBlockBytes >> 4) + 2 * (k & 3);
+            mma_ts(d2, a_tm + k * 8, smem_desc_join(b_lo, hi), kIdesc2Q, (h > 0 || k > 0) ? 1u : 0u);
+          }
           mma_commit(&bars->d1_free[p3]);
           p3 = p3 == kND1 - 1 ? 0 : p3 + 1;
           ppar ^= (p3 == 0);
         }
-        if (ok) mma_commit(&bars->d2_full[t & 1]);
+        if (ok) mma_commit(&bars->d2_full);
       }
     }
-  } else if (warp >= kReluWarp0 && warp < kAuxWarp0) {
+  } else if (warp < kEpiWarp0Q) {
+    reg_dec<kRegsReluQ>();
     const int g = (warp - kReluWarp0) >> 2;
-    const int gt = threadIdx.x - 32 * kReluWarp0 - 128 * g;   // 0..127 inside the warpgroup
     const uint32_t lane_base = 32u * (warp & 3);
-    const int row = lane_base + lane;               // token within the tile = TMEM lane (== gt)
-    const float bw = fmaxf(beta[0], bw_floor);
-    const float epsp = eps * (float)m * bw * bw;
-    int next_out = g;                               // next tile this warpgroup writes out (tiles of parity g)
     bool ok = true;
     for (int u = g; u < units; u += 2) {
-      const int t = u / NH, h = u % NH;
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d1_full[u % 6], (u / 6) & 1, abort_flag, status, kErrRelu));
-      float dot = 0.f;
       if (ok) {
         tc_fence_after_sync();
-        dot = relu_unit<true>(tmem + (lane_base << 16) + (u % kND1) * 128, zs + h * 128);
+        relu_unit_plain(tmem + (lane_base << 16) + (u % kND1) * 128);
         tc_fence_before_sync();
         warp_arrive(&bars->phi_ready[u % kND1]);
       }
-      // write out this warpgroup's earlier tiles (all their units were handed to the MMA issuer before
-      // this one); this is also what frees the denominator slots waited for below.  Not conditional on
-      // `ok`: the group barriers inside must see all 128 threads.
-      for (; next_out < t; next_out += 2)
-        ok = qside_write_tile<NH, SL>(bars, smem, den, &map_o, tmem, epsp, next_out, blk0 * kBlk + next_out * kTile, n,
-                                      slab, g, gt, ok, abort_flag, status);
-      // the denominator slots of this tile parity must have been read by the epilogue of tile t-2
-      if (ok && t >= 2)
-        ok = __all_sync(0xffffffffu,
-                        mbar_wait(&bars->d2_free[t & 1], ((t >> 1) - 1) & 1, abort_flag, status, kErrRelu));
+    }
+  } else if (warp < kAuxWarp0Q) {
+    reg_inc<kRegsEpiQ>();
+    const int et = threadIdx.x - 32 * kEpiWarp0Q;     // 0..127 = token row of the tile = TMEM lane
+    const uint32_t lane_base = 32u * (warp & 3);
+    const float bw = fmaxf(beta[0], bw_floor);
+    const float epsp = eps * (float)m * bw * bw;
+    const uint32_t base = tmem + (lane_base << 16) + kAccCol;
+    bool ok = true;
+    for (int t = 0; t < ntiles; ++t) {
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d2_full, t & 1, abort_flag, status, kErrEpilogue));
+      uint32_t r0[32], r1[32], dd = 0;
       if (ok) {
-        den[((t & 1) * NH + h) * 128 + row] = dot;
-        warp_arrive(&bars->den_ready[t & 1]);
+        tc_fence_after_sync();
+        tmem_ld32(base, r0);
+        tmem_ld32(base + 32, r1);
+        tmem_ld1(base + 64, dd);
+        tmem_ld_wait();
+        reg_fence32(r0);
+        reg_fence32(r1);
+        tc_fence_before_sync();
+        warp_arrive(&bars->d2_free);
+      }
+      // the staging tile was last used by tile t - 2: its TMA store must have finished reading
+      if (et == 0) bulk_wait_group_read1();
+      named_bar_sync(kBarOut0, 128);
+      uint8_t* ost = smem + SL::ost + (t & 1) * kTileBytes;
+      if (ok) {
+        const float inv = 1.f / (__uint_as_float(dd) + epsp);
+        const f32x2 inv2 = pk2(inv, inv);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint4 v;
+          v.x = pack2_bf16(mul2(pk2(__uint_as_float(r0[8 * c]), __uint_as_float(r0[8 * c + 1])), inv2));
+          v.y = pack2_bf16(mul2(pk2(__uint_as_float(r0[8 * c + 2]), __uint_as_float(r0[8 * c + 3])), inv2));
+          v.z = pack2_bf16(mul2(pk2(__uint_as_float(r0[8 * c + 4]), __uint_as_float(r0[8 * c + 5])), inv2));
+          v.w = pack2_bf16(mul2(pk2(__uint_as_float(r0[8 * c + 6]), __uint_as_float(r0[8 * c + 7])), inv2));
+          *reinterpret_cast<uint4*>(ost + swz128(et, c)) = v;
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint4 v;
+          v.x = pack2_bf16(mul2(pk2(__uint_as_float(r1[8 * c]), __uint_as_float(r1[8 * c + 1])), inv2));
+          v.y = pack2_bf16(mul2(pk2(__uint_as_float(r1[8 * c + 2]), __uint_as_float(r1[8 * c + 3])), inv2));
+          v.z = pack2_bf16(mul2(pk2(__uint_as_float(r1[8 * c + 4]), __uint_as_float(r1[8 * c + 5])), inv2));
+          v.w = pack2_bf16(mul2(pk2(__uint_as_float(r1[8 * c + 6]), __uint_as_float(r1[8 * c + 7])), inv2));
+          *reinterpret_cast<uint4*>(ost + swz128(et, 4 + c)) = v;
+        }
+        fence_proxy_async_smem();
+      }
+      named_bar_sync(kBarOut0, 128);
+      const int row0 = blk0 * kBlk + t * kTile;
+      if (et == 0 && ok && row0 < n) {   // rows past n are clipped by the store
+        tma_store_3d(&map_o, ost, 0, row0, slab);
+        bulk_commit_group();
       }
     }
-    for (; next_out < ntiles; next_out += 2)
-      ok = qside_write_tile<NH, SL>(bars, smem, den, &map_o, tmem, epsp, next_out, blk0 * kBlk + next_out * kTile, n, slab,
-                                    g, gt, ok, abort_flag, status);
-    if (gt == 0) bulk_wait_group0();
+    if (et == 0) bulk_wait_group0();
   } else {
     reg_inc<kRegsAux>();
-    const int ht = threadIdx.x - 32 * kAuxWarp0;
+    const int ht = threadIdx.x - 32 * kAuxWarp0Q;
     f32x2* hcoef = reinterpret_cast<f32x2*>(smem + SL::hcoef);
     haar_coef_init(hcoef, f + (size_t)slab * (L + 1), L, ht);
     named_bar_sync(kBarCoef, 256);
@@ -868,14 +912,14 @@ cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const flo
     auto k = k_tc_qside<2>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, QsideSmem<2>::total)) != cudaSuccess)
       return err;
-    k<<<grid, kThreads, QsideSmem<2>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
+    k<<<grid, kThreadsQ, QsideSmem<2>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
                                                          p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks,
                                                          w.status);
   } else {
     auto k = k_tc_qside<1>;
     if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, QsideSmem<1>::total)) != cudaSuccess)
       return err;
-    k<<<grid, kThreads, QsideSmem<1>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
+    k<<<grid, kThreadsQ, QsideSmem<1>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
                                                          p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks,
                                                          w.status);
   }
