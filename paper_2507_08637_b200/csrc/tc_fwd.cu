@@ -17,10 +17,14 @@
 //
 // Work unit of the MMA pipeline: one 128-token tile times one 128-feature half ("unit").  Three D1
 // accumulators rotate, so the ReLU pass of a unit overlaps four MMAs of its neighbours.
-// Warp roles: warp 0 TMA producer (K or Q), warps 1 and 3 MMA issuers (one thread each: warp 1 issues
-// every MMA1 and runs up to three units ahead, warp 3 every MMA2), warp 2 TMA producer
-// (V, key side), warps 4-11 two ReLU warpgroups that alternate over the units (query side: they also
-// write out the finished tiles), warps 12-19 Haar filter.  All operand tiles use the 128-byte swizzle.
+// Issuing an MMA blocks the thread for about as long as the tensor pipe takes to accept it, so the pipe
+// only stays busy when several threads issue: the waits and commits of one overlap the MMAs of another.
+// Warp roles, key side (640 threads): warp 0 TMA producer (K and V rings), warp 1 issues every MMA1 and
+// runs up to three units ahead, warps 2 and 3 issue the MMA2 of feature half 0 and 1 (separate
+// accumulators, so the order between them does not matter), warps 4-11 two ReLU warpgroups that
+// alternate over the units, warps 12-19 Haar filter.  Query side (768 threads): warp 0 TMA producer,
+// warp 1 MMA1, warp 3 MMA2 (both halves add into one accumulator, hence one thread), warps 4-11 ReLU,
+// warps 12-15 epilogue, warps 16-23 Haar filter.  All operand tiles use the 128-byte swizzle.
 // Every wait on an mbarrier is bounded; a role whose wait expires keeps its control flow (so that
 // group barriers stay balanced) but skips all further work, and the host sees the status word.
 #include "common.cuh"
@@ -45,7 +49,8 @@ constexpr uint32_t kIdesc2 = make_idesc_bf16(128, 64, false, true);    // key si
 constexpr uint32_t kIdesc2Q = make_idesc_bf16(128, 80, false, false);  // query side: B = [S' | z' | 0]^T, K-major
 constexpr uint32_t kSztBlockBytes = 80 * 128;      // one 64-feature K block of that operand: 80 rows of 128 bytes
 
-constexpr int kWarpTma = 0, kWarpMma = 1, kWarpTmaV = 2, kWarpMma2 = 3;
+constexpr int kWarpTma = 0, kWarpMma = 1, kWarpMma2 = 2;   // key side: warps 2 and 3 issue MMA2 (one per half)
+constexpr int kWarpMma2Q = 3;                               // query side
 constexpr int kReluWarp0 = 4, kAuxWarp0 = 12;       // 8 ReLU warps, 8 Haar warps
 constexpr int kThreads = 32 * (kAuxWarp0 + 8);      // 640 threads, 96 registers each at launch
 // Registers per thread after the roles have traded: the Haar step holds a 256 x 64 block in registers
@@ -167,61 +172,56 @@ __device__ __forceinline__ uint32_t pack2_bf16(f32x2 v) {
 }
 
 // ReLU of 32 fp32 accumulator columns -> 16 packed bf16 pairs (one fused relu + round + pack per
-// pair).  The side sums use 2 relu(a) = a + |a| (one full-rate add), accumulated as packed pairs:
-// kDot = false: acc += 2 relu(a);  kDot = true: acc += 2 relu(a) * zrow[.]; relu_unit halves the total.
-template <bool kDot>
-__device__ __forceinline__ void relu_chunk(const uint32_t (&r)[32], uint32_t (&p)[16], const float* __restrict__ zrow,
-                                           f32x2 (&acc)[2]) {
+// pair).  Returns the sum of the 16 pairs as one bf16 pair (a tree of packed bf16 adds): the row sums
+// z' are taken over the same rounded values that MMA2 multiplies, and the rounding of the short tree
+// (relative 2^-9 per add, independent from tile to tile) averages out over the sequence.
+__device__ __forceinline__ uint32_t add_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ uint32_t relu_chunk(const uint32_t (&r)[32], uint32_t (&p)[16]) {
 #pragma unroll
-  for (int j4 = 0; j4 < 8; ++j4) {
-    const float a0 = __uint_as_float(r[4 * j4]), a1 = __uint_as_float(r[4 * j4 + 1]);
-    const float a2 = __uint_as_float(r[4 * j4 + 2]), a3 = __uint_as_float(r[4 * j4 + 3]);
-    p[2 * j4] = relu_pack_bf16x2(a0, a1);
-    p[2 * j4 + 1] = relu_pack_bf16x2(a2, a3);
-    const f32x2 r01 = pk2(a0 + fabsf(a0), a1 + fabsf(a1)), r23 = pk2(a2 + fabsf(a2), a3 + fabsf(a3));
-    if (kDot) {
-      const float4 zv = *reinterpret_cast<const float4*>(zrow + 4 * j4);
-      acc[0] = fma2(r01, pk2(zv.x, zv.y), acc[0]);
-      acc[1] = fma2(r23, pk2(zv.z, zv.w), acc[1]);
-    } else {
-      acc[0] = add2(acc[0], r01);
-      acc[1] = add2(acc[1], r23);
-    }
-  }
+  for (int j = 0; j < 16; ++j) p[j] = relu_pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+  uint32_t t[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) t[j] = add_bf16x2(p[2 * j], p[2 * j + 1]);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) t[j] = add_bf16x2(t[2 * j], t[2 * j + 1]);
+  return add_bf16x2(add_bf16x2(t[0], t[1]), add_bf16x2(t[2], t[3]));
 }
 
 // ReLU pass over one 128-column D1 accumulator: fp32 TMEM -> bf16 pairs back into columns [0, 64)
 // of the same accumulator.  The next 32 columns are in flight while the current 32 are processed.
-// Returns the row sum of the ReLU values (kDot = false) or their dot product with zrow[0..127].
-template <bool kDot>
-__device__ __forceinline__ float relu_unit(uint32_t taddr, const float* __restrict__ zrow) {
-  f32x2 acc[2] = {0ull, 0ull};
+// Returns the row sum of the (rounded) ReLU values, accumulated in fp32 from the four chunk sums.
+__device__ __forceinline__ float relu_unit(uint32_t taddr) {
   uint32_t a[32], b[32], p[16];
   tmem_ld32(taddr, a);
   tmem_ld_wait();
   reg_fence32(a);
   tmem_ld32(taddr + 32, b);
-  relu_chunk<kDot>(a, p, zrow, acc);
+  const uint32_t s0 = relu_chunk(a, p);
   tmem_st16(taddr, p);
   tmem_ld_wait();
   reg_fence32(b);
   tmem_ld32(taddr + 64, a);
-  relu_chunk<kDot>(b, p, kDot ? zrow + 32 : zrow, acc);
+  const uint32_t s1 = relu_chunk(b, p);
   tmem_st16(taddr + 16, p);
   tmem_ld_wait();
   reg_fence32(a);
   tmem_ld32(taddr + 96, b);
-  relu_chunk<kDot>(a, p, kDot ? zrow + 64 : zrow, acc);
+  const uint32_t s2 = relu_chunk(a, p);
   tmem_st16(taddr + 32, p);
   tmem_ld_wait();
   reg_fence32(b);
-  relu_chunk<kDot>(b, p, kDot ? zrow + 96 : zrow, acc);
+  const uint32_t s3 = relu_chunk(b, p);
   tmem_st16(taddr + 48, p);
   tmem_st_wait();
-  float s0, s1, s2, s3;
-  upk2(acc[0], s0, s1);
-  upk2(acc[1], s2, s3);
-  return 0.5f * ((s0 + s1) + (s2 + s3));
+  float sum = 0.f;
+  const uint32_t cs[4] = {s0, s1, s2, s3};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) sum += __uint_as_float(cs[i] << 16) + __uint_as_float(cs[i] & 0xFFFF0000u);
+  return sum;
 }
 
 // ---- Haar filter of one 256-token block in shared memory ------------------------------------------
@@ -388,14 +388,14 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
     for (int s = 0; s < kNF; ++s) mbar_init(&bars->xf_ready[s], 8);
     for (int s = 0; s < kNV; ++s) {
       mbar_init(&bars->v_full[s], 1);
-      mbar_init(&bars->v_empty[s], 1);
+      mbar_init(&bars->v_empty[s], NH);
     }
     for (int b = 0; b < 6; ++b) mbar_init(&bars->d1_full[b], 1);
     for (int b = 0; b < kND1; ++b) {
       mbar_init(&bars->phi_ready[b], 4);
       mbar_init(&bars->d1_free[b], 1);
     }
-    mbar_init(&bars->acc_done, 1);
+    mbar_init(&bars->acc_done, NH);
     bars->abort_flag = 0;
     fence_mbar_init();
   }
@@ -413,23 +413,42 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
 
   if (warp < kReluWarp0) {
     reg_dec<kRegsCtl>();
-    if ((warp == kWarpTma || warp == kWarpTmaV) && lane == 0) {
-      const bool is_v = warp == kWarpTmaV;
-      const int depth = is_v ? kNV : kNXK;
-      uint64_t* full = is_v ? bars->v_full : bars->x_full;
-      uint64_t* empty = is_v ? bars->v_empty : bars->x_empty;
-      uint8_t* ring = smem + (is_v ? SL::v : SL::x);
-      const CUtensorMap* map = is_v ? &map_v : &map_k;
-      int issued = 0;
-      for (int b = 0; b < 2 * nblk; ++b) {   // b counts 128-token tiles here
-        const int s = b % depth;
-        if (!mbar_wait(&empty[s], ((b / depth) & 1) ^ 1, abort_flag, status, kErrProducer)) break;
-        mbar_arrive_expect_tx(&full[s], kTileBytes);
-        tma_load_3d(ring + s * kTileBytes, map, 0, blk0 * kBlk + b * kTile, slab, &full[s]);
-        issued = b + 1;
+    if (warp == kWarpTma && lane == 0) {
+      // One producer for both rings: whichever ring has a free slot gets its next tile, so that a full
+      // V ring never holds back the K tiles (and the other way round).
+      int kb = 0, vb = 0;
+      const int total = 2 * nblk;   // 128-token tiles
+      const unsigned long long t0 = global_timer_ns();
+      uint32_t spins = 0;
+      bool ok = true;
+      while (ok && (kb < total || vb < total)) {
+        bool progress = false;
+        if (kb < total && mbar_try_wait(&bars->x_empty[kb % kNXK], ((kb / kNXK) & 1) ^ 1)) {
+          const int s = kb % kNXK;
+          mbar_arrive_expect_tx(&bars->x_full[s], kTileBytes);
+          tma_load_3d(smem + SL::x + s * kTileBytes, &map_k, 0, blk0 * kBlk + kb * kTile, slab, &bars->x_full[s]);
+          ++kb;
+          progress = true;
+        }
+        if (vb < total && mbar_try_wait(&bars->v_empty[vb % kNV], ((vb / kNV) & 1) ^ 1)) {
+          const int s = vb % kNV;
+          mbar_arrive_expect_tx(&bars->v_full[s], kTileBytes);
+          tma_load_3d(smem + SL::v + s * kTileBytes, &map_v, 0, blk0 * kBlk + vb * kTile, slab, &bars->v_full[s]);
+          ++vb;
+          progress = true;
+        }
+        if (!progress && (++spins & 255u) == 0) {
+          if (*abort_flag != 0) ok = false;
+          else if (global_timer_ns() - t0 > kWaitLimitNs * 4) {   // whole-kernel budget of this loop
+            *abort_flag = 1;
+            atomicCAS(status, 0, kErrProducer);
+            ok = false;
+          }
+        }
       }
       if (*abort_flag != 0) {   // let copies in flight land before the CTA's shared memory goes away
-        for (int b = max(0, issued - depth); b < issued; ++b) mbar_wait_drain(&full[b % depth], (b / depth) & 1);
+        for (int b = max(0, kb - kNXK); b < kb; ++b) mbar_wait_drain(&bars->x_full[b % kNXK], (b / kNXK) & 1);
+        for (int b = max(0, vb - kNV); b < vb; ++b) mbar_wait_drain(&bars->v_full[b % kNV], (b / kNV) & 1);
       }
     } else if (warp == kWarpMma && lane == 0) {
       // MMA1 of every unit.  Ring slots, D1 buffers and barrier phases are running counters, and the
@@ -470,31 +489,30 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
         fs = (fs + 1) & (kNF - 1);
         fpar ^= (fs == 0);
       }
-    } else if (warp == kWarpMma2 && lane == 0) {
-      // MMA2 of every unit: S'[half h] += Phi^T (the unit's D1 buffer, bf16 pairs) * V tile.
+    } else if (warp >= kWarpMma2 && warp - kWarpMma2 < NH && lane == 0) {
+      // MMA2 of the units of feature half h (one issuing thread per half, each with its own
+      // accumulator): S'[half h] += Phi^T (the unit's D1 buffer, bf16 pairs) * V tile.
+      const int h = warp - kWarpMma2;
       constexpr uint32_t kTileStep = kTileBytes >> 4;
       const uint32_t hi = smem_desc_hi(1024);
       const uint32_t v_lo = smem_desc_lo(smem_u32(smem + SL::v), 1024);
-      uint32_t vs = 0, vpar = 0, p3 = 0, ppar = 0;     // V ring slot / phase, D1 buffer / phi_ready phase
+      const uint32_t acc = tmem + kAccCol + h * 64;
+      uint32_t vs = 0, vpar = 0;                       // V ring slot / phase
       bool ok = true;
       for (int t = 0; t < 2 * nblk && ok; ++t) {
+        const int u = t * NH + h, p3 = u % kND1;
         ok = mbar_wait(&bars->v_full[vs], vpar, abort_flag, status, kErrMma);
         if (!ok) break;
+        ok = mbar_wait(&bars->phi_ready[p3], (u / kND1) & 1, abort_flag, status, kErrMma);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t a_tm = tmem + p3 * 128;
+        const uint32_t b_lo = v_lo + vs * kTileStep;
 #pragma unroll
-        for (int h = 0; h < NH; ++h) {
-          ok = mbar_wait(&bars->phi_ready[p3], ppar, abort_flag, status, kErrMma);
-          if (!ok) break;
-          tc_fence_after_sync();
-          const uint32_t acc = tmem + kAccCol + h * 64, a_tm = tmem + p3 * 128;
-          const uint32_t b_lo = v_lo + vs * kTileStep;
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            mma_ts(acc, a_tm + k * 8, smem_desc_join(b_lo + 128 * k, hi), kIdesc2, (t > 0 || k > 0) ? 1u : 0u);
-          mma_commit(&bars->d1_free[p3]);
-          p3 = p3 == kND1 - 1 ? 0 : p3 + 1;
-          ppar ^= (p3 == 0);
-        }
-        mma_commit(&bars->v_empty[vs]);
+        for (int k = 0; k < 8; ++k)
+          mma_ts(acc, a_tm + k * 8, smem_desc_join(b_lo + 128 * k, hi), kIdesc2, (t > 0 || k > 0) ? 1u : 0u);
+        mma_commit(&bars->d1_free[p3]);
+        mma_commit(&bars->v_empty[vs]);   // one arrival per half
         vs = vs == kNV - 1 ? 0 : vs + 1;
         vpar ^= (vs == 0);
       }
@@ -510,7 +528,7 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d1_full[u % 6], (u / 6) & 1, abort_flag, status, kErrRelu));
       if (ok) {
         tc_fence_after_sync();
-        zacc += relu_unit<false>(tmem + (lane_base << 16) + (u % kND1) * 128, nullptr);
+        zacc += relu_unit(tmem + (lane_base << 16) + (u % kND1) * 128);
         tc_fence_before_sync();
         warp_arrive(&bars->phi_ready[u % kND1]);
       }
@@ -718,7 +736,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
         fs = (fs + 1) & (kNF - 1);
         fpar ^= (fs == 0);
       }
-    } else if (warp == kWarpMma2 && lane == 0) {
+    } else if (warp == kWarpMma2Q && lane == 0) {
       // MMA2 of every unit: [N' | D'] (+)= Phi (the unit's D1 buffer, bf16 pairs) * [S' | z' | 0] half h.
       const uint32_t hi = smem_desc_hi(1024);
       const uint32_t s_lo = smem_desc_lo(smem_u32(smem + SL::simg), 16);
