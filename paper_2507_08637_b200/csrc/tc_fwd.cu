@@ -38,7 +38,7 @@ namespace {
 constexpr int kTile = 128;                        // tokens per MMA tile
 constexpr int kBlk = 256;                         // tokens per Haar block = one pipeline stage
 constexpr uint32_t kTileBytes = kTile * kD * 2;   // 128 x 64 bf16
-constexpr int kNXK = 6, kNV = 5;                  // key side: ring of K tiles, ring of V tiles
+constexpr int kNXK = 7, kNV = 4;                  // key side: ring of K tiles, ring of V tiles
 constexpr int kNXQ = 7;                           // query side: ring of Q tiles
 constexpr int kNF = 4;                            // "block filtered" barriers (block b uses b % 4)
 constexpr int kND1 = 3;                           // D1 accumulators in TMEM (columns 0, 128, 256)
@@ -299,19 +299,23 @@ __device__ __forceinline__ void haar_block_inplace(uint8_t* tile0, uint8_t* tile
     }
     named_bar_sync(kBarHaar, 256);
     if (ok) {
-      // lane (c, q = lane >> 3) combines the eight warps' sums of column pair q of chunk c, then the
-      // four lanes that share a chunk swap their pairs
+      // lane (c, q = lane >> 3) combines the eight warps' sums of column pair q of chunk c (two
+      // independent chains of four), then the four lanes that share a chunk swap their pairs
       const int qq = lane >> 3;
-      f32x2 acc = 0ull;
+      const f32x2* src = reinterpret_cast<const f32x2*>(xch + c * 8 + 2 * qq);
+      const f32x2* cf = hcoef + 8 + 8 * hw;
+      f32x2 acc0 = mul2(cf[0], src[0]), acc1 = mul2(cf[1], src[kD / 2]);
 #pragma unroll
-      for (int w = 0; w < 8; ++w)
-        acc = fma2(hcoef[8 + 8 * hw + w], *reinterpret_cast<const f32x2*>(xch + w * kD + c * 8 + 2 * qq), acc);
+      for (int w = 2; w < 8; w += 2) {
+        acc0 = fma2(cf[w], src[w * (kD / 2)], acc0);
+        acc1 = fma2(cf[w + 1], src[(w + 1) * (kD / 2)], acc1);
+      }
       float lo, hi_;
-      upk2(acc, lo, hi_);
+      upk2(add2(acc0, acc1), lo, hi_);
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const int src = (q << 3) | c;
-        hi[q] = add2(hi[q], pk2(__shfl_sync(0xffffffffu, lo, src), __shfl_sync(0xffffffffu, hi_, src)));
+        const int sl = (q << 3) | c;
+        hi[q] = add2(hi[q], pk2(__shfl_sync(0xffffffffu, lo, sl), __shfl_sync(0xffffffffu, hi_, sl)));
       }
     }
   }
@@ -333,11 +337,18 @@ __device__ __forceinline__ void haar_block_inplace(uint8_t* tile0, uint8_t* tile
       x[6][q] = fma2(f0, x[6][q], c13);
       x[7][q] = fma2(f0, x[7][q], c13);
     }
+    if (rg * 8 + 8 <= valid_rows) {   // the usual case: every row of this thread lies inside the sequence
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      uint4 out = make_uint4(pack2_bf16(x[j][0]), pack2_bf16(x[j][1]), pack2_bf16(x[j][2]), pack2_bf16(x[j][3]));
-      if (rg * 8 + j >= valid_rows) out = make_uint4(0u, 0u, 0u, 0u);
-      *reinterpret_cast<uint4*>(base + j * 128 + ((c ^ j) << 4)) = out;
+      for (int j = 0; j < 8; ++j)
+        *reinterpret_cast<uint4*>(base + j * 128 + ((c ^ j) << 4)) =
+            make_uint4(pack2_bf16(x[j][0]), pack2_bf16(x[j][1]), pack2_bf16(x[j][2]), pack2_bf16(x[j][3]));
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        uint4 out = make_uint4(pack2_bf16(x[j][0]), pack2_bf16(x[j][1]), pack2_bf16(x[j][2]), pack2_bf16(x[j][3]));
+        if (rg * 8 + j >= valid_rows) out = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(base + j * 128 + ((c ^ j) << 4)) = out;
+      }
     }
   }
 }
