@@ -22,8 +22,11 @@
 //   threads: dA_h = (G_h + dD' z'_h) (.) mask                           -> bf16 in place
 //   MMA4: dQ_F = sum_h dA_h * W_h^T (W^T image, N-major)                -> TMEM fp32 -> global
 // and at the end of the chunk the partial dS', dz' and sum of dD' go to the split-sequence buffers.
-// One CTA of 128 threads per SM walks a chunk of tiles one step at a time (thread 0 issues the copies
+// One CTA of 256 threads per SM walks a chunk of tiles one step at a time (thread 0 issues the copies
 // and the MMAs, everybody waits on one mbarrier); the copies of the next tile are in flight meanwhile.
+// The two warpgroups see the same 128 TMEM lanes and share every elementwise pass by columns: of the
+// 4 NH chunks of 32 accumulator columns, warpgroup g takes chunks 2 NH g .. 2 NH g + 2 NH - 1 (with
+// m = 256 that is feature half g), and of a 64-column result it takes columns 32 g .. 32 g + 31.
 // TMEM per CTA: 128 columns per feature half; the two 64-column results (dV, dK_F) reuse the upper
 // half of the first accumulator.  Every mbarrier wait is bounded; after an expired wait the CTA
 // leaves its loop (the decision is taken CTA-wide, so barriers stay balanced) and the host sees the
@@ -108,38 +111,82 @@ __device__ __forceinline__ void split_pack(float g0, float g1, uint32_t& p_hi, u
   p_lo = pack_bf16x2(g0 - __uint_as_float(p_hi << 16), g1 - __uint_as_float(p_hi & 0xFFFF0000u));
 }
 
-// Gradient through the ReLU of one 128-column accumulator (token = lane): x_j = (G_j + s * zr_j) where
-// mask bit j is set, else 0; written back as bf16 hi pairs in columns [0, 64) and lo pairs in columns
-// [64, 128) of the same accumulator (all 128 columns are read before the first one is overwritten).
-__device__ __forceinline__ void relu_grad_split(uint32_t taddr, const uint32_t (&mask)[4], float s,
-                                                const float* __restrict__ zr) {
-  uint32_t r[4][32];
+// ReLU pass over this warpgroup's 2 NH chunks of 32 fp32 accumulator columns: chunk (h, c) = columns
+// 128 h + 32 c .. + 31 becomes 16 bf16 pairs in columns 128 h + 16 c .. + 15 of the same accumulator.
+// `side(ii, h, c, r)` sees the 32 raw values of the warpgroup's ii-th chunk (mask bits, row sums).
+// With NH = 2 a warpgroup owns its accumulator and a chunk's pairs land in columns it has already
+// read; with NH = 1 the two warpgroups share one accumulator, so all pairs are held back until both
+// have read their columns (one CTA barrier).
+template <int NH, typename F>
+__device__ __forceinline__ void relu_pass(uint32_t trow, int wg, F&& side) {
+  uint32_t pp[NH == 1 ? 2 : 1][16];
 #pragma unroll
-  for (int c = 0; c < 4; ++c) tmem_ld32(taddr + 32 * c, r[c]);
+  for (int ii = 0; ii < 2 * NH; ++ii) {
+    const int i = wg * 2 * NH + ii, h = i >> 2, c = i & 3;
+    uint32_t r[32];
+    tmem_ld32(trow + h * 128 + 32 * c, r);
+    tmem_ld_wait();
+    reg_fence32(r);
+    side(ii, h, c, r);
+    uint32_t(&p)[16] = pp[NH == 1 ? ii : 0];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) p[j] = relu_pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+    if (NH != 1) tmem_st16(trow + h * 128 + 16 * c, p);
+  }
+  if (NH == 1) {
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+#pragma unroll
+    for (int ii = 0; ii < 2; ++ii) tmem_st16(trow + 16 * (wg * 2 + ii), pp[ii]);
+  }
+  tmem_st_wait();
+}
+
+// Gradient through the ReLU for this warpgroup's 2 NH chunks of 32 accumulator columns (token = lane):
+// x_j = (G_j + s * zr_j) where mask bit j is set, else 0; written back as bf16 hi pairs in columns
+// [0, 64) and lo pairs in columns [64, 128) of the same accumulator.  All columns are read before the
+// first one is overwritten; with NH = 1 the two warpgroups share one accumulator, so a CTA barrier
+// separates the reads from the writes.  `zr` points at the m values z'_f (or dz'_f).
+template <int NH>
+__device__ __forceinline__ void relu_grad_split(uint32_t trow, int wg, const uint32_t (&mask)[2 * NH], float s,
+                                                const float* __restrict__ zr) {
+  uint32_t r[2 * NH][32];
+#pragma unroll
+  for (int ii = 0; ii < 2 * NH; ++ii) {
+    const int i = wg * 2 * NH + ii;
+    tmem_ld32(trow + (i >> 2) * 128 + 32 * (i & 3), r[ii]);
+  }
   tmem_ld_wait();
 #pragma unroll
-  for (int c = 0; c < 4; ++c) reg_fence32(r[c]);
+  for (int ii = 0; ii < 2 * NH; ++ii) reg_fence32(r[ii]);
+  if (NH == 1) {
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+  }
 #pragma unroll
-  for (int c = 0; c < 4; ++c) {
+  for (int ii = 0; ii < 2 * NH; ++ii) {
+    const int i = wg * 2 * NH + ii, h = i >> 2, c = i & 3;
     uint32_t ph[16], pl[16];
-    const uint32_t bits = mask[c];
+    const uint32_t bits = mask[ii];
+    const float* z = zr + h * 128 + 32 * c;
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      const float g0 = ((bits >> (2 * j)) & 1u) ? fmaf(s, zr[32 * c + 2 * j], __uint_as_float(r[c][2 * j])) : 0.f;
-      const float g1 =
-          ((bits >> (2 * j + 1)) & 1u) ? fmaf(s, zr[32 * c + 2 * j + 1], __uint_as_float(r[c][2 * j + 1])) : 0.f;
+      const float g0 = ((bits >> (2 * j)) & 1u) ? fmaf(s, z[2 * j], __uint_as_float(r[ii][2 * j])) : 0.f;
+      const float g1 = ((bits >> (2 * j + 1)) & 1u) ? fmaf(s, z[2 * j + 1], __uint_as_float(r[ii][2 * j + 1])) : 0.f;
       split_pack(g0, g1, ph[j], pl[j]);
     }
-    tmem_st16(taddr + 16 * c, ph);
-    tmem_st16(taddr + 64 + 16 * c, pl);
+    tmem_st16(trow + h * 128 + 16 * c, ph);
+    tmem_st16(trow + h * 128 + 64 + 16 * c, pl);
   }
   tmem_st_wait();
 }
 
 // ---- key side -----------------------------------------------------------------------------------
-// grid (chunks, slabs), block 128.
+// grid (chunks, slabs), block 256.
 template <int NH, typename TG>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(256, 1)
 k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant__ CUtensorMap map_v,
                const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ dSbf,
                const float* __restrict__ dzg, TG* __restrict__ dV, float* __restrict__ dKF, int n, int chunk_tiles,
@@ -176,7 +223,8 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = bars->tmem_base;
-  const uint32_t trow = tmem + ((32u * warp) << 16);     // this warp's lane quarter
+  const int wg = warp >> 2, tl = threadIdx.x & 127;      // warpgroup; token of this thread = TMEM lane
+  const uint32_t trow = tmem + ((32u * (warp & 3)) << 16);   // this warp's lane quarter
   const uint32_t acc = NH * 128;                         // dV / dK_F
 
   const uint32_t hi = smem_desc_hi(1024);
@@ -207,7 +255,7 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
 
   for (int ti = 0; ti < ntiles && ok; ++ti) {
     const int row0 = (tile0 + ti) * kTile;
-    const int row = row0 + (int)threadIdx.x;
+    const int row = row0 + tl;
     const uint32_t x_k = stage_k + (ti & 1) * kStageStep, v_k = x_k + 3 * kTileStep;
     // ---- copies of the next tile (its stage was released by the barrier that ended tile ti - 1), MMA1
     if (threadIdx.x == 0 && ti + 1 < ntiles) {
@@ -233,25 +281,13 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
     if (!ok) break;
     tc_fence_after_sync();
     // ---- mask and Phi
-    uint32_t mask[NH][4];
+    uint32_t mask[2 * NH];
+    relu_pass<NH>(trow, wg, [&](int ii, int, int, const uint32_t(&r)[32]) {
+      uint32_t bits = 0;
 #pragma unroll
-    for (int h = 0; h < NH; ++h) {
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32], p[16];
-        tmem_ld32(trow + h * 128 + 32 * c, r);
-        tmem_ld_wait();
-        reg_fence32(r);
-        uint32_t bits = 0;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) bits |= (__uint_as_float(r[j]) > 0.f ? 1u : 0u) << j;
-        mask[h][c] = bits;
-#pragma unroll
-        for (int j = 0; j < 16; ++j) p[j] = relu_pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-        tmem_st16(trow + h * 128 + 16 * c, p);
-      }
-    }
-    tmem_st_wait();
+      for (int j = 0; j < 32; ++j) bits |= (__uint_as_float(r[j]) > 0.f ? 1u : 0u) << j;
+      mask[ii] = bits;
+    });
     tc_fence_before_sync();
     __syncthreads();
     // ---- MMA2: dV
@@ -269,13 +305,12 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
     mma_par ^= 1;
     if (!ok) break;
     tc_fence_after_sync();
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
+    {
       uint32_t r[32];
-      tmem_ld32(trow + acc + 32 * c, r);
+      tmem_ld32(trow + acc + 32 * wg, r);
       tmem_ld_wait();
       reg_fence32(r);
-      if (row < n) store_row32<TG>(dV + ((size_t)slab * n + row) * kD + 32 * c, r);
+      if (row < n) store_row32<TG>(dV + ((size_t)slab * n + row) * kD + 32 * wg, r);
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -295,8 +330,7 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
     if (!ok) break;
     tc_fence_after_sync();
     // ---- dB_h = (G_h + dz'_h) (.) mask, as bf16 hi + lo
-#pragma unroll
-    for (int h = 0; h < NH; ++h) relu_grad_split(trow + h * 128, mask[h], 1.f, dzs + h * 128);
+    relu_grad_split<NH>(trow, wg, mask, 1.f, dzs);
     tc_fence_before_sync();
     __syncthreads();
     // ---- MMA4: dK_F
@@ -316,13 +350,12 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
     mma_par ^= 1;
     if (!ok) break;
     tc_fence_after_sync();
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
+    {
       uint32_t r[32];
-      tmem_ld32(trow + acc + 32 * c, r);
+      tmem_ld32(trow + acc + 32 * wg, r);
       tmem_ld_wait();
       reg_fence32(r);
-      if (row < n) store_row32<float>(dKF + ((size_t)slab * n + row) * kD + 32 * c, r);
+      if (row < n) store_row32<float>(dKF + ((size_t)slab * n + row) * kD + 32 * wg, r);
     }
     tc_fence_before_sync();
     __syncthreads();   // the next tile's copies and MMA1 overwrite what this tile read
@@ -352,10 +385,13 @@ template <int NH> struct BwdQSmem {
   static constexpr uint32_t total = bars + 64 + 1024;
 };
 
-// grid (chunks, slabs), block 128.  TMEM: accumulator h at columns 128 h (A_h, A_h^T, G_h in turn; the
-// 64-column results N' and dQ_F sit at 384), dS'_h at 256 + 64 h.
+// grid (chunks, slabs), block 256.  TMEM: accumulator h at columns 128 h (A_h, A_h^T, G_h in turn; the
+// 64-column results N' and dQ_F sit at 384), dS'_h at 256 + 64 h.  Row quantities that both
+// warpgroups contribute to (D', dD', and with m = 128 dz') meet in the 128-float array `dds`:
+// warpgroup 1 leaves its part there, warpgroup 0 adds its own (always in this order) and leaves the
+// total there for everybody, with the CTA barriers of the step sequence in between.
 template <int NH>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(256, 1)
 k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant__ CUtensorMap map_do,
                const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ Sbf,
                const float* __restrict__ zg, const float* __restrict__ beta, float eps, float bw_floor,
@@ -396,7 +432,8 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = bars->tmem_base;
-  const uint32_t trow = tmem + ((32u * warp) << 16);
+  const int wg = warp >> 2, tl = threadIdx.x & 127;      // warpgroup; token / feature of this thread = TMEM lane
+  const uint32_t trow = tmem + ((32u * (warp & 3)) << 16);
   const uint32_t acc = 384;
   const float bw = fmaxf(beta[0], bw_floor);
   const float epsp = eps * (float)m * bw * bw;
@@ -438,7 +475,7 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
 
   for (int ti = 0; ti < ntiles && ok; ++ti) {
     const int row0 = (tile0 + ti) * kTile;
-    const int row = row0 + (int)threadIdx.x;
+    const int row = row0 + tl;
     const uint32_t x_k = stage_k + (ti & 1) * kStageStep;
     const uint8_t* do_tile = smem + SL::stage + (ti & 1) * SL::stage_bytes + 3 * kTileBytes;
     if (threadIdx.x == 0 && ti + 1 < ntiles) {
@@ -462,33 +499,26 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
     }
     if (!(ok = wait_mma())) break;
     // ---- mask, Phi, denominator
-    uint32_t mask[NH][4];
-    float den = epsp;
+    uint32_t mask[2 * NH];
+    float den = 0.f;
+    relu_pass<NH>(trow, wg, [&](int ii, int h, int c, const uint32_t(&r)[32]) {
+      uint32_t bits = 0;
+      const float* zr = zs + h * 128 + 32 * c;
 #pragma unroll
-    for (int h = 0; h < NH; ++h) {
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32], p[16];
-        tmem_ld32(trow + h * 128 + 32 * c, r);
-        tmem_ld_wait();
-        reg_fence32(r);
-        uint32_t bits = 0;
-        const float* zr = zs + h * 128 + 32 * c;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float a = __uint_as_float(r[j]);
-          bits |= (a > 0.f ? 1u : 0u) << j;
-          den = fmaf(fmaxf(a, 0.f), zr[j], den);
-        }
-        mask[h][c] = bits;
-#pragma unroll
-        for (int j = 0; j < 16; ++j) p[j] = relu_pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-        tmem_st16(trow + h * 128 + 16 * c, p);
+      for (int j = 0; j < 32; ++j) {
+        const float a = __uint_as_float(r[j]);
+        bits |= (a > 0.f ? 1u : 0u) << j;
+        den = fmaf(fmaxf(a, 0.f), zr[j], den);
       }
-    }
-    tmem_st_wait();
+      mask[ii] = bits;
+    });
+    if (wg == 1) dds[tl] = den;
     tc_fence_before_sync();
     __syncthreads();
+    if (wg == 0) {
+      den = epsp + (den + dds[tl]);
+      dds[tl] = den;
+    }
     // ---- MMA2: N'
     if (threadIdx.x == 0) {
       tc_fence_after_sync();
@@ -501,42 +531,43 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
       mma_commit(&bars->mma);
     }
     if (!(ok = wait_mma())) break;
-    // ---- O, dN' (-> smem tile, bf16), dD'
+    // ---- O, dN' (-> smem tile, bf16), dD': warpgroup g takes columns 32 g .. 32 g + 31
+    if (wg == 1) den = dds[tl];                    // the total left by warpgroup 0 before the last barrier
     const float inv = row < n ? 1.f / den : 0.f;   // rows past the end contribute nothing
     float dd = 0.f;
     {
       uint8_t* dn_tile = smem + SL::dn;
+      uint32_t r[32];
+      tmem_ld32(trow + acc + 32 * wg, r);
+      tmem_ld_wait();
+      reg_fence32(r);
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t r[32];
-        tmem_ld32(trow + acc + 32 * c, r);
-        tmem_ld_wait();
-        reg_fence32(r);
+      for (int q = 0; q < 4; ++q) {   // 16-byte chunk 4 g + q of this token's row: 8 columns
+        const uint4 raw = *reinterpret_cast<const uint4*>(do_tile + swz128(tl, 4 * wg + q));
+        const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+        uint32_t oh[4], ol[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {   // 16-byte chunk 4 c + q of this token's row: 8 columns
-          const uint4 raw = *reinterpret_cast<const uint4*>(do_tile + swz128(threadIdx.x, 4 * c + q));
-          const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
-          uint32_t oh[4], ol[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float g0 = __uint_as_float(u[i] << 16), g1 = __uint_as_float(u[i] & 0xFFFF0000u);
-            const float o0 = __uint_as_float(r[8 * q + 2 * i]) * inv, o1 = __uint_as_float(r[8 * q + 2 * i + 1]) * inv;
-            dd = fmaf(g0, o0, dd);
-            dd = fmaf(g1, o1, dd);
-            split_pack(g0 * inv, g1 * inv, oh[i], ol[i]);
-          }
-          *reinterpret_cast<uint4*>(dn_tile + swz128(threadIdx.x, 4 * c + q)) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
-          *reinterpret_cast<uint4*>(dn_tile + kTileBytes + swz128(threadIdx.x, 4 * c + q)) =
-              make_uint4(ol[0], ol[1], ol[2], ol[3]);
+        for (int i = 0; i < 4; ++i) {
+          const float g0 = __uint_as_float(u[i] << 16), g1 = __uint_as_float(u[i] & 0xFFFF0000u);
+          const float o0 = __uint_as_float(r[8 * q + 2 * i]) * inv, o1 = __uint_as_float(r[8 * q + 2 * i + 1]) * inv;
+          dd = fmaf(g0, o0, dd);
+          dd = fmaf(g1, o1, dd);
+          split_pack(g0 * inv, g1 * inv, oh[i], ol[i]);
         }
+        *reinterpret_cast<uint4*>(dn_tile + swz128(tl, 4 * wg + q)) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+        *reinterpret_cast<uint4*>(dn_tile + kTileBytes + swz128(tl, 4 * wg + q)) =
+            make_uint4(ol[0], ol[1], ol[2], ol[3]);
       }
     }
-    dd = -dd * inv;
-    dds[threadIdx.x] = dd;
-    sum_dd += dd;
+    if (wg == 1) dds[tl] = dd;                     // (the same thread has read D' from this slot above)
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
+    if (wg == 0) {
+      dd = -(dd + dds[tl]) * inv;
+      dds[tl] = dd;
+      sum_dd += dd;
+    }
     // ---- MMA1t: A_h^T (feature = lane), hi plane only
     if (threadIdx.x == 0) {
       tc_fence_after_sync();
@@ -549,26 +580,15 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
       mma_commit(&bars->mma);
     }
     if (!(ok = wait_mma())) break;
-    // ---- Phi^T, dz' partial
+    // ---- Phi^T, dz' partial (the barrier that ended the MMA wait also published dD')
+    if (wg == 1) dd = dds[tl];
+    relu_pass<NH>(trow, wg, [&](int, int h, int c, const uint32_t(&r)[32]) {
+      const float* ddr = dds + 32 * c;
+      float part = 0.f;
 #pragma unroll
-    for (int h = 0; h < NH; ++h) {
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32], p[16];
-        tmem_ld32(trow + h * 128 + 32 * c, r);
-        tmem_ld_wait();
-        reg_fence32(r);
-        const float* ddr = dds + 32 * c;
-        float part = 0.f;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) part = fmaf(fmaxf(__uint_as_float(r[j]), 0.f), ddr[j], part);
-        dzacc[h] += part;
-#pragma unroll
-        for (int j = 0; j < 16; ++j) p[j] = relu_pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-        tmem_st16(trow + h * 128 + 16 * c, p);
-      }
-    }
-    tmem_st_wait();
+      for (int j = 0; j < 32; ++j) part = fmaf(fmaxf(__uint_as_float(r[j]), 0.f), ddr[j], part);
+      dzacc[h] += part;
+    });
     tc_fence_before_sync();
     __syncthreads();
     // ---- MMA5: dS'_h += Phi_h^T dN'   and   MMA3: G_h = dN' S'_h^T (after MMA5 has read Phi_h^T)
@@ -594,8 +614,7 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
     }
     if (!(ok = wait_mma())) break;
     // ---- dA_h = (G_h + dD' z'_h) (.) mask, as bf16 hi + lo
-#pragma unroll
-    for (int h = 0; h < NH; ++h) relu_grad_split(trow + h * 128, mask[h], dd, zs + h * 128);
+    relu_grad_split<NH>(trow, wg, mask, dd, zs);
     tc_fence_before_sync();
     __syncthreads();
     // ---- MMA4: dQ_F
@@ -612,13 +631,12 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
       mma_commit(&bars->mma);
     }
     if (!(ok = wait_mma())) break;
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
+    {
       uint32_t r[32];
-      tmem_ld32(trow + acc + 32 * c, r);
+      tmem_ld32(trow + acc + 32 * wg, r);
       tmem_ld_wait();
       reg_fence32(r);
-      if (row < n) store_row32<float>(dQF + ((size_t)slab * n + row) * kD + 32 * c, r);
+      if (row < n) store_row32<float>(dQF + ((size_t)slab * n + row) * kD + 32 * wg, r);
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -627,24 +645,26 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
   const size_t pidx = (size_t)slab * gridDim.x + chunk;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sum_dd += __shfl_xor_sync(0xffffffffu, sum_dd, o);
-  if (lane == 0) red[warp] = sum_dd;
+  if (lane == 0 && wg == 0) red[warp] = sum_dd;
+  if (NH == 1 && wg == 1) dds[tl] = dzacc[0];      // with one feature half both warpgroups hold a part of dz'
   __syncthreads();
   if (threadIdx.x == 0) sumdD[pidx] = ok ? (red[0] + red[1]) + (red[2] + red[3]) : 0.f;
   if (ok && ntiles > 0) {
     tc_fence_after_sync();
+    // dS': of the 2 NH chunks of 32 columns (half h, columns 32 c ..), warpgroup g takes NH g .. NH g + NH - 1
 #pragma unroll
-    for (int h = 0; h < NH; ++h) {
-      const int feat = h * 128 + threadIdx.x;
-      float* dst = dspart + (pidx * m + feat) * kD;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t r[32];
-        tmem_ld32(trow + kAccS + h * 64 + 32 * c, r);
-        tmem_ld_wait();
-        reg_fence32(r);
-        store_row32<float>(dst + 32 * c, r);
-      }
-      dzpart[pidx * m + feat] = dzacc[h];
+    for (int ii = 0; ii < NH; ++ii) {
+      const int i = wg * NH + ii, h = i >> 1, c = i & 1;
+      uint32_t r[32];
+      tmem_ld32(trow + kAccS + h * 64 + 32 * c, r);
+      tmem_ld_wait();
+      reg_fence32(r);
+      store_row32<float>(dspart + (pidx * m + h * 128 + tl) * kD + 32 * c, r);
+    }
+    if (NH == 1) {
+      if (wg == 0) dzpart[pidx * m + tl] = dzacc[0] + dds[tl];
+    } else {
+      dzpart[pidx * m + wg * 128 + tl] = dzacc[NH - 1 < wg ? 0 : wg];
     }
   }
   if (!ok && threadIdx.x == 0) {
@@ -697,7 +717,7 @@ cudaError_t launch_kside(const Plan& p, const Ws& w, const CUtensorMap& map_kf, 
   cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdKSmem<NH>::total);
   if (err != cudaSuccess) return err;
   dim3 grid(p.bchunks, p.slabs);
-  k<<<grid, 128, BwdKSmem<NH>::total, st>>>(map_kf, map_v, w.Wt, w.dSbf, w.dz, static_cast<TG*>(dV), w.dKF,
+  k<<<grid, 256, BwdKSmem<NH>::total, st>>>(map_kf, map_v, w.Wt, w.dSbf, w.dz, static_cast<TG*>(dV), w.dKF,
                                             p.cfg.seq_len, p.bchunk_tiles, w.status);
   return cudaGetLastError();
 }
@@ -709,7 +729,7 @@ cudaError_t launch_qside(const Plan& p, const Ws& w, const CUtensorMap& map_qf, 
   cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdQSmem<NH>::total);
   if (err != cudaSuccess) return err;
   dim3 grid(p.bchunks, p.slabs);
-  k<<<grid, 128, BwdQSmem<NH>::total, st>>>(map_qf, map_do, w.Wt, w.Sbf, w.z, beta, p.cfg.eps, p.cfg.bw_floor, w.dQF,
+  k<<<grid, 256, BwdQSmem<NH>::total, st>>>(map_qf, map_do, w.Wt, w.Sbf, w.z, beta, p.cfg.eps, p.cfg.bw_floor, w.dQF,
                                             w.spart, w.zpart, w.sumdD, p.cfg.seq_len, p.bchunk_tiles, w.status);
   return cudaGetLastError();
 }
