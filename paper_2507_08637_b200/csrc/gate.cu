@@ -180,9 +180,10 @@ __global__ void __launch_bounds__(32) k_band_reduce(const float* __restrict__ ba
   if (j == 8 + L - 1) df[(size_t)slab * kBandVals + L] = s;
 }
 
-// Single CTA, 64 threads (thread c = column).  Chain rule through f = sigmoid(u) * omega,
-// u = gate(qbar): domega, dgate_b, dgate_w, dqbar; and the bandwidth gradient
-// dbeta = 2 eps m bw * sum_t dDh_t (ReLU is positively homogeneous, so beta only acts through eps).
+// Chain rule through f = sigmoid(u) * omega, u = gate(qbar): domega, dgate_b, dgate_w, dqbar; and the
+// bandwidth gradient dbeta = 2 eps m bw * sum_t dDh_t (ReLU is positively homogeneous, so beta only
+// acts through eps).  Grid H + 2, 64 threads: CTA h < H handles head h (thread c = column of q-bar,
+// loop over the batch), CTA H sums domega, CTA H + 1 sums dbeta; every sum has a fixed order.
 __global__ void __launch_bounds__(kD) k_gate_backward(
     const float* __restrict__ df, const float* __restrict__ sg, const float* __restrict__ qbar,
     const float* __restrict__ gate_w, const float* __restrict__ omega, const float* __restrict__ sumdD,
@@ -191,7 +192,9 @@ __global__ void __launch_bounds__(kD) k_gate_backward(
     float* __restrict__ domega, float* __restrict__ dqbar) {
   const int c = threadIdx.x;
   __shared__ float du[kMaxLevels + 1];
-  for (int h = 0; h < H; ++h) {
+  __shared__ float part[kD];
+  if ((int)blockIdx.x < H) {
+    const int h = blockIdx.x;
     float gw_acc[kMaxLevels + 1], gb_acc = 0.f;
 #pragma unroll
     for (int i = 0; i <= kMaxLevels; ++i) gw_acc[i] = 0.f;
@@ -226,29 +229,42 @@ __global__ void __launch_bounds__(kD) k_gate_backward(
         if (i < L1) dgate_w[((size_t)h * kD + c) * L1 + i] = gw_acc[i];
     }
     if (dgate_b != nullptr && c < L1) dgate_b[h * L1 + c] = (per_head || h == 0) ? gb_acc : 0.f;
-  }
-  if (domega != nullptr && c < L1) {
+  } else if ((int)blockIdx.x == H) {
+    // domega[i] = sum over slabs of df_i * sigmoid(u_i): thread (i = c & 15, q = c >> 4) takes the
+    // batch elements b = q, q + 4, ..., then the four parts are added in order
+    const int i = c & 15, q = c >> 4;
     float acc = 0.f;
-    for (int b = 0; b < B; ++b) {
-      if (per_head) {
-        for (int h = 0; h < H; ++h) {
-          const int slab = b * H + h;
-          acc += df[(size_t)slab * kBandVals + c] * sg[(size_t)slab * L1 + c];
+    if (domega != nullptr && i < L1) {
+      for (int b = q; b < B; b += 4) {
+        if (per_head) {
+          for (int h = 0; h < H; ++h) {
+            const int slab = b * H + h;
+            acc += df[(size_t)slab * kBandVals + i] * sg[(size_t)slab * L1 + i];
+          }
+        } else {
+          float dfi = 0.f;
+          for (int h = 0; h < H; ++h) dfi += df[((size_t)b * H + h) * kBandVals + i];
+          acc += dfi * sg[((size_t)b * H) * L1 + i];
         }
-      } else {
-        float dfi = 0.f;
-        for (int h = 0; h < H; ++h) dfi += df[((size_t)b * H + h) * kBandVals + c];
-        acc += dfi * sg[((size_t)b * H) * L1 + c];
       }
     }
-    domega[c] = acc;
-  }
-  if (dbeta != nullptr && c == 0) {
+    part[c] = acc;
+    __syncthreads();
+    if (domega != nullptr && c < L1) domega[c] = (part[c] + part[16 + c]) + (part[32 + c] + part[48 + c]);
+  } else {
     float tot = 0.f;
-    for (int i = 0; i < n_sumdD; ++i) tot += sumdD[i];
-    const float bt = beta[0];
-    const float bw = fmaxf(bt, bw_floor);
-    dbeta[0] = bt > bw_floor ? 2.f * eps * (float)m * bw * tot : 0.f;
+    for (int i = c; i < n_sumdD; i += kD) tot += sumdD[i];
+    part[c] = tot;
+    __syncthreads();
+    for (int o = kD / 2; o > 0; o >>= 1) {
+      if (c < o) part[c] += part[c + o];
+      __syncthreads();
+    }
+    if (dbeta != nullptr && c == 0) {
+      const float bt = beta[0];
+      const float bw = fmaxf(bt, bw_floor);
+      dbeta[0] = bt > bw_floor ? 2.f * eps * (float)m * bw * part[0] : 0.f;
+    }
   }
 }
 
@@ -331,7 +347,7 @@ cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, 
                                  float* domega, cudaStream_t st, int* launches) {
   float* df = w.dqbar + (size_t)p.slabs * kD;   // df lives behind dqbar in the same region
   k_band_reduce<<<p.slabs, 32, 0, st>>>(w.bands, p.slabs, p.htiles, p.cfg.levels, df);
-  k_gate_backward<<<1, kD, 0, st>>>(df, w.sg, w.qbar, gate_w, omega, w.sumdD, n_sumdD, beta,
+  k_gate_backward<<<p.cfg.heads + 2, kD, 0, st>>>(df, w.sg, w.qbar, gate_w, omega, w.sumdD, n_sumdD, beta,
                                     p.cfg.eps, p.cfg.bw_floor, p.cfg.features, p.cfg.batch, p.cfg.heads,
                                     p.L1, p.cfg.gate_per_head, dbeta, dgate_w, dgate_b, domega, w.dqbar);
   *launches += 2;
