@@ -162,11 +162,19 @@ __global__ void __launch_bounds__(256, 2) k_haar_filter_split3(const Tin* __rest
 //                        level-l detail coefficients (Delta_l = left half sum - right half sum);
 //   slot 8+l-1:          sum over blocks of s_l(G) * s_l(X) / 2^l, the product of the level-l
 //                        approximation coefficients.
+// G and X are loaded together (both copies in flight at once).  Levels 1-3 live in the thread's
+// 8 x 8 register tiles; the 8-row sums go to a pyramid in shared memory (per tensor and column: 32
+// sums of level 3, then 16, 8, 4, 2, 1 of levels 4-8), from which one thread per column takes the
+// level 4-8 products and every thread the coarse part of its output rows.
+constexpr int kPyr = 63;   // 32 + 16 + 8 + 4 + 2 + 1 block sums per column
+__device__ __forceinline__ int pyr_base(int l) { return 64 - (64 >> (l - 3)); }   // level 3 -> 0, 4 -> 32, 5 -> 48 ...
+
 template <typename Tin, typename Tout>
 __global__ void __launch_bounds__(256) k_haar_backward(const Tin* __restrict__ X, const float* __restrict__ G,
                                                        const float* __restrict__ f, Tout* __restrict__ dX,
                                                        float* __restrict__ bands, int n, int L) {
-  __shared__ float sh[8][kD];
+  __shared__ float pyr[2][kPyr][kD];    // [0] = G, [1] = X
+  __shared__ float hit[32][kD];         // coarse part of the output of row group rg, per column
   __shared__ float red[8][kBandVals];
   const int slab = blockIdx.y;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -176,65 +184,92 @@ __global__ void __launch_bounds__(256) k_haar_backward(const Tin* __restrict__ X
   float acc[kBandVals];
 #pragma unroll
   for (int i = 0; i < kBandVals; ++i) acc[i] = 0.f;
-  float g[8][8];
-  Sums sg;
+  float g[8][8], x[8][8];
   load_tile(G + (size_t)slab * n * kD, n, row0, g);
-  block_sums(g, sg, sh, L);
+  load_tile(X + (size_t)slab * n * kD, n, row0, x);
+  // levels 1-3: products from the register tiles, 8-row sums into the pyramid
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    float g1[4], x1[4];
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+      g1[p] = g[2 * p][c] + g[2 * p + 1][c];
+      x1[p] = x[2 * p][c] + x[2 * p + 1][c];
+      acc[0] += (g[2 * p][c] - g[2 * p + 1][c]) * (x[2 * p][c] - x[2 * p + 1][c]);
+      acc[8] += g1[p] * x1[p];
+    }
+    const float g20 = g1[0] + g1[1], g21 = g1[2] + g1[3], x20 = x1[0] + x1[1], x21 = x1[2] + x1[3];
+    acc[1] += (g1[0] - g1[1]) * (x1[0] - x1[1]) + (g1[2] - g1[3]) * (x1[2] - x1[3]);
+    acc[9] += g20 * x20 + g21 * x21;
+    const float g3 = g20 + g21, x3 = x20 + x21;
+    acc[2] += (g20 - g21) * (x20 - x21);
+    acc[10] += g3 * x3;
+    pyr[0][rg][cg * 8 + c] = g3;
+    pyr[1][rg][cg * 8 + c] = x3;
+  }
+  __syncthreads();
+  // levels 4-8 of the pyramid: thread (tensor = tid >> 6, column = tid & 63), tid < 128
+  if (threadIdx.x < 128) {
+    float(*py)[kD] = pyr[threadIdx.x >> 6];
+    const int col = threadIdx.x & 63;
+#pragma unroll
+    for (int l = 4; l <= 8; ++l) {
+      const int src = pyr_base(l - 1), dst = pyr_base(l), cnt = 256 >> l;
+      for (int b2 = 0; b2 < cnt; ++b2) py[dst + b2][col] = py[src + 2 * b2][col] + py[src + 2 * b2 + 1][col];
+    }
+  }
+  __syncthreads();
+  // level 4-8 products: one thread per column
+  if (threadIdx.x < kD) {
+    const int col = threadIdx.x;
+#pragma unroll
+    for (int l = 4; l <= 8; ++l) {
+      const int src = pyr_base(l - 1), dst = pyr_base(l), cnt = 256 >> l;
+      float dsum = 0.f, asum = 0.f;
+      for (int b2 = 0; b2 < cnt; ++b2) {
+        dsum += (pyr[0][src + 2 * b2][col] - pyr[0][src + 2 * b2 + 1][col]) *
+                (pyr[1][src + 2 * b2][col] - pyr[1][src + 2 * b2 + 1][col]);
+        asum += pyr[0][dst + b2][col] * pyr[1][dst + b2][col];
+      }
+      acc[l - 1] = dsum;
+      acc[8 + l - 1] = asum;
+    }
+  }
+  // coarse part of the output rows: hit[r][col] = sum_{l=3..8} k_l * s_l(block of row group r)
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int e = threadIdx.x + 256 * i, r = e >> 6, col = e & 63;
+    float v = k.k[3] * pyr[0][r][col];
+#pragma unroll
+    for (int l = 4; l <= 8; ++l) v += k.k[l] * pyr[0][pyr_base(l) + (r >> (l - 3))][col];
+    hit[r][col] = v;
+  }
+  __syncthreads();
   {
     Tout* dst = dX + (size_t)slab * n * kD + cg * 8;
-    // same expression as apply_filter, row by row, so that g survives for the band products
+    float hi[8], s1[4][8], s2[2][8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      hi[c] = hit[rg][cg * 8 + c];
+#pragma unroll
+      for (int p = 0; p < 4; ++p) s1[p][c] = g[2 * p][c] + g[2 * p + 1][c];
+      s2[0][c] = s1[0][c] + s1[1][c];
+      s2[1][c] = s1[2][c] + s1[3][c];
+    }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       float y[8];
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const float hi = k.k[3] * sg.s3[c] + k.k[4] * sg.s4[c] + k.k[5] * sg.s5[c] + k.k[6] * sg.s6[c] +
-                         k.k[7] * sg.s7[c] + k.k[8] * sg.s8[c];
-        y[c] = k.f0 * g[j][c] + k.k[1] * sg.s1[j >> 1][c] + k.k[2] * sg.s2[j >> 2][c] + hi;
-      }
+      for (int c = 0; c < 8; ++c) y[c] = k.f0 * g[j][c] + k.k[1] * s1[j >> 1][c] + k.k[2] * s2[j >> 2][c] + hi[c];
       if (row0 + j < n) store8(dst + (size_t)(row0 + j) * kD, y);
     }
   }
-  {
-    float x[8][8];
-    Sums sx;
-    load_tile(X + (size_t)slab * n * kD, n, row0, x);
-    block_sums(x, sx, sh, L);
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-#pragma unroll
-      for (int p = 0; p < 4; ++p) {
-        acc[0] += (g[2 * p][c] - g[2 * p + 1][c]) * (x[2 * p][c] - x[2 * p + 1][c]);
-        acc[8] += sg.s1[p][c] * sx.s1[p][c];
-      }
-#pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        acc[1] += (sg.s1[2 * q][c] - sg.s1[2 * q + 1][c]) * (sx.s1[2 * q][c] - sx.s1[2 * q + 1][c]);
-        acc[9] += sg.s2[q][c] * sx.s2[q][c];
-      }
-      acc[2] += (sg.s2[0][c] - sg.s2[1][c]) * (sx.s2[0][c] - sx.s2[1][c]);
-      acc[10] += sg.s3[c] * sx.s3[c];
-      // levels 4..8: every lane of a block holds the same block sum; the weights undo the
-      // replication (2, 4, 8, 16, 32 holders per column).
-      acc[3] += (sg.s3[c] - sg.p3[c]) * (sx.s3[c] - sx.p3[c]);
-      acc[11] += sg.s4[c] * sx.s4[c];
-      acc[4] += (sg.s4[c] - sg.p4[c]) * (sx.s4[c] - sx.p4[c]);
-      acc[12] += sg.s5[c] * sx.s5[c];
-      acc[5] += (sg.s5[c] - sg.p5[c]) * (sx.s5[c] - sx.p5[c]);
-      acc[13] += sg.s6[c] * sx.s6[c];
-      acc[6] += (sg.s6[c] - sg.p6[c]) * (sx.s6[c] - sx.p6[c]);
-      acc[14] += sg.s7[c] * sx.s7[c];
-      acc[7] += (sg.s7[c] - sg.p7[c]) * (sx.s7[c] - sx.p7[c]);
-      acc[15] += sg.s8[c] * sx.s8[c];
-    }
-  }
-  // 1/2^l normalisation times 1/replication.
-  const float wgt[8] = {0.5f, 0.25f, 0.125f, 0.0625f * 0.5f, 0.03125f * 0.25f, 0.015625f * 0.125f,
-                        0.0078125f * 0.0625f, 0.00390625f * 0.03125f};
+  // 1 / 2^l normalisation
 #pragma unroll
   for (int l = 0; l < 8; ++l) {
-    acc[l] *= wgt[l];
-    acc[8 + l] *= wgt[l];
+    const float wgt = 1.f / (float)(2 << l);
+    acc[l] *= wgt;
+    acc[8 + l] *= wgt;
   }
 #pragma unroll
   for (int i = 0; i < kBandVals; ++i) {
