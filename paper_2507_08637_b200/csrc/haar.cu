@@ -170,7 +170,7 @@ constexpr int kPyr = 63;   // 32 + 16 + 8 + 4 + 2 + 1 block sums per column
 __device__ __forceinline__ int pyr_base(int l) { return 64 - (64 >> (l - 3)); }   // level 3 -> 0, 4 -> 32, 5 -> 48 ...
 
 template <typename Tin, typename Tout>
-__global__ void __launch_bounds__(256) k_haar_backward(const Tin* __restrict__ X, const float* __restrict__ G,
+__global__ void __launch_bounds__(256, 2) k_haar_backward(const Tin* __restrict__ X, const float* __restrict__ G,
                                                        const float* __restrict__ f, Tout* __restrict__ dX,
                                                        float* __restrict__ bands, int n, int L) {
   __shared__ float pyr[2][kPyr][kD];    // [0] = G, [1] = X
