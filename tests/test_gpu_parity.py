@@ -252,6 +252,7 @@ BWD_SMALL = [
     dict(B=2, H=2, n=1024, d=64, L=5, m=128),
     dict(B=1, H=2, n=1000, d=64, L=8, m=256),
     dict(B=2, H=3, n=512, d=64, L=4, m=64, gate_per_head=0),
+    dict(B=5, H=1, n=300, d=64, L=4, m=128),   # more batch elements than the four-way split of the domega sum, ragged n
 ]
 
 
