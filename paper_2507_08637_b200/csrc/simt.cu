@@ -422,7 +422,24 @@ __global__ void __launch_bounds__(256) k_simt_bwd_kside(const float* __restrict_
   }
 }
 
-// S[slab][i] = sum_chunks part[slab][chunk][i] in chunk order.  One thread per element of [S | z].
+// S[slab][i] = sum over chunks of part[slab][chunk][i], always in the same order: four running sums
+// take the chunks k = 0, 1, 2, 3 (mod 4) in increasing k (four loads in flight instead of one) and are
+// added as (a0 + a1) + (a2 + a3).  One thread per element of [S | z].
+__device__ __forceinline__ float sum_chunks4(const float* __restrict__ p, size_t stride, int chunks) {
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+  int k = 0;
+  for (; k + 4 <= chunks; k += 4) {
+    a0 += p[(size_t)k * stride];
+    a1 += p[(size_t)(k + 1) * stride];
+    a2 += p[(size_t)(k + 2) * stride];
+    a3 += p[(size_t)(k + 3) * stride];
+  }
+  if (k < chunks) a0 += p[(size_t)k * stride];
+  if (k + 1 < chunks) a1 += p[(size_t)(k + 1) * stride];
+  if (k + 2 < chunks) a2 += p[(size_t)(k + 2) * stride];
+  return (a0 + a1) + (a2 + a3);
+}
+
 __global__ void __launch_bounds__(256) k_reduce_partials(const float* __restrict__ spart,
                                                          const float* __restrict__ zpart, int chunks, int m,
                                                          float* __restrict__ S, float* __restrict__ z,
@@ -431,15 +448,12 @@ __global__ void __launch_bounds__(256) k_reduce_partials(const float* __restrict
   const int i = blockIdx.x * 256 + threadIdx.x;
   const int ns = m * kD;
   if (i < ns) {
-    float s = 0.f;
-    for (int k = 0; k < chunks; ++k) s += spart[((size_t)slab * chunks + k) * ns + i];
+    const float s = sum_chunks4(spart + (size_t)slab * chunks * ns + i, ns, chunks);
     S[(size_t)slab * ns + i] = s;
     if (Sbf != nullptr) Sbf[(size_t)slab * ns + i] = __float2bfloat16_rn(s);
   } else if (i < ns + m) {
     const int r = i - ns;
-    float s = 0.f;
-    for (int k = 0; k < chunks; ++k) s += zpart[((size_t)slab * chunks + k) * m + r];
-    z[(size_t)slab * m + r] = s;
+    z[(size_t)slab * m + r] = sum_chunks4(zpart + (size_t)slab * chunks * m + r, m, chunks);
   }
 }
 
