@@ -6,14 +6,15 @@
 //
 // Key side  (Eq. 7, key summary):  S' = ReLU(K_F W)^T V,  z' = ReLU(K_F W)^T 1  per sequence chunk.
 //   MMA1: D1[128 features x 128 tokens] = W^T (smem, K-major) * K_F^T (smem, K-major)   -> TMEM fp32
-//   ReLU warps: TMEM -> registers -> max(.,0) -> bf16 -> back into the same TMEM columns
+//   ReLU warps: TMEM -> registers -> max(.,0) -> bf16 -> back into the same TMEM columns; the row sums
+//   z' come from a tree of packed bf16 adds over the rounded values
 //   MMA2: S'[128 features x 64] += Phi^T (TMEM operand, K = tokens) * V (smem, N-major)  -> TMEM fp32
 // Query side (Eq. 7, output):  O = ReLU(Q_F W) S' / (ReLU(Q_F W) z' + eps')
 //   MMA1: D1[128 tokens x 128 features] = Q_F (smem, K-major) * W (as W^T, K-major)
-//   ReLU warps as above, plus the row dot product with z' (denominator)
-//   MMA2: N'[128 tokens x 64] (+)= Phi (TMEM operand, K = features) * S' (smem bf16, N-major)
-//   epilogue (ReLU warpgroup t & 1 for tile t): TMEM -> registers -> * 1/(D' + eps') -> bf16 ->
-//   swizzled smem -> TMA store
+//   ReLU warps: TMEM -> registers -> max(.,0) -> bf16 -> TMEM, nothing else
+//   MMA2: [N' | D'][128 tokens x 80] (+)= Phi (TMEM operand, K = features) * [S' | z' | 0] (smem bf16
+//   image, K-major): column 64 of the accumulator is the denominator
+//   epilogue warps: TMEM -> registers -> * 1/(D' + eps') -> bf16 -> swizzled smem -> TMA store
 //
 // Work unit of the MMA pipeline: one 128-token tile times one 128-feature half ("unit").  Three D1
 // accumulators rotate, so the ReLU pass of a unit overlaps four MMAs of its neighbours.
