@@ -189,7 +189,7 @@ template <int NH, typename TG>
 __global__ void __launch_bounds__(256, 1)
 k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant__ CUtensorMap map_v,
                const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ dSbf,
-               const float* __restrict__ dzg, TG* __restrict__ dV, float* __restrict__ dKF, int n, int chunk_tiles,
+               const float* __restrict__ dzg, TG* __restrict__ dV, float* __restrict__ dKF, int n, int slabs,
                int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -197,10 +197,14 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
   BwdBars* bars = reinterpret_cast<BwdBars*>(smem + SL::bars);
   float* dzs = reinterpret_cast<float*>(smem + SL::dz);
   const int warp = threadIdx.x >> 5;
-  const int chunk = blockIdx.x, slab = blockIdx.y;
-  const int tiles_total = (n + kTile - 1) / kTile;
-  const int tile0 = chunk * chunk_tiles;
-  const int ntiles = min(chunk_tiles, tiles_total - tile0);
+  // The tiles of all slabs form one list (slab-major) that the CTAs share evenly: a tile of this side
+  // depends on no other tile, only on the dS' image and dz' of its slab, which are reloaded when the
+  // CTA's range crosses into the next slab.
+  const int tiles_per_slab = (n + kTile - 1) / kTile;
+  const long long tiles_all = (long long)tiles_per_slab * slabs;
+  const int g0 = (int)(tiles_all * blockIdx.x / gridDim.x);
+  const int ntiles = (int)(tiles_all * (blockIdx.x + 1) / gridDim.x) - g0;
+  int cur_slab = g0 / tiles_per_slab;
   constexpr int m = NH * 128;
   constexpr uint32_t kCols = NH * 256;            // TMEM columns: NH accumulators of 128, then dV / dK_F (64)
 
@@ -216,8 +220,8 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
     tmem_relinquish();
   }
   load_rows_swizzled(smem + SL::wt, Wt, m);
-  load_rows_swizzled(smem + SL::ds, dSbf + (size_t)slab * m * kD, m);
-  for (int i = threadIdx.x; i < m; i += blockDim.x) dzs[i] = dzg[(size_t)slab * m + i];
+  load_rows_swizzled(smem + SL::ds, dSbf + (size_t)cur_slab * m * kD, m);
+  for (int i = threadIdx.x; i < m; i += blockDim.x) dzs[i] = dzg[(size_t)cur_slab * m + i];
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
@@ -232,7 +236,6 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
   const uint32_t ds_k = smem_desc_lo(smem_u32(smem + SL::ds), 16), ds_n = smem_desc_lo(smem_u32(smem + SL::ds), 1024);
   const uint32_t stage_k = smem_desc_lo(smem_u32(smem + SL::stage), 16);
   constexpr uint32_t kTileStep = kTileBytes >> 4, kStageStep = SL::stage_bytes >> 4;
-  const int slabs = gridDim.y;
   uint32_t mma_par = 0;
   int issued = 0;
   bool ok = true;
@@ -242,7 +245,8 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
   auto issue_copies = [&](int t) {
     uint8_t* dst = smem + SL::stage + (t & 1) * SL::stage_bytes;
     uint64_t* bar = &bars->full[t & 1];
-    const int r0 = (tile0 + t) * kTile;
+    const int slab = (g0 + t) / tiles_per_slab;
+    const int r0 = ((g0 + t) - slab * tiles_per_slab) * kTile;
     mbar_arrive_expect_tx(bar, 4 * kTileBytes);
 #pragma unroll
     for (int pl = 0; pl < 3; ++pl) tma_load_3d(dst + pl * kTileBytes, &map_kf, 0, r0, pl * slabs + slab, bar);
@@ -254,9 +258,17 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
   }
 
   for (int ti = 0; ti < ntiles && ok; ++ti) {
-    const int row0 = (tile0 + ti) * kTile;
+    const int slab = (g0 + ti) / tiles_per_slab;
+    const int row0 = ((g0 + ti) - slab * tiles_per_slab) * kTile;
     const int row = row0 + tl;
     const uint32_t x_k = stage_k + (ti & 1) * kStageStep, v_k = x_k + 3 * kTileStep;
+    if (slab != cur_slab) {   // uniform over the CTA; every MMA of the previous tile has completed
+      cur_slab = slab;
+      load_rows_swizzled(smem + SL::ds, dSbf + (size_t)slab * m * kD, m);
+      for (int i = threadIdx.x; i < m; i += blockDim.x) dzs[i] = dzg[(size_t)slab * m + i];
+      fence_proxy_async_smem();
+      __syncthreads();
+    }
     // ---- copies of the next tile (its stage was released by the barrier that ended tile ti - 1), MMA1
     if (threadIdx.x == 0 && ti + 1 < ntiles) {
       issue_copies(ti + 1);
@@ -716,9 +728,10 @@ cudaError_t launch_kside(const Plan& p, const Ws& w, const CUtensorMap& map_kf, 
   auto k = k_tc_bwd_kside<NH, TG>;
   cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdKSmem<NH>::total);
   if (err != cudaSuccess) return err;
-  dim3 grid(p.bchunks, p.slabs);
+  const long long tiles_all = (long long)((p.cfg.seq_len + kTile - 1) / kTile) * p.slabs;
+  const unsigned grid = (unsigned)(tiles_all < 148 ? tiles_all : 148);   // one CTA per SM of a B200, one wave
   k<<<grid, 256, BwdKSmem<NH>::total, st>>>(map_kf, map_v, w.Wt, w.dSbf, w.dz, static_cast<TG*>(dV), w.dKF,
-                                            p.cfg.seq_len, p.bchunk_tiles, w.status);
+                                            p.cfg.seq_len, p.slabs, w.status);
   return cudaGetLastError();
 }
 
