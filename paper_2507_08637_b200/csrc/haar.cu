@@ -127,25 +127,64 @@ template <typename Tin>
 __global__ void __launch_bounds__(256, 2) k_haar_filter_split3(const Tin* __restrict__ X, const float* __restrict__ f,
                                                             __nv_bfloat16* __restrict__ XF3, size_t plane, int n,
                                                             int L) {
-  __shared__ float sh[8][kD];
+  // levels 4-8 through a pyramid of the 8-row sums in shared memory (per column: 32 sums of level 3,
+  // then 16, 8, 4, 2, 1), as in k_haar_backward
+  __shared__ float pyr[63][kD];
+  __shared__ float hit[32][kD];   // sum_{l=3..8} k_l * s_l(block of row group r), per column
   const int slab = blockIdx.y;
   const int cg = threadIdx.x & 7, rg = threadIdx.x >> 3;
   const int row0 = blockIdx.x * kHaarTile + rg * 8;
   const LevelCoef k = level_coef(f + (size_t)slab * (L + 1), L);
   float x[8][8];
   load_tile(X + (size_t)slab * n * kD, n, row0, x);
-  Sums s;
-  block_sums(x, s, sh, L);
-  apply_filter(x, s, k);
+#pragma unroll
+  for (int c = 0; c < 8; ++c)
+    pyr[rg][cg * 8 + c] = ((x[0][c] + x[1][c]) + (x[2][c] + x[3][c])) + ((x[4][c] + x[5][c]) + (x[6][c] + x[7][c]));
+  __syncthreads();
+  if (threadIdx.x < kD) {
+    const int col = threadIdx.x;
+    int src = 0, cnt = 16;
+#pragma unroll
+    for (int l = 4; l <= 8; ++l) {
+      const int dst = src + 2 * cnt;
+      for (int b2 = 0; b2 < cnt; ++b2) pyr[dst + b2][col] = pyr[src + 2 * b2][col] + pyr[src + 2 * b2 + 1][col];
+      src = dst;
+      cnt >>= 1;
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int e = threadIdx.x + 256 * i, r = e >> 6, col = e & 63;
+    float v = k.k[3] * pyr[r][col];
+    int base = 32;
+#pragma unroll
+    for (int l = 4; l <= 8; ++l) {
+      v += k.k[l] * pyr[base + (r >> (l - 3))][col];
+      base += 256 >> l;
+    }
+    hit[r][col] = v;
+  }
+  __syncthreads();
   __nv_bfloat16* dst = XF3 + (size_t)slab * n * kD + cg * 8;
+  float hi_c[8], s1[4][8], s2[2][8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    hi_c[c] = hit[rg][cg * 8 + c];
+#pragma unroll
+    for (int p = 0; p < 4; ++p) s1[p][c] = x[2 * p][c] + x[2 * p + 1][c];
+    s2[0][c] = s1[0][c] + s1[1][c];
+    s2[1][c] = s1[2][c] + s1[3][c];
+  }
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     if (row0 + j >= n) continue;
     float hi[8], mid[8], lo[8];
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
-      hi[c] = __bfloat162float(__float2bfloat16_rn(x[j][c]));
-      const float r1 = x[j][c] - hi[c];
+      const float y = k.f0 * x[j][c] + k.k[1] * s1[j >> 1][c] + k.k[2] * s2[j >> 2][c] + hi_c[c];
+      hi[c] = __bfloat162float(__float2bfloat16_rn(y));
+      const float r1 = y - hi[c];
       mid[c] = __bfloat162float(__float2bfloat16_rn(r1));
       lo[c] = r1 - mid[c];
     }
