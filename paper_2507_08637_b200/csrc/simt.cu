@@ -444,6 +444,9 @@ __global__ void __launch_bounds__(256) k_reduce_partials(const float* __restrict
                                                          const float* __restrict__ zpart, int chunks, int m,
                                                          float* __restrict__ S, float* __restrict__ z,
                                                          __nv_bfloat16* __restrict__ Sbf) {
+  // the kernel after this one in the stream may start now if it was launched as a programmatic
+  // dependent (it waits for this grid before it reads S, z, Sbf)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int slab = blockIdx.y;
   const int i = blockIdx.x * 256 + threadIdx.x;
   const int ns = m * kD;

@@ -77,6 +77,13 @@ __device__ __forceinline__ void mbar_wait_drain(uint64_t* bar, uint32_t parity) 
   }
 }
 
+// ---- programmatic dependent launch ----------------------------------------------------------------
+// A kernel launched with the programmatic-stream-serialization attribute may start while the kernel
+// before it in the stream is still running; what that kernel wrote is only visible after
+// griddep_wait().  A kernel lets its dependents start early with griddep_launch().
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- proxies and fences -------------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -81,7 +81,7 @@ struct alignas(8) KsideBars {
 };
 struct alignas(8) QsideBars {
   uint64_t x_full[kNXQ], x_empty[kNXQ], xf_ready[kNF];
-  uint64_t d1_full[6], phi_ready[kND1], d1_free[kND1], d2_full, d2_free;
+  uint64_t d1_full[6], phi_ready[kND1], d1_free[kND1], d2_full, d2_free, simg_ready;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -594,19 +594,20 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
 // Builds that image in shared memory from the bf16 S' (m x 64, row-major) and the fp32 z' of the slab:
 // 64-feature K blocks of 80 rows x 128 bytes (rows 0-63 = columns of S', row 64 = z', rows 65-79 = 0),
 // 128-byte swizzle.
+// Done by `nthr` threads numbered tid = 0 .. nthr - 1.
 __device__ __forceinline__ void load_szt_image(uint8_t* dst, const __nv_bfloat16* __restrict__ Sbf,
-                                               const float* __restrict__ z, int m) {
-  for (int i = threadIdx.x; i < m * (kD / 2); i += blockDim.x) {   // two adjacent columns of one feature
+                                               const float* __restrict__ z, int m, int tid, int nthr) {
+  for (int i = tid; i < m * (kD / 2); i += nthr) {   // two adjacent columns of one feature
     const int f = i / (kD / 2), c = 2 * (i % (kD / 2));
     const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(Sbf + (size_t)f * kD + c);
     uint8_t* blk = dst + (f >> 6) * kSztBlockBytes + (f & 7) * 2;
     *reinterpret_cast<__nv_bfloat16*>(blk + swz128(c, (f & 63) >> 3)) = v.x;
     *reinterpret_cast<__nv_bfloat16*>(blk + swz128(c + 1, (f & 63) >> 3)) = v.y;
   }
-  for (int f = threadIdx.x; f < m; f += blockDim.x)
+  for (int f = tid; f < m; f += nthr)
     *reinterpret_cast<__nv_bfloat16*>(dst + (f >> 6) * kSztBlockBytes + swz128(64, (f & 63) >> 3) + (f & 7) * 2) =
         __float2bfloat16_rn(z[f]);
-  for (int i = threadIdx.x; i < (m >> 6) * 15 * 8; i += blockDim.x) {   // 16-byte chunks of rows 65-79
+  for (int i = tid; i < (m >> 6) * 15 * 8; i += nthr) {   // 16-byte chunks of rows 65-79
     const int kb = i / 120, r = 65 + (i % 120) / 8, c = i & 7;
     *reinterpret_cast<uint4*>(dst + kb * kSztBlockBytes + r * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
   }
@@ -645,6 +646,20 @@ __device__ __forceinline__ void relu_unit_plain(uint32_t taddr) {
   tmem_st_wait();
 }
 
+// The ReLU and epilogue warps (idle while the pipeline fills) build the S' image: S' and z' come from
+// the kernel before this one in the stream, which may still be running (programmatic dependent
+// launch), everything else this kernel reads was complete before that kernel started.
+template <int NH>
+__device__ __forceinline__ void qside_build_simg(uint8_t* simg, const __nv_bfloat16* __restrict__ Sbf,
+                                                 const float* __restrict__ zg, int slab, uint64_t* ready) {
+  constexpr int m = NH * 128;
+  griddep_wait();
+  load_szt_image(simg, Sbf + (size_t)slab * m * kD, zg + (size_t)slab * m, m, threadIdx.x - 32 * kReluWarp0,
+                 32 * (kAuxWarp0Q - kReluWarp0));
+  fence_proxy_async_smem();
+  warp_arrive(ready);
+}
+
 // grid (chunks, slabs), block 768.  TMEM: D1[3] at columns 0 / 128 / 256, [N' | D'] of the current tile
 // at 384 .. 463.  Warps 12-15 are the epilogue: they drain the accumulator of a tile as soon as its
 // last MMA2 has completed (which frees it for the next tile), scale by 1 / (D' + eps'), round to bf16
@@ -680,6 +695,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     }
     mbar_init(&bars->d2_full, 1);
     mbar_init(&bars->d2_free, 4);
+    mbar_init(&bars->simg_ready, kAuxWarp0Q - kReluWarp0);
     bars->abort_flag = 0;
     fence_mbar_init();
   }
@@ -688,7 +704,6 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     tmem_relinquish();
   }
   load_rows_swizzled(smem + SL::wt, Wt, m);
-  load_szt_image(smem + SL::simg, Sbf + (size_t)slab * m * kD, zg + (size_t)slab * m, m);
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
@@ -754,7 +769,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       const uint32_t s_lo = smem_desc_lo(smem_u32(smem + SL::simg), 16);
       const uint32_t d2 = tmem + kAccCol;
       uint32_t p3 = 0, ppar = 0;
-      bool ok = true;
+      bool ok = mbar_wait(&bars->simg_ready, 0, abort_flag, status, kErrMma);   // the [S' | z' | 0]^T image is in place
       for (int t = 0; t < ntiles && ok; ++t) {
         if (t >= 1) {   // the accumulator of tile t - 1 must have been drained
           ok = mbar_wait(&bars->d2_free, (t - 1) & 1, abort_flag, status, kErrMma);
@@ -781,6 +796,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     }
   } else if (warp < kEpiWarp0Q) {
     reg_dec<kRegsReluQ>();
+    qside_build_simg<NH>(smem + SL::simg, Sbf, zg, slab, &bars->simg_ready);
     const int g = (warp - kReluWarp0) >> 2;
     const uint32_t lane_base = 32u * (warp & 3);
     bool ok = true;
@@ -795,6 +811,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     }
   } else if (warp < kAuxWarp0Q) {
     reg_inc<kRegsEpiQ>();
+    qside_build_simg<NH>(smem + SL::simg, Sbf, zg, slab, &bars->simg_ready);
     const int et = threadIdx.x - 32 * kEpiWarp0Q;     // 0..127 = token row of the tile = TMEM lane
     const uint32_t lane_base = 32u * (warp & 3);
     const float bw = fmaxf(beta[0], bw_floor);
@@ -931,30 +948,39 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
   return cudaGetLastError();
 }
 
+// Launched so that it may start while the kernel before it (the reduction that produces S', z') is
+// still running; the kernel waits for that kernel where it first needs its results.
+template <int NH>
+static cudaError_t launch_qside_pdl(const Plan& p, const Ws& w, const CUtensorMap& map_q, const CUtensorMap& map_o,
+                                    const float* beta, cudaStream_t st) {
+  auto k = k_tc_qside<NH>;
+  cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, QsideSmem<NH>::total);
+  if (err != cudaSuccess) return err;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.tchunks, p.slabs);
+  cfg.blockDim = dim3(kThreadsQ);
+  cfg.dynamicSmemBytes = QsideSmem<NH>::total;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k, map_q, map_o, (const __nv_bfloat16*)w.Wt, (const __nv_bfloat16*)w.Sbf,
+                            (const float*)w.z, (const float*)w.f, beta, p.cfg.eps, p.cfg.bw_floor, p.cfg.seq_len,
+                            p.cfg.levels, p.tchunk_blocks, w.status);
+}
+
 cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const float* beta, void* O, cudaStream_t st,
                             int* launches) {
   CUtensorMap map_q, map_o;
   cudaError_t err;
   if ((err = make_tile_map(Q, p.slabs, p.cfg.seq_len, kTile, &map_q)) != cudaSuccess) return err;
   if ((err = make_tile_map(O, p.slabs, p.cfg.seq_len, kTile, &map_o)) != cudaSuccess) return err;
-  dim3 grid(p.tchunks, p.slabs);
-  if (p.cfg.features == 256) {
-    auto k = k_tc_qside<2>;
-    if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, QsideSmem<2>::total)) != cudaSuccess)
-      return err;
-    k<<<grid, kThreadsQ, QsideSmem<2>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
-                                                         p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks,
-                                                         w.status);
-  } else {
-    auto k = k_tc_qside<1>;
-    if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, QsideSmem<1>::total)) != cudaSuccess)
-      return err;
-    k<<<grid, kThreadsQ, QsideSmem<1>::total, st>>>(map_q, map_o, w.Wt, w.Sbf, w.z, w.f, beta, p.cfg.eps,
-                                                         p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks,
-                                                         w.status);
-  }
+  err = p.cfg.features == 256 ? launch_qside_pdl<2>(p, w, map_q, map_o, beta, st)
+                              : launch_qside_pdl<1>(p, w, map_q, map_o, beta, st);
   *launches += 1;
-  return cudaGetLastError();
+  return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 }  // namespace wersa
