@@ -99,6 +99,9 @@ __global__ void __launch_bounds__(256) k_qmean_gate(const T* __restrict__ Q, flo
                                                     int* __restrict__ slab_count, int* __restrict__ batch_count,
                                                     const __nv_bfloat16* __restrict__ W, __nv_bfloat16* __restrict__ Wt,
                                                     int m) {
+  // the key-side kernel may be staged now (programmatic dependent launch; it waits for this grid
+  // before it reads W^T or the gate)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if ((int)blockIdx.y == slabs) {
     for (int i = blockIdx.x * 256 + threadIdx.x; i < m * kD; i += gridDim.x * 256) {
       const int r = i / kD, c = i - r * kD;

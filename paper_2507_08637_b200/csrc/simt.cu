@@ -444,9 +444,11 @@ __global__ void __launch_bounds__(256) k_reduce_partials(const float* __restrict
                                                          const float* __restrict__ zpart, int chunks, int m,
                                                          float* __restrict__ S, float* __restrict__ z,
                                                          __nv_bfloat16* __restrict__ Sbf) {
-  // the kernel after this one in the stream may start now if it was launched as a programmatic
-  // dependent (it waits for this grid before it reads S, z, Sbf)
+  // Programmatic dependent launch: the kernel after this one may be staged now (it waits for this grid
+  // before it reads S, z, Sbf), and this kernel may itself have been staged early: the partials are
+  // complete once the kernel before it has finished.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int slab = blockIdx.y;
   const int i = blockIdx.x * 256 + threadIdx.x;
   const int ns = m * kD;
@@ -501,9 +503,18 @@ cudaError_t launch_reduce_partials(const Plan& p, const float* spart, const floa
                                    float* z, __nv_bfloat16* Sbf, cudaStream_t st, int* launches) {
   const int m = p.cfg.features;
   dim3 grid((m * kD + m + 255) / 256, p.slabs);
-  k_reduce_partials<<<grid, 256, 0, st>>>(spart, zpart, chunks, m, S, z, Sbf);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(256);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t err = cudaLaunchKernelEx(&cfg, k_reduce_partials, spart, zpart, chunks, m, S, z, Sbf);
   *launches += 1;
-  return cudaGetLastError();
+  return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 cudaError_t launch_simt_qside(const Plan& p, const Ws& w, const void* W, const float* beta, void* O,

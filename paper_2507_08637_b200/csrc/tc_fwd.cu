@@ -410,11 +410,26 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
     mbar_init(&bars->acc_done, NH);
     bars->abort_flag = 0;
     fence_mbar_init();
+    // K and V are inputs: the first copies of both rings go out before the dependency wait below
+    for (int b = 0; b < min(2 * nblk, kNXK); ++b) {
+      mbar_arrive_expect_tx(&bars->x_full[b], kTileBytes);
+      tma_load_3d(smem + SL::x + b * kTileBytes, &map_k, 0, blk0 * kBlk + b * kTile, slab, &bars->x_full[b]);
+    }
+    for (int b = 0; b < min(2 * nblk, kNV); ++b) {
+      mbar_arrive_expect_tx(&bars->v_full[b], kTileBytes);
+      tma_load_3d(smem + SL::v + b * kTileBytes, &map_v, 0, blk0 * kBlk + b * kTile, slab, &bars->v_full[b]);
+    }
   }
   if (warp == kWarpMma) {
     tmem_alloc(&bars->tmem_base, kTmemCols);
     tmem_relinquish();
   }
+  // Programmatic dependent launch: this kernel may have started while the mean-pool / gate kernel was
+  // still running, and W^T and the gate coefficients f are that kernel's results.  Only then may the
+  // kernels after this one be staged: the reduction waits for this grid itself, but it lets the query
+  // side start in turn, whose set-up reads W^T and f without a wait of its own.
+  griddep_wait();
+  griddep_launch();
   load_rows_swizzled(smem + SL::wt, Wt, m);
   fence_proxy_async_smem();
   tc_fence_before_sync();
@@ -428,8 +443,8 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
     if (warp == kWarpTma && lane == 0) {
       // One producer for both rings: whichever ring has a free slot gets its next tile, so that a full
       // V ring never holds back the K tiles (and the other way round).
-      int kb = 0, vb = 0;
       const int total = 2 * nblk;   // 128-token tiles
+      int kb = min(total, kNXK), vb = min(total, kNV);   // the first ring of each went out during set-up
       const unsigned long long t0 = global_timer_ns();
       uint32_t spins = 0;
       bool ok = true;
@@ -924,6 +939,24 @@ bool tc_supported(const wersa_config& cfg) {
   return cfg.dtype == WERSA_BF16 && (cfg.features == 128 || cfg.features == 256) && cfg.head_dim == kD;
 }
 
+// Both tensor-core kernels are launched as programmatic dependents of the kernel before them.
+template <typename... Args>
+static cudaError_t launch_pdl(void (*k)(Args...), dim3 grid, int threads, size_t smem, cudaStream_t st, Args... args) {
+  cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k, args...);
+}
+
 cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const void* V, cudaStream_t st,
                             int* launches) {
   CUtensorMap map_k, map_v;
@@ -931,44 +964,14 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
   if ((err = make_tile_map(K, p.slabs, p.cfg.seq_len, kTile, &map_k)) != cudaSuccess) return err;
   if ((err = make_tile_map(V, p.slabs, p.cfg.seq_len, kTile, &map_v)) != cudaSuccess) return err;
   dim3 grid(p.tchunks, p.slabs);
-  if (p.cfg.features == 256) {
-    auto k = k_tc_kside<2>;
-    if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, KsideSmem<2>::total)) != cudaSuccess)
-      return err;
-    k<<<grid, kThreads, KsideSmem<2>::total, st>>>(map_k, map_v, w.Wt, w.f, w.spart, w.zpart, p.cfg.seq_len,
-                                                         p.cfg.levels, p.tchunk_blocks, w.status);
-  } else {
-    auto k = k_tc_kside<1>;
-    if ((err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, KsideSmem<1>::total)) != cudaSuccess)
-      return err;
-    k<<<grid, kThreads, KsideSmem<1>::total, st>>>(map_k, map_v, w.Wt, w.f, w.spart, w.zpart, p.cfg.seq_len,
-                                                         p.cfg.levels, p.tchunk_blocks, w.status);
-  }
+  if (p.cfg.features == 256)
+    err = launch_pdl(k_tc_kside<2>, grid, kThreads, KsideSmem<2>::total, st, map_k, map_v, (const __nv_bfloat16*)w.Wt,
+                     (const float*)w.f, w.spart, w.zpart, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
+  else
+    err = launch_pdl(k_tc_kside<1>, grid, kThreads, KsideSmem<1>::total, st, map_k, map_v, (const __nv_bfloat16*)w.Wt,
+                     (const float*)w.f, w.spart, w.zpart, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
   *launches += 1;
-  return cudaGetLastError();
-}
-
-// Launched so that it may start while the kernel before it (the reduction that produces S', z') is
-// still running; the kernel waits for that kernel where it first needs its results.
-template <int NH>
-static cudaError_t launch_qside_pdl(const Plan& p, const Ws& w, const CUtensorMap& map_q, const CUtensorMap& map_o,
-                                    const float* beta, cudaStream_t st) {
-  auto k = k_tc_qside<NH>;
-  cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, QsideSmem<NH>::total);
-  if (err != cudaSuccess) return err;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(p.tchunks, p.slabs);
-  cfg.blockDim = dim3(kThreadsQ);
-  cfg.dynamicSmemBytes = QsideSmem<NH>::total;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, k, map_q, map_o, (const __nv_bfloat16*)w.Wt, (const __nv_bfloat16*)w.Sbf,
-                            (const float*)w.z, (const float*)w.f, beta, p.cfg.eps, p.cfg.bw_floor, p.cfg.seq_len,
-                            p.cfg.levels, p.tchunk_blocks, w.status);
+  return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const float* beta, void* O, cudaStream_t st,
@@ -977,8 +980,17 @@ cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const flo
   cudaError_t err;
   if ((err = make_tile_map(Q, p.slabs, p.cfg.seq_len, kTile, &map_q)) != cudaSuccess) return err;
   if ((err = make_tile_map(O, p.slabs, p.cfg.seq_len, kTile, &map_o)) != cudaSuccess) return err;
-  err = p.cfg.features == 256 ? launch_qside_pdl<2>(p, w, map_q, map_o, beta, st)
-                              : launch_qside_pdl<1>(p, w, map_q, map_o, beta, st);
+  // (the query side may start while the reduction that produces S', z' is still running; it waits for
+  // that kernel where it first needs its results)
+  dim3 grid(p.tchunks, p.slabs);
+  if (p.cfg.features == 256)
+    err = launch_pdl(k_tc_qside<2>, grid, kThreadsQ, QsideSmem<2>::total, st, map_q, map_o, (const __nv_bfloat16*)w.Wt,
+                     (const __nv_bfloat16*)w.Sbf, (const float*)w.z, (const float*)w.f, beta, p.cfg.eps,
+                     p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
+  else
+    err = launch_pdl(k_tc_qside<1>, grid, kThreadsQ, QsideSmem<1>::total, st, map_q, map_o, (const __nv_bfloat16*)w.Wt,
+                     (const __nv_bfloat16*)w.Sbf, (const float*)w.z, (const float*)w.f, beta, p.cfg.eps,
+                     p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
   *launches += 1;
   return err != cudaSuccess ? err : cudaGetLastError();
 }
