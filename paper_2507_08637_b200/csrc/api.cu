@@ -106,7 +106,7 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
     p->off_dS = take(sizeof(float) * slabs * m * kD);
     p->off_dz = take(sizeof(float) * slabs * m);
     p->off_sumdD = take(sizeof(float) * slabs * p->schunks);
-    p->off_bands = take(sizeof(float) * 2 * slabs * p->htiles * kBandVals);
+    p->off_bands = take(sizeof(float) * 2 * slabs * 2 * p->htiles * kBandVals);   // Q and K; two column halves per tile
     p->off_dqbar = take(sizeof(float) * slabs * (kD + kBandVals));
     p->off_dQF = take(sizeof(float) * slab_elems);
     p->off_dKF = take(sizeof(float) * slab_elems);

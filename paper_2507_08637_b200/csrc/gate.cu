@@ -349,7 +349,7 @@ cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, 
                                  const float* omega, int n_sumdD, float* dbeta, float* dgate_w, float* dgate_b,
                                  float* domega, cudaStream_t st, int* launches) {
   float* df = w.dqbar + (size_t)p.slabs * kD;   // df lives behind dqbar in the same region
-  k_band_reduce<<<p.slabs, 32, 0, st>>>(w.bands, p.slabs, p.htiles, p.cfg.levels, df);
+  k_band_reduce<<<p.slabs, 32, 0, st>>>(w.bands, p.slabs, 2 * p.htiles, p.cfg.levels, df);   // two partials per tile
   k_gate_backward<<<p.cfg.heads + 2, kD, 0, st>>>(df, w.sg, w.qbar, gate_w, omega, w.sumdD, n_sumdD, beta,
                                     p.cfg.eps, p.cfg.bw_floor, p.cfg.features, p.cfg.batch, p.cfg.heads,
                                     p.L1, p.cfg.gate_per_head, dbeta, dgate_w, dgate_b, domega, w.dqbar);

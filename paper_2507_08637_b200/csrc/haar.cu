@@ -201,34 +201,73 @@ __global__ void __launch_bounds__(256, 2) k_haar_filter_split3(const Tin* __rest
 //                        level-l detail coefficients (Delta_l = left half sum - right half sum);
 //   slot 8+l-1:          sum over blocks of s_l(G) * s_l(X) / 2^l, the product of the level-l
 //                        approximation coefficients.
-// G and X are loaded together (both copies in flight at once).  Levels 1-3 live in the thread's
-// 8 x 8 register tiles; the 8-row sums go to a pyramid in shared memory (per tensor and column: 32
-// sums of level 3, then 16, 8, 4, 2, 1 of levels 4-8), from which one thread per column takes the
-// level 4-8 products and every thread the coarse part of its output rows.
-constexpr int kPyr = 63;   // 32 + 16 + 8 + 4 + 2 + 1 block sums per column
+// The transform acts on every column separately, so one CTA takes 256 rows x 32 columns (half of the
+// head dimension): 8 rows x 4 columns per thread, a small register tile (three CTAs per SM keep loads,
+// arithmetic and stores of different tiles overlapped).  G and X are loaded together.  Levels 1-3 live
+// in the register tiles; the 8-row sums go to a pyramid in shared memory (per tensor and column: 32
+// sums of level 3, then 16, 8, 4, 2, 1 of levels 4-8), from which one thread per column takes the level
+// 4-8 products and every thread the coarse part of its output rows.
+// grid (2 * htiles, slabs): blockIdx.x = 2 * tile + column half; one band partial per CTA.
+constexpr int kPyr = 63;    // 32 + 16 + 8 + 4 + 2 + 1 block sums per column
+constexpr int kHalfD = kD / 2;
 __device__ __forceinline__ int pyr_base(int l) { return 64 - (64 >> (l - 3)); }   // level 3 -> 0, 4 -> 32, 5 -> 48 ...
 
+__device__ __forceinline__ void load4(const float* p, float (&v)[4]) {
+  const float4 a = *reinterpret_cast<const float4*>(p);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&v)[4]) {
+  const uint2 raw = *reinterpret_cast<const uint2*>(p);
+  v[0] = __uint_as_float(raw.x << 16);
+  v[1] = __uint_as_float(raw.x & 0xFFFF0000u);
+  v[2] = __uint_as_float(raw.y << 16);
+  v[3] = __uint_as_float(raw.y & 0xFFFF0000u);
+}
+__device__ __forceinline__ void store4(float* p, const float (&v)[4]) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+__device__ __forceinline__ void store4(__nv_bfloat16* p, const float (&v)[4]) {
+  const __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b2 = __floats2bfloat162_rn(v[2], v[3]);
+  uint2 raw;
+  raw.x = *reinterpret_cast<const uint32_t*>(&a);
+  raw.y = *reinterpret_cast<const uint32_t*>(&b2);
+  *reinterpret_cast<uint2*>(p) = raw;
+}
+
 template <typename Tin, typename Tout>
-__global__ void __launch_bounds__(256, 2) k_haar_backward(const Tin* __restrict__ X, const float* __restrict__ G,
-                                                       const float* __restrict__ f, Tout* __restrict__ dX,
-                                                       float* __restrict__ bands, int n, int L) {
-  __shared__ float pyr[2][kPyr][kD];    // [0] = G, [1] = X
-  __shared__ float hit[32][kD];         // coarse part of the output of row group rg, per column
+__global__ void __launch_bounds__(256, 3) k_haar_backward(const Tin* __restrict__ X, const float* __restrict__ G,
+                                                          const float* __restrict__ f, Tout* __restrict__ dX,
+                                                          float* __restrict__ bands, int n, int L) {
+  __shared__ float pyr[2][kPyr][kHalfD];   // [0] = G, [1] = X
+  __shared__ float hit[32][kHalfD];        // coarse part of the output of row group rg, per column
   __shared__ float red[8][kBandVals];
-  const int slab = blockIdx.y;
+  const int slab = blockIdx.y, half = blockIdx.x & 1;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int cg = threadIdx.x & 7, rg = threadIdx.x >> 3;
-  const int row0 = blockIdx.x * kHaarTile + rg * 8;
+  const int row0 = (blockIdx.x >> 1) * kHaarTile + rg * 8;
+  const int col0 = half * kHalfD + cg * 4;   // first of this thread's four columns
   const LevelCoef k = level_coef(f + (size_t)slab * (L + 1), L);
   float acc[kBandVals];
 #pragma unroll
   for (int i = 0; i < kBandVals; ++i) acc[i] = 0.f;
-  float g[8][8], x[8][8];
-  load_tile(G + (size_t)slab * n * kD, n, row0, g);
-  load_tile(X + (size_t)slab * n * kD, n, row0, x);
+  float g[8][4], x[8][4];
+  {
+    const float* gp = G + (size_t)slab * n * kD + col0;
+    const Tin* xp = X + (size_t)slab * n * kD + col0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (row0 + j < n) {
+        load4(gp + (size_t)(row0 + j) * kD, g[j]);
+        load4(xp + (size_t)(row0 + j) * kD, x[j]);
+      } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) g[j][c] = x[j][c] = 0.f;
+      }
+    }
+  }
   // levels 1-3: products from the register tiles, 8-row sums into the pyramid
 #pragma unroll
-  for (int c = 0; c < 8; ++c) {
+  for (int c = 0; c < 4; ++c) {
     float g1[4], x1[4];
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
@@ -243,14 +282,14 @@ __global__ void __launch_bounds__(256, 2) k_haar_backward(const Tin* __restrict_
     const float g3 = g20 + g21, x3 = x20 + x21;
     acc[2] += (g20 - g21) * (x20 - x21);
     acc[10] += g3 * x3;
-    pyr[0][rg][cg * 8 + c] = g3;
-    pyr[1][rg][cg * 8 + c] = x3;
+    pyr[0][rg][cg * 4 + c] = g3;
+    pyr[1][rg][cg * 4 + c] = x3;
   }
   __syncthreads();
-  // levels 4-8 of the pyramid: thread (tensor = tid >> 6, column = tid & 63), tid < 128
-  if (threadIdx.x < 128) {
-    float(*py)[kD] = pyr[threadIdx.x >> 6];
-    const int col = threadIdx.x & 63;
+  // levels 4-8 of the pyramid: thread (tensor = tid >> 5, column = tid & 31), tid < 64
+  if (threadIdx.x < 2 * kHalfD) {
+    float(*py)[kHalfD] = pyr[threadIdx.x >> 5];
+    const int col = threadIdx.x & 31;
 #pragma unroll
     for (int l = 4; l <= 8; ++l) {
       const int src = pyr_base(l - 1), dst = pyr_base(l), cnt = 256 >> l;
@@ -259,7 +298,7 @@ __global__ void __launch_bounds__(256, 2) k_haar_backward(const Tin* __restrict_
   }
   __syncthreads();
   // level 4-8 products: one thread per column
-  if (threadIdx.x < kD) {
+  if (threadIdx.x < kHalfD) {
     const int col = threadIdx.x;
 #pragma unroll
     for (int l = 4; l <= 8; ++l) {
@@ -276,8 +315,8 @@ __global__ void __launch_bounds__(256, 2) k_haar_backward(const Tin* __restrict_
   }
   // coarse part of the output rows: hit[r][col] = sum_{l=3..8} k_l * s_l(block of row group r)
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int e = threadIdx.x + 256 * i, r = e >> 6, col = e & 63;
+  for (int i = 0; i < 4; ++i) {
+    const int e = threadIdx.x + 256 * i, r = e >> 5, col = e & 31;
     float v = k.k[3] * pyr[0][r][col];
 #pragma unroll
     for (int l = 4; l <= 8; ++l) v += k.k[l] * pyr[0][pyr_base(l) + (r >> (l - 3))][col];
@@ -285,11 +324,11 @@ __global__ void __launch_bounds__(256, 2) k_haar_backward(const Tin* __restrict_
   }
   __syncthreads();
   {
-    Tout* dst = dX + (size_t)slab * n * kD + cg * 8;
-    float hi[8], s1[4][8], s2[2][8];
+    Tout* dst = dX + (size_t)slab * n * kD + col0;
+    float hi[4], s1[4][4], s2[2][4];
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      hi[c] = hit[rg][cg * 8 + c];
+    for (int c = 0; c < 4; ++c) {
+      hi[c] = hit[rg][cg * 4 + c];
 #pragma unroll
       for (int p = 0; p < 4; ++p) s1[p][c] = g[2 * p][c] + g[2 * p + 1][c];
       s2[0][c] = s1[0][c] + s1[1][c];
@@ -297,10 +336,10 @@ __global__ void __launch_bounds__(256, 2) k_haar_backward(const Tin* __restrict_
     }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      float y[8];
+      float y[4];
 #pragma unroll
-      for (int c = 0; c < 8; ++c) y[c] = k.f0 * g[j][c] + k.k[1] * s1[j >> 1][c] + k.k[2] * s2[j >> 2][c] + hi[c];
-      if (row0 + j < n) store8(dst + (size_t)(row0 + j) * kD, y);
+      for (int c = 0; c < 4; ++c) y[c] = k.f0 * g[j][c] + k.k[1] * s1[j >> 1][c] + k.k[2] * s2[j >> 2][c] + hi[c];
+      if (row0 + j < n) store4(dst + (size_t)(row0 + j) * kD, y);
     }
   }
   // 1 / 2^l normalisation
@@ -360,9 +399,9 @@ cudaError_t launch_haar_filter_split3(const Plan& p, const void* X, int in_kind,
 
 cudaError_t launch_haar_backward(const Plan& p, const Ws& w, const void* X, int in_kind, const float* G,
                                  void* dX, int out_kind, int which, cudaStream_t st, int* launches) {
-  dim3 grid(p.htiles, p.slabs);
+  dim3 grid(2 * p.htiles, p.slabs);   // two column halves per 256-row tile
   const int n = p.cfg.seq_len, L = p.cfg.levels;
-  float* bands = w.bands + (size_t)which * p.slabs * p.htiles * kBandVals;
+  float* bands = w.bands + (size_t)which * p.slabs * 2 * p.htiles * kBandVals;
   if (in_kind == 1 && out_kind == 1)
     k_haar_backward<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
         (const __nv_bfloat16*)X, G, w.f, (__nv_bfloat16*)dX, bands, n, L);
