@@ -354,9 +354,106 @@ __device__ __forceinline__ void haar_block_inplace(uint8_t* tile0, uint8_t* tile
   }
 }
 
+// The same filter with plain fp32 registers instead of packed pairs (bit-identical: the packed operations
+// round each half like the scalar ones).  Which of the two compiles into the faster stage differs between
+// the two kernels: the key side uses this one, the query side the packed one.
+__device__ __forceinline__ void haar_block_inplace_scalar(uint8_t* tile0, uint8_t* tile1, const f32x2* hcoef, bool cross,
+                                                   float* xch, int ht, int valid_rows, bool ok) {
+  const int c = ht & 7, rg = ht >> 3, lane = ht & 31, hw = ht >> 5;
+  uint8_t* base = (rg < 16 ? tile0 : tile1) + (rg & 15) * 1024;   // rows 0-127 / 128-255 of the block
+  const float* hc = reinterpret_cast<const float*>(hcoef);        // entry i of the pair table = hc[2 i]
+  float x[8][8];   // 8 rows x 8 columns
+  float hi[8], s5[8];
+  if (ok) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {   // row 8 rg + j has swizzle phase j
+      const uint4 raw = *reinterpret_cast<const uint4*>(base + j * 128 + ((c ^ j) << 4));
+      const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        x[j][2 * i] = __uint_as_float(u[i] << 16);
+        x[j][2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
+      }
+    }
+    const float k3 = hc[6], k4 = hc[8], k5 = hc[10];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const float s3 = ((x[0][q] + x[1][q]) + (x[2][q] + x[3][q])) + ((x[4][q] + x[5][q]) + (x[6][q] + x[7][q]));
+      const float s4 = s3 + __shfl_xor_sync(0xffffffffu, s3, 8);
+      s5[q] = s4 + __shfl_xor_sync(0xffffffffu, s4, 16);
+      hi[q] = fmaf(k3, s3, fmaf(k4, s4, k5 * s5[q]));
+    }
+  }
+  if (cross) {   // uniform over the kernel: L > 5
+    if (ok && (lane >> 3) == 0) {
+      float4* dst = reinterpret_cast<float4*>(xch + hw * kD + c * 8);
+      dst[0] = make_float4(s5[0], s5[1], s5[2], s5[3]);
+      dst[1] = make_float4(s5[4], s5[5], s5[6], s5[7]);
+    }
+    named_bar_sync(kBarHaar, 256);
+    if (ok) {
+      // lane (c, q = lane >> 3) combines the eight warps' sums of columns 2 q, 2 q + 1 of chunk c (two
+      // independent chains of four), then the four lanes that share a chunk swap their pairs
+      const int qq = lane >> 3;
+      const float2* src = reinterpret_cast<const float2*>(xch + c * 8 + 2 * qq);
+      const float* cf = hc + 2 * (8 + 8 * hw);
+      float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; w += 2) {
+        const float2 v0 = src[w * (kD / 2)], v1 = src[(w + 1) * (kD / 2)];
+        a0 = fmaf(cf[2 * w], v0.x, a0);
+        a1 = fmaf(cf[2 * w], v0.y, a1);
+        b0 = fmaf(cf[2 * w + 2], v1.x, b0);
+        b1 = fmaf(cf[2 * w + 2], v1.y, b1);
+      }
+      const float lo = a0 + b0, hi_ = a1 + b1;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int sl = (q << 3) | c;
+        hi[2 * q] += __shfl_sync(0xffffffffu, lo, sl);
+        hi[2 * q + 1] += __shfl_sync(0xffffffffu, hi_, sl);
+      }
+    }
+  }
+  if (ok) {
+    const float f0 = hc[0], k1 = hc[2], k2 = hc[4];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const float a0 = x[0][q] + x[1][q], a1 = x[2][q] + x[3][q];
+      const float a2 = x[4][q] + x[5][q], a3 = x[6][q] + x[7][q];
+      const float c20 = fmaf(k2, a0 + a1, hi[q]), c21 = fmaf(k2, a2 + a3, hi[q]);
+      const float c10 = fmaf(k1, a0, c20), c11 = fmaf(k1, a1, c20);
+      const float c12 = fmaf(k1, a2, c21), c13 = fmaf(k1, a3, c21);
+      x[0][q] = fmaf(f0, x[0][q], c10);
+      x[1][q] = fmaf(f0, x[1][q], c10);
+      x[2][q] = fmaf(f0, x[2][q], c11);
+      x[3][q] = fmaf(f0, x[3][q], c11);
+      x[4][q] = fmaf(f0, x[4][q], c12);
+      x[5][q] = fmaf(f0, x[5][q], c12);
+      x[6][q] = fmaf(f0, x[6][q], c13);
+      x[7][q] = fmaf(f0, x[7][q], c13);
+    }
+    if (rg * 8 + 8 <= valid_rows) {   // the usual case: every row of this thread lies inside the sequence
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        *reinterpret_cast<uint4*>(base + j * 128 + ((c ^ j) << 4)) =
+            make_uint4(pack_bf16x2(x[j][0], x[j][1]), pack_bf16x2(x[j][2], x[j][3]), pack_bf16x2(x[j][4], x[j][5]),
+                       pack_bf16x2(x[j][6], x[j][7]));
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        uint4 out = make_uint4(pack_bf16x2(x[j][0], x[j][1]), pack_bf16x2(x[j][2], x[j][3]),
+                               pack_bf16x2(x[j][4], x[j][5]), pack_bf16x2(x[j][6], x[j][7]));
+        if (rg * 8 + j >= valid_rows) out = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(base + j * 128 + ((c ^ j) << 4)) = out;
+      }
+    }
+  }
+}
+
 // One Haar step: wait for the two raw tiles of block b, filter them in place, hand the block to the
 // MMA issuer.  NX = number of tile slots in the ring.
-template <int NX, typename Bars>
+template <int NX, bool kScalar, typename Bars>
 __device__ __forceinline__ bool haar_step(uint8_t* xring, Bars* bars, float* xch, const f32x2* hcoef, bool cross,
                                           int b, int rows_left, int ht, bool ok, volatile int* abort_flag,
                                           int* status) {
@@ -364,8 +461,12 @@ __device__ __forceinline__ bool haar_step(uint8_t* xring, Bars* bars, float* xch
   const int s0 = t0 % NX, s1 = t1 % NX;
   if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[s0], (t0 / NX) & 1, abort_flag, status, kErrHaar));
   if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[s1], (t1 / NX) & 1, abort_flag, status, kErrHaar));
-  haar_block_inplace(xring + s0 * kTileBytes, xring + s1 * kTileBytes, hcoef, cross, xch + (b & 1) * 8 * kD, ht,
-                     rows_left - b * kBlk, ok);
+  if (kScalar)
+    haar_block_inplace_scalar(xring + s0 * kTileBytes, xring + s1 * kTileBytes, hcoef, cross, xch + (b & 1) * 8 * kD, ht,
+                              rows_left - b * kBlk, ok);
+  else
+    haar_block_inplace(xring + s0 * kTileBytes, xring + s1 * kTileBytes, hcoef, cross, xch + (b & 1) * 8 * kD, ht,
+                       rows_left - b * kBlk, ok);
   if (ok) {
     fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
     warp_arrive(&bars->xf_ready[b & (kNF - 1)]);
@@ -591,7 +692,7 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
     named_bar_sync(kBarCoef, 256);
     bool ok = true;
     for (int b = 0; b < nblk; ++b)
-      ok = haar_step<kNXK>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
+      ok = haar_step<kNXK, true>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
                      ht, ok, abort_flag, status);
   }
   tc_fence_before_sync();
@@ -890,7 +991,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     named_bar_sync(kBarCoef, 256);
     bool ok = true;
     for (int b = 0; b < nblk; ++b)
-      ok = haar_step<kNXQ>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
+      ok = haar_step<kNXQ, false>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
                      ht, ok, abort_flag, status);
   }
   tc_fence_before_sync();
