@@ -44,7 +44,7 @@ constexpr int kNXQ = 7;                           // query side: ring of Q tiles
 constexpr int kNF = 4;                            // "block filtered" barriers (block b uses b % 4)
 constexpr int kND1 = 3;                           // D1 accumulators in TMEM (columns 0, 128, 256)
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kAccCol = 384;                 // S' halves (key side) / N' of two tiles (query side)
+constexpr uint32_t kAccCol = 384;                 // S' halves (key side) / [N' | D'] of the current tile (query side)
 constexpr uint32_t kIdesc1 = make_idesc_bf16(128, 128, false, false);  // both operands K-major
 constexpr uint32_t kIdesc2 = make_idesc_bf16(128, 64, false, true);    // key side: B = V, N-major
 constexpr uint32_t kIdesc2Q = make_idesc_bf16(128, 80, false, false);  // query side: B = [S' | z' | 0]^T, K-major
@@ -70,7 +70,7 @@ static_assert(4 * kRegsCtlQ + 8 * kRegsReluQ + 4 * kRegsEpiQ + 8 * kRegsAux <= (
 static_assert(4 * kRegsCtl + 8 * 96 + 8 * kRegsAux <= (kThreads / 32) * 96, "key-side register split");
 
 // Named barriers (id 0 is __syncthreads).
-enum { kBarZsum = 1, kBarCoef = 3, kBarHaar = 4, kBarOut0 = 5 /* and 6: one per ReLU warpgroup */ };
+enum { kBarZsum = 1, kBarCoef = 3, kBarHaar = 4, kBarOut0 = 5 };
 enum { kErrProducer = 11, kErrMma = 12, kErrRelu = 13, kErrEpilogue = 14, kErrHaar = 15 };
 
 struct alignas(8) KsideBars {
