@@ -277,8 +277,9 @@ wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const v
              launch_qmean_gate(p, w, Q, gate_w, gate_b, omega, p.use_tc ? W : nullptr, st, &launches));
   if (p.use_tc) {
     WERSA_STEP(0, "tc_kside", launch_tc_kside(p, w, K, V, st, &launches));
-    WERSA_STEP(0, "reduce_partials",
-               launch_reduce_partials(p, w.spart, w.zpart, p.tchunks, w.S, w.z, w.Sbf, st, &launches));
+    if (p.tchunks > 1)   // with one chunk per slab the key-side kernel has written S', z' and the image itself
+      WERSA_STEP(0, "reduce_partials",
+                 launch_reduce_partials(p, w.spart, w.zpart, p.tchunks, w.S, w.z, w.Sbf, st, &launches));
     WERSA_STEP(0, "tc_qside", launch_tc_qside(p, w, Q, beta, O, st, &launches));
   } else {
     WERSA_STEP(0, "haar_filter_q", launch_haar_filter(p, Q, kind, w.f, w.QF, 0, st, &launches));

@@ -480,7 +480,8 @@ template <int NH>
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
            const __nv_bfloat16* __restrict__ Wt, const float* __restrict__ f, float* __restrict__ spart,
-           float* __restrict__ zpart, int n, int L, int chunk_blocks, int* __restrict__ status) {
+           float* __restrict__ zpart, __nv_bfloat16* __restrict__ sbf, int n, int L, int chunk_blocks,
+           int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   using SL = KsideSmem<NH>;
@@ -681,6 +682,16 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
 #pragma unroll
         for (int j = 0; j < 8; ++j)
           *reinterpret_cast<uint4*>(dst + 32 * c + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+        if (sbf != nullptr) {   // one chunk per slab: this is S' itself, leave its bf16 image as well
+          __nv_bfloat16* bdst = sbf + (pidx * m + feat) * kD + 32 * c;
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            *reinterpret_cast<uint4*>(bdst + 8 * j) =
+                make_uint4(pack_bf16x2(__uint_as_float(r[8 * j]), __uint_as_float(r[8 * j + 1])),
+                           pack_bf16x2(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3])),
+                           pack_bf16x2(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5])),
+                           pack_bf16x2(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7])));
+        }
       }
       zpart[pidx * m + feat] = zacc;
     }
@@ -1065,12 +1076,18 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
   if ((err = make_tile_map(K, p.slabs, p.cfg.seq_len, kTile, &map_k)) != cudaSuccess) return err;
   if ((err = make_tile_map(V, p.slabs, p.cfg.seq_len, kTile, &map_v)) != cudaSuccess) return err;
   dim3 grid(p.tchunks, p.slabs);
+  // With one chunk per slab the "partial" is the result: the kernel writes S', z' and the bf16 image
+  // itself and no reduction follows.
+  const bool single = p.tchunks == 1;
+  float* sp = single ? w.S : w.spart;
+  float* zp = single ? w.z : w.zpart;
+  __nv_bfloat16* sb = single ? w.Sbf : nullptr;
   if (p.cfg.features == 256)
     err = launch_pdl(k_tc_kside<2>, grid, kThreads, KsideSmem<2>::total, st, map_k, map_v, (const __nv_bfloat16*)w.Wt,
-                     (const float*)w.f, w.spart, w.zpart, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
+                     (const float*)w.f, sp, zp, sb, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
   else
     err = launch_pdl(k_tc_kside<1>, grid, kThreads, KsideSmem<1>::total, st, map_k, map_v, (const __nv_bfloat16*)w.Wt,
-                     (const float*)w.f, w.spart, w.zpart, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
+                     (const float*)w.f, sp, zp, sb, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
   *launches += 1;
   return err != cudaSuccess ? err : cudaGetLastError();
 }
