@@ -75,13 +75,13 @@ enum { kErrProducer = 11, kErrMma = 12, kErrRelu = 13, kErrEpilogue = 14, kErrHa
 
 struct alignas(8) KsideBars {
   uint64_t x_full[kNXK], x_empty[kNXK], xf_ready[kNF], v_full[kNV], v_empty[kNV];
-  uint64_t d1_full[6], phi_ready[kND1], d1_free[kND1], acc_done;
+  uint64_t d1_full[6], phi_ready[kND1], d1_free[kND1], acc_done, w_full;
   uint32_t tmem_base;
   int abort_flag;
 };
 struct alignas(8) QsideBars {
   uint64_t x_full[kNXQ], x_empty[kNXQ], xf_ready[kNF];
-  uint64_t d1_full[6], phi_ready[kND1], d1_free[kND1], d2_full, d2_free, simg_ready;
+  uint64_t d1_full[6], phi_ready[kND1], d1_free[kND1], d2_full, d2_free, simg_ready, w_full;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -106,15 +106,6 @@ template <int NH> struct QsideSmem {
   static constexpr uint32_t bars = hcoef + 1024;
   static constexpr uint32_t total = bars + 512 + 1024;
 };
-
-// (rows x 64) bf16 row-major in global memory -> 128B-swizzled rows of 128 bytes in shared memory.
-__device__ __forceinline__ void load_rows_swizzled(uint8_t* dst, const __nv_bfloat16* src, int rows) {
-  for (int i = threadIdx.x; i < rows * 8; i += blockDim.x) {
-    const int r = i >> 3, c = i & 7;
-    const uint4 val = *reinterpret_cast<const uint4*>(src + (size_t)r * kD + c * 8);
-    *reinterpret_cast<uint4*>(dst + swz128(r, c)) = val;
-  }
-}
 
 // Ties the 32 registers of an asynchronous TMEM load to the point behind its wait, so that no use
 // of them is scheduled ahead of the wait.
@@ -479,7 +470,7 @@ __device__ __forceinline__ bool haar_step(uint8_t* xring, Bars* bars, float* xch
 template <int NH>
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-           const __nv_bfloat16* __restrict__ Wt, const float* __restrict__ f, float* __restrict__ spart,
+           const __grid_constant__ CUtensorMap map_w, const float* __restrict__ f, float* __restrict__ spart,
            float* __restrict__ zpart, __nv_bfloat16* __restrict__ sbf, int n, int L, int chunk_blocks,
            int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
@@ -510,6 +501,7 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       mbar_init(&bars->d1_free[b], 1);
     }
     mbar_init(&bars->acc_done, NH);
+    mbar_init(&bars->w_full, 1);
     bars->abort_flag = 0;
     fence_mbar_init();
     // K and V are inputs: the first copies of both rings go out before the dependency wait below
@@ -532,7 +524,11 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
   // side start in turn, whose set-up reads W^T and f without a wait of its own.
   griddep_wait();
   griddep_launch();
-  load_rows_swizzled(smem + SL::wt, Wt, m);
+  if (threadIdx.x == 0) {   // the W^T image (m rows of 64 bf16) arrives by TMA; only the MMA1 issuer waits for it
+    mbar_arrive_expect_tx(&bars->w_full, NH * kTileBytes);
+#pragma unroll
+    for (int h = 0; h < NH; ++h) tma_load_3d(smem + SL::wt + h * kTileBytes, &map_w, 0, h * kTile, 0, &bars->w_full);
+  }
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
@@ -578,6 +574,7 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       if (*abort_flag != 0) {   // let copies in flight land before the CTA's shared memory goes away
         for (int b = max(0, kb - kNXK); b < kb; ++b) mbar_wait_drain(&bars->x_full[b % kNXK], (b / kNXK) & 1);
         for (int b = max(0, vb - kNV); b < vb; ++b) mbar_wait_drain(&bars->v_full[b % kNV], (b / kNV) & 1);
+        mbar_wait_drain(&bars->w_full, 0);
       }
     } else if (warp == kWarpMma && lane == 0) {
       // MMA1 of every unit.  Ring slots, D1 buffers and barrier phases are running counters, and the
@@ -588,7 +585,7 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       const uint32_t x_lo = smem_desc_lo(smem_u32(smem + SL::x), 16);
       uint32_t xs = 0, fs = 0, fpar = 0;               // K ring slot; "block filtered" barrier and phase
       uint32_t c3 = 0, c6 = 0, round = 0;              // D1 buffer, d1_full barrier, uses of buffer 0 so far
-      bool ok = true;
+      bool ok = mbar_wait(&bars->w_full, 0, abort_flag, status, kErrMma);
       for (int b = 0; b < nblk && ok; ++b) {
         ok = mbar_wait(&bars->xf_ready[fs], fpar, abort_flag, status, kErrMma);
         if (!ok) break;
@@ -794,7 +791,7 @@ __device__ __forceinline__ void qside_build_simg(uint8_t* simg, const __nv_bfloa
 template <int NH>
 __global__ void __launch_bounds__(kThreadsQ, 1)
 k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
-           const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ Sbf,
+           const __grid_constant__ CUtensorMap map_w, const __nv_bfloat16* __restrict__ Sbf,
            const float* __restrict__ zg, const float* __restrict__ f, const float* __restrict__ beta, float eps,
            float bw_floor, int n, int L, int chunk_blocks, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
@@ -823,14 +820,18 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     mbar_init(&bars->d2_full, 1);
     mbar_init(&bars->d2_free, 4);
     mbar_init(&bars->simg_ready, kAuxWarp0Q - kReluWarp0);
+    mbar_init(&bars->w_full, 1);
     bars->abort_flag = 0;
     fence_mbar_init();
+    // W^T was complete before the kernel ahead of this one started: its image can be fetched at once
+    mbar_arrive_expect_tx(&bars->w_full, NH * kTileBytes);
+#pragma unroll
+    for (int h = 0; h < NH; ++h) tma_load_3d(smem + SL::wt + h * kTileBytes, &map_w, 0, h * kTile, 0, &bars->w_full);
   }
   if (warp == kWarpMma) {
     tmem_alloc(&bars->tmem_base, kTmemCols);
     tmem_relinquish();
   }
-  load_rows_swizzled(smem + SL::wt, Wt, m);
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
@@ -851,6 +852,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       }
       if (*abort_flag != 0) {
         for (int b = max(0, issued - kNXQ); b < issued; ++b) mbar_wait_drain(&bars->x_full[b % kNXQ], (b / kNXQ) & 1);
+        mbar_wait_drain(&bars->w_full, 0);
       }
     } else if (warp == kWarpMma && lane == 0) {
       // MMA1 of every unit (see the key side).
@@ -860,7 +862,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       const uint32_t x_lo = smem_desc_lo(smem_u32(smem + SL::x), 16);
       uint32_t xs = 0, fs = 0, fpar = 0;
       uint32_t c3 = 0, c6 = 0, round = 0;
-      bool ok = true;
+      bool ok = mbar_wait(&bars->w_full, 0, abort_flag, status, kErrMma);
       for (int b = 0; b < nblk && ok; ++b) {
         ok = mbar_wait(&bars->xf_ready[fs], fpar, abort_flag, status, kErrMma);
         if (!ok) break;
@@ -1075,6 +1077,8 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
   cudaError_t err;
   if ((err = make_tile_map(K, p.slabs, p.cfg.seq_len, kTile, &map_k)) != cudaSuccess) return err;
   if ((err = make_tile_map(V, p.slabs, p.cfg.seq_len, kTile, &map_v)) != cudaSuccess) return err;
+  CUtensorMap map_w;   // W^T (m x 64) as one slab of m rows
+  if ((err = make_tile_map(w.Wt, 1, p.cfg.features, kTile, &map_w)) != cudaSuccess) return err;
   dim3 grid(p.tchunks, p.slabs);
   // With one chunk per slab the "partial" is the result: the kernel writes S', z' and the bf16 image
   // itself and no reduction follows.
@@ -1083,10 +1087,10 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
   float* zp = single ? w.z : w.zpart;
   __nv_bfloat16* sb = single ? w.Sbf : nullptr;
   if (p.cfg.features == 256)
-    err = launch_pdl(k_tc_kside<2>, grid, kThreads, KsideSmem<2>::total, st, map_k, map_v, (const __nv_bfloat16*)w.Wt,
+    err = launch_pdl(k_tc_kside<2>, grid, kThreads, KsideSmem<2>::total, st, map_k, map_v, map_w,
                      (const float*)w.f, sp, zp, sb, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
   else
-    err = launch_pdl(k_tc_kside<1>, grid, kThreads, KsideSmem<1>::total, st, map_k, map_v, (const __nv_bfloat16*)w.Wt,
+    err = launch_pdl(k_tc_kside<1>, grid, kThreads, KsideSmem<1>::total, st, map_k, map_v, map_w,
                      (const float*)w.f, sp, zp, sb, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
   *launches += 1;
   return err != cudaSuccess ? err : cudaGetLastError();
@@ -1100,13 +1104,15 @@ cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const flo
   if ((err = make_tile_map(O, p.slabs, p.cfg.seq_len, kTile, &map_o)) != cudaSuccess) return err;
   // (the query side may start while the reduction that produces S', z' is still running; it waits for
   // that kernel where it first needs its results)
+  CUtensorMap map_w;
+  if ((err = make_tile_map(w.Wt, 1, p.cfg.features, kTile, &map_w)) != cudaSuccess) return err;
   dim3 grid(p.tchunks, p.slabs);
   if (p.cfg.features == 256)
-    err = launch_pdl(k_tc_qside<2>, grid, kThreadsQ, QsideSmem<2>::total, st, map_q, map_o, (const __nv_bfloat16*)w.Wt,
+    err = launch_pdl(k_tc_qside<2>, grid, kThreadsQ, QsideSmem<2>::total, st, map_q, map_o, map_w,
                      (const __nv_bfloat16*)w.Sbf, (const float*)w.z, (const float*)w.f, beta, p.cfg.eps,
                      p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
   else
-    err = launch_pdl(k_tc_qside<1>, grid, kThreadsQ, QsideSmem<1>::total, st, map_q, map_o, (const __nv_bfloat16*)w.Wt,
+    err = launch_pdl(k_tc_qside<1>, grid, kThreadsQ, QsideSmem<1>::total, st, map_q, map_o, map_w,
                      (const __nv_bfloat16*)w.Sbf, (const float*)w.z, (const float*)w.f, beta, p.cfg.eps,
                      p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
   *launches += 1;
