@@ -668,8 +668,13 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       if (g == 0) zacc += zx[row];
     }
     if (ok && (NH == 2 || g == 0)) {
-      const int feat = (NH == 2 ? g * 128 : 0) + row;
-      float* dst = spart + (pidx * m + feat) * kD;
+      // The accumulator row of a thread is one feature's 64 values; written straight from the registers a
+      // warp would touch 32 different 256-byte rows per store.  Each warp instead turns its 32 x 32 chunk
+      // around in shared memory (the K ring is idle by now; rows padded to 33 floats) and writes whole
+      // 128-byte row segments.
+      const int feat0 = (NH == 2 ? g * 128 : 0) + (int)lane_base;   // first feature of this warp
+      float* stage = reinterpret_cast<float*>(smem + SL::x) + (warp - kReluWarp0) * (32 * 33);
+      float* dst = spart + (pidx * m + feat0) * kD;
 #pragma unroll 1
       for (int c = 0; c < 2; ++c) {
         uint32_t r[32];
@@ -677,20 +682,21 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
         tmem_ld_wait();
         reg_fence32(r);
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          *reinterpret_cast<uint4*>(dst + 32 * c + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+        for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = __uint_as_float(r[j]);
+        __syncwarp();
+#pragma unroll 8
+        for (int rr = 0; rr < 32; ++rr) dst[(size_t)rr * kD + 32 * c + lane] = stage[rr * 33 + lane];
         if (sbf != nullptr) {   // one chunk per slab: this is S' itself, leave its bf16 image as well
-          __nv_bfloat16* bdst = sbf + (pidx * m + feat) * kD + 32 * c;
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            *reinterpret_cast<uint4*>(bdst + 8 * j) =
-                make_uint4(pack_bf16x2(__uint_as_float(r[8 * j]), __uint_as_float(r[8 * j + 1])),
-                           pack_bf16x2(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3])),
-                           pack_bf16x2(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5])),
-                           pack_bf16x2(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7])));
+          __nv_bfloat16* bdst = sbf + (pidx * m + feat0) * kD + 32 * c;
+#pragma unroll 8
+          for (int rr = 0; rr < 32; rr += 2) {   // two rows per instruction, a pair of columns per lane
+            const int rw = rr + (lane >> 4), cc = 2 * (lane & 15);
+            *reinterpret_cast<uint32_t*>(bdst + (size_t)rw * kD + cc) = pack_bf16x2(stage[rw * 33 + cc], stage[rw * 33 + cc + 1]);
+          }
         }
+        __syncwarp();
       }
-      zpart[pidx * m + feat] = zacc;
+      zpart[pidx * m + feat0 + lane] = zacc;
     }
   } else {
     reg_inc<kRegsAux>();
