@@ -296,7 +296,7 @@ def main():
     # DRAM bytes per token-head of one launch, from the ncu capture summarised in
     # profiles/forward_cfg5_ncu_full_set.md (dram__bytes_read.sum + dram__bytes_write.sum on the cfg5
     # forward, 524288 token-heads; traffic grows in proportion to the token-heads of a launch)
-    ncu_bytes_per_th = {"qmean_gate": 128.6, "tc_kside": 263.8, "tc_qside": 165.4}
+    ncu_bytes_per_th = {"qmean_gate": 128.8, "tc_kside": 264.0, "tc_qside": 165.9}
     if dom in flops:
         if dom.startswith("tc_"):
             bound, peak, unit = "tensor", float(peaks["bf16_tflops"]), "TFLOP/s"
