@@ -125,6 +125,7 @@ TC_SMALL = [
     dict(B=2, H=1, n=1000, d=64, L=3, m=128),     # ragged: last block is partly past the end
     dict(B=1, H=2, n=4100, d=64, L=8, m=256),     # ragged tail of 4 rows in a 256-row Haar block
     dict(B=1, H=1, n=77, d=64, L=2, m=128),       # shorter than one tile
+    dict(B=10, H=8, n=1024, d=64, L=6, m=256),    # 80 slabs: one chunk of four blocks per slab, no reduction launch
 ]
 
 
