@@ -307,6 +307,61 @@ def test_config5_training_step_bf16():
     assert abs(db - ref["dbeta_closed"]) <= 0.1 * abs(ref["dbeta_closed"]) + 1e-12
 
 
+# ---------------------------------------------------------------- seeded random shapes
+def _random_shapes(seed, count, backward):
+    """Shapes drawn from a fixed seed: ragged n, every L, both feature counts, few and many slabs (so that
+    a slab is cut into several chunks, or handled by one CTA without a reduction launch)."""
+    import random
+    rng = random.Random(seed)
+    out = []
+    for _ in range(count):
+        m = rng.choice([128, 256])
+        L = rng.randint(1, 8)
+        B, H = rng.choice([(1, 1), (1, 3), (2, 2), (3, 5), (5, 1), (6, 7)] if backward else
+                          [(1, 1), (1, 3), (2, 2), (3, 5), (9, 9), (20, 8), (2, 40)])
+        nmax = (1500 if B * H <= 6 else 500) if backward else (5000 if B * H <= 10 else (1500 if B * H <= 40 else 700))
+        out.append(dict(B=B, H=H, n=rng.randint(1 << L, nmax), d=64, L=L, m=m, gate_per_head=rng.choice([1, 1, 0])))
+    return out
+
+
+FWD_RANDOM = _random_shapes(11, 10, backward=False)
+BWD_RANDOM = _random_shapes(12, 5, backward=True)
+
+
+@pytest.mark.parametrize("case", range(len(FWD_RANDOM)))
+def test_forward_random_shapes_tensor_core(case):
+    import torch
+    cfg = dict(FWD_RANDOM[case], dtype="bf16")
+    inp = wi.make_inputs(**cfg, seed=5000 + case, w_seed=6000 + case, gate_std=0.3, gate_seed=7000 + case,
+                         mean_shift=0.25, scale=0.7)
+    ctx = _ctx(cfg)
+    assert ctx.uses_tensor_cores()
+    dev = device_inputs(inp, "bf16")
+    args = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    O = ctx.forward(*args).clone()
+    O2 = ctx.forward(*args)
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    assert torch.equal(O, O2), "two runs on the same inputs differ"
+    _check(to_numpy64(O), _oracle_forward(cfg, inp), "bf16", "O")
+
+
+@pytest.mark.parametrize("case", range(len(BWD_RANDOM)))
+def test_backward_random_shapes_tensor_core(case):
+    import torch
+    cfg = dict(BWD_RANDOM[case], dtype="bf16", eps=1e-3)
+    inp = wi.make_inputs(**cfg, seed=8000 + case, w_seed=8100 + case, gate_std=0.3, gate_seed=8200 + case,
+                         mean_shift=0.25, scale=0.7, backward=True)
+    ctx = _ctx(cfg)
+    dev = device_inputs(inp, "bf16")
+    args = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    ctx.forward(*args)
+    grads = ctx.backward(*args, dev["dO"])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    _check_backward(cfg, inp, grads)
+
+
 # ---------------------------------------------------------------- error paths that need a device
 def test_error_paths_on_device():
     import paper_2507_08637_b200 as wersa
