@@ -102,6 +102,21 @@ wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const v
                            const float* gate_b, const float* omega, void* O,
                            void* cuda_stream);
 
+/* The same forward for tensors that live in HOST memory (the end-to-end path: Sec. 3.1 steps 3-8 with
+ * the transfers a caller without device-resident activations has to pay).  Enqueues on cuda_stream, in
+ * this order: copies of hQ, hK, hV (host; batch*heads*seq_len*head_dim elements of cfg.dtype each) into
+ * the device staging buffers dQ, dK, dV; wersa_forward on them into the device buffer dO; a copy of dO
+ * into hO (host).  The four staging buffers are caller-owned device memory of the same size, 16-byte
+ * aligned; the library allocates nothing.  W, beta, gate_w, gate_b, omega are DEVICE pointers as for
+ * wersa_forward (parameters stay resident).  With page-locked host buffers the call returns once the
+ * work is enqueued; with pageable ones the copies may block.  hO is valid after cuda_stream has been
+ * synchronised.  Errors: WERSA_ERR_INVALID_ARG on a NULL or misaligned pointer (nothing enqueued),
+ * WERSA_ERR_CUDA if a copy cannot be enqueued, else wersa_forward's status. */
+wersa_status wersa_forward_host(wersa_ctx* ctx, const void* hQ, const void* hK, const void* hV,
+                                void* dQ, void* dK, void* dV, const void* W, const float* beta,
+                                const float* gate_w, const float* gate_b, const float* omega,
+                                void* dO, void* hO, void* cuda_stream);
+
 /* Backward pass: gradients of sum(dO (.) O) with respect to Q, K, V (cfg.grad_dtype), beta
  * (1 float), gate_w (heads, head_dim, levels+1), gate_b (heads, levels+1; rows >= 1 are zero
  * when gate_per_head = 0) and omega (levels+1).  The paper does not write the backward pass;

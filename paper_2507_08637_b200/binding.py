@@ -54,6 +54,8 @@ def _lib():
     lib.wersa_create.argtypes = [ctypes.POINTER(wersa_config), vp, ctypes.c_size_t, ctypes.POINTER(vp)]
     lib.wersa_forward.restype = ctypes.c_int
     lib.wersa_forward.argtypes = [vp, vp, vp, vp, vp, fp, fp, fp, fp, vp, vp]
+    lib.wersa_forward_host.restype = ctypes.c_int
+    lib.wersa_forward_host.argtypes = [vp] + [vp] * 3 + [vp] * 3 + [vp] + [fp] * 4 + [vp, vp, vp]
     lib.wersa_backward.restype = ctypes.c_int
     lib.wersa_backward.argtypes = [vp] + [vp] * 4 + [fp] * 4 + [vp] * 4 + [fp] * 4 + [vp]
     lib.wersa_haar_filter.restype = ctypes.c_int
@@ -115,6 +117,14 @@ def _ptr(t, dtype=None, name="tensor", optional=False):
     return ctypes.c_void_p(t.data_ptr())
 
 
+def _host_ptr(t, dtype, name):
+    if t is None or t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous host tensor")
+    if t.dtype != dtype:
+        raise ValueError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
 def _stream_ptr(stream):
     if stream is None:
         stream = torch.cuda.current_stream()
@@ -155,6 +165,22 @@ class WersaContext:
         if st != WERSA_OK:
             raise WersaError(st, "wersa_forward")
         return out
+
+    def forward_host(self, hQ, hK, hV, dQ, dK, dV, W, beta, gate_w, gate_b, omega, dO, hO, stream=None):
+        """wersa_forward_host: hQ, hK, hV, hO are contiguous HOST tensors (page-locked for asynchronous
+        copies), dQ, dK, dV, dO device staging tensors of the same shape and dtype.  Everything is
+        enqueued on `stream`; hO is valid once the stream has been synchronised."""
+        dt = self.io_dtype
+        st = _lib().wersa_forward_host(self._h, _host_ptr(hQ, dt, "hQ"), _host_ptr(hK, dt, "hK"),
+                                       _host_ptr(hV, dt, "hV"), _ptr(dQ, dt, "dQ"), _ptr(dK, dt, "dK"),
+                                       _ptr(dV, dt, "dV"), _ptr(W, dt, "W"), _ptr(beta, torch.float32, "beta"),
+                                       _ptr(gate_w, torch.float32, "gate_w", optional=True),
+                                       _ptr(gate_b, torch.float32, "gate_b", optional=True),
+                                       _ptr(omega, torch.float32, "omega"), _ptr(dO, dt, "dO"),
+                                       _host_ptr(hO, dt, "hO"), _stream_ptr(stream))
+        if st != WERSA_OK:
+            raise WersaError(st, "wersa_forward_host")
+        return hO
 
     def backward(self, Q, K, V, W, beta, gate_w, gate_b, omega, dO, stream=None):
         dt, gd = self.io_dtype, self.grad_dtype
@@ -244,6 +270,10 @@ def wersa_create(batch, heads, seq_len, head_dim, levels, features, **kw):
 
 def wersa_forward(ctx, Q, K, V, W, beta, gate_w, gate_b, omega, out=None, stream=None):
     return ctx.forward(Q, K, V, W, beta, gate_w, gate_b, omega, out=out, stream=stream)
+
+
+def wersa_forward_host(ctx, hQ, hK, hV, dQ, dK, dV, W, beta, gate_w, gate_b, omega, dO, hO, stream=None):
+    return ctx.forward_host(hQ, hK, hV, dQ, dK, dV, W, beta, gate_w, gate_b, omega, dO, hO, stream=stream)
 
 
 def wersa_backward(ctx, Q, K, V, W, beta, gate_w, gate_b, omega, dO, stream=None):

@@ -294,6 +294,28 @@ wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const v
   return WERSA_OK;
 }
 
+wersa_status wersa_forward_host(wersa_ctx* ctx, const void* hQ, const void* hK, const void* hV, void* dQ,
+                                void* dK, void* dV, const void* W, const float* beta, const float* gate_w,
+                                const float* gate_b, const float* omega, void* dO, void* hO, void* cuda_stream) {
+  if (ctx == nullptr || hQ == nullptr || hK == nullptr || hV == nullptr || hO == nullptr || dQ == nullptr ||
+      dK == nullptr || dV == nullptr || dO == nullptr || W == nullptr || beta == nullptr || omega == nullptr)
+    return WERSA_ERR_INVALID_ARG;
+  if (!aligned16(dQ) || !aligned16(dK) || !aligned16(dV) || !aligned16(dO) || !aligned16(W))
+    return WERSA_ERR_INVALID_ARG;
+  const Plan& p = ctx->plan;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t bytes = (size_t)p.slabs * p.cfg.seq_len * kD * (p.bf16 ? 2 : 4);
+  DeviceGuard guard(p.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  WERSA_CUDA(cudaMemcpyAsync(dQ, hQ, bytes, cudaMemcpyHostToDevice, st));
+  WERSA_CUDA(cudaMemcpyAsync(dK, hK, bytes, cudaMemcpyHostToDevice, st));
+  WERSA_CUDA(cudaMemcpyAsync(dV, hV, bytes, cudaMemcpyHostToDevice, st));
+  const wersa_status s = wersa_forward(ctx, dQ, dK, dV, W, beta, gate_w, gate_b, omega, dO, cuda_stream);
+  if (s != WERSA_OK) return s;
+  WERSA_CUDA(cudaMemcpyAsync(hO, dO, bytes, cudaMemcpyDeviceToHost, st));
+  return WERSA_OK;
+}
+
 wersa_status wersa_backward(wersa_ctx* ctx, const void* Q, const void* K, const void* V, const void* W,
                             const float* beta, const float* gate_w, const float* gate_b, const float* omega,
                             const void* dO, void* dQ, void* dK, void* dV, float* dbeta, float* dgate_w,

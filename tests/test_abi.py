@@ -78,6 +78,10 @@ def test_create_rejects_bad_arguments_without_a_device(lib):
     lib.wersa_forward.restype = ctypes.c_int
     lib.wersa_forward.argtypes = [ctypes.c_void_p] * 11
     assert lib.wersa_forward(handle, None, None, None, None, None, None, None, None, None, None) == 1
+    lib.wersa_forward_host.restype = ctypes.c_int
+    lib.wersa_forward_host.argtypes = [ctypes.c_void_p] * 15
+    assert lib.wersa_forward_host(handle, *([None] * 14)) == 1
+    assert lib.wersa_forward_host(None, *([ctypes.c_void_p(256)] * 14)) == 1
     lib.wersa_destroy.argtypes = [ctypes.c_void_p]
     assert lib.wersa_destroy(handle) == 0
     assert lib.wersa_destroy(None) == 0

@@ -166,6 +166,40 @@ def test_forward_is_bit_identical_run_to_run():
         assert torch.equal(a.view(torch.int16), b.view(torch.int16))
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_forward_host_matches_device_forward_and_oracle(dtype):
+    """The end-to-end entry point (host tensors in, host tensor out) gives the device-resident forward's
+    bits, page-locked or pageable, and meets the oracle at the same tolerance."""
+    import torch
+    cfg = dict(B=2, H=3, n=1500, d=64, L=5, m=128, dtype=dtype)
+    inp = wi.make_inputs(**cfg, seed=41, w_seed=42, gate_std=0.2, gate_seed=43, mean_shift=0.2)
+    ctx = _ctx(cfg)
+    dev = device_inputs(inp, dtype)
+    params = (dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    O = ctx.forward(dev["Q"], dev["K"], dev["V"], *params).clone()
+    torch.cuda.synchronize()
+    for pinned in (True, False):
+        host = [dev[k].cpu() for k in ("Q", "K", "V")]
+        hO = torch.zeros_like(host[0])
+        if pinned:
+            host = [t.pin_memory() for t in host]
+            hO = hO.pin_memory()
+        stage = [torch.zeros_like(dev["Q"]) for _ in range(4)]
+        out = ctx.forward_host(*host, *stage[:3], *params, stage[3], hO)
+        torch.cuda.synchronize()
+        assert ctx.query_status() == 0
+        assert out is hO and torch.equal(hO, O.cpu())
+        assert torch.equal(stage[0], dev["Q"]) and torch.equal(stage[3], O)
+    _check(to_numpy64(hO), _oracle_forward(cfg, inp), dtype, "O")
+    import paper_2507_08637_b200 as wersa
+    with pytest.raises(ValueError):
+        ctx.forward_host(dev["Q"], *host[1:], *stage[:3], *params, stage[3], hO)   # device tensor as host input
+    with pytest.raises(wersa.WersaError) as e:
+        big = torch.zeros(dev["Q"].numel() + 1, device="cuda", dtype=dev["Q"].dtype)
+        ctx.forward_host(*host, big[1:].view_as(dev["Q"]), *stage[1:3], *params, stage[3], hO)
+    assert e.value.status == 1
+
+
 # ---------------------------------------------------------------- the five configurations
 def _run_config(name, flags=0, **overrides):
     import torch
