@@ -86,13 +86,29 @@ __device__ __forceinline__ bool cta_wait(uint64_t* bar, uint32_t parity, BwdBars
   return __syncthreads_and(ok) != 0;
 }
 
-template <typename TG> __device__ __forceinline__ void store_row32(TG* dst, const uint32_t (&r)[32]);
-template <> __device__ __forceinline__ void store_row32<float>(float* dst, const uint32_t (&r)[32]) {
+__device__ __forceinline__ void store_row32(float* dst, const uint32_t (&r)[32]) {
 #pragma unroll
   for (int j = 0; j < 8; ++j)
     *reinterpret_cast<uint4*>(dst + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
 }
-template <> __device__ __forceinline__ void store_row32<__nv_bfloat16>(__nv_bfloat16* dst, const uint32_t (&r)[32]) {
+
+// A 128 x 64 result tile leaves through shared memory and a TMA store: written straight from the
+// registers (one token row per lane) every store instruction of a warp would touch 32 different
+// 128-byte lines, and the load/store unit stays busy with them for about 2,000 cycles per tile, during
+// which the barrier polls and MMA issues of the next step queue behind them.
+// stage_row32: columns 32 wg .. 32 wg + 31 of row tl into the staging image, in the 128-byte-swizzled
+// layout the store's tensor map describes: fp32 = two boxes of 128 rows x 32 columns (16 KB each, box
+// wg), bf16 = one box of 128 rows x 64 columns (16-byte chunks 4 wg .. 4 wg + 3 of the row).
+template <typename TG>
+__device__ __forceinline__ void stage_row32(uint8_t* stage, int tl, int wg, const uint32_t (&r)[32]);
+template <> __device__ __forceinline__ void stage_row32<float>(uint8_t* stage, int tl, int wg, const uint32_t (&r)[32]) {
+  uint8_t* box = stage + wg * kTileBytes;
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    *reinterpret_cast<uint4*>(box + swz128(tl, j)) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+}
+template <>
+__device__ __forceinline__ void stage_row32<__nv_bfloat16>(uint8_t* stage, int tl, int wg, const uint32_t (&r)[32]) {
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     uint4 v;
@@ -100,8 +116,16 @@ template <> __device__ __forceinline__ void store_row32<__nv_bfloat16>(__nv_bflo
     v.y = pack_bf16x2(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
     v.z = pack_bf16x2(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
     v.w = pack_bf16x2(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
-    *reinterpret_cast<uint4*>(dst + 8 * j) = v;
+    *reinterpret_cast<uint4*>(stage + swz128(tl, 4 * wg + j)) = v;
   }
+}
+// Issued by one thread after the CTA barrier that follows the staging writes (each writer has fenced its
+// writes for the async proxy).  Rows past the end of the slab are clipped by the tensor map.
+template <typename TG>
+__device__ __forceinline__ void store_tile(const CUtensorMap* map, const uint8_t* stage, int row0, int slab) {
+  tma_store_3d(map, stage, 0, row0, slab);
+  if (sizeof(TG) == 4) tma_store_3d(map, stage + kTileBytes, 32, row0, slab);
+  bulk_commit_group();
 }
 
 // bf16 hi + lo split of a pair of fp32 values: hi = bf16(x), lo = bf16(x - hi).  Feeding both to the
@@ -189,8 +213,8 @@ template <int NH, typename TG>
 __global__ void __launch_bounds__(256, 1)
 k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant__ CUtensorMap map_v,
                const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ dSbf,
-               const float* __restrict__ dzg, TG* __restrict__ dV, float* __restrict__ dKF, int n, int slabs,
-               int* __restrict__ status) {
+               const float* __restrict__ dzg, const __grid_constant__ CUtensorMap map_dv,
+               const __grid_constant__ CUtensorMap map_dkf, int n, int slabs, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   using SL = BwdKSmem<NH>;
@@ -260,8 +284,10 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
   for (int ti = 0; ti < ntiles && ok; ++ti) {
     const int slab = (g0 + ti) / tiles_per_slab;
     const int row0 = ((g0 + ti) - slab * tiles_per_slab) * kTile;
-    const int row = row0 + tl;
     const uint32_t x_k = stage_k + (ti & 1) * kStageStep, v_k = x_k + 3 * kTileStep;
+    // results leave through this tile's own stage: dV over planes 0-1 (read for the last time by MMA1),
+    // dK_F over plane 2 and the V tile (read for the last time by MMA3)
+    uint8_t* out_stage = smem + SL::stage + (ti & 1) * SL::stage_bytes;
     if (slab != cur_slab) {   // uniform over the CTA; every MMA of the previous tile has completed
       cur_slab = slab;
       load_rows_swizzled(smem + SL::ds, dSbf + (size_t)slab * m * kD, m);
@@ -269,11 +295,8 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
       fence_proxy_async_smem();
       __syncthreads();
     }
-    // ---- copies of the next tile (its stage was released by the barrier that ended tile ti - 1), MMA1
-    if (threadIdx.x == 0 && ti + 1 < ntiles) {
-      issue_copies(ti + 1);
-      issued = ti + 2;
-    }
+    // ---- MMA1, then the copies of the next tile: its stage is the one tile ti - 1 left its results in,
+    // so the stores of that tile must have read it first
     ok = cta_wait(&bars->full[ti & 1], (ti >> 1) & 1, bars, status, kErrBwdCopy);
     if (!ok) break;
     if (threadIdx.x == 0) {
@@ -287,6 +310,11 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
             mma_ss(tmem + h * 128, smem_desc_join(x_k + pl * kTileStep + 2 * k, hi),
                    smem_desc_join(wt_k + h * kTileStep + 2 * k, hi), kIdescP, (pl > 0 || k > 0) ? 1u : 0u);
       mma_commit(&bars->mma);
+      if (ti + 1 < ntiles) {
+        bulk_wait_group_read0();
+        issue_copies(ti + 1);
+        issued = ti + 2;
+      }
     }
     ok = cta_wait(&bars->mma, mma_par, bars, status, kErrBwdMma);
     mma_par ^= 1;
@@ -322,12 +350,14 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
       tmem_ld32(trow + acc + 32 * wg, r);
       tmem_ld_wait();
       reg_fence32(r);
-      if (row < n) store_row32<TG>(dV + ((size_t)slab * n + row) * kD + 32 * wg, r);
+      stage_row32<TG>(out_stage, tl, wg, r);
     }
+    fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
     // ---- MMA3: G_h = V dS'_h^T
     if (threadIdx.x == 0) {
+      store_tile<TG>(&map_dv, out_stage, row0, slab);
       tc_fence_after_sync();
 #pragma unroll
       for (int h = 0; h < NH; ++h)
@@ -367,13 +397,17 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
       tmem_ld32(trow + acc + 32 * wg, r);
       tmem_ld_wait();
       reg_fence32(r);
-      if (row < n) store_row32<float>(dKF + ((size_t)slab * n + row) * kD + 32 * wg, r);
+      stage_row32<float>(out_stage + 2 * kTileBytes, tl, wg, r);
     }
+    fence_proxy_async_smem();
     tc_fence_before_sync();
-    __syncthreads();   // the next tile's copies and MMA1 overwrite what this tile read
+    __syncthreads();   // the next tile's MMA1 overwrites what this tile read
+    if (threadIdx.x == 0) store_tile<float>(&map_dkf, out_stage + 2 * kTileBytes, row0, slab);
   }
-  if (!ok && threadIdx.x == 0) {   // copies may still be in flight
-    for (int t = max(0, issued - 2); t < issued; ++t) mbar_wait_drain(&bars->full[t & 1], (t >> 1) & 1);
+  if (threadIdx.x == 0) {
+    if (!ok)   // copies may still be in flight
+      for (int t = max(0, issued - 2); t < issued; ++t) mbar_wait_drain(&bars->full[t & 1], (t >> 1) & 1);
+    bulk_wait_group0();   // the result stores read this CTA's shared memory
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -407,8 +441,9 @@ __global__ void __launch_bounds__(256, 1)
 k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant__ CUtensorMap map_do,
                const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ Sbf,
                const float* __restrict__ zg, const float* __restrict__ beta, float eps, float bw_floor,
-               float* __restrict__ dQF, float* __restrict__ dspart, float* __restrict__ dzpart,
-               float* __restrict__ sumdD, int n, int chunk_tiles, int* __restrict__ status) {
+               const __grid_constant__ CUtensorMap map_dqf, float* __restrict__ dspart,
+               float* __restrict__ dzpart, float* __restrict__ sumdD, int n, int chunk_tiles,
+               int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   using SL = BwdQSmem<NH>;
@@ -533,6 +568,7 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
     }
     // ---- MMA2: N'
     if (threadIdx.x == 0) {
+      bulk_wait_group_read0();   // dQ_F of the previous tile has left the dN' tiles, which are written next
       tc_fence_after_sync();
 #pragma unroll
       for (int h = 0; h < NH; ++h)
@@ -648,10 +684,12 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
       tmem_ld32(trow + acc + 32 * wg, r);
       tmem_ld_wait();
       reg_fence32(r);
-      if (row < n) store_row32<float>(dQF + ((size_t)slab * n + row) * kD + 32 * wg, r);
+      stage_row32<float>(smem + SL::dn, tl, wg, r);   // the dN' tiles are free: MMA5 and MMA3 have completed
     }
+    fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
+    if (threadIdx.x == 0) store_tile<float>(&map_dqf, smem + SL::dn, row0, slab);
   }
   // ---- partial dS', dz', sum dD' of this chunk (zeros if the chunk gave up)
   const size_t pidx = (size_t)slab * gridDim.x + chunk;
@@ -671,7 +709,7 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
       tmem_ld32(trow + kAccS + h * 64 + 32 * c, r);
       tmem_ld_wait();
       reg_fence32(r);
-      store_row32<float>(dspart + (pidx * m + h * 128 + tl) * kD + 32 * c, r);
+      store_row32(dspart + (pidx * m + h * 128 + tl) * kD + 32 * c, r);
     }
     if (NH == 1) {
       if (wg == 0) dzpart[pidx * m + tl] = dzacc[0] + dds[tl];
@@ -679,8 +717,10 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
       dzpart[pidx * m + wg * 128 + tl] = dzacc[NH - 1 < wg ? 0 : wg];
     }
   }
-  if (!ok && threadIdx.x == 0) {
-    for (int t = max(0, issued - 2); t < issued; ++t) mbar_wait_drain(&bars->full[t & 1], (t >> 1) & 1);
+  if (threadIdx.x == 0) {
+    if (!ok)
+      for (int t = max(0, issued - 2); t < issued; ++t) mbar_wait_drain(&bars->full[t & 1], (t >> 1) & 1);
+    bulk_wait_group0();   // the dQ_F stores read this CTA's shared memory
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -722,16 +762,36 @@ cudaError_t make_tile_map(const void* base, int slabs, int n, CUtensorMap* out) 
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+// Store map of a (slabs x n x 64) result tensor: fp32 in boxes of 128 rows x 32 columns (128 bytes, the
+// widest a 128-byte swizzle takes), bf16 in boxes of 128 rows x 64 columns; rows past n are not written.
+cudaError_t make_out_map(void* base, int slabs, int n, bool bf16, CUtensorMap* out) {
+  if (bf16) return make_tile_map(base, slabs, n, out);
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return cudaErrorNotSupported;
+  const cuuint64_t dims[3] = {kD, (cuuint64_t)n, (cuuint64_t)slabs};
+  const cuuint64_t strides[2] = {kD * 4, (cuuint64_t)n * kD * 4};
+  const cuuint32_t box[3] = {32, kTile, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 template <int NH, typename TG>
 cudaError_t launch_kside(const Plan& p, const Ws& w, const CUtensorMap& map_kf, const CUtensorMap& map_v, void* dV,
                          cudaStream_t st) {
+  CUtensorMap map_dv, map_dkf;
+  cudaError_t merr;
+  if ((merr = make_out_map(dV, p.slabs, p.cfg.seq_len, sizeof(TG) == 2, &map_dv)) != cudaSuccess) return merr;
+  if ((merr = make_out_map(w.dKF, p.slabs, p.cfg.seq_len, false, &map_dkf)) != cudaSuccess) return merr;
   auto k = k_tc_bwd_kside<NH, TG>;
   cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdKSmem<NH>::total);
   if (err != cudaSuccess) return err;
   const long long tiles_all = (long long)((p.cfg.seq_len + kTile - 1) / kTile) * p.slabs;
   const unsigned grid = (unsigned)(tiles_all < 148 ? tiles_all : 148);   // one CTA per SM of a B200, one wave
-  k<<<grid, 256, BwdKSmem<NH>::total, st>>>(map_kf, map_v, w.Wt, w.dSbf, w.dz, static_cast<TG*>(dV), w.dKF,
-                                            p.cfg.seq_len, p.slabs, w.status);
+  k<<<grid, 256, BwdKSmem<NH>::total, st>>>(map_kf, map_v, w.Wt, w.dSbf, w.dz, map_dv, map_dkf, p.cfg.seq_len, p.slabs,
+                                            w.status);
   return cudaGetLastError();
 }
 
@@ -741,8 +801,10 @@ cudaError_t launch_qside(const Plan& p, const Ws& w, const CUtensorMap& map_qf, 
   auto k = k_tc_bwd_qside<NH>;
   cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdQSmem<NH>::total);
   if (err != cudaSuccess) return err;
+  CUtensorMap map_dqf;
+  if ((err = make_out_map(w.dQF, p.slabs, p.cfg.seq_len, false, &map_dqf)) != cudaSuccess) return err;
   dim3 grid(p.bchunks, p.slabs);
-  k<<<grid, 256, BwdQSmem<NH>::total, st>>>(map_qf, map_do, w.Wt, w.Sbf, w.z, beta, p.cfg.eps, p.cfg.bw_floor, w.dQF,
+  k<<<grid, 256, BwdQSmem<NH>::total, st>>>(map_qf, map_do, w.Wt, w.Sbf, w.z, beta, p.cfg.eps, p.cfg.bw_floor, map_dqf,
                                             w.spart, w.zpart, w.sumdD, p.cfg.seq_len, p.bchunk_tiles, w.status);
   return cudaGetLastError();
 }
