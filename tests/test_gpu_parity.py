@@ -308,6 +308,44 @@ def test_backward_small(case, dtype):
     _check_backward(cfg, inp, grads)
 
 
+@pytest.mark.parametrize("case", [1, 2, 4])
+@pytest.mark.parametrize("simt", [False, True])
+def test_backward_bf16_gradients(case, simt):
+    """grad_dtype = bf16: dQ, dK, dV are the fp32-gradient run rounded to bf16 on the way out (the same
+    arithmetic, another store), and meet the oracle at the bf16 tolerance."""
+    import paper_2507_08637_b200 as wersa
+    import torch
+    cfg = dict(BWD_SMALL[case], dtype="bf16", eps=1e-3)
+    inp = wi.make_inputs(**cfg, seed=450 + case, w_seed=550 + case, gate_std=0.3, gate_seed=650 + case,
+                         mean_shift=0.25, scale=0.7, backward=True)
+    dev = device_inputs(inp, "bf16")
+    args = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    flags = wersa.WERSA_FLAG_SIMT_ONLY if simt else 0
+    out = {}
+    for gd in ("f32", "bf16"):
+        ctx = _ctx(cfg, grad_dtype=gd, flags=flags)
+        assert ctx.uses_tensor_cores() == (not simt)
+        ctx.forward(*args)
+        out[gd] = ctx.backward(*args, dev["dO"])
+        torch.cuda.synchronize()
+        assert ctx.query_status() == 0
+    for key in ("dQ", "dK", "dV"):
+        assert out["bf16"][key].dtype == torch.bfloat16
+        err = normalised_error(to_numpy64(out["bf16"][key]), to_numpy64(out["f32"][key]))
+        assert err.max() <= 2.0 ** -7, (key, err.max())   # dQ is rounded twice (filter, then the mean-pool term)
+    if not simt:   # dV goes from the fp32 accumulator to its store in one rounding
+        assert torch.equal(out["bf16"]["dV"], out["f32"]["dV"].to(torch.bfloat16))
+    for key in ("dbeta", "dgate_w", "dgate_b", "domega"):
+        assert torch.equal(out["bf16"][key], out["f32"][key]), key
+    # Against the oracle: the fp32-stored gradients meet the bf16 tolerance as they are; the bf16-stored ones
+    # get the storage roundings on top (one for dK and dV, two for dQ; 2^-9 of the value each).
+    ref = _check_backward(cfg, inp, out["f32"])
+    for key in ("dQ", "dK", "dV"):
+        err = normalised_error(to_numpy64(out["bf16"][key]), ref[key])
+        assert err.max() <= BF16_MAX + 2.0 ** -8, (key, "max", err.max())
+        assert err.mean() <= BF16_MEAN + 2.0 ** -10, (key, "mean", err.mean())
+
+
 def test_config5_training_step_bf16():
     import torch
     # full configuration on the GPU ...
