@@ -6,10 +6,10 @@
 //   MMA1: B_h = K_F (smem, K-major; three bf16 planes hi + mid + lo that add up to the fp32 K_F, so
 //         that the mask below does not flip through rounding) * W_h (as W^T, K-major) -> TMEM fp32
 //   threads: mask = 1[B_h > 0] (bits in registers), Phi_h = ReLU(B_h) -> bf16 pairs in place
-//   MMA2: dV = sum_h Phi_h (TMEM operand) * dS'_h (smem bf16, N-major) -> TMEM fp32 -> global
+//   MMA2: dV = sum_h Phi_h (TMEM operand) * dS'_h (smem bf16, N-major) -> TMEM fp32 -> smem -> TMA store
 //   MMA3: G_h = V (smem, K-major) * dS'_h^T (same image, K-major)      -> TMEM fp32
 //   threads: dB_h = (G_h + dz'_h) (.) mask                              -> bf16 pairs in place
-//   MMA4: dK_F = sum_h dB_h (TMEM operand) * W_h^T (W^T image, N-major) -> TMEM fp32 -> global
+//   MMA4: dK_F = sum_h dB_h (TMEM operand) * W_h^T (W^T image, N-major) -> TMEM fp32 -> smem -> TMA store
 // Query side, per 128-token tile:
 //   MMA1: A_h = Q_F (three planes) * W_h                                -> TMEM fp32 (token = lane)
 //   threads: mask, Phi_h -> bf16 in place, D' = sum_h Phi_h . z'_h + eps'
@@ -20,7 +20,7 @@
 //   MMA5: dS'_h += Phi_h^T (TMEM operand) * dN' (smem tile, N-major)    -> TMEM fp32, kept for the chunk
 //   MMA3: G_h = dN' (smem, K-major) * S'_h^T (same image, K-major)      -> TMEM fp32 (token = lane)
 //   threads: dA_h = (G_h + dD' z'_h) (.) mask                           -> bf16 in place
-//   MMA4: dQ_F = sum_h dA_h * W_h^T (W^T image, N-major)                -> TMEM fp32 -> global
+//   MMA4: dQ_F = sum_h dA_h * W_h^T (W^T image, N-major)                -> TMEM fp32 -> smem -> TMA store
 // and at the end of the chunk the partial dS', dz' and sum of dD' go to the split-sequence buffers.
 // One CTA of 256 threads per SM walks a chunk of tiles one step at a time (thread 0 issues the copies
 // and the MMAs, everybody waits on one mbarrier); the copies of the next tile are in flight meanwhile.
