@@ -304,6 +304,12 @@ def main():
 
     # ---- roofline of the dominant kernel -----------------------------------------------------
     peaks, peak_kind = load_peaks()
+    # Which bf16 peak is the denominator: the burst figure while the clocks stay at their maximum, the
+    # sustained one once the timed region is long enough for the power cap to pull them down.
+    sustained = ("sw_power_cap" in clocks.get("reasons", []) and clocks.get("sm_mhz") and clocks.get("sm_max_mhz")
+                 and clocks["sm_mhz"] < 0.985 * clocks["sm_max_mhz"] and "bf16_tflops_sustained" in peaks)
+    tensor_peak = float(peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"])
+    regime = "sustained" if sustained else "burst"
     TH = cfg["B"] * cfg["H"] * cfg["n"]
     d, m = cfg["d"], cfg["m"]
     s_bytes = 2 if dtype == "bf16" else 4
@@ -323,7 +329,7 @@ def main():
     ncu_bytes_per_th = {"qmean_gate": 128.8, "tc_kside": 264.0, "tc_qside": 165.9}
     if dom in flops:
         if dom.startswith("tc_"):
-            bound, peak, unit = "tensor", float(peaks["bf16_tflops"]), "TFLOP/s"
+            bound, peak, unit = "tensor", tensor_peak, "TFLOP/s"
         else:
             bound, peak, unit = "alu", FP32_ALU_TFLOPS, "TFLOP/s"
         achieved = flops[dom] / (avg[dom] * 1e-3) / 1e12
@@ -333,7 +339,7 @@ def main():
     traffic = ncu_bytes_per_th[dom] * TH if (tensor_cores and dtype == "bf16" and dom in ncu_bytes_per_th) else None
     roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
                 "frac": achieved / peak, "traffic": traffic,
-                "peak_source": f"{peak_kind} (burst)" if bound == "tensor" else
+                "peak_source": f"{peak_kind} ({regime})" if bound == "tensor" else
                                (peak_kind if bound == "hbm" else "derived: 148 SM x 128 FFMA x 2 x 1.965 GHz"),
                 "kernel_ms": avg, "kernel_share": {k: v / tot for k, v in avg.items()},
                 "timing": "CUDA events behind every kernel, second pass of K steps"}
@@ -343,9 +349,9 @@ def main():
     # whole-path roofline: slower of FLOPs at tensor peak and bytes at HBM bandwidth
     path_flops = TH * (8 * d * m + 4 * m)
     path_bytes = TH * 4 * d * s_bytes
-    t_roof = max(path_flops / (float(peaks["bf16_tflops"]) * 1e12), path_bytes / (float(peaks["hbm_gbs"]) * 1e9))
+    t_roof = max(path_flops / (tensor_peak * 1e12), path_bytes / (float(peaks["hbm_gbs"]) * 1e9))
     t_nom = max(path_flops / 2.25e15, path_bytes / 8.0e12)
-    path = {"roofline_us": t_roof * 1e6, "frac": t_roof / (ms_per_step * 1e-3), "peaks": peak_kind,
+    path = {"roofline_us": t_roof * 1e6, "frac": t_roof / (ms_per_step * 1e-3), "peaks": f"{peak_kind} ({regime})",
             "roofline_us_nominal": t_nom * 1e6, "frac_nominal": t_nom / (ms_per_step * 1e-3),
             "flops": path_flops, "bytes": path_bytes}
 
