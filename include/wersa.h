@@ -149,16 +149,20 @@ wersa_status wersa_haar_filter(wersa_ctx* ctx, const void* X, const float* f, vo
  *   cfg    as for wersa_create (only shapes, dtype, gate_per_head and device are used).
  *   Q      (batch, heads, seq_len, head_dim) of cfg->dtype; gate_w, gate_b may be NULL (zeros).
  *   qbar   out, (batch*heads, head_dim) floats;  f  out, (batch*heads, levels+1) floats.
- * Returns WERSA_ERR_TOO_LARGE, launching nothing, when batch*heads*(64*chunks + levels+2) + batch exceeds
- * 262144 array elements (chunks is the number of row chunks the mean pool splits the sequence into, about
- * 592/(batch*heads), at least 1): all five benchmark configurations fit.
+ * Returns WERSA_ERR_TOO_LARGE, launching nothing, when batch*heads*(64*chunks + levels+1) exceeds the
+ * 253952 floats the array leaves for sums (chunks is the number of row chunks the mean pool splits the
+ * sequence into, about 592/(batch*heads), at least 1), or when batch*heads + batch exceeds the 8192
+ * arrival counters kept in the array's last 8192 elements: all five benchmark configurations fit.
  * The first call on a device resolves the array's device address (once per device, with that
- * device made current); make that first call outside any CUDA stream capture.
- * Every call on a device shares the one array.  The partial sums and sigmoid values it reads are written
- * earlier in the same call; the small arrival counters at its end must be zero when a call starts -- they are
- * zero when the library is loaded and every call leaves them at zero, so nothing needs clearing between
- * calls.  Two calls that overlap on the GPU (different streams, no ordering between them) race on the array
- * and must be serialised by the caller. */
+ * device made current); make that first call outside any CUDA stream capture.  The address is kept for
+ * the life of the process: do not reset the device (cudaDeviceReset) while the library is loaded.
+ * Every call on a device shares the one array, and the array keeps what the last call left.  The partial
+ * sums and sigmoid values a call reads are written earlier in the same call.  The arrival counters live at
+ * a fixed place at the end of the array, whatever the problem's shape, and every call clears the ones it
+ * uses with a memset on cuda_stream ahead of its kernel: calls of different shapes may follow each other
+ * in any order, and a call that failed half way does not disturb the next.  Two calls that overlap on the
+ * GPU (different streams, no ordering between them) race on the array and must be serialised by the
+ * caller. */
 wersa_status wersa_gate_static(const wersa_config* cfg, const void* Q, const float* gate_w,
                                const float* gate_b, const float* omega, float* qbar, float* f,
                                void* cuda_stream);

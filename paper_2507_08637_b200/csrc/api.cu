@@ -384,7 +384,9 @@ wersa_status wersa_gate_static(const wersa_config* cfg, const void* Q, const flo
   Plan p;
   wersa_status s = make_plan(*cfg, &p);
   if (s != WERSA_OK) return s;
-  if (static_scratch_floats_needed(p) > static_scratch_capacity_floats()) return WERSA_ERR_TOO_LARGE;
+  if (static_scratch_floats_needed(p) > static_scratch_capacity_floats() ||
+      static_scratch_counters_needed(p) > static_scratch_counter_capacity())
+    return WERSA_ERR_TOO_LARGE;
   DeviceGuard guard(p.cfg.device);
   if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
   float* scratch = nullptr;
@@ -479,7 +481,7 @@ const char* wersa_status_string(wersa_status status) {
     case WERSA_ERR_CUDA: return "CUDA runtime error";
     case WERSA_ERR_TIMEOUT: return "bounded device wait expired";
     case WERSA_ERR_STATE: return "backward or saved-tensor query without a preceding forward";
-    case WERSA_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of wersa_gate_static (262144 floats)";
+    case WERSA_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of wersa_gate_static (253952 floats + 8192 counters)";
   }
   return "unknown status";
 }

@@ -69,8 +69,10 @@ cudaError_t launch_add_rowvec(const Plan& p, const Ws& w, void* dQ, cudaStream_t
 
 // Mean pool + gate with their scratch in a file-scope device array (no caller workspace).
 cudaError_t static_scratch_address(int device, float** out);
-size_t static_scratch_capacity_floats();
+size_t static_scratch_capacity_floats();      // floats available to the partial sums and sigmoids
+size_t static_scratch_counter_capacity();     // ints reserved for the arrival counters
 size_t static_scratch_floats_needed(const Plan& p);
+size_t static_scratch_counters_needed(const Plan& p);
 cudaError_t launch_qmean_gate_static(const Plan& p, float* scratch, const void* Q, const float* gate_w,
                                      const float* gate_b, const float* omega, float* qbar, float* f,
                                      cudaStream_t st);

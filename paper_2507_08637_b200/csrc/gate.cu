@@ -6,8 +6,11 @@
 namespace wersa {
 namespace {
 
-// Scratch of wersa_gate_static: lives in the library image of every GPU that loads it.
+// Scratch of wersa_gate_static: lives in the library image of every GPU that loads it.  The last
+// kStaticCounterInts elements are reserved for the arrival counters, at a place that does not depend on
+// the problem, so that no float of any call's layout can ever land on them.
 constexpr size_t kStaticScratchFloats = 262144;   // 1 MiB
+constexpr size_t kStaticCounterInts = 8192;       // slab counters, then batch counters
 static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
 constexpr int kMaxDevices = 64;
 float* g_static_scratch_addr[kMaxDevices] = {nullptr};
@@ -328,22 +331,28 @@ cudaError_t static_scratch_address(int device, float** out) {
   return cudaSuccess;
 }
 
-size_t static_scratch_capacity_floats() { return kStaticScratchFloats; }
+size_t static_scratch_capacity_floats() { return kStaticScratchFloats - kStaticCounterInts; }
+size_t static_scratch_counter_capacity() { return kStaticCounterInts; }
 
 cudaError_t launch_qmean_gate_static(const Plan& p, float* scratch, const void* Q, const float* gate_w,
                                      const float* gate_b, const float* omega, float* qbar, float* f,
                                      cudaStream_t st) {
-  // scratch = [ partial column sums: slabs x qchunks x 64 | sigmoid(u): slabs x (L+1) | arrival counters:
-  //             slabs + batch ints, zero when the library is loaded and left at zero by every call ]
+  // scratch = [ partial column sums: slabs x qchunks x 64 | sigmoid(u): slabs x (L+1) | unused ...
+  //             | arrival counters in the last kStaticCounterInts elements: slabs, then batch ints ]
+  // The counters this call uses are cleared on the stream first (a memset allocates nothing): a call
+  // then starts from zero whatever an earlier call of another shape, or one that failed half way, left.
   float* qpart = scratch;
   float* sg = scratch + (size_t)p.slabs * p.qchunks * kD;
-  int* counters = reinterpret_cast<int*>(sg + (size_t)p.slabs * p.L1);
+  int* counters = reinterpret_cast<int*>(scratch + (kStaticScratchFloats - kStaticCounterInts));
+  cudaError_t err = cudaMemsetAsync(counters, 0, sizeof(int) * ((size_t)p.slabs + (size_t)p.cfg.batch), st);
+  if (err != cudaSuccess) return err;
   return launch_qmean_gate_impl(p, Q, qpart, gate_w, gate_b, omega, qbar, sg, f, counters, nullptr, nullptr, st);
 }
 
 size_t static_scratch_floats_needed(const Plan& p) {
-  return (size_t)p.slabs * p.qchunks * kD + (size_t)p.slabs * p.L1 + (size_t)p.slabs + (size_t)p.cfg.batch;
+  return (size_t)p.slabs * p.qchunks * kD + (size_t)p.slabs * p.L1;
 }
+size_t static_scratch_counters_needed(const Plan& p) { return (size_t)p.slabs + (size_t)p.cfg.batch; }
 
 cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, const float* gate_w,
                                  const float* omega, int n_sumdD, float* dbeta, float* dgate_w, float* dgate_b,
