@@ -25,8 +25,11 @@ if ROOT not in sys.path:
 METRIC = "WERSA attn tokens/sec on 1 B200 at n=128k (device-timed), % of roofline"
 DEFAULT_WORKLOAD = "cfg4_long_bf16"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# fp32 FFMA peak of the fp32 kernels: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (max SM clock)
-FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def fp32_alu_tflops(sms, sm_max_mhz):
+    """fp32 FFMA peak behind the fp32 kernels: SMs x 128 lanes x 2 flop x maximum SM clock."""
+    return sms * 128 * 2 * sm_max_mhz * 1e6 / 1e12
 
 
 def load_peaks():
@@ -36,6 +39,36 @@ def load_peaks():
             p = json.load(fh)
         return p, "measured"
     return dict(FALLBACK_PEAKS), "fallback"
+
+
+def load_traffic():
+    """DRAM bytes per token-head per forward kernel from the tracked ncu summary, or ({}, reason) when the
+    kernel sources have changed since the counters were taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "forward_dram_traffic.txt")
+    if not os.path.exists(path):
+        return {}, "no capture on file"
+    fields = {}
+    with open(path) as fh:
+        for line in fh:
+            if line.startswith("#") or ":" not in line:
+                continue
+            key, val = line.split(":", 1)
+            fields[key.strip()] = val.strip()
+    h = hashlib.sha256()
+    for rel in fields.get("source_files", "").split():
+        with open(os.path.join(ROOT, rel), "rb") as fh:
+            h.update(fh.read())
+    where = f"profiles/forward_dram_traffic.txt (ncu capture at commit {fields.get('captured_at_commit', '?')}, scaled by token-heads)"
+    if h.hexdigest() != fields.get("source_sha256"):
+        return {}, "stale: kernel sources changed since " + where
+    out = {}
+    for key, val in fields.items():
+        try:
+            out[key] = float(val)
+        except ValueError:
+            pass
+    return out, where
 
 
 def workload_string(cfg):
@@ -141,7 +174,8 @@ def run_reference(args, cfg, inp, rank):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / len(times),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic", "config": {"workload": workload_string(cfg)},
-        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": used, "kind": "oracle", "sample": desc},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": used, "kind": "oracle", "sample": desc,
+                         "host_cores": os.cpu_count()},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -178,7 +212,7 @@ def main():
     import torch
 
     import paper_2507_08637_b200 as wersa
-    from tests.util import device_inputs
+    from wersa_inputs import device_inputs
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
@@ -304,6 +338,8 @@ def main():
 
     # ---- roofline of the dominant kernel -----------------------------------------------------
     peaks, peak_kind = load_peaks()
+    sms = torch.cuda.get_device_properties(local_rank).multi_processor_count
+    sm_max_mhz = float(clocks.get("sm_max_mhz") or peaks.get("sm_max_mhz") or 1965.0)
     # Which bf16 peak is the denominator: the burst figure while the clocks stay at their maximum, the
     # sustained one once the timed region is long enough for the power cap to pull them down.
     sustained = ("sw_power_cap" in clocks.get("reasons", []) and clocks.get("sm_mhz") and clocks.get("sm_max_mhz")
@@ -323,24 +359,21 @@ def main():
               "haar_filter_k": TH * d * (s_bytes + 4),
               "tc_kside": 2 * TH * d * s_bytes,      # K and V read once
               "tc_qside": 2 * TH * d * s_bytes}      # Q read once, O written once
-    # DRAM bytes per token-head of one launch, from the ncu capture summarised in
-    # profiles/forward_cfg5_ncu_full_set.md (dram__bytes_read.sum + dram__bytes_write.sum on the cfg5
-    # forward, 524288 token-heads; traffic grows in proportion to the token-heads of a launch)
-    ncu_bytes_per_th = {"qmean_gate": 128.8, "tc_kside": 264.0, "tc_qside": 165.9}
+    ncu_bytes_per_th, traffic_source = load_traffic()
     if dom in flops:
         if dom.startswith("tc_"):
             bound, peak, unit = "tensor", tensor_peak, "TFLOP/s"
         else:
-            bound, peak, unit = "alu", FP32_ALU_TFLOPS, "TFLOP/s"
+            bound, peak, unit = "alu", fp32_alu_tflops(sms, sm_max_mhz), "TFLOP/s"
         achieved = flops[dom] / (avg[dom] * 1e-3) / 1e12
     else:
         bound, peak, unit = "hbm", float(peaks["hbm_gbs"]), "GB/s"
         achieved = bytes_.get(dom, 0) / (avg[dom] * 1e-3) / 1e9
     traffic = ncu_bytes_per_th[dom] * TH if (tensor_cores and dtype == "bf16" and dom in ncu_bytes_per_th) else None
     roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
-                "frac": achieved / peak, "traffic": traffic,
+                "frac": achieved / peak, "traffic": traffic, "traffic_source": traffic_source,
                 "peak_source": f"{peak_kind} ({regime})" if bound == "tensor" else
-                               (peak_kind if bound == "hbm" else "derived: 148 SM x 128 FFMA x 2 x 1.965 GHz"),
+                               (peak_kind if bound == "hbm" else f"derived: {sms} SM x 128 FFMA x 2 x {sm_max_mhz:.0f} MHz"),
                 "kernel_ms": avg, "kernel_share": {k: v / tot for k, v in avg.items()},
                 "timing": "CUDA events behind every kernel, second pass of K steps"}
     if dom in flops and dom in bytes_:   # the tensor-core kernels sit on the ridge: report the HBM side too
@@ -393,7 +426,7 @@ def main():
     if not args.no_cpu_baseline:
         rate, desc, used, _ = oracle_sample_rate(cfg, inp, 15.0)
         line["cpu_baseline"] = {"value": rate, "unit": "tokens/s", "cores": used, "kind": "oracle",
-                                "sample": desc}
+                                "sample": desc, "host_cores": os.cpu_count()}
     else:
         line["cpu_baseline"] = None
     print(json.dumps(line), flush=True)

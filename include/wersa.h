@@ -151,7 +151,7 @@ wersa_status wersa_haar_filter(wersa_ctx* ctx, const void* X, const float* f, vo
  *   qbar   out, (batch*heads, head_dim) floats;  f  out, (batch*heads, levels+1) floats.
  * Returns WERSA_ERR_TOO_LARGE, launching nothing, when batch*heads*(64*chunks + levels+1) exceeds the
  * 253952 floats the array leaves for sums (chunks is the number of row chunks the mean pool splits the
- * sequence into, about 592/(batch*heads), at least 1), or when batch*heads + batch exceeds the 8192
+ * sequence into, about four per multiprocessor over all slabs -- 592/(batch*heads) on a B200 --, at least 1), or when batch*heads + batch exceeds the 8192
  * arrival counters kept in the array's last 8192 elements: all five benchmark configurations fit.
  * The first call on a device resolves the array's device address (once per device, with that
  * device made current); make that first call outside any CUDA stream capture.  The address is kept for
@@ -179,6 +179,18 @@ wersa_status wersa_saved(wersa_ctx* ctx, int which, const float** device_ptr, si
  * up on a bounded wait, WERSA_ERR_CUDA on a sticky CUDA error, else WERSA_OK.  Clears the
  * device-side error word. */
 wersa_status wersa_query_status(wersa_ctx* ctx, void* cuda_stream);
+
+/* Self-test of the error path behind WERSA_ERR_TIMEOUT (the paper has no counterpart).  Every wait of the
+ * tensor-core kernels on a shared-memory barrier is bounded; when one runs out, the waiting role records
+ * a code in the context's device status word, raises the CTA's abort flag and every role leaves without
+ * touching further data.  This call enqueues one small CTA that runs exactly that path: it waits, for at
+ * most limit_us microseconds (1..100000), on a barrier that is one arrival short, while a second role
+ * waits for a hand-off that therefore never comes.  Nothing faults and nothing waits longer than the
+ * limit.  observed: DEVICE pointer to 3 ints, written by the kernel: [0] the abort flag (1), [1] and [2]
+ * whether the two roles' waits succeeded (0 and 0).  Afterwards wersa_query_status returns
+ * WERSA_ERR_TIMEOUT once and WERSA_OK from then on. */
+wersa_status wersa_selftest_wait_timeout(wersa_ctx* ctx, uint32_t limit_us, int32_t* observed,
+                                         void* cuda_stream);
 
 /* Releases the host-side context.  Does not touch the workspace.  NULL is accepted. */
 wersa_status wersa_destroy(wersa_ctx* ctx);

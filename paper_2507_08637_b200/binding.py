@@ -72,6 +72,8 @@ def _lib():
     lib.wersa_launch_count.argtypes = [vp, ctypes.c_int]
     lib.wersa_gate_static.restype = ctypes.c_int
     lib.wersa_gate_static.argtypes = [ctypes.POINTER(wersa_config), vp, fp, fp, fp, fp, fp, vp]
+    lib.wersa_selftest_wait_timeout.restype = ctypes.c_int
+    lib.wersa_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint32, vp, vp]
     lib.wersa_uses_tensor_cores.restype = ctypes.c_int32
     lib.wersa_uses_tensor_cores.argtypes = [vp]
     lib.wersa_set_step_timing.restype = ctypes.c_int
@@ -229,6 +231,16 @@ class WersaContext:
 
     def query_status(self, stream=None):
         return int(_lib().wersa_query_status(self._h, _stream_ptr(stream)))
+
+    def selftest_wait_timeout(self, limit_us=1000, stream=None):
+        """wersa_selftest_wait_timeout: returns the three ints the kernel observed (abort flag, and whether
+        the two roles' waits succeeded) as a CUDA int32 tensor; read it after synchronising."""
+        observed = torch.full((3,), -1, dtype=torch.int32, device=self.device)
+        st = _lib().wersa_selftest_wait_timeout(self._h, int(limit_us), _ptr(observed, torch.int32, "observed"),
+                                                _stream_ptr(stream))
+        if st != WERSA_OK:
+            raise WersaError(st, "wersa_selftest_wait_timeout")
+        return observed
 
     def set_step_timing(self, enable):
         st = _lib().wersa_set_step_timing(self._h, int(bool(enable)))

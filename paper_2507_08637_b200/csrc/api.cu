@@ -17,6 +17,16 @@ int next_pow2(int n) {
   while (p < n) p <<= 1;
   return p;
 }
+// Streaming multiprocessors of the device the plan is made for: the chunk counts below aim at whole
+// waves of CTAs.  Without a device (host-only sizing queries) the count of a B200 is assumed.
+int device_sm_count(int device) {
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 1) {
+    cudaGetLastError();   // a failed query leaves no sticky error behind
+    sms = 148;
+  }
+  return sms;
+}
 
 }  // namespace
 
@@ -41,8 +51,9 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   p->with_backward = !(c.flags & WERSA_FLAG_FORWARD_ONLY);
   p->use_tc = p->bf16 && !(c.flags & WERSA_FLAG_SIMT_ONLY) && tc_supported(c);
   const int n = c.seq_len, m = c.features;
+  p->sms = device_sm_count(c.device);
 
-  p->qchunks = ceil_div(592, p->slabs);
+  p->qchunks = ceil_div(4 * p->sms, p->slabs);
   if (p->qchunks > ceil_div(n, 128)) p->qchunks = ceil_div(n, 128);
   if (p->qchunks < 1) p->qchunks = 1;
   p->qchunk_rows = ceil_div(ceil_div(n, p->qchunks), 32) * 32;
@@ -51,7 +62,7 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   p->htiles = ceil_div(n, kHaarTile);
 
   const int tiles32 = ceil_div(n, kSimtTile);
-  p->schunks = ceil_div(296, p->slabs);
+  p->schunks = ceil_div(2 * p->sms, p->slabs);
   if (p->schunks > tiles32) p->schunks = tiles32;
   p->schunk_tiles = ceil_div(tiles32, p->schunks);
   p->schunks = ceil_div(tiles32, p->schunk_tiles);
@@ -60,7 +71,7 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   p->tchunk_blocks = 0;
   if (p->use_tc) {
     const int blocks = ceil_div(n, 256);
-    p->tchunks = 148 / p->slabs;
+    p->tchunks = p->sms / p->slabs;
     if (p->tchunks < 1) p->tchunks = 1;
     if (p->tchunks > blocks) p->tchunks = blocks;
     p->tchunk_blocks = ceil_div(blocks, p->tchunks);
@@ -68,7 +79,7 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   }
   {
     const int tiles128 = ceil_div(n, 128);
-    p->bchunks = 148 / p->slabs;   // one CTA per SM, a single wave
+    p->bchunks = p->sms / p->slabs;   // one CTA per SM, a single wave
     if (p->bchunks < 1) p->bchunks = 1;
     if (p->bchunks > tiles128) p->bchunks = tiles128;
     p->bchunk_tiles = ceil_div(tiles128, p->bchunks);
@@ -426,6 +437,17 @@ wersa_status wersa_query_status(wersa_ctx* ctx, void* cuda_stream) {
     WERSA_CUDA(cudaStreamSynchronize(st));
     return WERSA_ERR_TIMEOUT;
   }
+  return WERSA_OK;
+}
+
+wersa_status wersa_selftest_wait_timeout(wersa_ctx* ctx, uint32_t limit_us, int32_t* observed, void* cuda_stream) {
+  if (ctx == nullptr || observed == nullptr || limit_us == 0 || limit_us > 100000) return WERSA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DeviceGuard guard(ctx->plan.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  wersa_status s = clear_status_once(ctx, st);
+  if (s != WERSA_OK) return s;
+  WERSA_CUDA(launch_selftest_wait(ctx->ws, 1000ull * limit_us, observed, st));
   return WERSA_OK;
 }
 

@@ -20,6 +20,7 @@ constexpr int kBandVals = 16;    // per-tile band inner products kept by the Haa
 struct Plan {
   wersa_config cfg;
   int slabs;          // B*H
+  int sms;            // streaming multiprocessors of cfg.device
   int L1;             // levels + 1
   bool bf16;          // storage type of Q,K,V,W,O,dO
   bool grad_bf16;     // storage type of dQ,dK,dV
@@ -120,6 +121,11 @@ cudaError_t launch_tc_bwd_qside(const Plan& p, const Ws& w, const void* QF3, con
                                 cudaStream_t st, int* launches);
 cudaError_t launch_tc_bwd_kside(const Plan& p, const Ws& w, const void* KF3, const void* V, void* dV,
                                 cudaStream_t st, int* launches);
+
+// ---- selftest.cu ---------------------------------------------------------------------------
+// One CTA whose bounded wait runs out after limit_ns: sets the status word; observed[0] = abort flag,
+// observed[1], observed[2] = whether the two roles' waits succeeded (both must read 0).
+cudaError_t launch_selftest_wait(const Ws& w, unsigned long long limit_ns, int* observed, cudaStream_t st);
 
 // ---- device helpers ------------------------------------------------------------------------
 __device__ __forceinline__ float to_f32(float x) { return x; }

@@ -789,7 +789,7 @@ cudaError_t launch_kside(const Plan& p, const Ws& w, const CUtensorMap& map_kf, 
   cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdKSmem<NH>::total);
   if (err != cudaSuccess) return err;
   const long long tiles_all = (long long)((p.cfg.seq_len + kTile - 1) / kTile) * p.slabs;
-  const unsigned grid = (unsigned)(tiles_all < 148 ? tiles_all : 148);   // one CTA per SM of a B200, one wave
+  const unsigned grid = (unsigned)(tiles_all < p.sms ? tiles_all : p.sms);   // one CTA per SM, one wave
   k<<<grid, 256, BwdKSmem<NH>::total, st>>>(map_kf, map_v, w.Wt, w.dSbf, w.dz, map_dv, map_dkf, p.cfg.seq_len, p.slabs,
                                             w.status);
   return cudaGetLastError();

@@ -222,48 +222,63 @@ def test_config1_single_head_fp32():
     print("cfg1 max err", err.max())
 
 
+_ORACLE_CACHE = {}
+
+
+def _oracle_forward_cached(name, cfg, inp):
+    """Full-tensor oracle forward of a named configuration, computed once per test session (both arithmetic
+    paths of the library are compared with the same reference)."""
+    if name not in _ORACLE_CACHE:
+        _ORACLE_CACHE[name] = _oracle_forward(cfg, inp, want_aux=True)
+    return _ORACLE_CACHE[name]
+
+
+def _check_config_forward(name, flags):
+    """Every element of O, of every slab, against the oracle; the key summary and the normaliser too."""
+    cfg, inp, dev, ctx, O = _run_config(name, flags=flags)
+    ref, aux = _oracle_forward_cached(name, cfg, inp)
+    err = _check(to_numpy64(O), ref, cfg["dtype"], name)
+    c = 1.0 / (max(float(inp["beta"][0]), 1e-6) * np.sqrt(cfg["m"]))
+    errS = normalised_error(to_numpy64(ctx.saved("S")).reshape(aux["S"].shape) * c, aux["S"])
+    errz = normalised_error(to_numpy64(ctx.saved("z")).reshape(aux["z"].shape) * c, aux["z"])
+    tolS = 2e-2 if not flags else 1e-4
+    assert errS.max() <= tolS and errz.max() <= (5e-3 if not flags else 1e-4), (errS.max(), errz.max())
+    # the stated bound also holds as a plain relative error wherever the reference is not small
+    big = np.abs(ref) > np.sqrt(np.mean(ref ** 2, axis=(2, 3), keepdims=True))
+    rel = np.abs(to_numpy64(O) - ref)[big] / np.abs(ref)[big]
+    assert rel.max() <= BF16_MAX, rel.max()
+    print(f"{name} flags={flags}: max {err.max():.3e} mean {err.mean():.3e} rel(|ref|>rms) {rel.max():.3e} "
+          f"S {errS.max():.3e} z {errz.max():.3e}")
+    return cfg, inp, dev, ctx, O
+
+
 @pytest.mark.parametrize("flags", [0, 1])
 def test_config2_text_bf16(flags):
-    cfg, inp, dev, ctx, O = _run_config("cfg2_text_bf16", flags=flags)
-    # oracle on a sample of slabs (every slab is independent given its head's gate parameters)
-    got = to_numpy64(O)
-    for (b, h) in [(0, 0), (3, 5), (7, 7)]:
-        sub = {k: (v[b:b + 1, h:h + 1] if k in ("Q", "K", "V") else v) for k, v in inp.items()}
-        sub["gate_w"], sub["gate_b"] = inp["gate_w"][h:h + 1], inp["gate_b"][h:h + 1]
-        ref = _oracle_forward(dict(cfg, B=1, H=1), sub)
-        _check(got[b:b + 1, h:h + 1], ref, "bf16", f"cfg2 slab {b},{h}")
+    _check_config_forward("cfg2_text_bf16", flags)
 
 
 @pytest.mark.parametrize("flags", [0, 1])
 def test_config3_vision_bf16(flags):
-    cfg, inp, dev, ctx, O = _run_config("cfg3_vision_bf16", flags=flags)
-    got = to_numpy64(O)
-    for (b, h) in [(0, 0), (17, 3), (63, 11), (40, 8)]:
-        sub = {k: (v[b:b + 1, h:h + 1] if k in ("Q", "K", "V") else v) for k, v in inp.items()}
-        sub["gate_w"], sub["gate_b"] = inp["gate_w"][h:h + 1], inp["gate_b"][h:h + 1]
-        ref = _oracle_forward(dict(cfg, B=1, H=1), sub)
-        _check(got[b:b + 1, h:h + 1], ref, "bf16", f"cfg3 slab {b},{h}")
+    _check_config_forward("cfg3_vision_bf16", flags)
 
 
 @pytest.mark.parametrize("flags", [0, 1])
 def test_config4_long_sequence_bf16(flags):
-    cfg, inp, dev, ctx, O = _run_config("cfg4_long_bf16", flags=flags)
-    got = to_numpy64(O)
-    n = cfg["n"]
-    rng = np.random.default_rng(0)
-    # whole 256-row Haar blocks at both ends and the middle plus scattered rows
-    rows = np.unique(np.concatenate([np.arange(0, 256), np.arange(n // 2 - 128, n // 2 + 128),
-                                     np.arange(n - 256, n), rng.integers(0, n, 1200)]))
-    for h in (0, 5):
-        sub = {k: (v[:, h:h + 1] if k in ("Q", "K", "V") else v) for k, v in inp.items()}
-        sub["gate_w"], sub["gate_b"] = inp["gate_w"][h:h + 1], inp["gate_b"][h:h + 1]
-        ref, aux = _oracle_forward(dict(cfg, H=1), sub, sample_rows=rows, want_aux=True)
-        # normalise by the rms of the sampled reference rows
-        err = normalised_error(got[:, h:h + 1, rows], ref[:, :, rows])
-        assert err.max() <= BF16_MAX and err.mean() <= BF16_MEAN, (h, err.max(), err.mean())
-        c = 1.0 / np.sqrt(cfg["m"])
-        S = to_numpy64(ctx.saved("S"))[:, h:h + 1] * c
-        assert normalised_error(S, aux["S"]).max() < 2e-2
+    _check_config_forward("cfg4_long_bf16", flags)
+
+
+def _dbeta_error(cfg, inp, got, ref_closed):
+    """Error of the bandwidth gradient, normalised like every other error here: by max(|ref|, natural scale).
+    dbeta = c sum_t dD_t with c = 2 eps / bw is a sum of signed terms that largely cancel (sum |dD_t| is
+    3.4e3 times |sum dD_t| on the training configuration), so a per-term relative error delta moves the sum by
+    about delta * sqrt(sum dD_t^2), whatever the size the sum happens to have.  That root-sum-square of the
+    terms, from the oracle's own O and D (dD_t = -sum_c dO[t,c] O[t,c] / D[t]), is the scale; the error is
+    |got - ref| / max(|ref|, c * sqrt(sum dD_t^2))."""
+    O, aux = _oracle_forward(cfg, inp, want_aux=True)
+    dD = -(np.asarray(inp["dO"], dtype=np.float64) * O).sum(-1) / aux["D"]
+    bw = max(float(inp["beta"][0]), 1e-6)
+    scale = 2.0 * cfg.get("eps", 1e-6) / bw * np.sqrt((dD ** 2).sum())
+    return abs(got - ref_closed) / max(abs(ref_closed), scale, 1e-300)
 
 
 def _check_backward(cfg, inp, grads, sub_slabs=None):
@@ -278,7 +293,10 @@ def _check_backward(cfg, inp, grads, sub_slabs=None):
         err = small_vector_error(to_numpy64(grads[key]), ref[key])
         assert err.max() <= tol, (key, err.max())
     db = float(grads["dbeta"].cpu()[0])
-    assert abs(db - ref["dbeta_closed"]) <= tol * max(abs(ref["dbeta_closed"]), 1e-30) * 5, (db, ref["dbeta_closed"])
+    rel = abs(db - ref["dbeta_closed"]) / max(abs(ref["dbeta_closed"]), 1e-300)
+    err = _dbeta_error(cfg, inp, db, ref["dbeta_closed"])
+    print(f"dbeta {db:.6e} ref {ref['dbeta_closed']:.6e} plain rel {rel:.3e} normalised {err:.3e}")
+    assert err <= tol, (db, ref["dbeta_closed"], err)
     return ref
 
 
@@ -346,37 +364,55 @@ def test_backward_bf16_gradients(case, simt):
         assert err.mean() <= BF16_MEAN + 2.0 ** -10, (key, "mean", err.mean())
 
 
-def test_config5_training_step_bf16():
+@pytest.mark.parametrize("flags", [0, 1])
+def test_config5_training_step_bf16(flags):
+    """The whole training configuration, every slab: O, dQ, dK, dV element by element, and the parameter
+    gradients (sums over all 32 slabs) of the same run, against the oracle."""
     import torch
-    # full configuration on the GPU ...
-    cfg, inp, dev, ctx, O = _run_config("cfg5_train_bf16")
+    name = "cfg5_train_bf16"
+    cfg, inp, dev, ctx, O = _check_config_forward(name, flags)
     args = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
     grads = ctx.backward(*args, dev["dO"])
     torch.cuda.synchronize()
     assert ctx.query_status() == 0
-    # ... oracle on two slabs (a slab depends only on its own rows and its head's gate)
-    b, hs = 1, slice(2, 4)
-    sub = {k: (v[b:b + 1, hs] if k in ("Q", "K", "V", "dO") else v) for k, v in inp.items()}
-    sub["gate_w"], sub["gate_b"] = inp["gate_w"][hs], inp["gate_b"][hs]
-    scfg = dict(cfg, B=1, H=2)
-    ref = orc.backward(sub["Q"], sub["K"], sub["V"], sub["W"], float(sub["beta"][0]), sub["gate_w"],
-                       sub["gate_b"], sub["omega"], sub["dO"], scfg["L"])
+    if name + "/bwd" not in _ORACLE_CACHE:
+        _ORACLE_CACHE[name + "/bwd"] = orc.backward(
+            inp["Q"], inp["K"], inp["V"], inp["W"], float(inp["beta"][0]), inp["gate_w"], inp["gate_b"],
+            inp["omega"], inp["dO"], cfg["L"])
+    ref = _ORACLE_CACHE[name + "/bwd"]
     for key in ("dQ", "dK", "dV"):
-        _check(to_numpy64(grads[key])[b:b + 1, hs], ref[key], "bf16", key)
-    refO = _oracle_forward(scfg, sub)
-    _check(to_numpy64(O)[b:b + 1, hs], refO, "bf16", "O")
-    # parameter gradients sum over slabs: compare them on the two-slab problem run on its own
-    sctx = _ctx(scfg)
-    sdev = device_inputs(sub, "bf16")
-    sargs = (sdev["Q"], sdev["K"], sdev["V"], sdev["W"], sdev["beta"], sdev["gate_w"], sdev["gate_b"], sdev["omega"])
-    sctx.forward(*sargs)
-    sg = sctx.backward(*sargs, sdev["dO"])
-    torch.cuda.synchronize()
+        err = _check(to_numpy64(grads[key]), ref[key], "bf16", key)
+        print(f"cfg5 flags={flags} {key}: max {err.max():.3e} mean {err.mean():.3e}")
     for key in ("dgate_w", "dgate_b", "domega"):
-        err = small_vector_error(to_numpy64(sg[key]), ref[key])
-        assert err.max() <= 2e-2, (key, err.max())
-    db = float(sg["dbeta"].cpu()[0])
-    assert abs(db - ref["dbeta_closed"]) <= 0.1 * abs(ref["dbeta_closed"]) + 1e-12
+        err = small_vector_error(to_numpy64(grads[key]), ref[key])
+        print(f"cfg5 flags={flags} {key}: max {err.max():.3e}")
+        assert err.max() <= BF16_MAX, (key, err.max())
+    db = float(grads["dbeta"].cpu()[0])
+    rel = abs(db - ref["dbeta_closed"]) / abs(ref["dbeta_closed"])
+    ref_O, ref_aux = _ORACLE_CACHE[name]
+    dD = -(np.asarray(inp["dO"], dtype=np.float64) * ref_O).sum(-1) / ref_aux["D"]
+    scale = 2.0 * 1e-6 * np.sqrt((dD ** 2).sum())   # see _dbeta_error
+    err = abs(db - ref["dbeta_closed"]) / max(abs(ref["dbeta_closed"]), scale)
+    print(f"cfg5 flags={flags} dbeta {db:.6e} ref {ref['dbeta_closed']:.6e} plain rel {rel:.3e} normalised {err:.3e}")
+    assert err <= BF16_MAX, (db, ref["dbeta_closed"], err)
+
+
+@pytest.mark.parametrize("dtype,flags", [("f32", 0), ("bf16", 0), ("bf16", 1)])
+def test_backward_at_the_configurations_epsilon(dtype, flags):
+    """Backward with the denominator constant of the configurations (1e-6) instead of the larger one the
+    small cases use: dbeta, which only acts through that constant, is then ~1e-6 of the other gradients."""
+    import torch
+    cfg = dict(B=2, H=2, n=1536, d=64, L=6, m=256 if dtype == "bf16" else 64, dtype=dtype)
+    inp = wi.make_inputs(**cfg, seed=460, w_seed=461, gate_std=0.3, gate_seed=462, mean_shift=0.25, scale=0.7,
+                         backward=True)
+    ctx = _ctx(cfg, flags=flags)
+    dev = device_inputs(inp, dtype)
+    args = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    ctx.forward(*args)
+    grads = ctx.backward(*args, dev["dO"])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    _check_backward(cfg, inp, grads)
 
 
 # ---------------------------------------------------------------- seeded random shapes
@@ -432,6 +468,32 @@ def test_backward_random_shapes_tensor_core(case):
     torch.cuda.synchronize()
     assert ctx.query_status() == 0
     _check_backward(cfg, inp, grads)
+
+
+# ---------------------------------------------------------------- a bounded wait that runs out
+def test_bounded_wait_runs_out_and_is_reported_once():
+    """The error path of the tensor-core kernels' waits, on a one-CTA self-test kernel: a wait limited to a
+    millisecond on a barrier that is one arrival short gives up, the status word and the abort flag are set,
+    the second role leaves through the abort flag, the kernel returns; the host sees WERSA_ERR_TIMEOUT once,
+    then WERSA_OK, and the context still computes correctly afterwards."""
+    import time
+    import torch
+    cfg = dict(B=1, H=1, n=256, d=64, L=3, m=128, dtype="bf16")
+    inp = wi.make_inputs(**cfg, seed=3, w_seed=4)
+    dev = device_inputs(inp, "bf16")
+    ctx = _ctx(cfg)
+    args = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    want = ctx.forward(*args).clone()
+    assert ctx.query_status() == 0
+    t0 = time.perf_counter()
+    observed = ctx.selftest_wait_timeout(limit_us=1000)
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 1.0          # the kernel returned by itself, well within a second
+    assert observed.cpu().tolist() == [1, 0, 0]
+    assert ctx.query_status() == 5                  # WERSA_ERR_TIMEOUT, reported once
+    assert ctx.query_status() == 0
+    assert torch.equal(ctx.forward(*args), want)
+    assert ctx.query_status() == 0
 
 
 # ---------------------------------------------------------------- error paths that need a device

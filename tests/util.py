@@ -5,23 +5,7 @@ import numpy as np
 import wersa_inputs as wi
 
 
-def to_device(x, dtype, device="cuda"):
-    """float32 numpy array (bf16-representable when dtype is bf16) -> torch CUDA tensor."""
-    import torch
-    if dtype == "bf16":
-        bits = wi.to_bf16_bits(x).view(np.int16)
-        return torch.from_numpy(bits.copy()).to(device).view(torch.bfloat16)
-    return torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(device)
-
-
-def device_inputs(inp, dtype, device="cuda"):
-    out = {}
-    for key in ("Q", "K", "V", "W", "dO"):
-        if key in inp:
-            out[key] = to_device(inp[key], dtype, device)
-    for key in ("beta", "gate_w", "gate_b", "omega"):
-        out[key] = None if inp.get(key) is None else to_device(inp[key], "f32", device)
-    return out
+from wersa_inputs import device_inputs, to_device  # noqa: E402,F401  (re-exported for the tests)
 
 
 def to_numpy64(t):

@@ -85,3 +85,24 @@ def make_config(name, **overrides):
     cfg = dict(CONFIGS[name])
     cfg.update(overrides)
     return cfg, make_inputs(**cfg)
+
+
+def to_device(x, dtype, device="cuda"):
+    """float32 numpy array (bf16-representable when dtype is bf16) -> torch CUDA tensor of that storage type.
+    Pure data movement: the bf16 tensor is built from the 16-bit image of the values."""
+    import torch
+    if dtype == "bf16":
+        bits = to_bf16_bits(x).view(np.int16)
+        return torch.from_numpy(bits.copy()).to(device).view(torch.bfloat16)
+    return torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(device)
+
+
+def device_inputs(inp, dtype, device="cuda"):
+    """Device copies of one problem instance: Q, K, V, W, dO in the storage type, parameters as float32."""
+    out = {}
+    for key in ("Q", "K", "V", "W", "dO"):
+        if key in inp:
+            out[key] = to_device(inp[key], dtype, device)
+    for key in ("beta", "gate_w", "gate_b", "omega"):
+        out[key] = None if inp.get(key) is None else to_device(inp[key], "f32", device)
+    return out
