@@ -48,6 +48,23 @@ constexpr uint32_t kAccCol = 384;                 // S' halves (key side) / [N' 
 constexpr uint32_t kIdesc1 = make_idesc_bf16(128, 128, false, false);  // both operands K-major
 constexpr uint32_t kIdesc2 = make_idesc_bf16(128, 64, false, true);    // key side: B = V, N-major
 constexpr uint32_t kIdesc2Q = make_idesc_bf16(128, 80, false, false);  // query side: B = [S' | z' | 0]^T, K-major
+// Query side: one MMA1 covers a 128-token tile and all m = 128 NH features (N = m), into one of two
+// 256-column TMEM buffers.  The ReLU pass packs the bf16 features of 32-column chunks [0, CH) to the front
+// of the buffer and those of chunks [CH, 4 NH) to the front of their own span, which leaves 80 free
+// columns in between (m = 256) for the [N' | D'] accumulator of the same tile.
+constexpr uint32_t kQBufCols = 256;
+template <int NH> struct QTmem {
+  static constexpr int kChunks = 4 * NH;                 // 32-column fp32 chunks of D1
+  static constexpr int kHeavy = NH == 2 ? 5 : 2;         // chunks packed by the first warp of a lane quarter
+  static constexpr uint32_t kLightCol = 32 * kHeavy;     // where the second warp's span starts (input and output)
+  static constexpr uint32_t kAcc = NH == 2 ? 80 : 128;   // first column of [N' | D'] inside the buffer
+  // first TMEM column (inside the buffer) of the 8 columns that hold features 16 k .. 16 k + 15 as bf16 pairs
+  __host__ __device__ static constexpr uint32_t phi_col(int k) {
+    return (k >> 1) < kHeavy ? 8u * k : kLightCol + 8u * (k - 2 * kHeavy);
+  }
+};
+static_assert(QTmem<2>::phi_col(9) + 8 <= QTmem<2>::kAcc && QTmem<2>::kAcc + 80 <= QTmem<2>::kLightCol,
+              "accumulator must sit between the two packed spans");
 constexpr uint32_t kSztBlockBytes = 80 * 128;      // one 64-feature K block of that operand: 80 rows of 128 bytes
 
 constexpr int kWarpTma = 0, kWarpMma = 1, kWarpMma2 = 2;   // key side: warps 2 and 3 issue MMA2 (one per half)
@@ -81,7 +98,7 @@ struct alignas(8) KsideBars {
 };
 struct alignas(8) QsideBars {
   uint64_t x_full[kNXQ], x_empty[kNXQ], xf_ready[kNF];
-  uint64_t d1_full[6], phi_ready[kND1], d1_free[kND1], d2_full, d2_free, simg_ready, w_full;
+  uint64_t d1_full[2], phi_ready[2], d2_full[2], buf_free[2], simg_ready, w_full;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -743,8 +760,8 @@ __device__ __forceinline__ void load_szt_image(uint8_t* dst, const __nv_bfloat16
   }
 }
 
-// ReLU pass over one 128-column D1 accumulator in 16-column steps (a smaller register footprint than
-// relu_unit): fp32 TMEM -> bf16 pairs back into columns [0, 64) of the same accumulator.
+// ReLU pass in 16-column steps (a smaller register footprint than relu_unit): fp32 TMEM columns -> bf16
+// pairs in half as many columns.
 __device__ __forceinline__ void reg_fence16(uint32_t (&r)[16]) {
   asm volatile(""
                : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
@@ -757,21 +774,25 @@ __device__ __forceinline__ void relu_pack16(const uint32_t (&r)[16], uint32_t (&
 #pragma unroll
   for (int j = 0; j < 8; ++j) p[j] = relu_pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
 }
-__device__ __forceinline__ void relu_unit_plain(uint32_t taddr) {
+// STEPS steps of 16 fp32 columns starting at `in` -> 8 columns of bf16 pairs each starting at `out`
+// (out <= in: a step's store lands at or below columns that were read before it was issued).
+template <int STEPS>
+__device__ __forceinline__ void relu_span(uint32_t in, uint32_t out) {
+  static_assert(STEPS % 2 == 0, "two steps per iteration");
   uint32_t a[16], b[16], p[8];
-  tmem_ld16(taddr, a);
+  tmem_ld16(in, a);
 #pragma unroll
-  for (int c = 0; c < 8; c += 2) {
+  for (int c = 0; c < STEPS; c += 2) {
     tmem_ld_wait();
     reg_fence16(a);
-    tmem_ld16(taddr + 16 * (c + 1), b);
+    tmem_ld16(in + 16 * (c + 1), b);
     relu_pack16(a, p);
-    tmem_st8(taddr + 8 * c, p);
+    tmem_st8(out + 8 * c, p);
     tmem_ld_wait();
     reg_fence16(b);
-    if (c + 2 < 8) tmem_ld16(taddr + 16 * (c + 2), a);
+    if (c + 2 < STEPS) tmem_ld16(in + 16 * (c + 2), a);
     relu_pack16(b, p);
-    tmem_st8(taddr + 8 * (c + 1), p);
+    tmem_st8(out + 8 * (c + 1), p);
   }
   tmem_st_wait();
 }
@@ -790,10 +811,11 @@ __device__ __forceinline__ void qside_build_simg(uint8_t* simg, const __nv_bfloa
   warp_arrive(ready);
 }
 
-// grid (chunks, slabs), block 768.  TMEM: D1[3] at columns 0 / 128 / 256, [N' | D'] of the current tile
-// at 384 .. 463.  Warps 12-15 are the epilogue: they drain the accumulator of a tile as soon as its
-// last MMA2 has completed (which frees it for the next tile), scale by 1 / (D' + eps'), round to bf16
-// into one of two staging tiles and store it with TMA.
+// grid (chunks, slabs), block 768.  TMEM: two buffers of 256 columns; tile t uses buffer t & 1 for its D1
+// (128 tokens x m features, fp32), then for the packed bf16 features and the [N' | D'] accumulator (see
+// QTmem).  Per tile: MMA1 (warp 1) -> ReLU pass (warps 4-11, two warps per lane quarter that split the
+// feature columns) -> MMA2 (warp 3) -> epilogue (warps 12-15: drain the accumulator, which frees the buffer
+// for tile t + 2, scale by 1 / (D' + eps'), round to bf16 into one of two staging tiles, TMA store).
 template <int NH>
 __global__ void __launch_bounds__(kThreadsQ, 1)
 k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
@@ -803,14 +825,15 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   using SL = QsideSmem<NH>;
+  using TM = QTmem<NH>;
   QsideBars* bars = reinterpret_cast<QsideBars*>(smem + SL::bars);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunk = blockIdx.x, slab = blockIdx.y;
   const int blk0 = chunk * chunk_blocks;
   const int nblk = min(chunk_blocks, (n + kBlk - 1) / kBlk - blk0);
   const int ntiles = nblk * 2;
-  const int units = ntiles * NH;
   constexpr int m = NH * 128;
+  constexpr uint32_t kIdesc1Q = make_idesc_bf16(128, m, false, false);   // Q_F tile x all features
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kNXQ; ++s) {
@@ -818,13 +841,12 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       mbar_init(&bars->x_empty[s], 1);
     }
     for (int s = 0; s < kNF; ++s) mbar_init(&bars->xf_ready[s], 8);
-    for (int b = 0; b < 6; ++b) mbar_init(&bars->d1_full[b], 1);
-    for (int b = 0; b < kND1; ++b) {
-      mbar_init(&bars->phi_ready[b], 4);
-      mbar_init(&bars->d1_free[b], 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&bars->d1_full[b], 1);
+      mbar_init(&bars->phi_ready[b], 8);
+      mbar_init(&bars->d2_full[b], 1);
+      mbar_init(&bars->buf_free[b], 4);
     }
-    mbar_init(&bars->d2_full, 1);
-    mbar_init(&bars->d2_free, 4);
     mbar_init(&bars->simg_ready, kAuxWarp0Q - kReluWarp0);
     mbar_init(&bars->w_full, 1);
     bars->abort_flag = 0;
@@ -861,72 +883,56 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
         mbar_wait_drain(&bars->w_full, 0);
       }
     } else if (warp == kWarpMma && lane == 0) {
-      // MMA1 of every unit (see the key side).
+      // MMA1 of every tile: D1[128 tokens x m] = Q_F tile (K-major) * W (as W^T rows, K-major), one
+      // instruction per 16 columns of the head dimension.  The W^T image is m contiguous 128-byte rows.
       constexpr uint32_t kTileStep = kTileBytes >> 4;
       const uint32_t hi = smem_desc_hi(1024);
       const uint32_t wt_lo = smem_desc_lo(smem_u32(smem + SL::wt), 16);
       const uint32_t x_lo = smem_desc_lo(smem_u32(smem + SL::x), 16);
       uint32_t xs = 0, fs = 0, fpar = 0;
-      uint32_t c3 = 0, c6 = 0, round = 0;
+      int t = 0;
       bool ok = mbar_wait(&bars->w_full, 0, abort_flag, status, kErrMma);
       for (int b = 0; b < nblk && ok; ++b) {
         ok = mbar_wait(&bars->xf_ready[fs], fpar, abort_flag, status, kErrMma);
         if (!ok) break;
         tc_fence_after_sync();
 #pragma unroll
-        for (int j = 0; j < 2 * NH; ++j) {
-          const int h = j % NH;
-          if (round > 0) {
-            ok = mbar_wait(&bars->d1_free[c3], (round - 1) & 1, abort_flag, status, kErrMma);
+        for (int j = 0; j < 2; ++j, ++t) {
+          const int buf = t & 1;
+          if (t >= 2) {   // the epilogue must have drained the accumulator of tile t - 2 (same buffer)
+            ok = mbar_wait(&bars->buf_free[buf], ((t >> 1) - 1) & 1, abort_flag, status, kErrMma);
             if (!ok) break;
             tc_fence_after_sync();
           }
-          const uint32_t a_lo = x_lo + xs * kTileStep, b_lo = wt_lo + h * kTileStep;
-          const uint32_t d1 = tmem + c3 * 128;
+          const uint32_t a_lo = x_lo + xs * kTileStep;
+          const uint32_t d1 = tmem + buf * kQBufCols;
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            mma_ss(d1, smem_desc_join(a_lo + 2 * k, hi), smem_desc_join(b_lo + 2 * k, hi), kIdesc1, k > 0);
-          mma_commit(&bars->d1_full[c6]);
-          if (h == NH - 1) {   // last MMA1 that reads this tile
-            mma_commit(&bars->x_empty[xs]);
-            xs = xs == kNXQ - 1 ? 0 : xs + 1;
-          }
-          c3 = c3 == kND1 - 1 ? 0 : c3 + 1;
-          round += (c3 == 0);
-          c6 = c6 == 5 ? 0 : c6 + 1;
+            mma_ss(d1, smem_desc_join(a_lo + 2 * k, hi), smem_desc_join(wt_lo + 2 * k, hi), kIdesc1Q, k > 0);
+          mma_commit(&bars->d1_full[buf]);
+          mma_commit(&bars->x_empty[xs]);
+          xs = xs == kNXQ - 1 ? 0 : xs + 1;
         }
         fs = (fs + 1) & (kNF - 1);
         fpar ^= (fs == 0);
       }
     } else if (warp == kWarpMma2Q && lane == 0) {
-      // MMA2 of every unit: [N' | D'] (+)= Phi (the unit's D1 buffer, bf16 pairs) * [S' | z' | 0] half h.
+      // MMA2 of every tile: [N' | D'] = Phi (bf16 pairs in the tile's buffer) * [S' | z' | 0].
       const uint32_t hi = smem_desc_hi(1024);
       const uint32_t s_lo = smem_desc_lo(smem_u32(smem + SL::simg), 16);
-      const uint32_t d2 = tmem + kAccCol;
-      uint32_t p3 = 0, ppar = 0;
       bool ok = mbar_wait(&bars->simg_ready, 0, abort_flag, status, kErrMma);   // the [S' | z' | 0]^T image is in place
       for (int t = 0; t < ntiles && ok; ++t) {
-        if (t >= 1) {   // the accumulator of tile t - 1 must have been drained
-          ok = mbar_wait(&bars->d2_free, (t - 1) & 1, abort_flag, status, kErrMma);
-          if (!ok) break;
-          tc_fence_after_sync();
-        }
+        const int buf = t & 1;
+        ok = mbar_wait(&bars->phi_ready[buf], (t >> 1) & 1, abort_flag, status, kErrMma);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t base = tmem + buf * kQBufCols;
 #pragma unroll
-        for (int h = 0; h < NH; ++h) {
-          ok = mbar_wait(&bars->phi_ready[p3], ppar, abort_flag, status, kErrMma);
-          if (!ok) break;
-          tc_fence_after_sync();
-          const uint32_t a_tm = tmem + p3 * 128;
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {   // K block 2 h + k / 4, 32 bytes per step of 16 features inside it
-            const uint32_t b_lo = s_lo + (2 * h + (k >> 2)) * (kSztBlockBytes >> 4) + 2 * (k & 3);
-            mma_ts(d2, a_tm + k * 8, smem_desc_join(b_lo, hi), kIdesc2Q, (h > 0 || k > 0) ? 1u : 0u);
-          }
-          mma_commit(&bars->d1_free[p3]);
-          p3 = p3 == kND1 - 1 ? 0 : p3 + 1;
-          ppar ^= (p3 == 0);
+        for (int k = 0; k < 8 * NH; ++k) {   // K block k / 4 of the image, 32 bytes per step of 16 features inside it
+          const uint32_t b_lo = s_lo + (k >> 2) * (kSztBlockBytes >> 4) + 2 * (k & 3);
+          mma_ts(base + TM::kAcc, base + TM::phi_col(k), smem_desc_join(b_lo, hi), kIdesc2Q, k > 0 ? 1u : 0u);
         }
-        if (ok) mma_commit(&bars->d2_full);
+        mma_commit(&bars->d2_full[buf]);
       }
     }
   } else if (warp < kEpiWarp0Q) {
@@ -935,13 +941,18 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     const int g = (warp - kReluWarp0) >> 2;
     const uint32_t lane_base = 32u * (warp & 3);
     bool ok = true;
-    for (int u = g; u < units; u += 2) {
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d1_full[u % 6], (u / 6) & 1, abort_flag, status, kErrRelu));
+    for (int t = 0; t < ntiles; ++t) {
+      const int buf = t & 1;
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d1_full[buf], (t >> 1) & 1, abort_flag, status, kErrRelu));
       if (ok) {
         tc_fence_after_sync();
-        relu_unit_plain(tmem + (lane_base << 16) + (u % kND1) * 128);
+        const uint32_t base = tmem + (lane_base << 16) + buf * kQBufCols;
+        // the two warps of a lane quarter split the columns (5 : 3 chunks with m = 256) and swap parts from
+        // tile to tile
+        if (((g ^ t) & 1) == 0) relu_span<2 * TM::kHeavy>(base, base);
+        else relu_span<2 * (TM::kChunks - TM::kHeavy)>(base + TM::kLightCol, base + TM::kLightCol);
         tc_fence_before_sync();
-        warp_arrive(&bars->phi_ready[u % kND1]);
+        warp_arrive(&bars->phi_ready[buf]);
       }
     }
   } else if (warp < kAuxWarp0Q) {
@@ -951,10 +962,11 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     const uint32_t lane_base = 32u * (warp & 3);
     const float bw = fmaxf(beta[0], bw_floor);
     const float epsp = eps * (float)m * bw * bw;
-    const uint32_t base = tmem + (lane_base << 16) + kAccCol;
     bool ok = true;
     for (int t = 0; t < ntiles; ++t) {
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d2_full, t & 1, abort_flag, status, kErrEpilogue));
+      const int buf = t & 1;
+      const uint32_t base = tmem + (lane_base << 16) + buf * kQBufCols + TM::kAcc;
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d2_full[buf], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
       uint32_t r0[32], r1[32], dd = 0;
       if (ok) {
         tc_fence_after_sync();
@@ -965,7 +977,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
         reg_fence32(r0);
         reg_fence32(r1);
         tc_fence_before_sync();
-        warp_arrive(&bars->d2_free);
+        warp_arrive(&bars->buf_free[buf]);
       }
       // the staging tile was last used by tile t - 2: its TMA store must have finished reading
       if (et == 0) bulk_wait_group_read1();

@@ -281,13 +281,56 @@ def _dbeta_error(cfg, inp, got, ref_closed):
     return abs(got - ref_closed) / max(abs(ref_closed), scale, 1e-300)
 
 
+AMBIGUOUS_MARGIN = 1e-6
+
+
+def _ambiguous_rows(cfg, inp, key):
+    """Rows of Q (key="Q") or K whose ReLU decision is not unique in working precision: the gradient of
+    ReLU, 1[a > 0], is a 0/1 decision on a = x_F . w, and the kernels take it in fp32 while the oracle takes it
+    in fp64.  Where |a| is below fp32 resolution (|a| <= 1e-6 |x_F| |w| for some feature; a dot product of 64
+    terms carries about 64 * 2^-24 = 4e-6 of relative rounding) either answer is a correct one and the row's
+    gradient differs by that feature's whole rank-one term.  Returns a boolean (B, H, n) mask of such rows,
+    from the oracle's own filter and a float64 matmul."""
+    qbar, f = orc.gate(inp["Q"], inp["gate_w"], inp["gate_b"], inp["omega"], cfg["L"],
+                       gate_per_head=cfg.get("gate_per_head", 1))
+    W = np.asarray(inp["W"], dtype=np.float64)
+    wn = np.linalg.norm(W, axis=0)
+    X = inp[key]
+    out = np.zeros(X.shape[:3], dtype=bool)
+    for b in range(X.shape[0]):
+        for h in range(X.shape[1]):
+            XF = orc.haar_filter(X[b, h].astype(np.float64), f[b, h])
+            A = np.abs(XF @ W)
+            scale = np.linalg.norm(XF, axis=1)[:, None] * wn[None, :]
+            out[b, h] = (A <= AMBIGUOUS_MARGIN * scale).any(axis=1)
+    return out
+
+
+def _check_grad(got, ref, dtype, what, ambiguous=None):
+    """Element-by-element check of dQ / dK / dV.  Rows whose ReLU decision is ambiguous (see _ambiguous_rows)
+    are compared at a validity bound instead of the tolerance: one flipped feature moves the row by a
+    rank-one term, well below the row's own size."""
+    err = normalised_error(got, ref)
+    if ambiguous is not None and ambiguous.any():
+        assert ambiguous.mean() <= 0.02, (what, "too many ambiguous rows", ambiguous.mean())
+        assert err[ambiguous].max() <= 1.0, (what, "ambiguous rows", err[ambiguous].max())
+        err = err[~ambiguous]
+    if dtype == "f32":
+        assert err.max() <= F32_MAX, (what, err.max())
+    else:
+        assert err.max() <= BF16_MAX, (what, "max", err.max())
+        assert err.mean() <= BF16_MEAN, (what, "mean", err.mean())
+    return err
+
+
 def _check_backward(cfg, inp, grads, sub_slabs=None):
     ref = orc.backward(inp["Q"], inp["K"], inp["V"], inp["W"], float(inp["beta"][0]), inp["gate_w"],
                        inp["gate_b"], inp["omega"], inp["dO"], cfg["L"], eps=cfg.get("eps", 1e-6),
                        gate_per_head=cfg.get("gate_per_head", 1))
     dtype = cfg["dtype"]
-    for key in ("dQ", "dK", "dV"):
-        _check(to_numpy64(grads[key]), ref[key], dtype, key)
+    _check_grad(to_numpy64(grads["dQ"]), ref["dQ"], dtype, "dQ", _ambiguous_rows(cfg, inp, "Q"))
+    _check_grad(to_numpy64(grads["dK"]), ref["dK"], dtype, "dK", _ambiguous_rows(cfg, inp, "K"))
+    _check_grad(to_numpy64(grads["dV"]), ref["dV"], dtype, "dV")
     tol = 1e-4 if dtype == "f32" else 2e-2
     for key in ("dgate_w", "dgate_b", "domega"):
         err = small_vector_error(to_numpy64(grads[key]), ref[key])
@@ -381,8 +424,10 @@ def test_config5_training_step_bf16(flags):
             inp["omega"], inp["dO"], cfg["L"])
     ref = _ORACLE_CACHE[name + "/bwd"]
     for key in ("dQ", "dK", "dV"):
-        err = _check(to_numpy64(grads[key]), ref[key], "bf16", key)
-        print(f"cfg5 flags={flags} {key}: max {err.max():.3e} mean {err.mean():.3e}")
+        amb = _ambiguous_rows(cfg, inp, key[1]) if key != "dV" else None
+        err = _check_grad(to_numpy64(grads[key]), ref[key], "bf16", key, amb)
+        print(f"cfg5 flags={flags} {key}: max {err.max():.3e} mean {err.mean():.3e} "
+              f"(rows with an ambiguous ReLU decision: {0 if amb is None else int(amb.sum())} of {amb.size if amb is not None else 0})")
     for key in ("dgate_w", "dgate_b", "domega"):
         err = small_vector_error(to_numpy64(grads[key]), ref[key])
         print(f"cfg5 flags={flags} {key}: max {err.max():.3e}")
