@@ -108,7 +108,7 @@ template <int NH> struct KsideSmem {
   static constexpr uint32_t x = wt + NH * kTileBytes;
   static constexpr uint32_t v = x + kNXK * kTileBytes;
   static constexpr uint32_t xch = v + kNV * kTileBytes;           // 2 x 8 x 64 floats
-  static constexpr uint32_t hcoef = xch + 4096;                  // kHaarCoefPairs pairs
+  static constexpr uint32_t hcoef = xch + 4096;                  // kHaarCoefs floats
   static constexpr uint32_t zx = hcoef + 1024;                   // 128 floats
   static constexpr uint32_t bars = zx + 512;
   static constexpr uint32_t total = bars + 512 + 1024;           // + alignment slack
@@ -119,7 +119,7 @@ template <int NH> struct QsideSmem {
   static constexpr uint32_t x = simg + 2 * NH * kSztBlockBytes;
   static constexpr uint32_t ost = x + kNXQ * kTileBytes;           // 2 output staging tiles
   static constexpr uint32_t xch = ost + 2 * kTileBytes;          // 2 x 8 x 64 floats
-  static constexpr uint32_t hcoef = xch + 4096;                  // kHaarCoefPairs pairs
+  static constexpr uint32_t hcoef = xch + 4096;                  // kHaarCoefs floats
   static constexpr uint32_t bars = hcoef + 1024;
   static constexpr uint32_t total = bars + 512 + 1024;
 };
@@ -159,19 +159,9 @@ __device__ __forceinline__ f32x2 pk2(float lo, float hi) {
 __device__ __forceinline__ void upk2(f32x2 v, float& lo, float& hi) {
   asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
 }
-__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
-  f32x2 r;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
 __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
   f32x2 r;
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
-  f32x2 r;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
   return r;
 }
 __device__ __forceinline__ uint32_t pack2_bf16(f32x2 v) {
@@ -237,33 +227,57 @@ __device__ __forceinline__ float relu_unit(uint32_t taddr) {
 // T_f x = f_0 x + sum_{i=1..L} (f_i - f_{i-1}) * blockmean_{2^i}(x): the detail projector of level l
 // is blockmean_{2^(l-1)} - blockmean_{2^l} and the approximation projector of level L is
 // blockmean_{2^L}, so only aligned block sums of 2, 4, ..., 2^L rows are needed.
-// Filter coefficients as (v, v) pairs in shared memory, written once per CTA by the aux warps:
-//   hcoef[0] = f_0, hcoef[i] = k_i = (f_i - f_{i-1}) / 2^i for i = 1..5 (0 beyond L),
-//   hcoef[8 + 8 hw + w] = weight of warp w's 32-row sum in warp hw's levels 6-8 term
-//                       = k_8 + [same 128-row group] k_7 + [same 64-row group] k_6.
-constexpr int kHaarCoefPairs = 8 + 64;
-static_assert(kHaarCoefPairs * 8 <= 1024, "coefficient table must fit its shared-memory slot");
+//
+// The block is filtered on packed bf16 pairs wherever that costs no accuracy that matters: the sums of
+// row pairs (level 1) are packed bf16 adds, everything coarser is fp32 on those 32 sums per thread, and
+// the last step, f_0 x + c, is one packed bf16 fma per two elements (one rounding, like a conversion of
+// the fp32 result) with c rounded to bf16 first.  A packed fma needs f_0 as a bf16 value; instead of
+// rounding the coefficient (a systematic error), the stage computes r T_f x with r = bf16(f_0) / f_0: the
+// coefficient of x is then exact and every other coefficient is scaled by r in fp32.  ReLU is positively
+// homogeneous and r > 0, so the features come out scaled by r as well and the kernels take the factor
+// out again where they leave results (S', z': divided by r; output: eps' scaled by r).
+//
+// Coefficient table in shared memory, written once per CTA by the Haar warps:
+//   hc[0] = bf16(f_0) in both halves (bit pattern), hc[i] = r k_i = r (f_i - f_{i-1}) / 2^i for i = 1..5
+//   (0 beyond L), hc[8 + 8 hw + w] = weight of warp w's 32-row sum in warp hw's levels 6-8 term
+//                                  = r (k_8 + [same 128-row group] k_7 + [same 64-row group] k_6).
+constexpr int kHaarCoefs = 8 + 64;
+static_assert(kHaarCoefs * 4 <= 1024, "coefficient table must fit its shared-memory slot");
 
-__device__ __forceinline__ void haar_coef_init(f32x2* hcoef, const float* __restrict__ f, int L, int ht) {
+// r = bf16(f_0) / f_0 (1 when f_0 = 0): the factor by which the filtered block, and with it the features, come
+// out scaled.  Every role that needs it computes it from f_0 with these same operations.
+__device__ __forceinline__ float haar_scale(float f0) {
+  const float f0b = __uint_as_float(pack_bf16x2(f0, f0) << 16);
+  return f0 != 0.f ? f0b / f0 : 1.f;
+}
+
+__device__ __forceinline__ void haar_coef_init(float* hc, const float* __restrict__ f, int L, int ht) {
+  const float r = haar_scale(f[0]);
   float k[kMaxLevels + 1];
   k[0] = f[0];
-  float scale = 0.5f;
+  float scale = 0.5f * r;
 #pragma unroll
   for (int i = 1; i <= kMaxLevels; ++i) {
     k[i] = (i <= L) ? (f[i] - f[i - 1]) * scale : 0.f;
     scale *= 0.5f;
   }
-  if (ht < 6) {
-    float v = k[0];
+  if (ht == 0) hc[0] = __uint_as_float(pack_bf16x2(k[0], k[0]));
+  if (ht >= 1 && ht < 6) {
+    float v = k[1];
 #pragma unroll
-    for (int i = 1; i < 6; ++i) v = (ht == i) ? k[i] : v;
-    hcoef[ht] = pk2(v, v);
+    for (int i = 2; i < 6; ++i) v = (ht == i) ? k[i] : v;
+    hc[ht] = v;
   }
   if (ht < 64) {
     const int hw = ht >> 3, w = ht & 7;
-    const float v = k[8] + ((w >> 2) == (hw >> 2) ? k[7] : 0.f) + ((w >> 1) == (hw >> 1) ? k[6] : 0.f);
-    hcoef[8 + ht] = pk2(v, v);
+    hc[8 + ht] = k[8] + ((w >> 2) == (hw >> 2) ? k[7] : 0.f) + ((w >> 1) == (hw >> 1) ? k[6] : 0.f);
   }
+}
+
+__device__ __forceinline__ uint32_t fma_bf16x2(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t r;
+  asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  return r;
 }
 
 // 256 threads (ht = 0..255) filter the block (two 128-row tiles) in place.  Thread (c = ht & 7, rg = ht >> 3) owns rows
@@ -274,119 +288,31 @@ __device__ __forceinline__ void haar_coef_init(f32x2* hcoef, const float* __rest
 // barrier balanced; with ok = false no memory is touched.  Rows >= valid_rows lie past the end of the
 // sequence: they arrive as zeros (the zero padding of Algorithm 2) and leave as zeros (the trim
 // before the feature map).
-__device__ __forceinline__ void haar_block_inplace(uint8_t* tile0, uint8_t* tile1, const f32x2* hcoef, bool cross,
+__device__ __forceinline__ void haar_block_inplace(uint8_t* tile0, uint8_t* tile1, const float* hc, bool cross,
                                                    float* xch, int ht, int valid_rows, bool ok) {
   const int c = ht & 7, rg = ht >> 3, lane = ht & 31, hw = ht >> 5;
   uint8_t* base = (rg < 16 ? tile0 : tile1) + (rg & 15) * 1024;   // rows 0-127 / 128-255 of the block
-  f32x2 x[8][4];   // 8 rows x 4 column pairs
-  f32x2 hi[4], s5[4];
-  if (ok) {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {   // row 8 rg + j has swizzle phase j
-      const uint4 raw = *reinterpret_cast<const uint4*>(base + j * 128 + ((c ^ j) << 4));
-      const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) x[j][i] = pk2(__uint_as_float(u[i] << 16), __uint_as_float(u[i] & 0xFFFF0000u));
-    }
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const f32x2 s3 = add2(add2(add2(x[0][q], x[1][q]), add2(x[2][q], x[3][q])),
-                            add2(add2(x[4][q], x[5][q]), add2(x[6][q], x[7][q])));
-      float lo, hi_;
-      upk2(s3, lo, hi_);
-      const f32x2 s4 = add2(s3, pk2(__shfl_xor_sync(0xffffffffu, lo, 8), __shfl_xor_sync(0xffffffffu, hi_, 8)));
-      upk2(s4, lo, hi_);
-      s5[q] = add2(s4, pk2(__shfl_xor_sync(0xffffffffu, lo, 16), __shfl_xor_sync(0xffffffffu, hi_, 16)));
-      hi[q] = fma2(hcoef[3], s3, fma2(hcoef[4], s4, mul2(hcoef[5], s5[q])));
-    }
-  }
-  if (cross) {   // uniform over the kernel: L > 5
-    if (ok && (lane >> 3) == 0) {
-      ulonglong2* dst = reinterpret_cast<ulonglong2*>(xch + hw * kD + c * 8);
-      dst[0] = make_ulonglong2(s5[0], s5[1]);
-      dst[1] = make_ulonglong2(s5[2], s5[3]);
-    }
-    named_bar_sync(kBarHaar, 256);
-    if (ok) {
-      // lane (c, q = lane >> 3) combines the eight warps' sums of column pair q of chunk c (two
-      // independent chains of four), then the four lanes that share a chunk swap their pairs
-      const int qq = lane >> 3;
-      const f32x2* src = reinterpret_cast<const f32x2*>(xch + c * 8 + 2 * qq);
-      const f32x2* cf = hcoef + 8 + 8 * hw;
-      f32x2 acc0 = mul2(cf[0], src[0]), acc1 = mul2(cf[1], src[kD / 2]);
-#pragma unroll
-      for (int w = 2; w < 8; w += 2) {
-        acc0 = fma2(cf[w], src[w * (kD / 2)], acc0);
-        acc1 = fma2(cf[w + 1], src[(w + 1) * (kD / 2)], acc1);
-      }
-      float lo, hi_;
-      upk2(add2(acc0, acc1), lo, hi_);
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int sl = (q << 3) | c;
-        hi[q] = add2(hi[q], pk2(__shfl_sync(0xffffffffu, lo, sl), __shfl_sync(0xffffffffu, hi_, sl)));
-      }
-    }
-  }
-  if (ok) {
-    const f32x2 f0 = hcoef[0], k1 = hcoef[1], k2 = hcoef[2];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const f32x2 a0 = add2(x[0][q], x[1][q]), a1 = add2(x[2][q], x[3][q]);
-      const f32x2 a2 = add2(x[4][q], x[5][q]), a3 = add2(x[6][q], x[7][q]);
-      const f32x2 c20 = fma2(k2, add2(a0, a1), hi[q]), c21 = fma2(k2, add2(a2, a3), hi[q]);
-      const f32x2 c10 = fma2(k1, a0, c20), c11 = fma2(k1, a1, c20);
-      const f32x2 c12 = fma2(k1, a2, c21), c13 = fma2(k1, a3, c21);
-      x[0][q] = fma2(f0, x[0][q], c10);
-      x[1][q] = fma2(f0, x[1][q], c10);
-      x[2][q] = fma2(f0, x[2][q], c11);
-      x[3][q] = fma2(f0, x[3][q], c11);
-      x[4][q] = fma2(f0, x[4][q], c12);
-      x[5][q] = fma2(f0, x[5][q], c12);
-      x[6][q] = fma2(f0, x[6][q], c13);
-      x[7][q] = fma2(f0, x[7][q], c13);
-    }
-    if (rg * 8 + 8 <= valid_rows) {   // the usual case: every row of this thread lies inside the sequence
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        *reinterpret_cast<uint4*>(base + j * 128 + ((c ^ j) << 4)) =
-            make_uint4(pack2_bf16(x[j][0]), pack2_bf16(x[j][1]), pack2_bf16(x[j][2]), pack2_bf16(x[j][3]));
-    } else {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        uint4 out = make_uint4(pack2_bf16(x[j][0]), pack2_bf16(x[j][1]), pack2_bf16(x[j][2]), pack2_bf16(x[j][3]));
-        if (rg * 8 + j >= valid_rows) out = make_uint4(0u, 0u, 0u, 0u);
-        *reinterpret_cast<uint4*>(base + j * 128 + ((c ^ j) << 4)) = out;
-      }
-    }
-  }
-}
-
-// The same filter with plain fp32 registers instead of packed pairs (bit-identical: the packed operations
-// round each half like the scalar ones).  Which of the two compiles into the faster stage differs between
-// the two kernels: the key side uses this one, the query side the packed one.
-__device__ __forceinline__ void haar_block_inplace_scalar(uint8_t* tile0, uint8_t* tile1, const f32x2* hcoef, bool cross,
-                                                   float* xch, int ht, int valid_rows, bool ok) {
-  const int c = ht & 7, rg = ht >> 3, lane = ht & 31, hw = ht >> 5;
-  uint8_t* base = (rg < 16 ? tile0 : tile1) + (rg & 15) * 1024;   // rows 0-127 / 128-255 of the block
-  const float* hc = reinterpret_cast<const float*>(hcoef);        // entry i of the pair table = hc[2 i]
-  float x[8][8];   // 8 rows x 8 columns
+  uint32_t u[8][4];   // 8 rows x 4 column pairs, as loaded
+  float a[4][8];      // sums of row pairs, then the additive term c of each row pair
   float hi[8], s5[8];
   if (ok) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) {   // row 8 rg + j has swizzle phase j
       const uint4 raw = *reinterpret_cast<const uint4*>(base + j * 128 + ((c ^ j) << 4));
-      const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+      u[j][0] = raw.x; u[j][1] = raw.y; u[j][2] = raw.z; u[j][3] = raw.w;
+    }
+#pragma unroll
+    for (int p = 0; p < 4; ++p)
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        x[j][2 * i] = __uint_as_float(u[i] << 16);
-        x[j][2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
+        const uint32_t s = add_bf16x2(u[2 * p][i], u[2 * p + 1][i]);
+        a[p][2 * i] = __uint_as_float(s << 16);
+        a[p][2 * i + 1] = __uint_as_float(s & 0xFFFF0000u);
       }
-    }
-    const float k3 = hc[6], k4 = hc[8], k5 = hc[10];
+    const float k3 = hc[3], k4 = hc[4], k5 = hc[5];
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
-      const float s3 = ((x[0][q] + x[1][q]) + (x[2][q] + x[3][q])) + ((x[4][q] + x[5][q]) + (x[6][q] + x[7][q]));
+      const float s3 = (a[0][q] + a[1][q]) + (a[2][q] + a[3][q]);
       const float s4 = s3 + __shfl_xor_sync(0xffffffffu, s3, 8);
       s5[q] = s4 + __shfl_xor_sync(0xffffffffu, s4, 16);
       hi[q] = fmaf(k3, s3, fmaf(k4, s4, k5 * s5[q]));
@@ -404,15 +330,15 @@ __device__ __forceinline__ void haar_block_inplace_scalar(uint8_t* tile0, uint8_
       // independent chains of four), then the four lanes that share a chunk swap their pairs
       const int qq = lane >> 3;
       const float2* src = reinterpret_cast<const float2*>(xch + c * 8 + 2 * qq);
-      const float* cf = hc + 2 * (8 + 8 * hw);
+      const float* cf = hc + 8 + 8 * hw;
       float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
 #pragma unroll
       for (int w = 0; w < 8; w += 2) {
         const float2 v0 = src[w * (kD / 2)], v1 = src[(w + 1) * (kD / 2)];
-        a0 = fmaf(cf[2 * w], v0.x, a0);
-        a1 = fmaf(cf[2 * w], v0.y, a1);
-        b0 = fmaf(cf[2 * w + 2], v1.x, b0);
-        b1 = fmaf(cf[2 * w + 2], v1.y, b1);
+        a0 = fmaf(cf[w], v0.x, a0);
+        a1 = fmaf(cf[w], v0.y, a1);
+        b0 = fmaf(cf[w + 1], v1.x, b0);
+        b1 = fmaf(cf[w + 1], v1.y, b1);
       }
       const float lo = a0 + b0, hi_ = a1 + b1;
 #pragma unroll
@@ -424,34 +350,32 @@ __device__ __forceinline__ void haar_block_inplace_scalar(uint8_t* tile0, uint8_
     }
   }
   if (ok) {
-    const float f0 = hc[0], k1 = hc[2], k2 = hc[4];
+    const float k1 = hc[1], k2 = hc[2];
+    const uint32_t f0 = __float_as_uint(hc[0]);
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
-      const float a0 = x[0][q] + x[1][q], a1 = x[2][q] + x[3][q];
-      const float a2 = x[4][q] + x[5][q], a3 = x[6][q] + x[7][q];
-      const float c20 = fmaf(k2, a0 + a1, hi[q]), c21 = fmaf(k2, a2 + a3, hi[q]);
-      const float c10 = fmaf(k1, a0, c20), c11 = fmaf(k1, a1, c20);
-      const float c12 = fmaf(k1, a2, c21), c13 = fmaf(k1, a3, c21);
-      x[0][q] = fmaf(f0, x[0][q], c10);
-      x[1][q] = fmaf(f0, x[1][q], c10);
-      x[2][q] = fmaf(f0, x[2][q], c11);
-      x[3][q] = fmaf(f0, x[3][q], c11);
-      x[4][q] = fmaf(f0, x[4][q], c12);
-      x[5][q] = fmaf(f0, x[5][q], c12);
-      x[6][q] = fmaf(f0, x[6][q], c13);
-      x[7][q] = fmaf(f0, x[7][q], c13);
+      const float c20 = fmaf(k2, a[0][q] + a[1][q], hi[q]), c21 = fmaf(k2, a[2][q] + a[3][q], hi[q]);
+      a[0][q] = fmaf(k1, a[0][q], c20);
+      a[1][q] = fmaf(k1, a[1][q], c20);
+      a[2][q] = fmaf(k1, a[2][q], c21);
+      a[3][q] = fmaf(k1, a[3][q], c21);
     }
+#pragma unroll
+    for (int p = 0; p < 4; ++p)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t cp = pack_bf16x2(a[p][2 * i], a[p][2 * i + 1]);
+        u[2 * p][i] = fma_bf16x2(f0, u[2 * p][i], cp);
+        u[2 * p + 1][i] = fma_bf16x2(f0, u[2 * p + 1][i], cp);
+      }
     if (rg * 8 + 8 <= valid_rows) {   // the usual case: every row of this thread lies inside the sequence
 #pragma unroll
       for (int j = 0; j < 8; ++j)
-        *reinterpret_cast<uint4*>(base + j * 128 + ((c ^ j) << 4)) =
-            make_uint4(pack_bf16x2(x[j][0], x[j][1]), pack_bf16x2(x[j][2], x[j][3]), pack_bf16x2(x[j][4], x[j][5]),
-                       pack_bf16x2(x[j][6], x[j][7]));
+        *reinterpret_cast<uint4*>(base + j * 128 + ((c ^ j) << 4)) = make_uint4(u[j][0], u[j][1], u[j][2], u[j][3]);
     } else {
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        uint4 out = make_uint4(pack_bf16x2(x[j][0], x[j][1]), pack_bf16x2(x[j][2], x[j][3]),
-                               pack_bf16x2(x[j][4], x[j][5]), pack_bf16x2(x[j][6], x[j][7]));
+        uint4 out = make_uint4(u[j][0], u[j][1], u[j][2], u[j][3]);
         if (rg * 8 + j >= valid_rows) out = make_uint4(0u, 0u, 0u, 0u);
         *reinterpret_cast<uint4*>(base + j * 128 + ((c ^ j) << 4)) = out;
       }
@@ -461,20 +385,16 @@ __device__ __forceinline__ void haar_block_inplace_scalar(uint8_t* tile0, uint8_
 
 // One Haar step: wait for the two raw tiles of block b, filter them in place, hand the block to the
 // MMA issuer.  NX = number of tile slots in the ring.
-template <int NX, bool kScalar, typename Bars>
-__device__ __forceinline__ bool haar_step(uint8_t* xring, Bars* bars, float* xch, const f32x2* hcoef, bool cross,
+template <int NX, typename Bars>
+__device__ __forceinline__ bool haar_step(uint8_t* xring, Bars* bars, float* xch, const float* hcoef, bool cross,
                                           int b, int rows_left, int ht, bool ok, volatile int* abort_flag,
                                           int* status) {
   const int t0 = 2 * b, t1 = 2 * b + 1;
   const int s0 = t0 % NX, s1 = t1 % NX;
   if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[s0], (t0 / NX) & 1, abort_flag, status, kErrHaar));
   if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[s1], (t1 / NX) & 1, abort_flag, status, kErrHaar));
-  if (kScalar)
-    haar_block_inplace_scalar(xring + s0 * kTileBytes, xring + s1 * kTileBytes, hcoef, cross, xch + (b & 1) * 8 * kD, ht,
-                              rows_left - b * kBlk, ok);
-  else
-    haar_block_inplace(xring + s0 * kTileBytes, xring + s1 * kTileBytes, hcoef, cross, xch + (b & 1) * 8 * kD, ht,
-                       rows_left - b * kBlk, ok);
+  haar_block_inplace(xring + s0 * kTileBytes, xring + s1 * kTileBytes, hcoef, cross, xch + (b & 1) * 8 * kD, ht,
+                     rows_left - b * kBlk, ok);
   if (ok) {
     fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
     warp_arrive(&bars->xf_ready[b & (kNF - 1)]);
@@ -690,6 +610,8 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       // around in shared memory (the K ring is idle by now; rows padded to 33 floats) and writes whole
       // 128-byte row segments.
       const int feat0 = (NH == 2 ? g * 128 : 0) + (int)lane_base;   // first feature of this warp
+      // the filter stage left K_F, and with it the features, scaled by r (see haar_block_inplace)
+      const float inv_r = 1.f / haar_scale(f[(size_t)slab * (L + 1)]);
       float* stage = reinterpret_cast<float*>(smem + SL::x) + (warp - kReluWarp0) * (32 * 33);
       float* dst = spart + (pidx * m + feat0) * kD;
 #pragma unroll 1
@@ -699,7 +621,7 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
         tmem_ld_wait();
         reg_fence32(r);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = __uint_as_float(r[j]);
+        for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = __uint_as_float(r[j]) * inv_r;
         __syncwarp();
 #pragma unroll 8
         for (int rr = 0; rr < 32; ++rr) dst[(size_t)rr * kD + 32 * c + lane] = stage[rr * 33 + lane];
@@ -713,17 +635,17 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
         }
         __syncwarp();
       }
-      zpart[pidx * m + feat0 + lane] = zacc;
+      zpart[pidx * m + feat0 + lane] = zacc * inv_r;
     }
   } else {
     reg_inc<kRegsAux>();
     const int ht = threadIdx.x - 32 * kAuxWarp0;
-    f32x2* hcoef = reinterpret_cast<f32x2*>(smem + SL::hcoef);
+    float* hcoef = reinterpret_cast<float*>(smem + SL::hcoef);
     haar_coef_init(hcoef, f + (size_t)slab * (L + 1), L, ht);
     named_bar_sync(kBarCoef, 256);
     bool ok = true;
     for (int b = 0; b < nblk; ++b)
-      ok = haar_step<kNXK, true>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
+      ok = haar_step<kNXK>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
                      ht, ok, abort_flag, status);
   }
   tc_fence_before_sync();
@@ -961,7 +883,8 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     const int et = threadIdx.x - 32 * kEpiWarp0Q;     // 0..127 = token row of the tile = TMEM lane
     const uint32_t lane_base = 32u * (warp & 3);
     const float bw = fmaxf(beta[0], bw_floor);
-    const float epsp = eps * (float)m * bw * bw;
+    // the filter stage left Q_F, and with it N' and D', scaled by r (see haar_block_inplace): eps' follows
+    const float epsp = eps * (float)m * bw * bw * haar_scale(f[(size_t)slab * (L + 1)]);
     bool ok = true;
     for (int t = 0; t < ntiles; ++t) {
       const int buf = t & 1;
@@ -1017,12 +940,12 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
   } else {
     reg_inc<kRegsAux>();
     const int ht = threadIdx.x - 32 * kAuxWarp0Q;
-    f32x2* hcoef = reinterpret_cast<f32x2*>(smem + SL::hcoef);
+    float* hcoef = reinterpret_cast<float*>(smem + SL::hcoef);
     haar_coef_init(hcoef, f + (size_t)slab * (L + 1), L, ht);
     named_bar_sync(kBarCoef, 256);
     bool ok = true;
     for (int b = 0; b < nblk; ++b)
-      ok = haar_step<kNXQ, false>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
+      ok = haar_step<kNXQ>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
                      ht, ok, abort_flag, status);
   }
   tc_fence_before_sync();
