@@ -31,59 +31,6 @@ __device__ __forceinline__ LevelCoef level_coef(const float* __restrict__ f, int
   return c;
 }
 
-// Block sums of the 8x8 register tile and of its partners.  s1[4], s2[2], s3..s8 per column.
-struct Sums {
-  float s1[4][8], s2[2][8], s3[8], s4[8], s5[8], s6[8], s7[8], s8[8];
-  float p3[8], p4[8], p5[8], p6[8], p7[8];   // the partner's half at levels 4..8 (for details)
-};
-
-__device__ __forceinline__ void block_sums(const float (&x)[8][8], Sums& s, float (*sh)[kD], int L) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, cg = threadIdx.x & 7;
-#pragma unroll
-  for (int c = 0; c < 8; ++c) {
-#pragma unroll
-    for (int p = 0; p < 4; ++p) s.s1[p][c] = x[2 * p][c] + x[2 * p + 1][c];
-    s.s2[0][c] = s.s1[0][c] + s.s1[1][c];
-    s.s2[1][c] = s.s1[2][c] + s.s1[3][c];
-    s.s3[c] = s.s2[0][c] + s.s2[1][c];
-    s.p3[c] = __shfl_xor_sync(0xffffffffu, s.s3[c], 8);
-    s.s4[c] = s.s3[c] + s.p3[c];
-    s.p4[c] = __shfl_xor_sync(0xffffffffu, s.s4[c], 16);
-    s.s5[c] = s.s4[c] + s.p4[c];
-    s.s6[c] = s.s7[c] = s.s8[c] = 0.f;
-    s.p5[c] = s.p6[c] = s.p7[c] = 0.f;
-  }
-  if (L > 5) {   // uniform over the grid
-    __syncthreads();   // previous use of sh is over
-    if ((lane >> 3) == 0) {
-#pragma unroll
-      for (int c = 0; c < 8; ++c) sh[warp][cg * 8 + c] = s.s5[c];
-    }
-    __syncthreads();
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const int col = cg * 8 + c;
-      s.p5[c] = sh[warp ^ 1][col];
-      s.s6[c] = s.s5[c] + s.p5[c];
-      s.p6[c] = sh[warp ^ 2][col] + sh[warp ^ 3][col];
-      s.s7[c] = s.s6[c] + s.p6[c];
-      s.p7[c] = (sh[warp ^ 4][col] + sh[warp ^ 5][col]) + (sh[warp ^ 6][col] + sh[warp ^ 7][col]);
-      s.s8[c] = s.s7[c] + s.p7[c];
-    }
-  }
-}
-
-__device__ __forceinline__ void apply_filter(float (&x)[8][8], const Sums& s, const LevelCoef& k) {
-#pragma unroll
-  for (int c = 0; c < 8; ++c) {
-    const float hi = k.k[3] * s.s3[c] + k.k[4] * s.s4[c] + k.k[5] * s.s5[c] + k.k[6] * s.s6[c] +
-                     k.k[7] * s.s7[c] + k.k[8] * s.s8[c];
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-      x[j][c] = k.f0 * x[j][c] + k.k[1] * s.s1[j >> 1][c] + k.k[2] * s.s2[j >> 2][c] + hi;
-  }
-}
-
 template <typename T>
 __device__ __forceinline__ void load_tile(const T* __restrict__ X, int n, int row0, float (&x)[8][8]) {
   const int cg = threadIdx.x & 7;
@@ -99,24 +46,218 @@ __device__ __forceinline__ void load_tile(const T* __restrict__ X, int n, int ro
   }
 }
 
-// grid (htiles, slabs), block 256.
+constexpr int kPyr = 63;    // 32 + 16 + 8 + 4 + 2 + 1 block sums per column
+constexpr int kHalfD = kD / 2;
+__device__ __forceinline__ int pyr_base(int l) { return 64 - (64 >> (l - 3)); }   // level 3 -> 0, 4 -> 32, 5 -> 48 ...
+
+__device__ __forceinline__ void load4(const float* p, float (&v)[4]) {
+  const float4 a = *reinterpret_cast<const float4*>(p);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&v)[4]) {
+  const uint2 raw = *reinterpret_cast<const uint2*>(p);
+  v[0] = __uint_as_float(raw.x << 16);
+  v[1] = __uint_as_float(raw.x & 0xFFFF0000u);
+  v[2] = __uint_as_float(raw.y << 16);
+  v[3] = __uint_as_float(raw.y & 0xFFFF0000u);
+}
+__device__ __forceinline__ void store4(float* p, const float (&v)[4]) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+__device__ __forceinline__ void store4(__nv_bfloat16* p, const float (&v)[4]) {
+  const __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b2 = __floats2bfloat162_rn(v[2], v[3]);
+  uint2 raw;
+  raw.x = *reinterpret_cast<const uint32_t*>(&a);
+  raw.y = *reinterpret_cast<const uint32_t*>(&b2);
+  *reinterpret_cast<uint2*>(p) = raw;
+}
+
+
+// Stand-alone filter pass, XF = T_f(X).  The transform acts on every column separately, so one CTA takes
+// 256 rows x 32 columns (half of the head dimension), 8 rows x 4 columns per thread: a register tile of
+// 32 values lets several CTAs share an SM, so that the loads of one overlap the arithmetic and stores of
+// the others (the pass is bound by memory bandwidth).  Levels 1-3 come from the register tile; the 8-row
+// sums go to a pyramid in shared memory (per column 32 sums of level 3, then 16, 8, 4, 2, 1 of levels
+// 4-8), from which every thread takes the coarse part of its output rows.
+// grid (2 * htiles, slabs): blockIdx.x = 2 * tile + column half; block 256.
 template <typename Tin, typename Tout>
-__global__ void __launch_bounds__(256, 2) k_haar_filter(const Tin* __restrict__ X, const float* __restrict__ f,
+__global__ void __launch_bounds__(256, 4) k_haar_filter(const Tin* __restrict__ X, const float* __restrict__ f,
                                                      Tout* __restrict__ XF, int n, int L) {
-  __shared__ float sh[8][kD];
+  __shared__ float pyr[kPyr][kHalfD];
+  __shared__ float hit[32][kHalfD];   // sum_{l=3..8} k_l * s_l(block of row group r), per column
+  const int slab = blockIdx.y, half = blockIdx.x & 1;
+  const int cg = threadIdx.x & 7, rg = threadIdx.x >> 3;
+  const int row0 = (blockIdx.x >> 1) * kHaarTile + rg * 8;
+  const int col0 = half * kHalfD + cg * 4;   // first of this thread's four columns
+  const LevelCoef k = level_coef(f + (size_t)slab * (L + 1), L);
+  float x[8][4];
+  {
+    const Tin* xp = X + (size_t)slab * n * kD + col0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (row0 + j < n) {
+        load4(xp + (size_t)(row0 + j) * kD, x[j]);
+      } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) x[j][c] = 0.f;
+      }
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < 4; ++c)
+    pyr[rg][cg * 4 + c] = ((x[0][c] + x[1][c]) + (x[2][c] + x[3][c])) + ((x[4][c] + x[5][c]) + (x[6][c] + x[7][c]));
+  __syncthreads();
+  if (threadIdx.x < kHalfD) {   // levels 4-8 of the pyramid, one thread per column
+    const int col = threadIdx.x;
+#pragma unroll
+    for (int l = 4; l <= 8; ++l) {
+      const int src = pyr_base(l - 1), dst = pyr_base(l), cnt = 256 >> l;
+      for (int b2 = 0; b2 < cnt; ++b2) pyr[dst + b2][col] = pyr[src + 2 * b2][col] + pyr[src + 2 * b2 + 1][col];
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int e = threadIdx.x + 256 * i, r = e >> 5, col = e & 31;
+    float v = k.k[3] * pyr[r][col];
+#pragma unroll
+    for (int l = 4; l <= 8; ++l) v += k.k[l] * pyr[pyr_base(l) + (r >> (l - 3))][col];
+    hit[r][col] = v;
+  }
+  __syncthreads();
+  Tout* dst = XF + (size_t)slab * n * kD + col0;
+#pragma unroll
+  for (int j = 0; j < 8; j += 4) {   // four rows (one level-2 block) at a time
+    float y[4][4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const float a0 = x[j][c] + x[j + 1][c], a1 = x[j + 2][c] + x[j + 3][c];
+      const float c2 = fmaf(k.k[2], a0 + a1, hit[rg][cg * 4 + c]);
+      const float c10 = fmaf(k.k[1], a0, c2), c11 = fmaf(k.k[1], a1, c2);
+      y[0][c] = fmaf(k.f0, x[j][c], c10);
+      y[1][c] = fmaf(k.f0, x[j + 1][c], c10);
+      y[2][c] = fmaf(k.f0, x[j + 2][c], c11);
+      y[3][c] = fmaf(k.f0, x[j + 3][c], c11);
+    }
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj)
+      if (row0 + j + jj < n) store4(dst + (size_t)(row0 + j + jj) * kD, y[jj]);
+  }
+}
+
+// The same pass for bf16 input: a thread keeps its 8 rows x 8 columns as the 32 packed words it loaded
+// (16-byte loads; unpacked where they are used, twice), so that three CTAs of 256 rows x 64 columns share an
+// SM with 16-byte accesses in flight.  grid (htiles, slabs), block 256.
+__device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+
+template <typename Tout>
+__global__ void __launch_bounds__(256, 3) k_haar_filter_bf16(const __nv_bfloat16* __restrict__ X,
+                                                             const float* __restrict__ f, Tout* __restrict__ XF,
+                                                             int n, int L) {
+  __shared__ float pyr[kPyr][kD];
+  __shared__ float hit[32][kD];   // sum_{l=3..8} k_l * s_l(block of row group r), per column
   const int slab = blockIdx.y;
   const int cg = threadIdx.x & 7, rg = threadIdx.x >> 3;
   const int row0 = blockIdx.x * kHaarTile + rg * 8;
   const LevelCoef k = level_coef(f + (size_t)slab * (L + 1), L);
-  float x[8][8];
-  load_tile(X + (size_t)slab * n * kD, n, row0, x);
-  Sums s;
-  block_sums(x, s, sh, L);
-  apply_filter(x, s, k);
-  Tout* dst = XF + (size_t)slab * n * kD + cg * 8;
+  uint32_t u[8][4];
+  {
+    const __nv_bfloat16* xp = X + (size_t)slab * n * kD + cg * 8;
 #pragma unroll
-  for (int j = 0; j < 8; ++j)
-    if (row0 + j < n) store8(dst + (size_t)(row0 + j) * kD, x[j]);
+    for (int j = 0; j < 8; ++j) {
+      uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+      if (row0 + j < n) raw = *reinterpret_cast<const uint4*>(xp + (size_t)(row0 + j) * kD);
+      u[j][0] = raw.x; u[j][1] = raw.y; u[j][2] = raw.z; u[j][3] = raw.w;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float lo = 0.f, hi = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; j += 2) {   // pairs first, as the other kernels add them
+      lo += bf_lo(u[j][i]) + bf_lo(u[j + 1][i]);
+      hi += bf_hi(u[j][i]) + bf_hi(u[j + 1][i]);
+    }
+    pyr[rg][cg * 8 + 2 * i] = lo;
+    pyr[rg][cg * 8 + 2 * i + 1] = hi;
+  }
+  __syncthreads();
+  if (threadIdx.x < kD) {   // levels 4-8 of the pyramid, one thread per column
+    const int col = threadIdx.x;
+#pragma unroll
+    for (int l = 4; l <= 8; ++l) {
+      const int src = pyr_base(l - 1), dst = pyr_base(l), cnt = 256 >> l;
+      for (int b2 = 0; b2 < cnt; ++b2) pyr[dst + b2][col] = pyr[src + 2 * b2][col] + pyr[src + 2 * b2 + 1][col];
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int e = threadIdx.x + 256 * i, r = e >> 6, col = e & 63;
+    float v = k.k[3] * pyr[r][col];
+#pragma unroll
+    for (int l = 4; l <= 8; ++l) v += k.k[l] * pyr[pyr_base(l) + (r >> (l - 3))][col];
+    hit[r][col] = v;
+  }
+  __syncthreads();
+  Tout* dst = XF + (size_t)slab * n * kD + cg * 8;
+  if constexpr (sizeof(Tout) == 2) {
+    // bf16 out: the results replace the packed inputs column pair by column pair, rows are stored whole
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float h0 = hit[rg][cg * 8 + 2 * i], h1 = hit[rg][cg * 8 + 2 * i + 1];
+#pragma unroll
+      for (int j = 0; j < 8; j += 4) {
+        float y[4][2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float x0 = h ? bf_hi(u[j][i]) : bf_lo(u[j][i]), x1 = h ? bf_hi(u[j + 1][i]) : bf_lo(u[j + 1][i]);
+          const float x2 = h ? bf_hi(u[j + 2][i]) : bf_lo(u[j + 2][i]), x3 = h ? bf_hi(u[j + 3][i]) : bf_lo(u[j + 3][i]);
+          const float a0 = x0 + x1, a1 = x2 + x3;
+          const float c2 = fmaf(k.k[2], a0 + a1, h ? h1 : h0);
+          const float c10 = fmaf(k.k[1], a0, c2), c11 = fmaf(k.k[1], a1, c2);
+          y[0][h] = fmaf(k.f0, x0, c10);
+          y[1][h] = fmaf(k.f0, x1, c10);
+          y[2][h] = fmaf(k.f0, x2, c11);
+          y[3][h] = fmaf(k.f0, x3, c11);
+        }
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          const __nv_bfloat162 pk = __floats2bfloat162_rn(y[jj][0], y[jj][1]);
+          u[j + jj][i] = *reinterpret_cast<const uint32_t*>(&pk);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (row0 + j < n)
+        *reinterpret_cast<uint4*>(dst + (size_t)(row0 + j) * kD) = make_uint4(u[j][0], u[j][1], u[j][2], u[j][3]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; j += 4) {   // four rows (one level-2 block) at a time
+      float y[4][8];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int c = 2 * i + h;
+          const float x0 = h ? bf_hi(u[j][i]) : bf_lo(u[j][i]), x1 = h ? bf_hi(u[j + 1][i]) : bf_lo(u[j + 1][i]);
+          const float x2 = h ? bf_hi(u[j + 2][i]) : bf_lo(u[j + 2][i]), x3 = h ? bf_hi(u[j + 3][i]) : bf_lo(u[j + 3][i]);
+          const float a0 = x0 + x1, a1 = x2 + x3;
+          const float c2 = fmaf(k.k[2], a0 + a1, hit[rg][cg * 8 + c]);
+          const float c10 = fmaf(k.k[1], a0, c2), c11 = fmaf(k.k[1], a1, c2);
+          y[0][c] = fmaf(k.f0, x0, c10);
+          y[1][c] = fmaf(k.f0, x1, c10);
+          y[2][c] = fmaf(k.f0, x2, c11);
+          y[3][c] = fmaf(k.f0, x3, c11);
+        }
+      }
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj)
+        if (row0 + j + jj < n) store8(dst + (size_t)(row0 + j + jj) * kD, y[jj]);
+    }
+  }
 }
 
 // The same filter with the result written as three bf16 planes hi + mid + lo (each slabs x n x 64):
@@ -208,32 +349,6 @@ __global__ void __launch_bounds__(256, 2) k_haar_filter_split3(const Tin* __rest
 // sums of level 3, then 16, 8, 4, 2, 1 of levels 4-8), from which one thread per column takes the level
 // 4-8 products and every thread the coarse part of its output rows.
 // grid (2 * htiles, slabs): blockIdx.x = 2 * tile + column half; one band partial per CTA.
-constexpr int kPyr = 63;    // 32 + 16 + 8 + 4 + 2 + 1 block sums per column
-constexpr int kHalfD = kD / 2;
-__device__ __forceinline__ int pyr_base(int l) { return 64 - (64 >> (l - 3)); }   // level 3 -> 0, 4 -> 32, 5 -> 48 ...
-
-__device__ __forceinline__ void load4(const float* p, float (&v)[4]) {
-  const float4 a = *reinterpret_cast<const float4*>(p);
-  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
-}
-__device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&v)[4]) {
-  const uint2 raw = *reinterpret_cast<const uint2*>(p);
-  v[0] = __uint_as_float(raw.x << 16);
-  v[1] = __uint_as_float(raw.x & 0xFFFF0000u);
-  v[2] = __uint_as_float(raw.y << 16);
-  v[3] = __uint_as_float(raw.y & 0xFFFF0000u);
-}
-__device__ __forceinline__ void store4(float* p, const float (&v)[4]) {
-  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
-}
-__device__ __forceinline__ void store4(__nv_bfloat16* p, const float (&v)[4]) {
-  const __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b2 = __floats2bfloat162_rn(v[2], v[3]);
-  uint2 raw;
-  raw.x = *reinterpret_cast<const uint32_t*>(&a);
-  raw.y = *reinterpret_cast<const uint32_t*>(&b2);
-  *reinterpret_cast<uint2*>(p) = raw;
-}
-
 template <typename Tin, typename Tout>
 __global__ void __launch_bounds__(256, 3) k_haar_backward(const Tin* __restrict__ X, const float* __restrict__ G,
                                                           const float* __restrict__ f, Tout* __restrict__ dX,
@@ -369,13 +484,13 @@ __global__ void __launch_bounds__(256, 3) k_haar_backward(const Tin* __restrict_
 
 cudaError_t launch_haar_filter(const Plan& p, const void* X, int in_kind, const float* f, void* XF,
                                int out_kind, cudaStream_t st, int* launches) {
-  dim3 grid(p.htiles, p.slabs);
+  dim3 grid(2 * p.htiles, p.slabs);   // fp32 input: two column halves per 256-row tile
+  dim3 grid_bf(p.htiles, p.slabs);
   const int n = p.cfg.seq_len, L = p.cfg.levels;
   if (in_kind == 1 && out_kind == 1)
-    k_haar_filter<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, f,
-                                                                       (__nv_bfloat16*)XF, n, L);
+    k_haar_filter_bf16<__nv_bfloat16><<<grid_bf, 256, 0, st>>>((const __nv_bfloat16*)X, f, (__nv_bfloat16*)XF, n, L);
   else if (in_kind == 1 && out_kind == 0)
-    k_haar_filter<__nv_bfloat16, float><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, f, (float*)XF, n, L);
+    k_haar_filter_bf16<float><<<grid_bf, 256, 0, st>>>((const __nv_bfloat16*)X, f, (float*)XF, n, L);
   else if (in_kind == 0 && out_kind == 0)
     k_haar_filter<float, float><<<grid, 256, 0, st>>>((const float*)X, f, (float*)XF, n, L);
   else
