@@ -124,8 +124,9 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
     p->off_dSbf = take(sizeof(__nv_bfloat16) * slabs * m * kD);
     p->off_KF3 = take(p->use_tc ? 3 * sizeof(__nv_bfloat16) * slab_elems : 0);
     p->off_QF3 = take(p->use_tc ? 3 * sizeof(__nv_bfloat16) * slab_elems : 0);
+    p->off_Slo = take(p->use_tc ? sizeof(__nv_bfloat16) * slabs * m * kD : 0);
   } else {
-    p->off_dS = p->off_dz = p->off_sumdD = p->off_bands = p->off_dqbar = p->off_dQF = p->off_dKF = p->off_dSbf = p->off_KF3 = p->off_QF3 = 0;
+    p->off_dS = p->off_dz = p->off_sumdD = p->off_bands = p->off_dqbar = p->off_dQF = p->off_dKF = p->off_dSbf = p->off_KF3 = p->off_QF3 = p->off_Slo = 0;
   }
   p->total = off;
   return WERSA_OK;
@@ -158,6 +159,7 @@ Ws resolve(const Plan& p, void* workspace) {
   w.dSbf = reinterpret_cast<__nv_bfloat16*>(b + p.off_dSbf);
   w.KF3 = reinterpret_cast<__nv_bfloat16*>(b + p.off_KF3);
   w.QF3 = reinterpret_cast<__nv_bfloat16*>(b + p.off_QF3);
+  w.Slo = reinterpret_cast<__nv_bfloat16*>(b + p.off_Slo);
   return w;
 }
 

@@ -39,7 +39,7 @@ struct Plan {
   // workspace offsets (bytes)
   size_t off_status, off_counters, status_bytes, off_qpart, off_qbar, off_sg, off_f, off_spart, off_zpart, off_S, off_z,
       off_Sbf, off_Wt, off_dS, off_dz, off_sumdD, off_bands, off_dqbar, off_QF, off_KF, off_dQF,
-      off_dKF, off_dSbf, off_KF3, off_QF3, total;
+      off_dKF, off_dSbf, off_KF3, off_QF3, off_Slo, total;
   int part_chunks;    // max(schunks, tchunks): leading extent of the partial buffers
 };
 
@@ -50,7 +50,7 @@ struct Ws {   // resolved workspace pointers
   int* status;
   int* counters;   // arrival counters (slabs + batch + slabs ints), zero between launches
   float *qpart, *qbar, *sg, *f, *spart, *zpart, *S, *z, *dS, *dz, *sumdD, *bands, *dqbar;
-  __nv_bfloat16 *Sbf, *Wt, *dSbf, *KF3, *QF3;
+  __nv_bfloat16 *Sbf, *Wt, *dSbf, *KF3, *QF3, *Slo;   // Slo = bf16(S' - bf16(S')), built by the backward
   float *QF, *KF, *dQF, *dKF;
 };
 Ws resolve(const Plan& p, void* workspace);

@@ -46,7 +46,7 @@ constexpr uint32_t kIdescC = make_idesc_bf16(128, 64, false, true);    // contra
 enum { kErrBwdCopy = 21, kErrBwdMma = 22 };
 
 struct alignas(8) BwdBars {
-  uint64_t full[2], mma;
+  uint64_t full[2], mma, slo;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -439,7 +439,8 @@ template <int NH> struct BwdQSmem {
 template <int NH>
 __global__ void __launch_bounds__(256, 1)
 k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant__ CUtensorMap map_do,
-               const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ Sbf,
+               const __grid_constant__ CUtensorMap map_slo, const __nv_bfloat16* __restrict__ Wt,
+               const __nv_bfloat16* __restrict__ Sbf,
                const float* __restrict__ zg, const float* __restrict__ beta, float eps, float bw_floor,
                const __grid_constant__ CUtensorMap map_dqf, float* __restrict__ dspart,
                float* __restrict__ dzpart, float* __restrict__ sumdD, int n, int chunk_tiles,
@@ -464,6 +465,7 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
     mbar_init(&bars->full[0], 1);
     mbar_init(&bars->full[1], 1);
     mbar_init(&bars->mma, 1);
+    mbar_init(&bars->slo, 1);
     bars->abort_flag = 0;
     fence_mbar_init();
   }
@@ -493,7 +495,7 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
   constexpr uint32_t kTileStep = kTileBytes >> 4, kStageStep = SL::stage_bytes >> 4;
   const int slabs = gridDim.y;
   uint32_t mma_par = 0;
-  int issued = 0;
+  int issued = 0, slo_issued = 0;
   bool ok = true;
   float dzacc[NH];                                // feature = thread: dz'_h partial of this chunk
 #pragma unroll
@@ -545,6 +547,16 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
       mma_commit(&bars->mma);
     }
     if (!(ok = wait_mma())) break;
+    // The mid and lo planes of this tile's stage are dead from here on (MMA1 has read them; the transposed
+    // projection below takes the hi plane only): the low-order image of S' of this slab, bf16(S' - bf16(S')),
+    // is fetched into their place for MMA3.  (Shared memory has no room to hold it for the whole chunk.)
+    if (threadIdx.x == 0) {
+      uint8_t* dst = smem + SL::stage + (ti & 1) * SL::stage_bytes + kTileBytes;
+      mbar_arrive_expect_tx(&bars->slo, NH * kTileBytes);
+#pragma unroll
+      for (int h = 0; h < NH; ++h) tma_load_3d(dst + h * kTileBytes, &map_slo, 0, h * kTile, slab, &bars->slo);
+      slo_issued = ti + 1;
+    }
     // ---- mask, Phi, denominator
     uint32_t mask[2 * NH];
     float den = 0.f;
@@ -658,6 +670,16 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
           for (int k = 0; k < 4; ++k)
             mma_ss(tmem + h * 128, smem_desc_join(dn_k + part * kTileStep + 2 * k, hi),
                    smem_desc_join(s_k + h * kTileStep + 2 * k, hi), kIdescP, (part > 0 || k > 0) ? 1u : 0u);
+      // + dN'(hi) S'(lo)^T: the single bf16 rounding of S' was the largest error of dQ_F
+      if (mbar_wait(&bars->slo, ti & 1, &bars->abort_flag, status, kErrBwdCopy)) {
+        const uint32_t slo_k = x_k + kTileStep;
+#pragma unroll
+        for (int h = 0; h < NH; ++h)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            mma_ss(tmem + h * 128, smem_desc_join(dn_k + 2 * k, hi), smem_desc_join(slo_k + h * kTileStep + 2 * k, hi),
+                   kIdescP, 1u);
+      }
       mma_commit(&bars->mma);
     }
     if (!(ok = wait_mma())) break;
@@ -718,8 +740,10 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
     }
   }
   if (threadIdx.x == 0) {
-    if (!ok)
+    if (!ok) {
       for (int t = max(0, issued - 2); t < issued; ++t) mbar_wait_drain(&bars->full[t & 1], (t >> 1) & 1);
+      if (slo_issued > 0) mbar_wait_drain(&bars->slo, (slo_issued - 1) & 1);
+    }
     bulk_wait_group0();   // the dQ_F stores read this CTA's shared memory
   }
   tc_fence_before_sync();
@@ -728,6 +752,13 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
     tc_fence_after_sync();
     tmem_dealloc(tmem, kCols);
   }
+}
+
+// lo = bf16(x - hi) for hi = bf16(x) as the forward left it: the second half of a hi + lo pair for S'.
+__global__ void __launch_bounds__(256) k_split_lo(const float* __restrict__ x, const __nv_bfloat16* __restrict__ hi_img,
+                                                   __nv_bfloat16* __restrict__ lo_img, size_t count) {
+  const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+  if (i < count) lo_img[i] = __float2bfloat16_rn(x[i] - __bfloat162float(hi_img[i]));
 }
 
 // ---- host side ----------------------------------------------------------------------------------
@@ -798,13 +829,19 @@ cudaError_t launch_kside(const Plan& p, const Ws& w, const CUtensorMap& map_kf, 
 template <int NH>
 cudaError_t launch_qside(const Plan& p, const Ws& w, const CUtensorMap& map_qf, const CUtensorMap& map_do,
                          const float* beta, cudaStream_t st) {
+  // low-order bf16 image of S' (rows = features of a slab), fetched tile by tile by the kernel
+  const size_t count = (size_t)p.slabs * p.cfg.features * kD;
+  k_split_lo<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(w.S, w.Sbf, w.Slo, count);
+  CUtensorMap map_slo;
+  cudaError_t merr;
+  if ((merr = make_tile_map(w.Slo, p.slabs, p.cfg.features, &map_slo)) != cudaSuccess) return merr;
   auto k = k_tc_bwd_qside<NH>;
   cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdQSmem<NH>::total);
   if (err != cudaSuccess) return err;
   CUtensorMap map_dqf;
   if ((err = make_out_map(w.dQF, p.slabs, p.cfg.seq_len, false, &map_dqf)) != cudaSuccess) return err;
   dim3 grid(p.bchunks, p.slabs);
-  k<<<grid, 256, BwdQSmem<NH>::total, st>>>(map_qf, map_do, w.Wt, w.Sbf, w.z, beta, p.cfg.eps, p.cfg.bw_floor, map_dqf,
+  k<<<grid, 256, BwdQSmem<NH>::total, st>>>(map_qf, map_do, map_slo, w.Wt, w.Sbf, w.z, beta, p.cfg.eps, p.cfg.bw_floor, map_dqf,
                                             w.spart, w.zpart, w.sumdD, p.cfg.seq_len, p.bchunk_tiles, w.status);
   return cudaGetLastError();
 }
@@ -817,7 +854,7 @@ cudaError_t launch_tc_bwd_qside(const Plan& p, const Ws& w, const void* QF3, con
   cudaError_t err;
   if ((err = make_tile_map(QF3, 3 * p.slabs, p.cfg.seq_len, &map_qf)) != cudaSuccess) return err;
   if ((err = make_tile_map(dO, p.slabs, p.cfg.seq_len, &map_do)) != cudaSuccess) return err;
-  *launches += 1;
+  *launches += 2;   // the low-order image of S', then the kernel
   return p.cfg.features == 256 ? launch_qside<2>(p, w, map_qf, map_do, beta, st)
                                : launch_qside<1>(p, w, map_qf, map_do, beta, st);
 }
