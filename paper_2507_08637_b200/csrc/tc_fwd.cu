@@ -92,13 +92,13 @@ enum { kErrProducer = 11, kErrMma = 12, kErrRelu = 13, kErrEpilogue = 14, kErrHa
 
 struct alignas(8) KsideBars {
   uint64_t x_full[kNXK], x_empty[kNXK], xf_ready[kNF], v_full[kNV], v_empty[kNV];
-  uint64_t d1_full[6], phi_ready[kND1], d1_free[kND1], acc_done, w_full;
+  uint64_t d1_full[6], phi_ready[kND1], d1_free[kND1], acc_done, acc_free, w_full;
   uint32_t tmem_base;
   int abort_flag;
 };
 struct alignas(8) QsideBars {
   uint64_t x_full[kNXQ], x_empty[kNXQ], xf_ready[kNF];
-  uint64_t d1_full[2], phi_ready[2], d2_full[2], buf_free[2], simg_ready, w_full;
+  uint64_t d1_full[2], phi_ready[2], d2_full[2], buf_free[2], simg_ready, simg_next, w_full;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -383,18 +383,19 @@ __device__ __forceinline__ void haar_block_inplace(uint8_t* tile0, uint8_t* tile
   }
 }
 
-// One Haar step: wait for the two raw tiles of block b, filter them in place, hand the block to the
-// MMA issuer.  NX = number of tile slots in the ring.
+// One Haar step: wait for the two raw tiles of block b (counted over all the work items of the CTA, like
+// the ring slots and barrier phases), filter them in place, hand the block to the MMA issuer.  NX = number
+// of tile slots in the ring; valid_rows = rows of the block that lie inside the sequence.
 template <int NX, typename Bars>
 __device__ __forceinline__ bool haar_step(uint8_t* xring, Bars* bars, float* xch, const float* hcoef, bool cross,
-                                          int b, int rows_left, int ht, bool ok, volatile int* abort_flag,
+                                          int b, int valid_rows, int ht, bool ok, volatile int* abort_flag,
                                           int* status) {
   const int t0 = 2 * b, t1 = 2 * b + 1;
   const int s0 = t0 % NX, s1 = t1 % NX;
   if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[s0], (t0 / NX) & 1, abort_flag, status, kErrHaar));
   if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[s1], (t1 / NX) & 1, abort_flag, status, kErrHaar));
   haar_block_inplace(xring + s0 * kTileBytes, xring + s1 * kTileBytes, hcoef, cross, xch + (b & 1) * 8 * kD, ht,
-                     rows_left - b * kBlk, ok);
+                     valid_rows, ok);
   if (ok) {
     fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
     warp_arrive(&bars->xf_ready[b & (kNF - 1)]);
@@ -402,24 +403,38 @@ __device__ __forceinline__ bool haar_step(uint8_t* xring, Bars* bars, float* xch
   return ok;
 }
 
+// ---- work items ---------------------------------------------------------------------------------
+// Both kernels run one CTA per SM that walks work items: item = slab * chunks + chunk is one sequence
+// chunk of one slab, CTA c takes items c, c + gridDim.x, c + 2 gridDim.x, ...  Ring slots, accumulator
+// buffers and barrier phases count on across items, so the copies and the filter stage of the next item
+// run while the current one is still in the tensor pipe; only what belongs to a slab (filter
+// coefficients, accumulators, the S' image) is renewed at an item boundary.
+__device__ __forceinline__ int item_blocks(int item, int chunks, int chunk_blocks, int n) {
+  return min(chunk_blocks, (n + kBlk - 1) / kBlk - (item % chunks) * chunk_blocks);
+}
+
 // ---- key side -----------------------------------------------------------------------------------
-// grid (chunks, slabs), block 640.  TMEM: D1[3] at columns 0 / 128 / 256, S' half h at 384 + 64 h.
-template <int NH>
+// grid (chunks, slabs) when every CTA has one item, else (min(SMs, items)); block 640.  TMEM: D1[3] at columns 0 / 128 / 256, S' half h at 384 + 64 h.
+// kMulti = false: every CTA has exactly one work item (the item loops run once and the code of the item
+// boundaries drops out).
+template <int NH, bool kMulti>
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
            const __grid_constant__ CUtensorMap map_w, const float* __restrict__ f, float* __restrict__ spart,
-           float* __restrict__ zpart, __nv_bfloat16* __restrict__ sbf, int n, int L, int chunk_blocks,
-           int* __restrict__ status) {
+           float* __restrict__ zpart, __nv_bfloat16* __restrict__ sbf, int n, int L, int chunk_blocks, int chunks,
+           int items, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   using SL = KsideSmem<NH>;
   KsideBars* bars = reinterpret_cast<KsideBars*>(smem + SL::bars);
   float* zx = reinterpret_cast<float*>(smem + SL::zx);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int chunk = blockIdx.x, slab = blockIdx.y;
-  const int blk0 = chunk * chunk_blocks;
-  const int nblk = min(chunk_blocks, (n + kBlk - 1) / kBlk - blk0);
-  const int units = nblk * 2 * NH;
+  // item0 < items: the grid never exceeds the item count.  Without kMulti the step is a constant that ends
+  // every item loop after one pass, so that the compiler sees straight-line code.
+  const int item0 = blockIdx.y * gridDim.x + blockIdx.x, item_step = kMulti ? (int)gridDim.x : (1 << 30);
+  if (!kMulti) items = item0 + 1;
+  const int nblk0 = item_blocks(item0, chunks, chunk_blocks, n);
+  constexpr bool single_item = !kMulti;
   constexpr int m = NH * 128;
 
   if (threadIdx.x == 0) {
@@ -438,17 +453,20 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       mbar_init(&bars->d1_free[b], 1);
     }
     mbar_init(&bars->acc_done, NH);
+    mbar_init(&bars->acc_free, 8);
     mbar_init(&bars->w_full, 1);
     bars->abort_flag = 0;
     fence_mbar_init();
-    // K and V are inputs: the first copies of both rings go out before the dependency wait below
-    for (int b = 0; b < min(2 * nblk, kNXK); ++b) {
+    // K and V are inputs: the first copies of both rings (tiles of the first item) go out before the
+    // dependency wait below
+    const int slab = item0 / chunks, row0 = (item0 % chunks) * chunk_blocks * kBlk;
+    for (int b = 0; b < min(2 * nblk0, kNXK); ++b) {
       mbar_arrive_expect_tx(&bars->x_full[b], kTileBytes);
-      tma_load_3d(smem + SL::x + b * kTileBytes, &map_k, 0, blk0 * kBlk + b * kTile, slab, &bars->x_full[b]);
+      tma_load_3d(smem + SL::x + b * kTileBytes, &map_k, 0, row0 + b * kTile, slab, &bars->x_full[b]);
     }
-    for (int b = 0; b < min(2 * nblk, kNV); ++b) {
+    for (int b = 0; b < min(2 * nblk0, kNV); ++b) {
       mbar_arrive_expect_tx(&bars->v_full[b], kTileBytes);
-      tma_load_3d(smem + SL::v + b * kTileBytes, &map_v, 0, blk0 * kBlk + b * kTile, slab, &bars->v_full[b]);
+      tma_load_3d(smem + SL::v + b * kTileBytes, &map_v, 0, row0 + b * kTile, slab, &bars->v_full[b]);
     }
   }
   if (warp == kWarpMma) {
@@ -477,31 +495,58 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
     reg_dec<kRegsCtl>();
     if (warp == kWarpTma && lane == 0) {
       // One producer for both rings: whichever ring has a free slot gets its next tile, so that a full
-      // V ring never holds back the K tiles (and the other way round).
-      const int total = 2 * nblk;   // 128-token tiles
-      int kb = min(total, kNXK), vb = min(total, kNV);   // the first ring of each went out during set-up
-      const unsigned long long t0 = global_timer_ns();
+      // V ring never holds back the K tiles (and the other way round).  Each ring walks the tiles of this
+      // CTA's items on its own: (ik, tk) / (iv, tv) = item and tile of the next K / V copy, kb / vb = tiles
+      // sent so far (slot and phase of the ring).
+      int kb = min(2 * nblk0, kNXK), vb = min(2 * nblk0, kNV);   // the first ring of each went out during set-up
+      int ik = item0, tk = kb, iv = item0, tv = vb;
+      int nk = 2 * nblk0, nv = 2 * nblk0;                         // tiles of item ik / iv
+      if (tk == nk) {
+        ik += item_step;
+        tk = 0;
+        if (ik < items) nk = 2 * item_blocks(ik, chunks, chunk_blocks, n);
+      }
+      if (tv == nv) {
+        iv += item_step;
+        tv = 0;
+        if (iv < items) nv = 2 * item_blocks(iv, chunks, chunk_blocks, n);
+      }
+      unsigned long long t0 = global_timer_ns();
       uint32_t spins = 0;
       bool ok = true;
-      while (ok && (kb < total || vb < total)) {
+      while (ok && (ik < items || iv < items)) {
         bool progress = false;
-        if (kb < total && mbar_try_wait(&bars->x_empty[kb % kNXK], ((kb / kNXK) & 1) ^ 1)) {
+        if (ik < items && mbar_try_wait(&bars->x_empty[kb % kNXK], ((kb / kNXK) & 1) ^ 1)) {
           const int s = kb % kNXK;
           mbar_arrive_expect_tx(&bars->x_full[s], kTileBytes);
-          tma_load_3d(smem + SL::x + s * kTileBytes, &map_k, 0, blk0 * kBlk + kb * kTile, slab, &bars->x_full[s]);
+          tma_load_3d(smem + SL::x + s * kTileBytes, &map_k, 0, (ik % chunks) * chunk_blocks * kBlk + tk * kTile,
+                      ik / chunks, &bars->x_full[s]);
           ++kb;
+          if (++tk == nk) {
+            ik += item_step;
+            tk = 0;
+            if (ik < items) nk = 2 * item_blocks(ik, chunks, chunk_blocks, n);
+          }
           progress = true;
         }
-        if (vb < total && mbar_try_wait(&bars->v_empty[vb % kNV], ((vb / kNV) & 1) ^ 1)) {
+        if (iv < items && mbar_try_wait(&bars->v_empty[vb % kNV], ((vb / kNV) & 1) ^ 1)) {
           const int s = vb % kNV;
           mbar_arrive_expect_tx(&bars->v_full[s], kTileBytes);
-          tma_load_3d(smem + SL::v + s * kTileBytes, &map_v, 0, blk0 * kBlk + vb * kTile, slab, &bars->v_full[s]);
+          tma_load_3d(smem + SL::v + s * kTileBytes, &map_v, 0, (iv % chunks) * chunk_blocks * kBlk + tv * kTile,
+                      iv / chunks, &bars->v_full[s]);
           ++vb;
+          if (++tv == nv) {
+            iv += item_step;
+            tv = 0;
+            if (iv < items) nv = 2 * item_blocks(iv, chunks, chunk_blocks, n);
+          }
           progress = true;
         }
-        if (!progress && (++spins & 255u) == 0) {
+        if (progress) {
+          t0 = global_timer_ns();   // the limit bounds the time without progress
+        } else if ((++spins & 255u) == 0) {
           if (*abort_flag != 0) ok = false;
-          else if (global_timer_ns() - t0 > kWaitLimitNs * 4) {   // whole-kernel budget of this loop
+          else if (global_timer_ns() - t0 > kWaitLimitNs * 2) {
             *abort_flag = 1;
             atomicCAS(status, 0, kErrProducer);
             ok = false;
@@ -523,7 +568,9 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       uint32_t xs = 0, fs = 0, fpar = 0;               // K ring slot; "block filtered" barrier and phase
       uint32_t c3 = 0, c6 = 0, round = 0;              // D1 buffer, d1_full barrier, uses of buffer 0 so far
       bool ok = mbar_wait(&bars->w_full, 0, abort_flag, status, kErrMma);
-      for (int b = 0; b < nblk && ok; ++b) {
+      int blocks_all = 0;                              // blocks of all items of this CTA
+      for (int it = item0; it < items; it += item_step) blocks_all += item_blocks(it, chunks, chunk_blocks, n);
+      for (int b = 0; b < blocks_all && ok; ++b) {
         ok = mbar_wait(&bars->xf_ready[fs], fpar, abort_flag, status, kErrMma);
         if (!ok) break;
         tc_fence_after_sync();
@@ -561,92 +608,149 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
       const uint32_t v_lo = smem_desc_lo(smem_u32(smem + SL::v), 1024);
       const uint32_t acc = tmem + kAccCol + h * 64;
       uint32_t vs = 0, vpar = 0;                       // V ring slot / phase
+      int gt = 0, ic = 0;                              // tiles and items so far
       bool ok = true;
-      for (int t = 0; t < 2 * nblk && ok; ++t) {
-        const int u = t * NH + h, p3 = u % kND1;
-        ok = mbar_wait(&bars->v_full[vs], vpar, abort_flag, status, kErrMma);
-        if (!ok) break;
-        ok = mbar_wait(&bars->phi_ready[p3], (u / kND1) & 1, abort_flag, status, kErrMma);
-        if (!ok) break;
-        tc_fence_after_sync();
-        const uint32_t a_tm = tmem + p3 * 128;
-        const uint32_t b_lo = v_lo + vs * kTileStep;
+      for (int it = item0; it < items && ok; it += item_step, ++ic) {
+        const int ntl = 2 * item_blocks(it, chunks, chunk_blocks, n);
+        if (ic > 0) {   // the accumulators of the item before must have been read out
+          ok = mbar_wait(&bars->acc_free, (ic - 1) & 1, abort_flag, status, kErrMma);
+          if (!ok) break;
+          tc_fence_after_sync();
+        }
+        for (int t = 0; t < ntl && ok; ++t, ++gt) {
+          const int u = gt * NH + h, p3 = u % kND1;
+          ok = mbar_wait(&bars->v_full[vs], vpar, abort_flag, status, kErrMma);
+          if (!ok) break;
+          ok = mbar_wait(&bars->phi_ready[p3], (u / kND1) & 1, abort_flag, status, kErrMma);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t a_tm = tmem + p3 * 128;
+          const uint32_t b_lo = v_lo + vs * kTileStep;
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-          mma_ts(acc, a_tm + k * 8, smem_desc_join(b_lo + 128 * k, hi), kIdesc2, (t > 0 || k > 0) ? 1u : 0u);
-        mma_commit(&bars->d1_free[p3]);
-        mma_commit(&bars->v_empty[vs]);   // one arrival per half
-        vs = vs == kNV - 1 ? 0 : vs + 1;
-        vpar ^= (vs == 0);
+          for (int k = 0; k < 8; ++k)
+            mma_ts(acc, a_tm + k * 8, smem_desc_join(b_lo + 128 * k, hi), kIdesc2, (t > 0 || k > 0) ? 1u : 0u);
+          mma_commit(&bars->d1_free[p3]);
+          mma_commit(&bars->v_empty[vs]);   // one arrival per half
+          vs = vs == kNV - 1 ? 0 : vs + 1;
+          vpar ^= (vs == 0);
+        }
+        if (ok) mma_commit(&bars->acc_done);   // one phase per item
       }
-      mma_commit(&bars->acc_done);
     }
   } else if (warp >= kReluWarp0 && warp < kAuxWarp0) {
     const int g = (warp - kReluWarp0) >> 2;         // ReLU warpgroup 0 / 1
     const uint32_t lane_base = 32u * (warp & 3);
     const int row = lane_base + lane;               // feature within the half = TMEM lane
-    float zacc = 0.f;
     bool ok = true;
-    for (int u = g; u < units; u += 2) {
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d1_full[u % 6], (u / 6) & 1, abort_flag, status, kErrRelu));
-      if (ok) {
-        tc_fence_after_sync();
-        zacc += relu_unit(tmem + (lane_base << 16) + (u % kND1) * 128);
-        tc_fence_before_sync();
-        warp_arrive(&bars->phi_ready[u % kND1]);
+    int gu0 = 0, ic = 0;                            // units and items so far (an item has an even number of units)
+    for (int it = item0; it < items; it += item_step, ++ic) {
+      const int slab = it / chunks;
+      const int units = item_blocks(it, chunks, chunk_blocks, n) * 2 * NH;
+      float zacc = 0.f;
+      for (int u = g; u < units; u += 2) {
+        const int gu = gu0 + u;
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d1_full[gu % 6], (gu / 6) & 1, abort_flag, status, kErrRelu));
+        if (ok) {
+          tc_fence_after_sync();
+          zacc += relu_unit(tmem + (lane_base << 16) + (gu % kND1) * 128);
+          tc_fence_before_sync();
+          warp_arrive(&bars->phi_ready[gu % kND1]);
+        }
       }
-    }
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->acc_done, 0, abort_flag, status, kErrRelu));
-    if (ok) tc_fence_after_sync();
-    const size_t pidx = (size_t)slab * gridDim.x + chunk;
-    if (NH == 1) {   // both warpgroups saw the same 128 features on alternating tiles
-      if (g == 1) zx[row] = zacc;
-      named_bar_sync(kBarZsum, 256);
-      if (g == 0) zacc += zx[row];
-    }
-    if (ok && (NH == 2 || g == 0)) {
-      // The accumulator row of a thread is one feature's 64 values; written straight from the registers a
-      // warp would touch 32 different 256-byte rows per store.  Each warp instead turns its 32 x 32 chunk
-      // around in shared memory (the K ring is idle by now; rows padded to 33 floats) and writes whole
-      // 128-byte row segments.
-      const int feat0 = (NH == 2 ? g * 128 : 0) + (int)lane_base;   // first feature of this warp
-      // the filter stage left K_F, and with it the features, scaled by r (see haar_block_inplace)
-      const float inv_r = 1.f / haar_scale(f[(size_t)slab * (L + 1)]);
-      float* stage = reinterpret_cast<float*>(smem + SL::x) + (warp - kReluWarp0) * (32 * 33);
-      float* dst = spart + (pidx * m + feat0) * kD;
+      gu0 += units;
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->acc_done, ic & 1, abort_flag, status, kErrRelu));
+      if (ok) tc_fence_after_sync();
+      const size_t pidx = (size_t)it;                 // = slab * chunks + chunk
+      if (NH == 1) {   // both warpgroups saw the same 128 features on alternating tiles
+        if (ic > 0) named_bar_sync(kBarZsum, 256);    // the sums of the item before have been read
+        if (g == 1) zx[row] = zacc;
+        named_bar_sync(kBarZsum, 256);
+        if (g == 0) zacc += zx[row];
+      }
+      if (ok && (NH == 2 || g == 0)) {
+        const int feat0 = (NH == 2 ? g * 128 : 0) + (int)lane_base;   // first feature of this warp
+        // the filter stage left K_F, and with it the features, scaled by r (see haar_block_inplace)
+        const float inv_r = 1.f / haar_scale(f[(size_t)slab * (L + 1)]);
+        const uint32_t acc_addr = tmem + (lane_base << 16) + kAccCol + (NH == 2 ? g * 64 : 0);
+        if (single_item) {
+          // The accumulator row of a thread is one feature's 64 values; written straight from the registers
+          // a warp would touch 32 different 256-byte rows per store.  With one item per CTA the K ring is
+          // idle by now: each warp turns its 32 x 32 chunk around in it (rows padded to 33 floats) and
+          // writes whole 128-byte row segments.
+          float* stage = reinterpret_cast<float*>(smem + SL::x) + (warp - kReluWarp0) * (32 * 33);
+          float* dst = spart + (pidx * m + feat0) * kD;
 #pragma unroll 1
-      for (int c = 0; c < 2; ++c) {
-        uint32_t r[32];
-        tmem_ld32(tmem + (lane_base << 16) + kAccCol + (NH == 2 ? g * 64 : 0) + 32 * c, r);
-        tmem_ld_wait();
-        reg_fence32(r);
+          for (int c = 0; c < 2; ++c) {
+            uint32_t r[32];
+            tmem_ld32(acc_addr + 32 * c, r);
+            tmem_ld_wait();
+            reg_fence32(r);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = __uint_as_float(r[j]) * inv_r;
-        __syncwarp();
+            for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = __uint_as_float(r[j]) * inv_r;
+            __syncwarp();
 #pragma unroll 8
-        for (int rr = 0; rr < 32; ++rr) dst[(size_t)rr * kD + 32 * c + lane] = stage[rr * 33 + lane];
-        if (sbf != nullptr) {   // one chunk per slab: this is S' itself, leave its bf16 image as well
-          __nv_bfloat16* bdst = sbf + (pidx * m + feat0) * kD + 32 * c;
+            for (int rr = 0; rr < 32; ++rr) dst[(size_t)rr * kD + 32 * c + lane] = stage[rr * 33 + lane];
+            if (sbf != nullptr) {   // one chunk per slab: this is S' itself, leave its bf16 image as well
+              __nv_bfloat16* bdst = sbf + (pidx * m + feat0) * kD + 32 * c;
 #pragma unroll 8
-          for (int rr = 0; rr < 32; rr += 2) {   // two rows per instruction, a pair of columns per lane
-            const int rw = rr + (lane >> 4), cc = 2 * (lane & 15);
-            *reinterpret_cast<uint32_t*>(bdst + (size_t)rw * kD + cc) = pack_bf16x2(stage[rw * 33 + cc], stage[rw * 33 + cc + 1]);
+              for (int rr = 0; rr < 32; rr += 2) {   // two rows per instruction, a pair of columns per lane
+                const int rw = rr + (lane >> 4), cc = 2 * (lane & 15);
+                *reinterpret_cast<uint32_t*>(bdst + (size_t)rw * kD + cc) =
+                    pack_bf16x2(stage[rw * 33 + cc], stage[rw * 33 + cc + 1]);
+              }
+            }
+            __syncwarp();
+          }
+        } else {
+          // More items follow and the rings already hold their tiles: every thread writes its own row
+          // (16-byte stores; half-used sectors, but the accumulators are free again sooner).
+          float* dst = spart + (pidx * m + feat0 + lane) * kD;
+#pragma unroll 1
+          for (int c = 0; c < 2; ++c) {
+            uint32_t r[32];
+            tmem_ld32(acc_addr + 32 * c, r);
+            tmem_ld_wait();
+            reg_fence32(r);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * inv_r);
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              *reinterpret_cast<uint4*>(dst + 32 * c + 4 * q) = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+            if (sbf != nullptr) {
+              __nv_bfloat16* bdst = sbf + (pidx * m + feat0 + lane) * kD + 32 * c;
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                *reinterpret_cast<uint4*>(bdst + 8 * q) =
+                    make_uint4(pack_bf16x2(__uint_as_float(r[8 * q]), __uint_as_float(r[8 * q + 1])),
+                               pack_bf16x2(__uint_as_float(r[8 * q + 2]), __uint_as_float(r[8 * q + 3])),
+                               pack_bf16x2(__uint_as_float(r[8 * q + 4]), __uint_as_float(r[8 * q + 5])),
+                               pack_bf16x2(__uint_as_float(r[8 * q + 6]), __uint_as_float(r[8 * q + 7])));
+            }
           }
         }
-        __syncwarp();
+        zpart[pidx * m + feat0 + lane] = zacc * inv_r;
       }
-      zpart[pidx * m + feat0 + lane] = zacc * inv_r;
+      // the accumulators may be overwritten by the next item
+      tc_fence_before_sync();
+      if (ok) warp_arrive(&bars->acc_free);
     }
   } else {
     reg_inc<kRegsAux>();
     const int ht = threadIdx.x - 32 * kAuxWarp0;
     float* hcoef = reinterpret_cast<float*>(smem + SL::hcoef);
-    haar_coef_init(hcoef, f + (size_t)slab * (L + 1), L, ht);
-    named_bar_sync(kBarCoef, 256);
     bool ok = true;
-    for (int b = 0; b < nblk; ++b)
-      ok = haar_step<kNXK>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
-                     ht, ok, abort_flag, status);
+    int gb0 = 0;                                      // blocks of the items before
+    for (int it = item0; it < items; it += item_step) {
+      const int slab = it / chunks, blk0 = (it % chunks) * chunk_blocks;
+      const int nblk = item_blocks(it, chunks, chunk_blocks, n);
+      named_bar_sync(kBarCoef, 256);                  // nobody reads the coefficients of the item before any more
+      haar_coef_init(hcoef, f + (size_t)slab * (L + 1), L, ht);
+      named_bar_sync(kBarCoef, 256);
+      for (int b = 0; b < nblk; ++b)
+        ok = haar_step<kNXK>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, gb0 + b,
+                             n - (blk0 + b) * kBlk, ht, ok, abort_flag, status);
+      gb0 += nblk;
+    }
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -665,20 +769,41 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
 // 128-byte swizzle.
 // Done by `nthr` threads numbered tid = 0 .. nthr - 1.
 __device__ __forceinline__ void load_szt_image(uint8_t* dst, const __nv_bfloat16* __restrict__ Sbf,
-                                               const float* __restrict__ z, int m, int tid, int nthr) {
-  for (int i = tid; i < m * (kD / 2); i += nthr) {   // two adjacent columns of one feature
-    const int f = i / (kD / 2), c = 2 * (i % (kD / 2));
-    const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(Sbf + (size_t)f * kD + c);
-    uint8_t* blk = dst + (f >> 6) * kSztBlockBytes + (f & 7) * 2;
-    *reinterpret_cast<__nv_bfloat16*>(blk + swz128(c, (f & 63) >> 3)) = v.x;
-    *reinterpret_cast<__nv_bfloat16*>(blk + swz128(c + 1, (f & 63) >> 3)) = v.y;
+                                               const float* __restrict__ z, int m, int tid, int nthr,
+                                               bool zero_rows) {
+  // 16-byte loads of eight columns of one feature, two in flight per thread, scattered to eight rows
+  const int chunks16 = m * (kD / 8);
+  for (int i0 = tid; i0 < chunks16; i0 += 2 * nthr) {
+    uint4 v[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int i = i0 + u * nthr;
+      if (i < chunks16) v[u] = reinterpret_cast<const uint4*>(Sbf)[i];
+    }
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int i = i0 + u * nthr;
+      if (i < chunks16) {
+        const int f = i >> 3, c0 = (i & 7) * 8;
+        uint8_t* blk = dst + (f >> 6) * kSztBlockBytes + (f & 7) * 2;
+        const uint32_t kc = (f & 63) >> 3;
+        const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          *reinterpret_cast<uint16_t*>(blk + swz128(c0 + 2 * j, kc)) = (uint16_t)(w[j] & 0xFFFFu);
+          *reinterpret_cast<uint16_t*>(blk + swz128(c0 + 2 * j + 1, kc)) = (uint16_t)(w[j] >> 16);
+        }
+      }
+    }
   }
   for (int f = tid; f < m; f += nthr)
     *reinterpret_cast<__nv_bfloat16*>(dst + (f >> 6) * kSztBlockBytes + swz128(64, (f & 63) >> 3) + (f & 7) * 2) =
         __float2bfloat16_rn(z[f]);
-  for (int i = tid; i < (m >> 6) * 15 * 8; i += nthr) {   // 16-byte chunks of rows 65-79
-    const int kb = i / 120, r = 65 + (i % 120) / 8, c = i & 7;
-    *reinterpret_cast<uint4*>(dst + kb * kSztBlockBytes + r * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+  if (zero_rows) {   // rows 65-79 never change: written once per CTA
+    for (int i = tid; i < (m >> 6) * 15 * 8; i += nthr) {   // 16-byte chunks of rows 65-79
+      const int kb = i / 120, r = 65 + (i % 120) / 8, c = i & 7;
+      *reinterpret_cast<uint4*>(dst + kb * kSztBlockBytes + r * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+    }
   }
 }
 
@@ -728,32 +853,34 @@ __device__ __forceinline__ void qside_build_simg(uint8_t* simg, const __nv_bfloa
   constexpr int m = NH * 128;
   griddep_wait();
   load_szt_image(simg, Sbf + (size_t)slab * m * kD, zg + (size_t)slab * m, m, threadIdx.x - 32 * kReluWarp0,
-                 32 * (kAuxWarp0Q - kReluWarp0));
+                 32 * (kAuxWarp0Q - kReluWarp0), true);
   fence_proxy_async_smem();
   warp_arrive(ready);
 }
 
-// grid (chunks, slabs), block 768.  TMEM: two buffers of 256 columns; tile t uses buffer t & 1 for its D1
+// grid (min(SMs, items)), block 768; the CTA walks its work items as on the key side (tiles, buffers and
+// barrier phases count on across items; the S' image and the filter coefficients are renewed when an item
+// begins: the image of the first item by the ReLU and epilogue warps together, later ones by the epilogue
+// warps once the last MMA2 of the item before has completed).
+// TMEM: two buffers of 256 columns; tile t uses buffer t & 1 for its D1
 // (128 tokens x m features, fp32), then for the packed bf16 features and the [N' | D'] accumulator (see
 // QTmem).  Per tile: MMA1 (warp 1) -> ReLU pass (warps 4-11, two warps per lane quarter that split the
 // feature columns) -> MMA2 (warp 3) -> epilogue (warps 12-15: drain the accumulator, which frees the buffer
 // for tile t + 2, scale by 1 / (D' + eps'), round to bf16 into one of two staging tiles, TMA store).
-template <int NH>
+template <int NH, bool kMulti>
 __global__ void __launch_bounds__(kThreadsQ, 1)
 k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
            const __grid_constant__ CUtensorMap map_w, const __nv_bfloat16* __restrict__ Sbf,
            const float* __restrict__ zg, const float* __restrict__ f, const float* __restrict__ beta, float eps,
-           float bw_floor, int n, int L, int chunk_blocks, int* __restrict__ status) {
+           float bw_floor, int n, int L, int chunk_blocks, int chunks, int items, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   using SL = QsideSmem<NH>;
   using TM = QTmem<NH>;
   QsideBars* bars = reinterpret_cast<QsideBars*>(smem + SL::bars);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int chunk = blockIdx.x, slab = blockIdx.y;
-  const int blk0 = chunk * chunk_blocks;
-  const int nblk = min(chunk_blocks, (n + kBlk - 1) / kBlk - blk0);
-  const int ntiles = nblk * 2;
+  const int item0 = blockIdx.y * gridDim.x + blockIdx.x, item_step = kMulti ? (int)gridDim.x : (1 << 30);   // as on the key side
+  if (!kMulti) items = item0 + 1;
   constexpr int m = NH * 128;
   constexpr uint32_t kIdesc1Q = make_idesc_bf16(128, m, false, false);   // Q_F tile x all features
 
@@ -770,6 +897,7 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       mbar_init(&bars->buf_free[b], 4);
     }
     mbar_init(&bars->simg_ready, kAuxWarp0Q - kReluWarp0);
+    mbar_init(&bars->simg_next, kAuxWarp0Q - kEpiWarp0Q);
     mbar_init(&bars->w_full, 1);
     bars->abort_flag = 0;
     fence_mbar_init();
@@ -792,13 +920,19 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
   if (warp < kReluWarp0) {
     reg_dec<kRegsCtlQ>();
     if (warp == kWarpTma && lane == 0) {
-      int issued = 0;
-      for (int b = 0; b < ntiles; ++b) {   // b counts 128-token tiles here
-        const int s = b % kNXQ;
-        if (!mbar_wait(&bars->x_empty[s], ((b / kNXQ) & 1) ^ 1, abort_flag, status, kErrProducer)) break;
-        mbar_arrive_expect_tx(&bars->x_full[s], kTileBytes);
-        tma_load_3d(smem + SL::x + s * kTileBytes, &map_q, 0, blk0 * kBlk + b * kTile, slab, &bars->x_full[s]);
-        issued = b + 1;
+      int issued = 0;   // tiles sent so far, over all items (slot and phase of the ring)
+      bool ok = true;
+      for (int it = item0; it < items && ok; it += item_step) {
+        const int slab = it / chunks, row0 = (it % chunks) * chunk_blocks * kBlk;
+        const int ntl = 2 * item_blocks(it, chunks, chunk_blocks, n);
+        for (int b = 0; b < ntl; ++b) {   // b counts 128-token tiles here
+          const int s = issued % kNXQ;
+          ok = mbar_wait(&bars->x_empty[s], ((issued / kNXQ) & 1) ^ 1, abort_flag, status, kErrProducer);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&bars->x_full[s], kTileBytes);
+          tma_load_3d(smem + SL::x + s * kTileBytes, &map_q, 0, row0 + b * kTile, slab, &bars->x_full[s]);
+          ++issued;
+        }
       }
       if (*abort_flag != 0) {
         for (int b = max(0, issued - kNXQ); b < issued; ++b) mbar_wait_drain(&bars->x_full[b % kNXQ], (b / kNXQ) & 1);
@@ -814,7 +948,9 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       uint32_t xs = 0, fs = 0, fpar = 0;
       int t = 0;
       bool ok = mbar_wait(&bars->w_full, 0, abort_flag, status, kErrMma);
-      for (int b = 0; b < nblk && ok; ++b) {
+      int blocks_all = 0;   // blocks of all items of this CTA
+      for (int it = item0; it < items; it += item_step) blocks_all += item_blocks(it, chunks, chunk_blocks, n);
+      for (int b = 0; b < blocks_all && ok; ++b) {
         ok = mbar_wait(&bars->xf_ready[fs], fpar, abort_flag, status, kErrMma);
         if (!ok) break;
         tc_fence_after_sync();
@@ -842,28 +978,37 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       // MMA2 of every tile: [N' | D'] = Phi (bf16 pairs in the tile's buffer) * [S' | z' | 0].
       const uint32_t hi = smem_desc_hi(1024);
       const uint32_t s_lo = smem_desc_lo(smem_u32(smem + SL::simg), 16);
-      bool ok = mbar_wait(&bars->simg_ready, 0, abort_flag, status, kErrMma);   // the [S' | z' | 0]^T image is in place
-      for (int t = 0; t < ntiles && ok; ++t) {
-        const int buf = t & 1;
-        ok = mbar_wait(&bars->phi_ready[buf], (t >> 1) & 1, abort_flag, status, kErrMma);
-        if (!ok) break;
-        tc_fence_after_sync();
-        const uint32_t base = tmem + buf * kQBufCols;
+      bool ok = true;
+      int t = 0, ic = 0;   // tiles and items so far
+      for (int it = item0; it < items && ok; it += item_step, ++ic) {
+        const int ntl = 2 * item_blocks(it, chunks, chunk_blocks, n);
+        // the [S' | z' | 0]^T image of this item's slab is in place
+        ok = ic == 0 ? mbar_wait(&bars->simg_ready, 0, abort_flag, status, kErrMma)
+                     : mbar_wait(&bars->simg_next, (ic - 1) & 1, abort_flag, status, kErrMma);
+        for (int tt = 0; tt < ntl && ok; ++tt, ++t) {
+          const int buf = t & 1;
+          ok = mbar_wait(&bars->phi_ready[buf], (t >> 1) & 1, abort_flag, status, kErrMma);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t base = tmem + buf * kQBufCols;
 #pragma unroll
-        for (int k = 0; k < 8 * NH; ++k) {   // K block k / 4 of the image, 32 bytes per step of 16 features inside it
-          const uint32_t b_lo = s_lo + (k >> 2) * (kSztBlockBytes >> 4) + 2 * (k & 3);
-          mma_ts(base + TM::kAcc, base + TM::phi_col(k), smem_desc_join(b_lo, hi), kIdesc2Q, k > 0 ? 1u : 0u);
+          for (int k = 0; k < 8 * NH; ++k) {   // K block k / 4 of the image, 32 bytes per step of 16 features inside it
+            const uint32_t b_lo = s_lo + (k >> 2) * (kSztBlockBytes >> 4) + 2 * (k & 3);
+            mma_ts(base + TM::kAcc, base + TM::phi_col(k), smem_desc_join(b_lo, hi), kIdesc2Q, k > 0 ? 1u : 0u);
+          }
+          mma_commit(&bars->d2_full[buf]);
         }
-        mma_commit(&bars->d2_full[buf]);
       }
     }
   } else if (warp < kEpiWarp0Q) {
     reg_dec<kRegsReluQ>();
-    qside_build_simg<NH>(smem + SL::simg, Sbf, zg, slab, &bars->simg_ready);
+    qside_build_simg<NH>(smem + SL::simg, Sbf, zg, item0 / chunks, &bars->simg_ready);
     const int g = (warp - kReluWarp0) >> 2;
     const uint32_t lane_base = 32u * (warp & 3);
     bool ok = true;
-    for (int t = 0; t < ntiles; ++t) {
+    int tiles_all = 0;   // tiles of all items of this CTA
+    for (int it = item0; it < items; it += item_step) tiles_all += 2 * item_blocks(it, chunks, chunk_blocks, n);
+    for (int t = 0; t < tiles_all; ++t) {
       const int buf = t & 1;
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d1_full[buf], (t >> 1) & 1, abort_flag, status, kErrRelu));
       if (ok) {
@@ -879,14 +1024,28 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     }
   } else if (warp < kAuxWarp0Q) {
     reg_inc<kRegsEpiQ>();
-    qside_build_simg<NH>(smem + SL::simg, Sbf, zg, slab, &bars->simg_ready);
+    qside_build_simg<NH>(smem + SL::simg, Sbf, zg, item0 / chunks, &bars->simg_ready);
     const int et = threadIdx.x - 32 * kEpiWarp0Q;     // 0..127 = token row of the tile = TMEM lane
     const uint32_t lane_base = 32u * (warp & 3);
     const float bw = fmaxf(beta[0], bw_floor);
+    bool ok = true;
+    int t = 0, ic = 0;   // tiles and items so far
+    for (int it = item0; it < items; it += item_step, ++ic) {
+    const int slab = it / chunks, blk0 = (it % chunks) * chunk_blocks;
+    const int ntl = 2 * item_blocks(it, chunks, chunk_blocks, n);
+    if (ic > 0) {
+      // every MMA2 of the item before has completed (its last accumulator was drained above): the image of
+      // this item's slab takes the place of the old one
+      if (ok) {
+        if (slab != (it - item_step) / chunks)
+          load_szt_image(smem + SL::simg, Sbf + (size_t)slab * m * kD, zg + (size_t)slab * m, m, et, 128, false);
+        fence_proxy_async_smem();
+        warp_arrive(&bars->simg_next);
+      }
+    }
     // the filter stage left Q_F, and with it N' and D', scaled by r (see haar_block_inplace): eps' follows
     const float epsp = eps * (float)m * bw * bw * haar_scale(f[(size_t)slab * (L + 1)]);
-    bool ok = true;
-    for (int t = 0; t < ntiles; ++t) {
+    for (int tt = 0; tt < ntl; ++tt, ++t) {
       const int buf = t & 1;
       const uint32_t base = tmem + (lane_base << 16) + buf * kQBufCols + TM::kAcc;
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->d2_full[buf], (t >> 1) & 1, abort_flag, status, kErrEpilogue));
@@ -930,23 +1089,31 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
         fence_proxy_async_smem();
       }
       named_bar_sync(kBarOut0, 128);
-      const int row0 = blk0 * kBlk + t * kTile;
+      const int row0 = blk0 * kBlk + tt * kTile;
       if (et == 0 && ok && row0 < n) {   // rows past n are clipped by the store
         tma_store_3d(&map_o, ost, 0, row0, slab);
         bulk_commit_group();
       }
+    }
     }
     if (et == 0) bulk_wait_group0();
   } else {
     reg_inc<kRegsAux>();
     const int ht = threadIdx.x - 32 * kAuxWarp0Q;
     float* hcoef = reinterpret_cast<float*>(smem + SL::hcoef);
-    haar_coef_init(hcoef, f + (size_t)slab * (L + 1), L, ht);
-    named_bar_sync(kBarCoef, 256);
     bool ok = true;
-    for (int b = 0; b < nblk; ++b)
-      ok = haar_step<kNXQ>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, b, n - blk0 * kBlk,
-                     ht, ok, abort_flag, status);
+    int gb0 = 0;                                      // blocks of the items before
+    for (int it = item0; it < items; it += item_step) {
+      const int slab = it / chunks, blk0 = (it % chunks) * chunk_blocks;
+      const int nblk = item_blocks(it, chunks, chunk_blocks, n);
+      named_bar_sync(kBarCoef, 256);                  // nobody reads the coefficients of the item before any more
+      haar_coef_init(hcoef, f + (size_t)slab * (L + 1), L, ht);
+      named_bar_sync(kBarCoef, 256);
+      for (int b = 0; b < nblk; ++b)
+        ok = haar_step<kNXQ>(smem + SL::x, bars, reinterpret_cast<float*>(smem + SL::xch), hcoef, L > 5, gb0 + b,
+                             n - (blk0 + b) * kBlk, ht, ok, abort_flag, status);
+      gb0 += nblk;
+    }
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -1020,19 +1187,26 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
   if ((err = make_tile_map(V, p.slabs, p.cfg.seq_len, kTile, &map_v)) != cudaSuccess) return err;
   CUtensorMap map_w;   // W^T (m x 64) as one slab of m rows
   if ((err = make_tile_map(w.Wt, 1, p.cfg.features, kTile, &map_w)) != cudaSuccess) return err;
-  dim3 grid(p.tchunks, p.slabs);
+  const int items = p.tchunks * p.slabs;   // (slab, chunk) pairs; one CTA per SM walks them
+  dim3 grid(items < p.sms ? items : p.sms);
   // With one chunk per slab the "partial" is the result: the kernel writes S', z' and the bf16 image
   // itself and no reduction follows.
   const bool single = p.tchunks == 1;
   float* sp = single ? w.S : w.spart;
   float* zp = single ? w.z : w.zpart;
   __nv_bfloat16* sb = single ? w.Sbf : nullptr;
+  const bool multi = items > (int)grid.x;   // some CTA walks more than one item
+  // One item per CTA: a (chunks, slabs) grid.  The same CTAs as a one-dimensional grid measured 6 us more per
+  // config-4 forward (192 against 186 us), so the shape is kept where it has a choice.
+  if (!multi) grid = dim3(p.tchunks, p.slabs);
+  auto launch = [&](auto kernel, size_t smem_bytes) {
+    return launch_pdl(kernel, grid, kThreads, smem_bytes, st, map_k, map_v, map_w, (const float*)w.f, sp, zp, sb,
+                      p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, p.tchunks, items, w.status);
+  };
   if (p.cfg.features == 256)
-    err = launch_pdl(k_tc_kside<2>, grid, kThreads, KsideSmem<2>::total, st, map_k, map_v, map_w,
-                     (const float*)w.f, sp, zp, sb, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
+    err = multi ? launch(k_tc_kside<2, true>, KsideSmem<2>::total) : launch(k_tc_kside<2, false>, KsideSmem<2>::total);
   else
-    err = launch_pdl(k_tc_kside<1>, grid, kThreads, KsideSmem<1>::total, st, map_k, map_v, map_w,
-                     (const float*)w.f, sp, zp, sb, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
+    err = multi ? launch(k_tc_kside<1, true>, KsideSmem<1>::total) : launch(k_tc_kside<1, false>, KsideSmem<1>::total);
   *launches += 1;
   return err != cudaSuccess ? err : cudaGetLastError();
 }
@@ -1047,15 +1221,19 @@ cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const flo
   // that kernel where it first needs its results)
   CUtensorMap map_w;
   if ((err = make_tile_map(w.Wt, 1, p.cfg.features, kTile, &map_w)) != cudaSuccess) return err;
-  dim3 grid(p.tchunks, p.slabs);
+  const int items = p.tchunks * p.slabs;
+  dim3 grid(items < p.sms ? items : p.sms);
+  const bool multi = items > (int)grid.x;
+  if (!multi) grid = dim3(p.tchunks, p.slabs);   // see launch_tc_kside
+  auto launch = [&](auto kernel, size_t smem_bytes) {
+    return launch_pdl(kernel, grid, kThreadsQ, smem_bytes, st, map_q, map_o, map_w, (const __nv_bfloat16*)w.Sbf,
+                      (const float*)w.z, (const float*)w.f, beta, p.cfg.eps, p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels,
+                      p.tchunk_blocks, p.tchunks, items, w.status);
+  };
   if (p.cfg.features == 256)
-    err = launch_pdl(k_tc_qside<2>, grid, kThreadsQ, QsideSmem<2>::total, st, map_q, map_o, map_w,
-                     (const __nv_bfloat16*)w.Sbf, (const float*)w.z, (const float*)w.f, beta, p.cfg.eps,
-                     p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
+    err = multi ? launch(k_tc_qside<2, true>, QsideSmem<2>::total) : launch(k_tc_qside<2, false>, QsideSmem<2>::total);
   else
-    err = launch_pdl(k_tc_qside<1>, grid, kThreadsQ, QsideSmem<1>::total, st, map_q, map_o, map_w,
-                     (const __nv_bfloat16*)w.Sbf, (const float*)w.z, (const float*)w.f, beta, p.cfg.eps,
-                     p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, w.status);
+    err = multi ? launch(k_tc_qside<1, true>, QsideSmem<1>::total) : launch(k_tc_qside<1, false>, QsideSmem<1>::total);
   *launches += 1;
   return err != cudaSuccess ? err : cudaGetLastError();
 }
