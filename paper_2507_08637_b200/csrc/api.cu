@@ -109,6 +109,7 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   p->off_z = take(sizeof(float) * slabs * m);
   p->off_Sbf = take(sizeof(__nv_bfloat16) * slabs * m * kD);
   p->off_Wt = take(sizeof(__nv_bfloat16) * (size_t)m * kD);
+  p->off_Simg = take(p->use_tc ? slabs * simg_bytes(m) : 0);
   const size_t slab_elems = slabs * (size_t)n * kD;
   const bool need_xf = !p->use_tc;   // the tensor-core kernels filter on chip (forward) or read bf16 planes (backward)
   p->off_QF = take(need_xf ? sizeof(float) * slab_elems : 0);
@@ -147,6 +148,7 @@ Ws resolve(const Plan& p, void* workspace) {
   w.z = reinterpret_cast<float*>(b + p.off_z);
   w.Sbf = reinterpret_cast<__nv_bfloat16*>(b + p.off_Sbf);
   w.Wt = reinterpret_cast<__nv_bfloat16*>(b + p.off_Wt);
+  w.Simg = reinterpret_cast<uint8_t*>(b + p.off_Simg);
   w.QF = reinterpret_cast<float*>(b + p.off_QF);
   w.KF = reinterpret_cast<float*>(b + p.off_KF);
   w.dS = reinterpret_cast<float*>(b + p.off_dS);
@@ -292,14 +294,14 @@ wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const v
     WERSA_STEP(0, "tc_kside", launch_tc_kside(p, w, K, V, st, &launches));
     if (p.tchunks > 1)   // with one chunk per slab the key-side kernel has written S', z' and the image itself
       WERSA_STEP(0, "reduce_partials",
-                 launch_reduce_partials(p, w.spart, w.zpart, p.tchunks, w.S, w.z, w.Sbf, st, &launches));
+                 launch_reduce_partials(p, w.spart, w.zpart, p.tchunks, w.S, w.z, w.Sbf, w.Simg, st, &launches));
     WERSA_STEP(0, "tc_qside", launch_tc_qside(p, w, Q, beta, O, st, &launches));
   } else {
     WERSA_STEP(0, "haar_filter_q", launch_haar_filter(p, Q, kind, w.f, w.QF, 0, st, &launches));
     WERSA_STEP(0, "haar_filter_k", launch_haar_filter(p, K, kind, w.f, w.KF, 0, st, &launches));
     WERSA_STEP(0, "simt_kside", launch_simt_kside(p, w, V, W, st, &launches));
     WERSA_STEP(0, "reduce_partials",
-               launch_reduce_partials(p, w.spart, w.zpart, p.schunks, w.S, w.z, nullptr, st, &launches));
+               launch_reduce_partials(p, w.spart, w.zpart, p.schunks, w.S, w.z, nullptr, nullptr, st, &launches));
     WERSA_STEP(0, "simt_qside", launch_simt_qside(p, w, W, beta, O, st, &launches));
   }
   ctx->launches_fwd = launches;
@@ -361,7 +363,7 @@ wersa_status wersa_backward(wersa_ctx* ctx, const void* Q, const void* K, const 
     WERSA_STEP(1, "simt_bwd_qside", launch_simt_bwd_qside(p, w, W, beta, dO, st, &launches));
   }
   WERSA_STEP(1, "reduce_partials",
-             launch_reduce_partials(p, w.spart, w.zpart, bwd_chunks, w.dS, w.dz, p.use_tc ? w.dSbf : nullptr, st,
+             launch_reduce_partials(p, w.spart, w.zpart, bwd_chunks, w.dS, w.dz, p.use_tc ? w.dSbf : nullptr, nullptr, st,
                                     &launches));
   if (p.use_tc)
     WERSA_STEP(1, "tc_bwd_kside", launch_tc_bwd_kside(p, w, w.KF3, V, dV, st, &launches));

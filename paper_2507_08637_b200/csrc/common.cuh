@@ -39,7 +39,7 @@ struct Plan {
   // workspace offsets (bytes)
   size_t off_status, off_counters, status_bytes, off_qpart, off_qbar, off_sg, off_f, off_spart, off_zpart, off_S, off_z,
       off_Sbf, off_Wt, off_dS, off_dz, off_sumdD, off_bands, off_dqbar, off_QF, off_KF, off_dQF,
-      off_dKF, off_dSbf, off_KF3, off_QF3, off_Slo, total;
+      off_dKF, off_dSbf, off_KF3, off_QF3, off_Slo, off_Simg, total;
   int part_chunks;    // max(schunks, tchunks): leading extent of the partial buffers
 };
 
@@ -51,6 +51,7 @@ struct Ws {   // resolved workspace pointers
   int* counters;   // arrival counters (slabs + batch + slabs ints), zero between launches
   float *qpart, *qbar, *sg, *f, *spart, *zpart, *S, *z, *dS, *dz, *sumdD, *bands, *dqbar;
   __nv_bfloat16 *Sbf, *Wt, *dSbf, *KF3, *QF3, *Slo;   // Slo = bf16(S' - bf16(S')), built by the backward
+  uint8_t* Simg;   // [S' | z' | 0]^T operand images of the query-side kernel, one per slab (see simg_offset)
   float *QF, *KF, *dQF, *dKF;
 };
 Ws resolve(const Plan& p, void* workspace);
@@ -95,7 +96,7 @@ cudaError_t launch_simt_kside(const Plan& p, const Ws& w, const void* V, const v
                               cudaStream_t st, int* launches);
 // S = sum_chunks spart, z = sum_chunks zpart in chunk order (also used for dS, dz).
 cudaError_t launch_reduce_partials(const Plan& p, const float* spart, const float* zpart, int chunks,
-                                   float* S, float* z, __nv_bfloat16* Sbf, cudaStream_t st,
+                                   float* S, float* z, __nv_bfloat16* Sbf, uint8_t* Simg, cudaStream_t st,
                                    int* launches);
 cudaError_t launch_simt_qside(const Plan& p, const Ws& w, const void* W, const float* beta, void* O,
                               cudaStream_t st, int* launches);
@@ -126,6 +127,20 @@ cudaError_t launch_tc_bwd_kside(const Plan& p, const Ws& w, const void* KF3, con
 // One CTA whose bounded wait runs out after limit_ns: sets the status word; observed[0] = abort flag,
 // observed[1], observed[2] = whether the two roles' waits succeeded (both must read 0).
 cudaError_t launch_selftest_wait(const Ws& w, unsigned long long limit_ns, int* observed, cudaStream_t st);
+
+// ---- operand image of the query-side second contraction --------------------------------------
+// The query-side kernel multiplies the features by [S' | z' | 0] (m x 80) as a K-major bf16 operand: per
+// slab, m / 64 blocks of 80 rows x 128 bytes -- rows 0-63 are the columns of S', row 64 is z', rows 65-79
+// are zero, and a row holds 64 consecutive features in the 128-byte swizzle the tensor core reads (16-byte
+// chunk j of row r sits at chunk j ^ (r & 7)).  Whoever produces S' and z' leaves this image in global
+// memory in exactly that byte order, so that the kernel fetches it with one bulk copy.
+constexpr int kSimgRows = 80;
+constexpr size_t kSimgBlockBytes = kSimgRows * 128;
+__host__ __device__ inline size_t simg_bytes(int m) { return (size_t)(m / 64) * kSimgBlockBytes; }
+// byte offset of (feature f, row r) inside a slab's image
+__device__ __forceinline__ size_t simg_offset(int f, int r) {
+  return (size_t)(f >> 6) * kSimgBlockBytes + (size_t)r * 128 + (size_t)((((f & 63) >> 3) ^ (r & 7)) << 4) + (f & 7) * 2;
+}
 
 // ---- device helpers ------------------------------------------------------------------------
 __device__ __forceinline__ float to_f32(float x) { return x; }

@@ -440,26 +440,44 @@ __device__ __forceinline__ float sum_chunks4(const float* __restrict__ p, size_t
   return (a0 + a1) + (a2 + a3);
 }
 
-__global__ void __launch_bounds__(256) k_reduce_partials(const float* __restrict__ spart,
+// grid (m / 8, slabs), block 512: one CTA adds the partials of eight consecutive features (512 elements of
+// S', one per thread, and their eight entries of z') in chunk order.  With Sbf it also leaves the bf16 copy
+// of S', with Simg the operand image of the query-side kernel (see simg_offset): eight consecutive features
+// are one 16-byte chunk of an image row, so the 80 rows of the CTA's part go out as one 16-byte store each.
+__global__ void __launch_bounds__(512) k_reduce_partials(const float* __restrict__ spart,
                                                          const float* __restrict__ zpart, int chunks, int m,
                                                          float* __restrict__ S, float* __restrict__ z,
-                                                         __nv_bfloat16* __restrict__ Sbf) {
+                                                         __nv_bfloat16* __restrict__ Sbf, uint8_t* __restrict__ Simg) {
   // Programmatic dependent launch: the kernel after this one may be staged now (it waits for this grid
-  // before it reads S, z, Sbf), and this kernel may itself have been staged early: the partials are
+  // before it reads S, z, Sbf, Simg), and this kernel may itself have been staged early: the partials are
   // complete once the kernel before it has finished.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  const int slab = blockIdx.y;
-  const int i = blockIdx.x * 256 + threadIdx.x;
+  __shared__ __align__(16) __nv_bfloat16 tile[kSimgRows][8];   // [image row][feature - f0]
+  const int slab = blockIdx.y, f0 = blockIdx.x * 8;
   const int ns = m * kD;
-  if (i < ns) {
+  {
+    const int e = threadIdx.x;                    // element of the CTA's 8 x 64 part
+    const int i = f0 * kD + e;                    // element of S' (feature i / 64, column i % 64)
     const float s = sum_chunks4(spart + (size_t)slab * chunks * ns + i, ns, chunks);
     S[(size_t)slab * ns + i] = s;
-    if (Sbf != nullptr) Sbf[(size_t)slab * ns + i] = __float2bfloat16_rn(s);
-  } else if (i < ns + m) {
-    const int r = i - ns;
-    z[(size_t)slab * m + r] = sum_chunks4(zpart + (size_t)slab * chunks * m + r, m, chunks);
+    const __nv_bfloat16 sb = __float2bfloat16_rn(s);
+    if (Sbf != nullptr) Sbf[(size_t)slab * ns + i] = sb;
+    tile[e & (kD - 1)][e >> 6] = sb;
   }
+  if (threadIdx.x < 8) {
+    const int r = f0 + threadIdx.x;
+    const float zr = sum_chunks4(zpart + (size_t)slab * chunks * m + r, m, chunks);
+    z[(size_t)slab * m + r] = zr;
+    tile[kD][threadIdx.x] = __float2bfloat16_rn(zr);   // z' is row 64 of the image
+  } else if (threadIdx.x < 8 * (kSimgRows - kD)) {
+    tile[kD + (threadIdx.x >> 3)][threadIdx.x & 7] = __float2bfloat16_rn(0.f);   // rows 65-79 are zero
+  }
+  if (Simg == nullptr) return;
+  __syncthreads();
+  if (threadIdx.x < kSimgRows)
+    *reinterpret_cast<uint4*>(Simg + (size_t)slab * simg_bytes(m) + simg_offset(f0, threadIdx.x)) =
+        *reinterpret_cast<const uint4*>(&tile[threadIdx.x][0]);
 }
 
 template <typename K>
@@ -500,19 +518,19 @@ cudaError_t launch_simt_kside(const Plan& p, const Ws& w, const void* V, const v
 }
 
 cudaError_t launch_reduce_partials(const Plan& p, const float* spart, const float* zpart, int chunks, float* S,
-                                   float* z, __nv_bfloat16* Sbf, cudaStream_t st, int* launches) {
+                                   float* z, __nv_bfloat16* Sbf, uint8_t* Simg, cudaStream_t st, int* launches) {
   const int m = p.cfg.features;
-  dim3 grid((m * kD + m + 255) / 256, p.slabs);
+  dim3 grid(m / 8, p.slabs);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
-  cfg.blockDim = dim3(256);
+  cfg.blockDim = dim3(512);
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const cudaError_t err = cudaLaunchKernelEx(&cfg, k_reduce_partials, spart, zpart, chunks, m, S, z, Sbf);
+  const cudaError_t err = cudaLaunchKernelEx(&cfg, k_reduce_partials, spart, zpart, chunks, m, S, z, Sbf, Simg);
   *launches += 1;
   return err != cudaSuccess ? err : cudaGetLastError();
 }

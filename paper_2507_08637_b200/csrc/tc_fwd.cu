@@ -116,7 +116,11 @@ template <int NH> struct KsideSmem {
 template <int NH> struct QsideSmem {
   static constexpr uint32_t wt = 0;
   static constexpr uint32_t simg = wt + NH * kTileBytes;          // 2 NH K blocks of [S' | z' | 0]^T
-  static constexpr uint32_t x = simg + 2 * NH * kSztBlockBytes;
+  static constexpr uint32_t simg_bytes = 2 * NH * kSztBlockBytes;
+  // with m = 128 there is room for a second image: a CTA that walks several items builds the next item's
+  // image while the current one is in use
+  static constexpr bool two_images = NH == 1;
+  static constexpr uint32_t x = simg + (two_images ? 2 : 1) * simg_bytes;
   static constexpr uint32_t ost = x + kNXQ * kTileBytes;           // 2 output staging tiles
   static constexpr uint32_t xch = ost + 2 * kTileBytes;          // 2 x 8 x 64 floats
   static constexpr uint32_t hcoef = xch + 4096;                  // kHaarCoefs floats
@@ -421,8 +425,8 @@ template <int NH, bool kMulti>
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
            const __grid_constant__ CUtensorMap map_w, const float* __restrict__ f, float* __restrict__ spart,
-           float* __restrict__ zpart, __nv_bfloat16* __restrict__ sbf, int n, int L, int chunk_blocks, int chunks,
-           int items, int* __restrict__ status) {
+           float* __restrict__ zpart, __nv_bfloat16* __restrict__ sbf, uint8_t* __restrict__ simg_out, int n, int L,
+           int chunk_blocks, int chunks, int items, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   using SL = KsideSmem<NH>;
@@ -687,6 +691,13 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
             reg_fence32(r);
 #pragma unroll
             for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = __uint_as_float(r[j]) * inv_r;
+            if (sbf != nullptr) {   // ... and the operand image of the query side (features along a row)
+              uint8_t* img = simg_out + pidx * simg_bytes(m);
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                *reinterpret_cast<__nv_bfloat16*>(img + simg_offset(feat0 + lane, 32 * c + j)) =
+                    __float2bfloat16_rn(__uint_as_float(r[j]) * inv_r);
+            }
             __syncwarp();
 #pragma unroll 8
             for (int rr = 0; rr < 32; ++rr) dst[(size_t)rr * kD + 32 * c + lane] = stage[rr * 33 + lane];
@@ -717,6 +728,11 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
             for (int q = 0; q < 8; ++q)
               *reinterpret_cast<uint4*>(dst + 32 * c + 4 * q) = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
             if (sbf != nullptr) {
+              uint8_t* img = simg_out + pidx * simg_bytes(m);
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                *reinterpret_cast<__nv_bfloat16*>(img + simg_offset(feat0 + lane, 32 * c + j)) =
+                    __float2bfloat16_rn(__uint_as_float(r[j]));
               __nv_bfloat16* bdst = sbf + (pidx * m + feat0 + lane) * kD + 32 * c;
 #pragma unroll
               for (int q = 0; q < 4; ++q)
@@ -729,6 +745,13 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
           }
         }
         zpart[pidx * m + feat0 + lane] = zacc * inv_r;
+        if (sbf != nullptr) {   // z' is row 64 of the image, rows 65-79 are zero
+          uint8_t* img = simg_out + pidx * simg_bytes(m);
+          *reinterpret_cast<__nv_bfloat16*>(img + simg_offset(feat0 + lane, kD)) = __float2bfloat16_rn(zacc * inv_r);
+#pragma unroll
+          for (int row = kD + 1; row < kSimgRows; ++row)
+            *reinterpret_cast<uint16_t*>(img + simg_offset(feat0 + lane, row)) = 0;
+        }
       }
       // the accumulators may be overwritten by the next item
       tc_fence_before_sync();
@@ -764,48 +787,9 @@ k_tc_kside(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
 // The denominator rides on the tensor core: the B operand of MMA2 is the K-major image of
 // [S' | z' | 0]^T (80 rows of m features), so that column 64 of the accumulator is D' = Phi z'.
 //
-// Builds that image in shared memory from the bf16 S' (m x 64, row-major) and the fp32 z' of the slab:
-// 64-feature K blocks of 80 rows x 128 bytes (rows 0-63 = columns of S', row 64 = z', rows 65-79 = 0),
-// 128-byte swizzle.
-// Done by `nthr` threads numbered tid = 0 .. nthr - 1.
-__device__ __forceinline__ void load_szt_image(uint8_t* dst, const __nv_bfloat16* __restrict__ Sbf,
-                                               const float* __restrict__ z, int m, int tid, int nthr,
-                                               bool zero_rows) {
-  // 16-byte loads of eight columns of one feature, two in flight per thread, scattered to eight rows
-  const int chunks16 = m * (kD / 8);
-  for (int i0 = tid; i0 < chunks16; i0 += 2 * nthr) {
-    uint4 v[2];
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const int i = i0 + u * nthr;
-      if (i < chunks16) v[u] = reinterpret_cast<const uint4*>(Sbf)[i];
-    }
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const int i = i0 + u * nthr;
-      if (i < chunks16) {
-        const int f = i >> 3, c0 = (i & 7) * 8;
-        uint8_t* blk = dst + (f >> 6) * kSztBlockBytes + (f & 7) * 2;
-        const uint32_t kc = (f & 63) >> 3;
-        const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          *reinterpret_cast<uint16_t*>(blk + swz128(c0 + 2 * j, kc)) = (uint16_t)(w[j] & 0xFFFFu);
-          *reinterpret_cast<uint16_t*>(blk + swz128(c0 + 2 * j + 1, kc)) = (uint16_t)(w[j] >> 16);
-        }
-      }
-    }
-  }
-  for (int f = tid; f < m; f += nthr)
-    *reinterpret_cast<__nv_bfloat16*>(dst + (f >> 6) * kSztBlockBytes + swz128(64, (f & 63) >> 3) + (f & 7) * 2) =
-        __float2bfloat16_rn(z[f]);
-  if (zero_rows) {   // rows 65-79 never change: written once per CTA
-    for (int i = tid; i < (m >> 6) * 15 * 8; i += nthr) {   // 16-byte chunks of rows 65-79
-      const int kb = i / 120, r = 65 + (i % 120) / 8, c = i & 7;
-      *reinterpret_cast<uint4*>(dst + kb * kSztBlockBytes + r * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
-    }
-  }
-}
+// The image comes from global memory, where the kernel that produced S' and z' left it in the byte order of
+// the shared-memory operand (simg_offset): 64-feature K blocks of 80 rows x 128 bytes (rows 0-63 = columns of
+// S', row 64 = z', rows 65-79 = 0), 128-byte swizzle.  One bulk copy per work item fetches it.
 
 // ReLU pass in 16-column steps (a smaller register footprint than relu_unit): fp32 TMEM columns -> bf16
 // pairs in half as many columns.
@@ -844,24 +828,10 @@ __device__ __forceinline__ void relu_span(uint32_t in, uint32_t out) {
   tmem_st_wait();
 }
 
-// The ReLU and epilogue warps (idle while the pipeline fills) build the S' image: S' and z' come from
-// the kernel before this one in the stream, which may still be running (programmatic dependent
-// launch), everything else this kernel reads was complete before that kernel started.
-template <int NH>
-__device__ __forceinline__ void qside_build_simg(uint8_t* simg, const __nv_bfloat16* __restrict__ Sbf,
-                                                 const float* __restrict__ zg, int slab, uint64_t* ready) {
-  constexpr int m = NH * 128;
-  griddep_wait();
-  load_szt_image(simg, Sbf + (size_t)slab * m * kD, zg + (size_t)slab * m, m, threadIdx.x - 32 * kReluWarp0,
-                 32 * (kAuxWarp0Q - kReluWarp0), true);
-  fence_proxy_async_smem();
-  warp_arrive(ready);
-}
-
 // grid (min(SMs, items)), block 768; the CTA walks its work items as on the key side (tiles, buffers and
 // barrier phases count on across items; the S' image and the filter coefficients are renewed when an item
-// begins: the image of the first item by the ReLU and epilogue warps together, later ones by the epilogue
-// warps once the last MMA2 of the item before has completed).
+// begins: one thread of the epilogue warps sends the bulk copy of an item's image once the last MMA2 that
+// reads the buffer it goes to has completed).
 // TMEM: two buffers of 256 columns; tile t uses buffer t & 1 for its D1
 // (128 tokens x m features, fp32), then for the packed bf16 features and the [N' | D'] accumulator (see
 // QTmem).  Per tile: MMA1 (warp 1) -> ReLU pass (warps 4-11, two warps per lane quarter that split the
@@ -870,8 +840,8 @@ __device__ __forceinline__ void qside_build_simg(uint8_t* simg, const __nv_bfloa
 template <int NH, bool kMulti>
 __global__ void __launch_bounds__(kThreadsQ, 1)
 k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
-           const __grid_constant__ CUtensorMap map_w, const __nv_bfloat16* __restrict__ Sbf,
-           const float* __restrict__ zg, const float* __restrict__ f, const float* __restrict__ beta, float eps,
+           const __grid_constant__ CUtensorMap map_w, const uint8_t* __restrict__ simg_g,
+           const float* __restrict__ f, const float* __restrict__ beta, float eps,
            float bw_floor, int n, int L, int chunk_blocks, int chunks, int items, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -896,8 +866,8 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       mbar_init(&bars->d2_full[b], 1);
       mbar_init(&bars->buf_free[b], 4);
     }
-    mbar_init(&bars->simg_ready, kAuxWarp0Q - kReluWarp0);
-    mbar_init(&bars->simg_next, kAuxWarp0Q - kEpiWarp0Q);
+    mbar_init(&bars->simg_ready, 1);
+    mbar_init(&bars->simg_next, 1);
     mbar_init(&bars->w_full, 1);
     bars->abort_flag = 0;
     fence_mbar_init();
@@ -977,14 +947,16 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     } else if (warp == kWarpMma2Q && lane == 0) {
       // MMA2 of every tile: [N' | D'] = Phi (bf16 pairs in the tile's buffer) * [S' | z' | 0].
       const uint32_t hi = smem_desc_hi(1024);
-      const uint32_t s_lo = smem_desc_lo(smem_u32(smem + SL::simg), 16);
+      const uint32_t s_lo0 = smem_desc_lo(smem_u32(smem + SL::simg), 16);
       bool ok = true;
       int t = 0, ic = 0;   // tiles and items so far
       for (int it = item0; it < items && ok; it += item_step, ++ic) {
         const int ntl = 2 * item_blocks(it, chunks, chunk_blocks, n);
-        // the [S' | z' | 0]^T image of this item's slab is in place
+        // the [S' | z' | 0]^T image of this item's slab is in place (items alternate between two images
+        // where there are two)
         ok = ic == 0 ? mbar_wait(&bars->simg_ready, 0, abort_flag, status, kErrMma)
                      : mbar_wait(&bars->simg_next, (ic - 1) & 1, abort_flag, status, kErrMma);
+        const uint32_t s_lo = s_lo0 + ((kMulti && SL::two_images && (ic & 1)) ? (SL::simg_bytes >> 4) : 0u);
         for (int tt = 0; tt < ntl && ok; ++tt, ++t) {
           const int buf = t & 1;
           ok = mbar_wait(&bars->phi_ready[buf], (t >> 1) & 1, abort_flag, status, kErrMma);
@@ -1002,7 +974,6 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     }
   } else if (warp < kEpiWarp0Q) {
     reg_dec<kRegsReluQ>();
-    qside_build_simg<NH>(smem + SL::simg, Sbf, zg, item0 / chunks, &bars->simg_ready);
     const int g = (warp - kReluWarp0) >> 2;
     const uint32_t lane_base = 32u * (warp & 3);
     bool ok = true;
@@ -1024,27 +995,46 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     }
   } else if (warp < kAuxWarp0Q) {
     reg_inc<kRegsEpiQ>();
-    qside_build_simg<NH>(smem + SL::simg, Sbf, zg, item0 / chunks, &bars->simg_ready);
     const int et = threadIdx.x - 32 * kEpiWarp0Q;     // 0..127 = token row of the tile = TMEM lane
+    int img_sent = 0;                                 // bulk copies of images sent by thread 0 (first one included)
+    if (et == 0) {
+      // S' and z', and with them the image, come from the kernel before this one in the stream, which may
+      // still be running (programmatic dependent launch); everything else this kernel reads was complete
+      // before that kernel started.
+      griddep_wait();
+      mbar_arrive_expect_tx(&bars->simg_ready, SL::simg_bytes);
+      bulk_load_1d(smem + SL::simg, simg_g + (size_t)(item0 / chunks) * SL::simg_bytes, SL::simg_bytes, &bars->simg_ready);
+      img_sent = 1;
+    }
     const uint32_t lane_base = 32u * (warp & 3);
     const float bw = fmaxf(beta[0], bw_floor);
     bool ok = true;
     int t = 0, ic = 0;   // tiles and items so far
+    float f0 = f[(size_t)(item0 / chunks) * (L + 1)];   // f_0 of the item's slab, fetched one item ahead
     for (int it = item0; it < items; it += item_step, ++ic) {
     const int slab = it / chunks, blk0 = (it % chunks) * chunk_blocks;
     const int ntl = 2 * item_blocks(it, chunks, chunk_blocks, n);
-    if (ic > 0) {
-      // every MMA2 of the item before has completed (its last accumulator was drained above): the image of
-      // this item's slab takes the place of the old one
-      if (ok) {
-        if (slab != (it - item_step) / chunks)
-          load_szt_image(smem + SL::simg, Sbf + (size_t)slab * m * kD, zg + (size_t)slab * m, m, et, 128, false);
-        fence_proxy_async_smem();
-        warp_arrive(&bars->simg_next);
+    const int nxt = it + item_step;
+    if (kMulti && et == 0 && ok) {
+      if (SL::two_images) {
+        // Two images: the one of the next item is fetched now, into the buffer that the item before this one
+        // used (every MMA2 of that item has completed: its last accumulator was drained above).
+        if (nxt < items) {
+          mbar_arrive_expect_tx(&bars->simg_next, SL::simg_bytes);
+          bulk_load_1d(smem + SL::simg + ((ic + 1) & 1) * SL::simg_bytes, simg_g + (size_t)(nxt / chunks) * SL::simg_bytes,
+                       SL::simg_bytes, &bars->simg_next);
+          ++img_sent;
+        }
+      } else if (ic > 0) {
+        // One image: every MMA2 of the item before has completed, this item's image takes its place.
+        mbar_arrive_expect_tx(&bars->simg_next, SL::simg_bytes);
+        bulk_load_1d(smem + SL::simg, simg_g + (size_t)slab * SL::simg_bytes, SL::simg_bytes, &bars->simg_next);
+        ++img_sent;
       }
     }
     // the filter stage left Q_F, and with it N' and D', scaled by r (see haar_block_inplace): eps' follows
-    const float epsp = eps * (float)m * bw * bw * haar_scale(f[(size_t)slab * (L + 1)]);
+    const float epsp = eps * (float)m * bw * bw * haar_scale(f0);
+    if (kMulti && nxt < items) f0 = f[(size_t)(nxt / chunks) * (L + 1)];
     for (int tt = 0; tt < ntl; ++tt, ++t) {
       const int buf = t & 1;
       const uint32_t base = tmem + (lane_base << 16) + buf * kQBufCols + TM::kAcc;
@@ -1095,6 +1085,10 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
         bulk_commit_group();
       }
     }
+    }
+    if (et == 0 && *abort_flag != 0) {   // an image copy may still be in flight
+      if (img_sent >= 1) mbar_wait_drain(&bars->simg_ready, 0);
+      if (img_sent >= 2) mbar_wait_drain(&bars->simg_next, (img_sent - 2) & 1);
     }
     if (et == 0) bulk_wait_group0();
   } else {
@@ -1195,12 +1189,13 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
   float* sp = single ? w.S : w.spart;
   float* zp = single ? w.z : w.zpart;
   __nv_bfloat16* sb = single ? w.Sbf : nullptr;
+  uint8_t* si = single ? w.Simg : nullptr;
   const bool multi = items > (int)grid.x;   // some CTA walks more than one item
   // One item per CTA: a (chunks, slabs) grid.  The same CTAs as a one-dimensional grid measured 6 us more per
   // config-4 forward (192 against 186 us), so the shape is kept where it has a choice.
   if (!multi) grid = dim3(p.tchunks, p.slabs);
   auto launch = [&](auto kernel, size_t smem_bytes) {
-    return launch_pdl(kernel, grid, kThreads, smem_bytes, st, map_k, map_v, map_w, (const float*)w.f, sp, zp, sb,
+    return launch_pdl(kernel, grid, kThreads, smem_bytes, st, map_k, map_v, map_w, (const float*)w.f, sp, zp, sb, si,
                       p.cfg.seq_len, p.cfg.levels, p.tchunk_blocks, p.tchunks, items, w.status);
   };
   if (p.cfg.features == 256)
@@ -1226,8 +1221,8 @@ cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const flo
   const bool multi = items > (int)grid.x;
   if (!multi) grid = dim3(p.tchunks, p.slabs);   // see launch_tc_kside
   auto launch = [&](auto kernel, size_t smem_bytes) {
-    return launch_pdl(kernel, grid, kThreadsQ, smem_bytes, st, map_q, map_o, map_w, (const __nv_bfloat16*)w.Sbf,
-                      (const float*)w.z, (const float*)w.f, beta, p.cfg.eps, p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels,
+    return launch_pdl(kernel, grid, kThreadsQ, smem_bytes, st, map_q, map_o, map_w, (const uint8_t*)w.Simg,
+                      (const float*)w.f, beta, p.cfg.eps, p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels,
                       p.tchunk_blocks, p.tchunks, items, w.status);
   };
   if (p.cfg.features == 256)
