@@ -423,6 +423,25 @@ def main():
         line["training_step"] = {"ms_per_step": tms, "tokens_per_s": cfg["B"] * cfg["n"] / (tms * 1e-3),
                                  "what": "forward + backward, device-timed, 20 steps",
                                  "launches": ctx_t.launch_count(0) + ctx_t.launch_count(1)}
+    # the stand-alone Haar filter pass X -> T_f(X) on this workload's Q: a pure streaming kernel, read + write
+    hf = torch.linspace(0.5, 1.5, cfg["B"] * cfg["H"] * (cfg["L"] + 1), device=f"cuda:{local_rank}",
+                        dtype=torch.float32).view(cfg["B"] * cfg["H"], cfg["L"] + 1)
+    XF = torch.empty_like(dev["Q"])
+    for _ in range(3):
+        ctx.haar_filter(dev["Q"], hf, out=XF, stream=stream)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(20):
+        ctx.haar_filter(dev["Q"], hf, out=XF, stream=stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    hms = e0.elapsed_time(e1) / 20
+    hbytes = 2 * dev["Q"].numel() * dev["Q"].element_size()
+    line["haar_filter_pass"] = {"ms": hms, "bytes": hbytes, "achieved_gbs": hbytes / (hms * 1e-3) / 1e9,
+                                "peak_gbs": float(peaks["hbm_gbs"]),
+                                "frac": hbytes / (hms * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
+                                "what": "wersa_haar_filter on Q (read once, written once), 20 launches, device-timed"}
+    del XF
     if not args.no_cpu_baseline:
         rate, desc, used, _ = oracle_sample_rate(cfg, inp, 15.0)
         line["cpu_baseline"] = {"value": rate, "unit": "tokens/s", "cores": used, "kind": "oracle",

@@ -206,8 +206,9 @@ class WersaContext:
             raise WersaError(st, "wersa_backward")
         return dict(dQ=dQ, dK=dK, dV=dV, dbeta=dbeta, dgate_w=dgw, dgate_b=dgb, domega=dom)
 
-    def haar_filter(self, X, f, stream=None):
-        out = torch.empty_like(X)
+    def haar_filter(self, X, f, out=None, stream=None):
+        if out is None:
+            out = torch.empty_like(X)
         st = _lib().wersa_haar_filter(self._h, _ptr(X, self.io_dtype, "X"), _ptr(f, torch.float32, "f"),
                                       _ptr(out), _stream_ptr(stream))
         if st != WERSA_OK:
