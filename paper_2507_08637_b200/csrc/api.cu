@@ -369,12 +369,19 @@ wersa_status wersa_backward(wersa_ctx* ctx, const void* Q, const void* K, const 
     WERSA_STEP(1, "tc_bwd_kside", launch_tc_bwd_kside(p, w, w.KF3, V, dV, st, &launches));
   else
     WERSA_STEP(1, "simt_bwd_kside", launch_simt_bwd_kside(p, w, V, W, dV, st, &launches));
-  WERSA_STEP(1, "haar_backward_q", launch_haar_backward(p, w, Q, kind, w.dQF, dQ, gkind, 0, st, &launches));
+  // With gate weights dQ has a second term, d(qbar) / n on every row (Eq. 1), which is known only after the
+  // gate backward: the first pass over dQ_F then takes the band inner products alone, and dQ is written
+  // once, by a filter pass that adds the row vector.
+  const bool pooled_term = gate_w != nullptr;
+  WERSA_STEP(1, "haar_backward_q",
+             launch_haar_backward(p, w, Q, kind, w.dQF, pooled_term ? nullptr : dQ, gkind, 0, st, &launches));
   WERSA_STEP(1, "haar_backward_k", launch_haar_backward(p, w, K, kind, w.dKF, dK, gkind, 1, st, &launches));
   WERSA_STEP(1, "gate_backward",
              launch_gate_backward(p, w, beta, gate_w, omega, p.slabs * bwd_chunks, dbeta, dgate_w, dgate_b, domega, st,
                                   &launches));
-  if (gate_w != nullptr) WERSA_STEP(1, "add_rowvec", launch_add_rowvec(p, w, dQ, st, &launches));
+  if (pooled_term)
+    WERSA_STEP(1, "haar_filter_dq",
+               launch_haar_filter_addvec(p, w.dQF, w.f, w.dqbar, 1.f / (float)p.cfg.seq_len, dQ, gkind, st, &launches));
   ctx->launches_bwd = launches;
   return WERSA_OK;
 }

@@ -66,8 +66,6 @@ cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const f
 cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, const float* gate_w,
                                  const float* omega, int n_sumdD, float* dbeta, float* dgate_w, float* dgate_b,
                                  float* domega, cudaStream_t st, int* launches);
-// dQ[s,t,:] += dqbar[s,:] / n.
-cudaError_t launch_add_rowvec(const Plan& p, const Ws& w, void* dQ, cudaStream_t st, int* launches);
 
 // Mean pool + gate with their scratch in a file-scope device array (no caller workspace).
 cudaError_t static_scratch_address(int device, float** out);
@@ -86,7 +84,11 @@ cudaError_t launch_haar_filter(const Plan& p, const void* X, int in_kind, const 
 // XF3 = T_f(X) as three bf16 planes hi, mid, lo (each slabs x n x 64) whose sum is the fp32 result.
 cudaError_t launch_haar_filter_split3(const Plan& p, const void* X, int in_kind, const float* f,
                                       __nv_bfloat16* XF3, cudaStream_t st, int* launches);
-// dX = T_f(G) (G fp32) and per-tile band inner products of (G, X) into bands[which].
+// dX = T_f(G) + vec[slab] * vec_scale on every row (G fp32, vec = slabs x 64 floats).
+cudaError_t launch_haar_filter_addvec(const Plan& p, const float* G, const float* f, const float* vec,
+                                      float vec_scale, void* dX, int out_kind, cudaStream_t st, int* launches);
+// dX = T_f(G) (G fp32) and per-tile band inner products of (G, X) into bands[which]; dX == nullptr: only
+// the band inner products.
 cudaError_t launch_haar_backward(const Plan& p, const Ws& w, const void* X, int in_kind,
                                  const float* G, void* dX, int out_kind, int which, cudaStream_t st,
                                  int* launches);

@@ -274,21 +274,6 @@ __global__ void __launch_bounds__(kD) k_gate_backward(
   }
 }
 
-template <typename T>
-__global__ void __launch_bounds__(256) k_add_rowvec(T* __restrict__ dQ, const float* __restrict__ dqbar,
-                                                    int n, float inv_n) {
-  const int slab = blockIdx.y;
-  const size_t idx8 = (size_t)blockIdx.x * 256 + threadIdx.x;   // group of 8 elements in the slab
-  if (idx8 >= (size_t)n * (kD / 8)) return;
-  const int cg = (int)(idx8 & 7);
-  T* p = dQ + (size_t)slab * n * kD + idx8 * 8;
-  float v[8];
-  load8(p, v);
-#pragma unroll
-  for (int j = 0; j < 8; ++j) v[j] += dqbar[(size_t)slab * kD + cg * 8 + j] * inv_n;
-  store8(p, v);
-}
-
 }  // namespace
 
 // The launch shared by the workspace and the static-scratch variants.
@@ -363,18 +348,6 @@ cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, 
                                     p.cfg.eps, p.cfg.bw_floor, p.cfg.features, p.cfg.batch, p.cfg.heads,
                                     p.L1, p.cfg.gate_per_head, dbeta, dgate_w, dgate_b, domega, w.dqbar);
   *launches += 2;
-  return cudaGetLastError();
-}
-
-cudaError_t launch_add_rowvec(const Plan& p, const Ws& w, void* dQ, cudaStream_t st, int* launches) {
-  const size_t groups = (size_t)p.cfg.seq_len * (kD / 8);
-  dim3 grid((unsigned)((groups + 255) / 256), p.slabs);
-  const float inv_n = 1.f / (float)p.cfg.seq_len;
-  if (p.grad_bf16)
-    k_add_rowvec<__nv_bfloat16><<<grid, 256, 0, st>>>((__nv_bfloat16*)dQ, w.dqbar, p.cfg.seq_len, inv_n);
-  else
-    k_add_rowvec<float><<<grid, 256, 0, st>>>((float*)dQ, w.dqbar, p.cfg.seq_len, inv_n);
-  *launches += 1;
   return cudaGetLastError();
 }
 

@@ -79,10 +79,12 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, const float (&v)[4]) {
 // the others (the pass is bound by memory bandwidth).  Levels 1-3 come from the register tile; the 8-row
 // sums go to a pyramid in shared memory (per column 32 sums of level 3, then 16, 8, 4, 2, 1 of levels
 // 4-8), from which every thread takes the coarse part of its output rows.
+// With kAddVec every output row of slab s also gets vec[s][:] * vec_scale added (the mean-pool term of dQ).
 // grid (2 * htiles, slabs): blockIdx.x = 2 * tile + column half; block 256.
-template <typename Tin, typename Tout>
+template <typename Tin, typename Tout, bool kAddVec>
 __global__ void __launch_bounds__(256, 4) k_haar_filter(const Tin* __restrict__ X, const float* __restrict__ f,
-                                                     Tout* __restrict__ XF, int n, int L) {
+                                                     Tout* __restrict__ XF, int n, int L,
+                                                     const float* __restrict__ vec, float vec_scale) {
   __shared__ float pyr[kPyr][kHalfD];
   __shared__ float hit[32][kHalfD];   // sum_{l=3..8} k_l * s_l(block of row group r), per column
   const int slab = blockIdx.y, half = blockIdx.x & 1;
@@ -132,7 +134,8 @@ __global__ void __launch_bounds__(256, 4) k_haar_filter(const Tin* __restrict__ 
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       const float a0 = x[j][c] + x[j + 1][c], a1 = x[j + 2][c] + x[j + 3][c];
-      const float c2 = fmaf(k.k[2], a0 + a1, hit[rg][cg * 4 + c]);
+      float c2 = fmaf(k.k[2], a0 + a1, hit[rg][cg * 4 + c]);
+      if constexpr (kAddVec) c2 = fmaf(vec[(size_t)slab * kD + col0 + c], vec_scale, c2);
       const float c10 = fmaf(k.k[1], a0, c2), c11 = fmaf(k.k[1], a1, c2);
       y[0][c] = fmaf(k.f0, x[j][c], c10);
       y[1][c] = fmaf(k.f0, x[j + 1][c], c10);
@@ -349,7 +352,8 @@ __global__ void __launch_bounds__(256, 2) k_haar_filter_split3(const Tin* __rest
 // sums of level 3, then 16, 8, 4, 2, 1 of levels 4-8), from which one thread per column takes the level
 // 4-8 products and every thread the coarse part of its output rows.
 // grid (2 * htiles, slabs): blockIdx.x = 2 * tile + column half; one band partial per CTA.
-template <typename Tin, typename Tout>
+// kWrite = false leaves dX unwritten (only the band inner products are wanted).
+template <typename Tin, typename Tout, bool kWrite>
 __global__ void __launch_bounds__(256, 3) k_haar_backward(const Tin* __restrict__ X, const float* __restrict__ G,
                                                           const float* __restrict__ f, Tout* __restrict__ dX,
                                                           float* __restrict__ bands, int n, int L) {
@@ -429,16 +433,18 @@ __global__ void __launch_bounds__(256, 3) k_haar_backward(const Tin* __restrict_
     }
   }
   // coarse part of the output rows: hit[r][col] = sum_{l=3..8} k_l * s_l(block of row group r)
+  if constexpr (kWrite) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int e = threadIdx.x + 256 * i, r = e >> 5, col = e & 31;
-    float v = k.k[3] * pyr[0][r][col];
+    for (int i = 0; i < 4; ++i) {
+      const int e = threadIdx.x + 256 * i, r = e >> 5, col = e & 31;
+      float v = k.k[3] * pyr[0][r][col];
 #pragma unroll
-    for (int l = 4; l <= 8; ++l) v += k.k[l] * pyr[0][pyr_base(l) + (r >> (l - 3))][col];
-    hit[r][col] = v;
+      for (int l = 4; l <= 8; ++l) v += k.k[l] * pyr[0][pyr_base(l) + (r >> (l - 3))][col];
+      hit[r][col] = v;
+    }
+    __syncthreads();
   }
-  __syncthreads();
-  {
+  if constexpr (kWrite) {
     Tout* dst = dX + (size_t)slab * n * kD + col0;
     float hi[4], s1[4][4], s2[2][4];
 #pragma unroll
@@ -492,9 +498,22 @@ cudaError_t launch_haar_filter(const Plan& p, const void* X, int in_kind, const 
   else if (in_kind == 1 && out_kind == 0)
     k_haar_filter_bf16<float><<<grid_bf, 256, 0, st>>>((const __nv_bfloat16*)X, f, (float*)XF, n, L);
   else if (in_kind == 0 && out_kind == 0)
-    k_haar_filter<float, float><<<grid, 256, 0, st>>>((const float*)X, f, (float*)XF, n, L);
+    k_haar_filter<float, float, false><<<grid, 256, 0, st>>>((const float*)X, f, (float*)XF, n, L, nullptr, 0.f);
   else
-    k_haar_filter<float, __nv_bfloat16><<<grid, 256, 0, st>>>((const float*)X, f, (__nv_bfloat16*)XF, n, L);
+    k_haar_filter<float, __nv_bfloat16, false><<<grid, 256, 0, st>>>((const float*)X, f, (__nv_bfloat16*)XF, n, L,
+                                                                    nullptr, 0.f);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_haar_filter_addvec(const Plan& p, const float* G, const float* f, const float* vec,
+                                      float vec_scale, void* dX, int out_kind, cudaStream_t st, int* launches) {
+  dim3 grid(2 * p.htiles, p.slabs);
+  const int n = p.cfg.seq_len, L = p.cfg.levels;
+  if (out_kind == 0)
+    k_haar_filter<float, float, true><<<grid, 256, 0, st>>>(G, f, (float*)dX, n, L, vec, vec_scale);
+  else
+    k_haar_filter<float, __nv_bfloat16, true><<<grid, 256, 0, st>>>(G, f, (__nv_bfloat16*)dX, n, L, vec, vec_scale);
   *launches += 1;
   return cudaGetLastError();
 }
@@ -517,17 +536,23 @@ cudaError_t launch_haar_backward(const Plan& p, const Ws& w, const void* X, int 
   dim3 grid(2 * p.htiles, p.slabs);   // two column halves per 256-row tile
   const int n = p.cfg.seq_len, L = p.cfg.levels;
   float* bands = w.bands + (size_t)which * p.slabs * 2 * p.htiles * kBandVals;
-  if (in_kind == 1 && out_kind == 1)
-    k_haar_backward<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
+  if (dX == nullptr) {   // band inner products only
+    if (in_kind == 1)
+      k_haar_backward<__nv_bfloat16, float, false><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, G, w.f, nullptr,
+                                                                        bands, n, L);
+    else
+      k_haar_backward<float, float, false><<<grid, 256, 0, st>>>((const float*)X, G, w.f, nullptr, bands, n, L);
+  } else if (in_kind == 1 && out_kind == 1)
+    k_haar_backward<__nv_bfloat16, __nv_bfloat16, true><<<grid, 256, 0, st>>>(
         (const __nv_bfloat16*)X, G, w.f, (__nv_bfloat16*)dX, bands, n, L);
   else if (in_kind == 1 && out_kind == 0)
-    k_haar_backward<__nv_bfloat16, float><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, G, w.f, (float*)dX,
-                                                               bands, n, L);
+    k_haar_backward<__nv_bfloat16, float, true><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, G, w.f, (float*)dX,
+                                                                     bands, n, L);
   else if (in_kind == 0 && out_kind == 0)
-    k_haar_backward<float, float><<<grid, 256, 0, st>>>((const float*)X, G, w.f, (float*)dX, bands, n, L);
+    k_haar_backward<float, float, true><<<grid, 256, 0, st>>>((const float*)X, G, w.f, (float*)dX, bands, n, L);
   else
-    k_haar_backward<float, __nv_bfloat16><<<grid, 256, 0, st>>>((const float*)X, G, w.f, (__nv_bfloat16*)dX,
-                                                               bands, n, L);
+    k_haar_backward<float, __nv_bfloat16, true><<<grid, 256, 0, st>>>((const float*)X, G, w.f, (__nv_bfloat16*)dX,
+                                                                     bands, n, L);
   *launches += 1;
   return cudaGetLastError();
 }
