@@ -1191,8 +1191,8 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
   __nv_bfloat16* sb = single ? w.Sbf : nullptr;
   uint8_t* si = single ? w.Simg : nullptr;
   const bool multi = items > (int)grid.x;   // some CTA walks more than one item
-  // One item per CTA: a (chunks, slabs) grid.  The same CTAs as a one-dimensional grid measured 6 us more per
-  // config-4 forward (192 against 186 us), so the shape is kept where it has a choice.
+  // One item per CTA: a (chunks, slabs) grid (item = blockIdx.y * gridDim.x + blockIdx.x either way; other
+  // shapes with the same number of CTAs measured the same).
   if (!multi) grid = dim3(p.tchunks, p.slabs);
   auto launch = [&](auto kernel, size_t smem_bytes) {
     return launch_pdl(kernel, grid, kThreads, smem_bytes, st, map_k, map_v, map_w, (const float*)w.f, sp, zp, sb, si,
