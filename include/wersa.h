@@ -66,9 +66,14 @@ typedef struct wersa_config {
   int32_t batch;         /* B >= 1                                                      */
   int32_t heads;         /* H >= 1                                                      */
   int32_t seq_len;       /* n >= 2; 2^levels must not exceed the next power of two >= n */
-  int32_t head_dim;      /* d, must be 64                                               */
+  int32_t head_dim;      /* d: 8, 16, ... 64 (below 64 the tensors pass through zero-padded
+                            64-wide copies in the workspace, which leaves Eqs. 1-7 unchanged) */
   int32_t levels;        /* L, Haar levels, 1..8                                        */
-  int32_t features;      /* m, random features: 64, 128 or 256                          */
+  int32_t features;      /* m, random features: 64, 128 or 256; with dtype bf16 and without
+                            WERSA_FLAG_SIMT_ONLY also 512, 768 and 1024 (Sec. 3.3 uses 1024),
+                            forward only: the features run in groups of 256 whose outputs
+                            are combined by their denominators, wersa_backward then returns
+                            WERSA_ERR_UNSUPPORTED                                        */
   int32_t dtype;         /* wersa_dtype of Q, K, V, W, O, dO; accumulation is fp32      */
   int32_t grad_dtype;    /* wersa_dtype of dQ, dK, dV                                   */
   float eps;             /* denominator epsilon of Eq. 7 (paper: "small constant")      */
@@ -168,8 +173,9 @@ wersa_status wersa_gate_static(const wersa_config* cfg, const void* Q, const flo
                                void* cuda_stream);
 
 /* Device pointers into the workspace of quantities the last forward left there.
- * which: 0 = f (batch*heads, levels+1); 1 = qbar (batch*heads, head_dim);
- *        2 = S' (batch*heads, features, head_dim); 3 = z' (batch*heads, features),
+ * which: 0 = f (batch*heads, levels+1); 1 = qbar (batch*heads, 64);
+ *        2 = S' (batch*heads, features, 64); 3 = z' (batch*heads, features),
+ * the last axis of qbar and S' being the padded head dimension (columns >= head_dim are zero),
  * where S' = ReLU(K_F W)^T V and z' = ReLU(K_F W)^T 1 are the key summary and normaliser of
  * Eq. 7 without the 1/(bw sqrt(m)) factor of the feature map (S = S' / (bw sqrt(m))).
  * *count receives the number of floats. */

@@ -226,9 +226,10 @@ class WersaContext:
         flat = self.workspace[off:off + 4 * count.value].view(torch.float32).clone()
         c = self.cfg
         slabs = (c.batch, c.heads)
-        shape = {0: slabs + (c.levels + 1,), 1: slabs + (c.head_dim,), 2: slabs + (c.features, c.head_dim),
+        shape = {0: slabs + (c.levels + 1,), 1: slabs + (64,), 2: slabs + (c.features, 64),
                  3: slabs + (c.features,)}[idx]
-        return flat.view(shape)
+        out = flat.view(shape)
+        return out[..., :c.head_dim].contiguous() if idx in (1, 2) else out   # drop the padding columns
 
     def query_status(self, stream=None):
         return int(_lib().wersa_query_status(self._h, _stream_ptr(stream)))
@@ -250,7 +251,7 @@ class WersaContext:
 
     def step_times(self, which=0):
         """[(step name, milliseconds)] of the last forward (0) or backward (1); waits for it."""
-        cap = 16
+        cap = 32
         ms = (ctypes.c_float * cap)()
         names = (ctypes.c_char_p * cap)()
         count = ctypes.c_int()

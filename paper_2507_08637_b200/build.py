@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libwersa.so")
-SOURCES = ["api.cu", "gate.cu", "haar.cu", "simt.cu", "tc_fwd.cu", "tc_bwd.cu", "selftest.cu"]
+SOURCES = ["api.cu", "gate.cu", "haar.cu", "simt.cu", "tc_fwd.cu", "tc_bwd.cu", "selftest.cu", "glue.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 

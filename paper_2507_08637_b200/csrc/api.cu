@@ -38,9 +38,17 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   if (!(c.eps >= 0.f) || !(c.bw_floor > 0.f)) return WERSA_ERR_INVALID_ARG;
   if (c.device < 0) return WERSA_ERR_INVALID_ARG;
   if (c.levels <= 30 && (1LL << c.levels) > (long long)next_pow2(c.seq_len)) return WERSA_ERR_INVALID_ARG;
-  if (c.head_dim != kD) return WERSA_ERR_UNSUPPORTED;
+  // head dimensions 8, 16, ... 64 (narrower ones run zero-padded to 64 columns)
+  if (c.head_dim > kD || c.head_dim < 8 || c.head_dim % 8 != 0) return WERSA_ERR_UNSUPPORTED;
   if (c.levels > kMaxLevels) return WERSA_ERR_UNSUPPORTED;
-  if (c.features != 64 && c.features != 128 && c.features != 256) return WERSA_ERR_UNSUPPORTED;
+  // feature maps of 64, 128 or 256, and (bf16 tensor-core path, forward only) 512, 768, 1024 in groups of 256
+  const bool grouped = c.features > kGroupFeatures;
+  if (grouped) {
+    if (c.features % kGroupFeatures != 0 || c.features > 4 * kGroupFeatures) return WERSA_ERR_UNSUPPORTED;
+    if (c.dtype != WERSA_BF16 || (c.flags & WERSA_FLAG_SIMT_ONLY)) return WERSA_ERR_UNSUPPORTED;
+  } else if (c.features != 64 && c.features != 128 && c.features != 256) {
+    return WERSA_ERR_UNSUPPORTED;
+  }
   if ((long long)c.batch * c.heads > 65535) return WERSA_ERR_UNSUPPORTED;   // gridDim.y
 
   p->cfg = c;
@@ -48,7 +56,9 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   p->L1 = c.levels + 1;
   p->bf16 = c.dtype == WERSA_BF16;
   p->grad_bf16 = c.grad_dtype == WERSA_BF16;
-  p->with_backward = !(c.flags & WERSA_FLAG_FORWARD_ONLY);
+  p->with_backward = !(c.flags & WERSA_FLAG_FORWARD_ONLY) && !grouped;
+  p->dpad = c.head_dim < kD;
+  p->groups = grouped ? c.features / kGroupFeatures : 1;
   p->use_tc = p->bf16 && !(c.flags & WERSA_FLAG_SIMT_ONLY) && tc_supported(c);
   const int n = c.seq_len, m = c.features;
   p->sms = device_sm_count(c.device);
@@ -111,6 +121,17 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   p->off_Wt = take(sizeof(__nv_bfloat16) * (size_t)m * kD);
   p->off_Simg = take(p->use_tc ? slabs * simg_bytes(m) : 0);
   const size_t slab_elems = slabs * (size_t)n * kD;
+  const size_t io_bytes = p->bf16 ? 2 : 4, grad_bytes = p->grad_bf16 ? 2 : 4;
+  p->off_Qp = take(p->dpad ? io_bytes * slab_elems : 0);
+  p->off_Kp = take(p->dpad ? io_bytes * slab_elems : 0);
+  p->off_Vp = take(p->dpad ? io_bytes * slab_elems : 0);
+  p->off_Op = take(p->dpad ? io_bytes * slab_elems : 0);
+  p->off_Wp = take(p->dpad ? io_bytes * (size_t)kD * m : 0);
+  p->off_gwp = take(p->dpad ? sizeof(float) * (size_t)c.heads * kD * p->L1 : 0);
+  p->off_Og = take(grouped ? io_bytes * slab_elems * p->groups : 0);
+  p->off_den = take(grouped ? sizeof(float) * slabs * n * p->groups : 0);
+  p->off_Sout = take(grouped ? sizeof(float) * slabs * m * kD : 0);
+  p->off_zout = take(grouped ? sizeof(float) * slabs * m : 0);
   const bool need_xf = !p->use_tc;   // the tensor-core kernels filter on chip (forward) or read bf16 planes (backward)
   p->off_QF = take(need_xf ? sizeof(float) * slab_elems : 0);
   p->off_KF = take(need_xf ? sizeof(float) * slab_elems : 0);
@@ -126,8 +147,14 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
     p->off_KF3 = take(p->use_tc ? 3 * sizeof(__nv_bfloat16) * slab_elems : 0);
     p->off_QF3 = take(p->use_tc ? 3 * sizeof(__nv_bfloat16) * slab_elems : 0);
     p->off_Slo = take(p->use_tc ? sizeof(__nv_bfloat16) * slabs * m * kD : 0);
+    p->off_dOp = take(p->dpad ? io_bytes * slab_elems : 0);
+    p->off_dQp = take(p->dpad ? grad_bytes * slab_elems : 0);
+    p->off_dKp = take(p->dpad ? grad_bytes * slab_elems : 0);
+    p->off_dVp = take(p->dpad ? grad_bytes * slab_elems : 0);
+    p->off_dgwp = take(p->dpad ? sizeof(float) * (size_t)c.heads * kD * p->L1 : 0);
   } else {
     p->off_dS = p->off_dz = p->off_sumdD = p->off_bands = p->off_dqbar = p->off_dQF = p->off_dKF = p->off_dSbf = p->off_KF3 = p->off_QF3 = p->off_Slo = 0;
+    p->off_dOp = p->off_dQp = p->off_dKp = p->off_dVp = p->off_dgwp = 0;
   }
   p->total = off;
   return WERSA_OK;
@@ -162,6 +189,21 @@ Ws resolve(const Plan& p, void* workspace) {
   w.KF3 = reinterpret_cast<__nv_bfloat16*>(b + p.off_KF3);
   w.QF3 = reinterpret_cast<__nv_bfloat16*>(b + p.off_QF3);
   w.Slo = reinterpret_cast<__nv_bfloat16*>(b + p.off_Slo);
+  w.Qp = b + p.off_Qp;
+  w.Kp = b + p.off_Kp;
+  w.Vp = b + p.off_Vp;
+  w.Op = b + p.off_Op;
+  w.Wp = b + p.off_Wp;
+  w.gwp = reinterpret_cast<float*>(b + p.off_gwp);
+  w.dOp = b + p.off_dOp;
+  w.dQp = b + p.off_dQp;
+  w.dKp = b + p.off_dKp;
+  w.dVp = b + p.off_dVp;
+  w.dgwp = reinterpret_cast<float*>(b + p.off_dgwp);
+  w.Og = b + p.off_Og;
+  w.den = reinterpret_cast<float*>(b + p.off_den);
+  w.Sout = reinterpret_cast<float*>(b + p.off_Sout);
+  w.zout = reinterpret_cast<float*>(b + p.off_zout);
   return w;
 }
 
@@ -169,7 +211,7 @@ Ws resolve(const Plan& p, void* workspace) {
 
 using namespace wersa;
 
-constexpr int kMaxSteps = 16;
+constexpr int kMaxSteps = 32;
 
 // Optional per-step timing: an event before the first launch and one after every step.
 struct StepTimer {
@@ -232,6 +274,41 @@ wersa_status begin_pass(wersa_ctx* ctx, int which, cudaStream_t st) {
   return WERSA_OK;
 }
 
+// Feature group g of a map wider than 256 features: the plan of a 256-feature problem and the workspace
+// regions of that group (the kernels' buffers are kept group-major: [group][slab][...]).
+Plan group_plan(const Plan& p) {
+  Plan pg = p;
+  pg.cfg.features = kGroupFeatures;
+  return pg;
+}
+Ws group_view(const Plan& p, const Ws& w, int g) {
+  Ws v = w;
+  const size_t slabs = (size_t)p.slabs, mg = kGroupFeatures;
+  v.Wt = w.Wt + (size_t)g * mg * kD;
+  v.spart = w.spart + (size_t)g * slabs * p.tchunks * mg * kD;
+  v.zpart = w.zpart + (size_t)g * slabs * p.tchunks * mg;
+  v.S = w.S + (size_t)g * slabs * mg * kD;
+  v.z = w.z + (size_t)g * slabs * mg;
+  v.Sbf = w.Sbf + (size_t)g * slabs * mg * kD;
+  v.Simg = w.Simg + (size_t)g * slabs * simg_bytes((int)mg);
+  return v;
+}
+
+// Zero-padded 64-wide copies of the gate weights (heads x d x (L+1) -> heads x 64 x (L+1)) and of W (d x m -> 64 x m).
+cudaError_t pad_parameters(const Plan& p, const Ws& w, const void* W, const float* gate_w, cudaStream_t st) {
+  const int d = p.cfg.head_dim, m = p.cfg.features;
+  const size_t es = p.bf16 ? 2 : 4;
+  cudaError_t err = cudaMemsetAsync(w.Wp, 0, es * kD * m, st);
+  if (err == cudaSuccess) err = cudaMemcpyAsync(w.Wp, W, es * (size_t)d * m, cudaMemcpyDeviceToDevice, st);
+  if (err == cudaSuccess && gate_w != nullptr) {
+    const size_t row = sizeof(float) * p.L1;
+    err = cudaMemsetAsync(w.gwp, 0, row * kD * p.cfg.heads, st);
+    if (err == cudaSuccess)
+      err = cudaMemcpy2DAsync(w.gwp, row * kD, gate_w, row * d, row * d, p.cfg.heads, cudaMemcpyDeviceToDevice, st);
+  }
+  return err;
+}
+
 wersa_status clear_status_once(wersa_ctx* ctx, cudaStream_t st) {
   if (!ctx->status_cleared) {
     WERSA_CUDA(cudaMemsetAsync(ctx->ws.status, 0, ctx->plan.status_bytes, st));
@@ -288,22 +365,54 @@ wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const v
   int launches = 0;
   const int kind = p.bf16 ? 1 : 0;
   if ((s = begin_pass(ctx, 0, st)) != WERSA_OK) return s;
+  const size_t rows = (size_t)p.slabs * p.cfg.seq_len;
+  if (p.dpad) {   // run the zero-padded 64-wide problem (see glue.cu)
+    WERSA_STEP(0, "pad_q", launch_pad_cols(Q, w.Qp, rows, p.cfg.head_dim, kind, st, &launches));
+    WERSA_STEP(0, "pad_k", launch_pad_cols(K, w.Kp, rows, p.cfg.head_dim, kind, st, &launches));
+    WERSA_STEP(0, "pad_v", launch_pad_cols(V, w.Vp, rows, p.cfg.head_dim, kind, st, &launches));
+    WERSA_CUDA(pad_parameters(p, w, W, gate_w, st));
+    Q = w.Qp;
+    K = w.Kp;
+    V = w.Vp;
+    W = w.Wp;
+    if (gate_w != nullptr) gate_w = w.gwp;
+  }
+  void* Ocore = p.dpad ? w.Op : O;
   WERSA_STEP(0, "qmean_gate",
              launch_qmean_gate(p, w, Q, gate_w, gate_b, omega, p.use_tc ? W : nullptr, st, &launches));
-  if (p.use_tc) {
+  if (p.groups > 1) {
+    // feature groups of 256 (tensor-core path): every group runs the key side and the query side on its own
+    // rows of W^T; the query side leaves O_g and the denominators, which the last launch combines
+    const Plan pg = group_plan(p);
+    const size_t es = p.bf16 ? 2 : 4;
+    for (int g = 0; g < p.groups; ++g) {
+      const Ws wg = group_view(p, w, g);
+      WERSA_STEP(0, "tc_kside", launch_tc_kside(pg, wg, K, V, st, &launches));
+      if (p.tchunks > 1)
+        WERSA_STEP(0, "reduce_partials",
+                   launch_reduce_partials(pg, wg.spart, wg.zpart, p.tchunks, wg.S, wg.z, wg.Sbf, wg.Simg, st, &launches));
+      WERSA_STEP(0, "tc_qside",
+                 launch_tc_qside(pg, wg, Q, beta, static_cast<char*>(w.Og) + (size_t)g * rows * kD * es,
+                                 w.den + (size_t)g * rows, st, &launches));
+    }
+    WERSA_STEP(0, "combine_groups", launch_combine_groups(w.Og, w.den, Ocore, rows, p.groups, kind, st, &launches));
+    WERSA_STEP(0, "gather_groups",
+               launch_gather_groups(w.S, w.z, w.Sout, w.zout, p.slabs, p.groups, kGroupFeatures, st, &launches));
+  } else if (p.use_tc) {
     WERSA_STEP(0, "tc_kside", launch_tc_kside(p, w, K, V, st, &launches));
     if (p.tchunks > 1)   // with one chunk per slab the key-side kernel has written S', z' and the image itself
       WERSA_STEP(0, "reduce_partials",
                  launch_reduce_partials(p, w.spart, w.zpart, p.tchunks, w.S, w.z, w.Sbf, w.Simg, st, &launches));
-    WERSA_STEP(0, "tc_qside", launch_tc_qside(p, w, Q, beta, O, st, &launches));
+    WERSA_STEP(0, "tc_qside", launch_tc_qside(p, w, Q, beta, Ocore, nullptr, st, &launches));
   } else {
     WERSA_STEP(0, "haar_filter_q", launch_haar_filter(p, Q, kind, w.f, w.QF, 0, st, &launches));
     WERSA_STEP(0, "haar_filter_k", launch_haar_filter(p, K, kind, w.f, w.KF, 0, st, &launches));
     WERSA_STEP(0, "simt_kside", launch_simt_kside(p, w, V, W, st, &launches));
     WERSA_STEP(0, "reduce_partials",
                launch_reduce_partials(p, w.spart, w.zpart, p.schunks, w.S, w.z, nullptr, nullptr, st, &launches));
-    WERSA_STEP(0, "simt_qside", launch_simt_qside(p, w, W, beta, O, st, &launches));
+    WERSA_STEP(0, "simt_qside", launch_simt_qside(p, w, W, beta, Ocore, st, &launches));
   }
+  if (p.dpad) WERSA_STEP(0, "unpad_o", launch_unpad_cols(w.Op, O, rows, p.cfg.head_dim, kind, st, &launches));
   ctx->launches_fwd = launches;
   ctx->forward_done = true;
   return WERSA_OK;
@@ -319,7 +428,7 @@ wersa_status wersa_forward_host(wersa_ctx* ctx, const void* hQ, const void* hK, 
     return WERSA_ERR_INVALID_ARG;
   const Plan& p = ctx->plan;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const size_t bytes = (size_t)p.slabs * p.cfg.seq_len * kD * (p.bf16 ? 2 : 4);
+  const size_t bytes = (size_t)p.slabs * p.cfg.seq_len * p.cfg.head_dim * (p.bf16 ? 2 : 4);
   DeviceGuard guard(p.cfg.device);
   if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
   WERSA_CUDA(cudaMemcpyAsync(dQ, hQ, bytes, cudaMemcpyHostToDevice, st));
@@ -354,6 +463,26 @@ wersa_status wersa_backward(wersa_ctx* ctx, const void* Q, const void* K, const 
   wersa_status s = begin_pass(ctx, 1, st);
   if (s != WERSA_OK) return s;
   const int bwd_chunks = p.use_tc ? p.bchunks : p.schunks;   // chunks per slab of the dS', dz', sum dD' partials
+  const size_t rows = (size_t)p.slabs * p.cfg.seq_len;
+  void *dQ_out = dQ, *dK_out = dK, *dV_out = dV;
+  float* dgate_w_out = dgate_w;
+  if (p.dpad) {   // the zero-padded 64-wide problem: gradients come back 64 wide and are cut to head_dim columns
+    WERSA_STEP(1, "pad_q", launch_pad_cols(Q, w.Qp, rows, p.cfg.head_dim, kind, st, &launches));
+    WERSA_STEP(1, "pad_k", launch_pad_cols(K, w.Kp, rows, p.cfg.head_dim, kind, st, &launches));
+    WERSA_STEP(1, "pad_v", launch_pad_cols(V, w.Vp, rows, p.cfg.head_dim, kind, st, &launches));
+    WERSA_STEP(1, "pad_do", launch_pad_cols(dO, w.dOp, rows, p.cfg.head_dim, kind, st, &launches));
+    WERSA_CUDA(pad_parameters(p, w, W, gate_w, st));
+    Q = w.Qp;
+    K = w.Kp;
+    V = w.Vp;
+    W = w.Wp;
+    dO = w.dOp;
+    dQ = w.dQp;
+    dK = w.dKp;
+    dV = w.dVp;
+    if (gate_w != nullptr) gate_w = w.gwp;
+    if (dgate_w != nullptr) dgate_w = w.dgwp;
+  }
   if (p.use_tc) {
     // the tensor-core forward keeps Q_F, K_F on chip: rebuild them, as three bf16 planes each
     WERSA_STEP(1, "haar_filter_q", launch_haar_filter_split3(p, Q, kind, w.f, w.QF3, st, &launches));
@@ -382,6 +511,16 @@ wersa_status wersa_backward(wersa_ctx* ctx, const void* Q, const void* K, const 
   if (pooled_term)
     WERSA_STEP(1, "haar_filter_dq",
                launch_haar_filter_addvec(p, w.dQF, w.f, w.dqbar, 1.f / (float)p.cfg.seq_len, dQ, gkind, st, &launches));
+  if (p.dpad) {
+    WERSA_STEP(1, "unpad_dq", launch_unpad_cols(w.dQp, dQ_out, rows, p.cfg.head_dim, gkind, st, &launches));
+    WERSA_STEP(1, "unpad_dk", launch_unpad_cols(w.dKp, dK_out, rows, p.cfg.head_dim, gkind, st, &launches));
+    WERSA_STEP(1, "unpad_dv", launch_unpad_cols(w.dVp, dV_out, rows, p.cfg.head_dim, gkind, st, &launches));
+    if (dgate_w_out != nullptr) {
+      const size_t row = sizeof(float) * p.L1;
+      WERSA_CUDA(cudaMemcpy2DAsync(dgate_w_out, row * p.cfg.head_dim, w.dgwp, row * kD, row * p.cfg.head_dim,
+                                   p.cfg.heads, cudaMemcpyDeviceToDevice, st));
+    }
+  }
   ctx->launches_bwd = launches;
   return WERSA_OK;
 }
@@ -394,7 +533,15 @@ wersa_status wersa_haar_filter(wersa_ctx* ctx, const void* X, const float* f, vo
   if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
   int launches = 0;
   const int kind = p.bf16 ? 1 : 0;
-  WERSA_CUDA(launch_haar_filter(p, X, kind, f, XF, kind, static_cast<cudaStream_t>(cuda_stream), &launches));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (p.dpad) {
+    const size_t rows = (size_t)p.slabs * p.cfg.seq_len;
+    WERSA_CUDA(launch_pad_cols(X, ctx->ws.Qp, rows, p.cfg.head_dim, kind, st, &launches));
+    WERSA_CUDA(launch_haar_filter(p, ctx->ws.Qp, kind, f, ctx->ws.Op, kind, st, &launches));
+    WERSA_CUDA(launch_unpad_cols(ctx->ws.Op, XF, rows, p.cfg.head_dim, kind, st, &launches));
+    return WERSA_OK;
+  }
+  WERSA_CUDA(launch_haar_filter(p, X, kind, f, XF, kind, st, &launches));
   return WERSA_OK;
 }
 
@@ -406,6 +553,7 @@ wersa_status wersa_gate_static(const wersa_config* cfg, const void* Q, const flo
   Plan p;
   wersa_status s = make_plan(*cfg, &p);
   if (s != WERSA_OK) return s;
+  if (p.dpad) return WERSA_ERR_UNSUPPORTED;   // no workspace to pad into
   if (static_scratch_floats_needed(p) > static_scratch_capacity_floats() ||
       static_scratch_counters_needed(p) > static_scratch_counter_capacity())
     return WERSA_ERR_TOO_LARGE;
@@ -426,8 +574,8 @@ wersa_status wersa_saved(wersa_ctx* ctx, int which, const float** device_ptr, si
   switch (which) {
     case 0: *device_ptr = ctx->ws.f; *count = slabs * p.L1; break;
     case 1: *device_ptr = ctx->ws.qbar; *count = slabs * kD; break;
-    case 2: *device_ptr = ctx->ws.S; *count = slabs * p.cfg.features * kD; break;
-    case 3: *device_ptr = ctx->ws.z; *count = slabs * p.cfg.features; break;
+    case 2: *device_ptr = p.groups > 1 ? ctx->ws.Sout : ctx->ws.S; *count = slabs * p.cfg.features * kD; break;
+    case 3: *device_ptr = p.groups > 1 ? ctx->ws.zout : ctx->ws.z; *count = slabs * p.cfg.features; break;
     default: return WERSA_ERR_INVALID_ARG;
   }
   return WERSA_OK;

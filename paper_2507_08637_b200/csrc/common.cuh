@@ -10,7 +10,8 @@
 
 namespace wersa {
 
-constexpr int kD = 64;           // head dim (fixed)
+constexpr int kD = 64;           // head dim the kernels work on (narrower heads are zero-padded to it)
+constexpr int kGroupFeatures = 256;   // widest feature map of one kernel launch; wider maps run in groups
 constexpr int kMaxLevels = 8;    // Haar levels supported: block of 2^8 = 256 tokens
 constexpr int kHaarTile = 256;   // tokens per Haar tile (>= 2^kMaxLevels)
 constexpr int kSimtTile = 32;    // tokens per tile in the fp32 FFMA kernels
@@ -26,6 +27,8 @@ struct Plan {
   bool grad_bf16;     // storage type of dQ,dK,dV
   bool use_tc;        // bf16 tcgen05 forward kernels
   bool with_backward;
+  bool dpad;          // cfg.head_dim < 64: tensors pass through zero-padded 64-wide copies in the workspace
+  int groups;         // feature groups of kGroupFeatures (1 when cfg.features <= 256)
   // mean pool
   int qchunks, qchunk_rows;
   // haar tiles
@@ -39,7 +42,8 @@ struct Plan {
   // workspace offsets (bytes)
   size_t off_status, off_counters, status_bytes, off_qpart, off_qbar, off_sg, off_f, off_spart, off_zpart, off_S, off_z,
       off_Sbf, off_Wt, off_dS, off_dz, off_sumdD, off_bands, off_dqbar, off_QF, off_KF, off_dQF,
-      off_dKF, off_dSbf, off_KF3, off_QF3, off_Slo, off_Simg, total;
+      off_dKF, off_dSbf, off_KF3, off_QF3, off_Slo, off_Simg, off_Qp, off_Kp, off_Vp, off_Op, off_Wp, off_gwp,
+      off_dOp, off_dQp, off_dKp, off_dVp, off_dgwp, off_Og, off_den, off_Sout, off_zout, total;
   int part_chunks;    // max(schunks, tchunks): leading extent of the partial buffers
 };
 
@@ -53,6 +57,12 @@ struct Ws {   // resolved workspace pointers
   __nv_bfloat16 *Sbf, *Wt, *dSbf, *KF3, *QF3, *Slo;   // Slo = bf16(S' - bf16(S')), built by the backward
   uint8_t* Simg;   // [S' | z' | 0]^T operand images of the query-side kernel, one per slab (see simg_offset)
   float *QF, *KF, *dQF, *dKF;
+  // head_dim < 64: padded copies of the inputs and outputs (storage / gradient type), of W and of the gate weights
+  void *Qp, *Kp, *Vp, *Op, *Wp, *dOp, *dQp, *dKp, *dVp;
+  float *gwp, *dgwp;
+  // features > 256: per-group outputs and denominators, and the slab-major S', z' handed out by wersa_saved
+  void* Og;
+  float *den, *Sout, *zout;
 };
 Ws resolve(const Plan& p, void* workspace);
 
@@ -111,7 +121,8 @@ cudaError_t launch_simt_bwd_kside(const Plan& p, const Ws& w, const void* V, con
 // Both read the raw bf16 tensors and apply the Haar filter (coefficients from w.f) on chip.
 cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const void* V, cudaStream_t st,
                             int* launches);
-cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const float* beta, void* O,
+// den != nullptr (features == 256 only): also leaves every token's denominator in den[slab * n + token].
+cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const float* beta, void* O, float* den,
                             cudaStream_t st, int* launches);
 
 // ---- tc_bwd.cu -----------------------------------------------------------------------------
@@ -124,6 +135,17 @@ cudaError_t launch_tc_bwd_qside(const Plan& p, const Ws& w, const void* QF3, con
                                 cudaStream_t st, int* launches);
 cudaError_t launch_tc_bwd_kside(const Plan& p, const Ws& w, const void* KF3, const void* V, void* dV,
                                 cudaStream_t st, int* launches);
+
+// ---- glue.cu -------------------------------------------------------------------------------
+// kind: 0 = float, 1 = bf16.  rows x d <-> rows x 64 (zero-filled); d is a multiple of 8.
+cudaError_t launch_pad_cols(const void* src, void* dst, size_t rows, int d, int kind, cudaStream_t st, int* launches);
+cudaError_t launch_unpad_cols(const void* src, void* dst, size_t rows, int d, int kind, cudaStream_t st, int* launches);
+// O = sum_g Og[g] * den[g] / sum_g den[g] per token (Og: groups x tokens x 64, den: groups x tokens).
+cudaError_t launch_combine_groups(const void* Og, const float* den, void* O, size_t tokens, int groups, int kind,
+                                  cudaStream_t st, int* launches);
+// Group-major S', z' ([group][slab][mg][...]) -> slab-major ([slab][groups * mg][...]).
+cudaError_t launch_gather_groups(const float* Sg, const float* zg, float* S, float* z, int slabs, int groups, int mg,
+                                 cudaStream_t st, int* launches);
 
 // ---- selftest.cu ---------------------------------------------------------------------------
 // One CTA whose bounded wait runs out after limit_ns: sets the status word; observed[0] = abort flag,

@@ -837,12 +837,16 @@ __device__ __forceinline__ void relu_span(uint32_t in, uint32_t out) {
 // QTmem).  Per tile: MMA1 (warp 1) -> ReLU pass (warps 4-11, two warps per lane quarter that split the
 // feature columns) -> MMA2 (warp 3) -> epilogue (warps 12-15: drain the accumulator, which frees the buffer
 // for tile t + 2, scale by 1 / (D' + eps'), round to bf16 into one of two staging tiles, TMA store).
-template <int NH, bool kMulti>
+// kDen: the kernel also leaves every token's denominator D' + eps' (as it divides by it, i.e. carrying the
+// filter stage's factor r) in den_out[slab * n + token]: a caller that splits the features into groups
+// combines the groups' outputs with these weights.
+template <int NH, bool kMulti, bool kDen = false>
 __global__ void __launch_bounds__(kThreadsQ, 1)
 k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
            const __grid_constant__ CUtensorMap map_w, const uint8_t* __restrict__ simg_g,
            const float* __restrict__ f, const float* __restrict__ beta, float eps,
-           float bw_floor, int n, int L, int chunk_blocks, int chunks, int items, int* __restrict__ status) {
+           float bw_floor, int n, int L, int chunk_blocks, int chunks, int items, int* __restrict__ status,
+           float* __restrict__ den_out) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   using SL = QsideSmem<NH>;
@@ -1057,6 +1061,10 @@ k_tc_qside(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
       uint8_t* ost = smem + SL::ost + (t & 1) * kTileBytes;
       if (ok) {
         const float inv = 1.f / (__uint_as_float(dd) + epsp);
+        if constexpr (kDen) {
+          const int row = blk0 * kBlk + tt * kTile + et;
+          if (row < n) den_out[(size_t)slab * n + row] = __uint_as_float(dd) + epsp;
+        }
         const f32x2 inv2 = pk2(inv, inv);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -1151,8 +1159,12 @@ cudaError_t make_tile_map(const void* base, int slabs, int n, int box_rows, CUte
 
 }  // namespace
 
+// (the head dimension does not enter: narrower heads reach the kernels zero-padded to 64 columns, and
+// feature maps wider than 256 as groups of 256)
 bool tc_supported(const wersa_config& cfg) {
-  return cfg.dtype == WERSA_BF16 && (cfg.features == 128 || cfg.features == 256) && cfg.head_dim == kD;
+  return cfg.dtype == WERSA_BF16 &&
+         (cfg.features == 128 || cfg.features == 256 ||
+          (cfg.features > kGroupFeatures && cfg.features % kGroupFeatures == 0));
 }
 
 // Both tensor-core kernels are launched as programmatic dependents of the kernel before them.
@@ -1206,8 +1218,8 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
   return err != cudaSuccess ? err : cudaGetLastError();
 }
 
-cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const float* beta, void* O, cudaStream_t st,
-                            int* launches) {
+cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const float* beta, void* O, float* den,
+                            cudaStream_t st, int* launches) {
   CUtensorMap map_q, map_o;
   cudaError_t err;
   if ((err = make_tile_map(Q, p.slabs, p.cfg.seq_len, kTile, &map_q)) != cudaSuccess) return err;
@@ -1223,9 +1235,13 @@ cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const flo
   auto launch = [&](auto kernel, size_t smem_bytes) {
     return launch_pdl(kernel, grid, kThreadsQ, smem_bytes, st, map_q, map_o, map_w, (const uint8_t*)w.Simg,
                       (const float*)w.f, beta, p.cfg.eps, p.cfg.bw_floor, p.cfg.seq_len, p.cfg.levels,
-                      p.tchunk_blocks, p.tchunks, items, w.status);
+                      p.tchunk_blocks, p.tchunks, items, w.status, den);
   };
-  if (p.cfg.features == 256)
+  if (den != nullptr) {   // one group of 256 features of a wider feature map
+    if (p.cfg.features != 256) return cudaErrorInvalidValue;
+    err = multi ? launch(k_tc_qside<2, true, true>, QsideSmem<2>::total)
+                : launch(k_tc_qside<2, false, true>, QsideSmem<2>::total);
+  } else if (p.cfg.features == 256)
     err = multi ? launch(k_tc_qside<2, true>, QsideSmem<2>::total) : launch(k_tc_qside<2, false>, QsideSmem<2>::total);
   else
     err = multi ? launch(k_tc_qside<1, true>, QsideSmem<1>::total) : launch(k_tc_qside<1, false>, QsideSmem<1>::total);

@@ -47,10 +47,16 @@ def test_workspace_bytes_and_validation():
     fwd_only = w.wersa_workspace_bytes(_cfg(flags=w.WERSA_FLAG_FORWARD_ONLY))
     assert full % 256 == 0 and 0 < fwd_only < full
     # invalid or unsupported configurations give 0
-    for bad in (dict(batch=0), dict(heads=-1), dict(seq_len=1), dict(head_dim=32), dict(levels=0),
-                dict(levels=9), dict(features=100), dict(seq_len=100, levels=8), dict(eps=-1.0),
+    for bad in (dict(batch=0), dict(heads=-1), dict(seq_len=1), dict(head_dim=128), dict(head_dim=20), dict(levels=0),
+                dict(levels=9), dict(features=100), dict(features=1280), dict(features=512, dtype="f32"),
+                dict(features=512, flags=w.WERSA_FLAG_SIMT_ONLY), dict(seq_len=100, levels=8), dict(eps=-1.0),
                 dict(bw_floor=0.0)):
         assert w.wersa_workspace_bytes(_cfg(**bad)) == 0, bad
+    # narrower heads run zero-padded (more workspace); feature maps up to 1024 run in groups of 256 (bf16)
+    assert w.wersa_workspace_bytes(_cfg(head_dim=32)) > full
+    assert w.wersa_workspace_bytes(_cfg(head_dim=16, dtype="f32", features=64)) > 0
+    assert w.wersa_workspace_bytes(_cfg(features=1024)) > fwd_only
+    assert w.wersa_workspace_bytes(_cfg(features=512, head_dim=32)) > 0
     # 2^L may reach the next power of two above n (zero padding of the wavelet transform)
     assert w.wersa_workspace_bytes(_cfg(seq_len=200, levels=8)) > 0
 

@@ -150,6 +150,103 @@ def test_forward_small_tensor_core(case):
     _check(to_numpy64(O), ref, "bf16", "O")
 
 
+# ---------------------------------------------------------------- head dimensions below 64, more than 256 features
+NARROW = [
+    dict(B=2, H=2, n=640, d=32, L=2, m=128),       # the paper's head dimension of its text models (Sec. 4.1)
+    dict(B=1, H=3, n=1000, d=16, L=3, m=256),      # Sec. 4.5: 64 dimensions over 4 heads; ragged n
+    dict(B=2, H=1, n=300, d=32, L=4, m=64, gate_per_head=0),
+    dict(B=1, H=2, n=2304, d=8, L=8, m=256),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("case", range(len(NARROW)))
+def test_forward_and_backward_with_narrow_heads(case, dtype):
+    """head_dim < 64 (run as the zero-padded 64-wide problem) against the oracle on the narrow tensors
+    themselves: the output, the saved q-bar, S', z' and every gradient."""
+    import torch
+    cfg = dict(NARROW[case], dtype=dtype, eps=1e-3)
+    inp = wi.make_inputs(**cfg, seed=1400 + case, w_seed=1500 + case, gate_std=0.3, gate_seed=1600 + case,
+                         mean_shift=0.25, scale=0.7, backward=True)
+    ctx = _ctx(cfg)
+    assert ctx.uses_tensor_cores() == (dtype == "bf16" and cfg["m"] >= 128)
+    dev = device_inputs(inp, dtype)
+    args = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    O = ctx.forward(*args)
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0 and tuple(O.shape) == inp["Q"].shape
+    ref, aux = _oracle_forward(cfg, inp, want_aux=True)
+    _check(to_numpy64(O), ref, dtype, "O")
+    tol = 1e-4 if not ctx.uses_tensor_cores() else 2e-2
+    c = 1.0 / (max(float(inp["beta"][0]), 1e-6) * np.sqrt(cfg["m"]))
+    S = to_numpy64(ctx.saved("S"))
+    assert S.shape[-1] == cfg["d"]
+    assert normalised_error(S * c, aux["S"]).max() < tol
+    assert normalised_error(to_numpy64(ctx.saved("z")) * c, aux["z"]).max() < tol
+    assert to_numpy64(ctx.saved("qbar")).shape[-1] == cfg["d"]
+    grads = ctx.backward(*args, dev["dO"])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    assert tuple(grads["dQ"].shape) == inp["Q"].shape and tuple(grads["dgate_w"].shape) == inp["gate_w"].shape
+    _check_backward(cfg, inp, grads)
+
+
+def test_narrow_heads_equal_the_padded_problem_bit_for_bit():
+    """The narrow problem and the same tensors zero-padded to 64 columns by the caller give the same bits."""
+    import torch
+    cfg = dict(B=2, H=2, n=900, d=32, L=3, m=256, dtype="bf16")
+    inp = wi.make_inputs(**cfg, seed=1450, w_seed=1451, gate_std=0.3, gate_seed=1452, mean_shift=0.25, scale=0.7)
+    dev = device_inputs(inp, "bf16")
+    O = _ctx(cfg).forward(dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"],
+                          dev["omega"])
+    pad = lambda t, axis: torch.nn.functional.pad(t, (0, 0) * (t.dim() - 1 - axis) + (0, 32)).contiguous()
+    Qp, Kp, Vp = (pad(dev[k], 3) for k in ("Q", "K", "V"))
+    Wp = torch.cat([dev["W"], torch.zeros_like(dev["W"])], dim=0).contiguous()
+    gwp = torch.cat([dev["gate_w"], torch.zeros_like(dev["gate_w"])], dim=1).contiguous()
+    O64 = _ctx(dict(cfg, d=64)).forward(Qp, Kp, Vp, Wp, dev["beta"], gwp, dev["gate_b"], dev["omega"])
+    torch.cuda.synchronize()
+    assert torch.equal(O64[..., :32].contiguous().view(torch.int16), O.view(torch.int16))
+    assert float(O64[..., 32:].abs().max()) == 0.0
+
+
+WIDE = [
+    dict(B=1, H=2, n=1024, d=64, L=2, m=1024),       # Sec. 3.3: L = 2, m = 1024
+    dict(B=2, H=1, n=3000, d=64, L=5, m=512),        # several chunks per slab (reduction launch per group), ragged
+    dict(B=1, H=1, n=40000, d=64, L=8, m=768),       # many chunks, three groups
+    dict(B=12, H=16, n=512, d=64, L=4, m=512),       # 192 slabs: several work items per CTA, one chunk per slab
+    dict(B=2, H=4, n=700, d=32, L=2, m=1024, gate_per_head=0),   # the paper's text-model shape: d = 32, m = 1024
+]
+
+
+@pytest.mark.parametrize("case", range(len(WIDE)))
+def test_forward_with_wide_feature_maps(case):
+    """m = 512, 768, 1024 (groups of 256 features combined by their denominators) against the oracle on the
+    whole feature map: the output and the saved S', z'; twice, bit-identical."""
+    import paper_2507_08637_b200 as wersa
+    import torch
+    cfg = dict(WIDE[case], dtype="bf16")
+    inp = wi.make_inputs(**cfg, seed=1700 + case, w_seed=1800 + case, gate_std=0.3, gate_seed=1900 + case,
+                         mean_shift=0.25, scale=0.7)
+    ctx = _ctx(cfg)
+    assert ctx.uses_tensor_cores()
+    dev = device_inputs(inp, "bf16")
+    args = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    O = ctx.forward(*args).clone()
+    O2 = ctx.forward(*args)
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    assert torch.equal(O.view(torch.int16), O2.view(torch.int16))
+    ref, aux = _oracle_forward(cfg, inp, want_aux=True)
+    c = 1.0 / (max(float(inp["beta"][0]), 1e-6) * np.sqrt(cfg["m"]))
+    errS = normalised_error(to_numpy64(ctx.saved("S")) * c, aux["S"])
+    errz = normalised_error(to_numpy64(ctx.saved("z")) * c, aux["z"])
+    assert errS.max() < 2e-2 and errz.max() < 5e-3, (errS.max(), errz.max())
+    _check(to_numpy64(O), ref, "bf16", "O")
+    with pytest.raises(wersa.WersaError) as e:   # no backward for grouped feature maps
+        ctx.backward(*args, torch.zeros_like(dev["Q"]))
+    assert e.value.status == 2
+
+
 def test_forward_is_bit_identical_run_to_run():
     import paper_2507_08637_b200 as wersa
     import torch
