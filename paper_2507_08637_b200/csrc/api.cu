@@ -60,6 +60,7 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   p->dpad = c.head_dim < kD;
   p->groups = grouped ? c.features / kGroupFeatures : 1;
   p->use_tc = p->bf16 && !(c.flags & WERSA_FLAG_SIMT_ONLY) && tc_supported(c);
+  p->fwd_cols = p->use_tc ? c.head_dim : kD;
   const int n = c.seq_len, m = c.features;
   p->sms = device_sm_count(c.device);
 
@@ -366,7 +367,10 @@ wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const v
   const int kind = p.bf16 ? 1 : 0;
   if ((s = begin_pass(ctx, 0, st)) != WERSA_OK) return s;
   const size_t rows = (size_t)p.slabs * p.cfg.seq_len;
-  if (p.dpad) {   // run the zero-padded 64-wide problem (see glue.cu)
+  // Narrow heads: the tensor-core kernels and the mean pool read and write the narrow tensors themselves (the
+  // tensor maps zero-fill the missing columns); the fp32 path runs on zero-padded copies (see glue.cu).
+  const bool padded = p.dpad && p.fwd_cols == kD;
+  if (padded) {
     WERSA_STEP(0, "pad_q", launch_pad_cols(Q, w.Qp, rows, p.cfg.head_dim, kind, st, &launches));
     WERSA_STEP(0, "pad_k", launch_pad_cols(K, w.Kp, rows, p.cfg.head_dim, kind, st, &launches));
     WERSA_STEP(0, "pad_v", launch_pad_cols(V, w.Vp, rows, p.cfg.head_dim, kind, st, &launches));
@@ -377,9 +381,9 @@ wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const v
     W = w.Wp;
     if (gate_w != nullptr) gate_w = w.gwp;
   }
-  void* Ocore = p.dpad ? w.Op : O;
+  void* Ocore = padded ? w.Op : O;
   WERSA_STEP(0, "qmean_gate",
-             launch_qmean_gate(p, w, Q, gate_w, gate_b, omega, p.use_tc ? W : nullptr, st, &launches));
+             launch_qmean_gate(p, w, Q, gate_w, gate_b, omega, p.use_tc ? W : nullptr, p.fwd_cols, st, &launches));
   if (p.groups > 1) {
     // feature groups of 256 (tensor-core path): every group runs the key side and the query side on its own
     // rows of W^T; the query side leaves O_g and the denominators, which the last launch combines
@@ -395,7 +399,8 @@ wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const v
                  launch_tc_qside(pg, wg, Q, beta, static_cast<char*>(w.Og) + (size_t)g * rows * kD * es,
                                  w.den + (size_t)g * rows, st, &launches));
     }
-    WERSA_STEP(0, "combine_groups", launch_combine_groups(w.Og, w.den, Ocore, rows, p.groups, kind, st, &launches));
+    WERSA_STEP(0, "combine_groups",
+               launch_combine_groups(w.Og, w.den, Ocore, rows, p.groups, p.fwd_cols, kind, st, &launches));
     WERSA_STEP(0, "gather_groups",
                launch_gather_groups(w.S, w.z, w.Sout, w.zout, p.slabs, p.groups, kGroupFeatures, st, &launches));
   } else if (p.use_tc) {
@@ -412,7 +417,7 @@ wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const v
                launch_reduce_partials(p, w.spart, w.zpart, p.schunks, w.S, w.z, nullptr, nullptr, st, &launches));
     WERSA_STEP(0, "simt_qside", launch_simt_qside(p, w, W, beta, Ocore, st, &launches));
   }
-  if (p.dpad) WERSA_STEP(0, "unpad_o", launch_unpad_cols(w.Op, O, rows, p.cfg.head_dim, kind, st, &launches));
+  if (padded) WERSA_STEP(0, "unpad_o", launch_unpad_cols(w.Op, O, rows, p.cfg.head_dim, kind, st, &launches));
   ctx->launches_fwd = launches;
   ctx->forward_done = true;
   return WERSA_OK;

@@ -29,6 +29,8 @@ struct Plan {
   bool with_backward;
   bool dpad;          // cfg.head_dim < 64: tensors pass through zero-padded 64-wide copies in the workspace
   int groups;         // feature groups of kGroupFeatures (1 when cfg.features <= 256)
+  int fwd_cols;       // columns of Q, K, V, O as the forward kernels see them: head_dim on the tensor-core path
+                      // (the tensor maps zero-fill up to 64), 64 on the fp32 path (padded copies)
   // mean pool
   int qchunks, qchunk_rows;
   // haar tiles
@@ -69,8 +71,10 @@ Ws resolve(const Plan& p, void* workspace);
 // ---- gate.cu -------------------------------------------------------------------------------
 // Partial column sums of Q over row chunks, then qbar, sigmoid(u) and f per slab (Eqs. 1-3).
 // With W != nullptr the second launch also leaves the bf16 transpose of W (m x 64) in w.Wt.
+// cols: columns of Q as stored (64, or the head dimension when Q comes unpadded; then gate_w has cols rows
+// per head and W cols rows).
 cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const float* gate_w,
-                              const float* gate_b, const float* omega, const void* W, cudaStream_t st,
+                              const float* gate_b, const float* omega, const void* W, int cols, cudaStream_t st,
                               int* launches);
 // Gate backward: band inner products -> df -> domega, dgate_b, dgate_w, dqbar; dbeta.
 cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, const float* gate_w,
@@ -141,8 +145,9 @@ cudaError_t launch_tc_bwd_kside(const Plan& p, const Ws& w, const void* KF3, con
 cudaError_t launch_pad_cols(const void* src, void* dst, size_t rows, int d, int kind, cudaStream_t st, int* launches);
 cudaError_t launch_unpad_cols(const void* src, void* dst, size_t rows, int d, int kind, cudaStream_t st, int* launches);
 // O = sum_g Og[g] * den[g] / sum_g den[g] per token (Og: groups x tokens x 64, den: groups x tokens).
-cudaError_t launch_combine_groups(const void* Og, const float* den, void* O, size_t tokens, int groups, int kind,
-                                  cudaStream_t st, int* launches);
+// O has `cols` columns (the first `cols` of the 64 are written).
+cudaError_t launch_combine_groups(const void* Og, const float* den, void* O, size_t tokens, int groups, int cols,
+                                  int kind, cudaStream_t st, int* launches);
 // Group-major S', z' ([group][slab][mg][...]) -> slab-major ([slab][groups * mg][...]).
 cudaError_t launch_gather_groups(const float* Sg, const float* zg, float* S, float* z, int slabs, int groups, int mg,
                                  cudaStream_t st, int* launches);

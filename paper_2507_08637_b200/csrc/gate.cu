@@ -24,7 +24,7 @@ __device__ __forceinline__ void slab_gate(const float* __restrict__ qpart, int q
                                           int per_head, const float* __restrict__ gate_w,
                                           const float* __restrict__ gate_b, const float* __restrict__ omega,
                                           float* __restrict__ qbar, float* __restrict__ sg, float* __restrict__ f,
-                                          float (*red)[kD], float* qs) {
+                                          float (*red)[kD], float* qs, int dcols) {
   const int h = slab % H;
   const int c = threadIdx.x & (kD - 1), part = threadIdx.x >> 6;   // 4 interleaved partial sums per column
   float s = 0.f;
@@ -50,8 +50,8 @@ __device__ __forceinline__ void slab_gate(const float* __restrict__ qpart, int q
   if (gate_w != nullptr && i < L1) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const int kk = seg * 4 + j;
-      u += gate_w[((size_t)h * kD + kk) * L1 + i] * qs[kk];
+      const int kk = seg * 4 + j;   // gate_w is (heads, dcols, L1); columns >= dcols of qbar are zero padding
+      if (kk < dcols) u += gate_w[((size_t)h * dcols + kk) * L1 + i] * qs[kk];
     }
   }
 #pragma unroll
@@ -93,7 +93,10 @@ __device__ __forceinline__ void batch_gate(int b, int H, int L1, const float* __
 // result does not depend on which CTA comes last.  The counters start at zero and are left at zero.
 // Row y == slabs (only with W != nullptr): bf16 transpose Wt (m x 64) of W (64 x m) for the
 // tensor-core kernels.
-template <typename T>
+// kFull = false: Q has dcols < 64 columns (a multiple of 8), gate_w dcols rows per head and W dcols rows;
+// dcols / 8 threads share a row, 256 / (dcols / 8) rows are in flight per pass, and the partial sums, q-bar
+// and W^T come out 64 wide with zeros in the columns past dcols.
+template <typename T, bool kFull>
 __global__ void __launch_bounds__(256) k_qmean_gate(const T* __restrict__ Q, float* __restrict__ qpart, int n,
                                                     int chunk_rows, int slabs, int H, int L1, int per_head,
                                                     const float* __restrict__ gate_w, const float* __restrict__ gate_b,
@@ -101,52 +104,60 @@ __global__ void __launch_bounds__(256) k_qmean_gate(const T* __restrict__ Q, flo
                                                     float* __restrict__ sg, float* __restrict__ f,
                                                     int* __restrict__ slab_count, int* __restrict__ batch_count,
                                                     const __nv_bfloat16* __restrict__ W, __nv_bfloat16* __restrict__ Wt,
-                                                    int m) {
+                                                    int m, int dcols_arg) {
+  const int dcols = kFull ? kD : dcols_arg;
   // the key-side kernel may be staged now (programmatic dependent launch; it waits for this grid
   // before it reads W^T or the gate)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if ((int)blockIdx.y == slabs) {
     for (int i = blockIdx.x * 256 + threadIdx.x; i < m * kD; i += gridDim.x * 256) {
       const int r = i / kD, c = i - r * kD;
-      Wt[i] = W[(size_t)c * m + r];
+      Wt[i] = c < dcols ? W[(size_t)c * m + r] : __float2bfloat16_rn(0.f);
     }
     return;
   }
   const int chunk = blockIdx.x, slab = blockIdx.y;
-  const int cg = threadIdx.x & 7, rl = threadIdx.x >> 3;
+  const int cgs = kFull ? 8 : dcols >> 3;      // threads across a row
+  const int rp = kFull ? 32 : 256 / cgs;       // rows per pass
+  const int cg = kFull ? (threadIdx.x & 7) : (int)threadIdx.x % cgs;
+  const int rl = kFull ? (threadIdx.x >> 3) : (int)threadIdx.x / cgs;
   const int r0 = chunk * chunk_rows;
   const int r1 = min(n, r0 + chunk_rows);
-  const T* base = Q + (size_t)slab * n * kD + cg * 8;
+  const T* base = Q + (size_t)slab * n * dcols + cg * 8;
   float acc[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-  int r = r0 + rl;
-  for (; r + 96 < r1; r += 128) {
+  int r = rl < rp ? r0 + rl : r1;              // (256 need not be a multiple of cgs: the last threads idle)
+  for (; r + 3 * rp < r1; r += 4 * rp) {
     float v0[8], v1[8], v2[8], v3[8];
-    load8(base + (size_t)r * kD, v0);
-    load8(base + (size_t)(r + 32) * kD, v1);
-    load8(base + (size_t)(r + 64) * kD, v2);
-    load8(base + (size_t)(r + 96) * kD, v3);
+    load8(base + (size_t)r * dcols, v0);
+    load8(base + (size_t)(r + rp) * dcols, v1);
+    load8(base + (size_t)(r + 2 * rp) * dcols, v2);
+    load8(base + (size_t)(r + 3 * rp) * dcols, v3);
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] += (v0[j] + v1[j]) + (v2[j] + v3[j]);
   }
-  for (; r < r1; r += 32) {
+  for (; r < r1; r += rp) {
     float v0[8];
-    load8(base + (size_t)r * kD, v0);
+    load8(base + (size_t)r * dcols, v0);
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] += v0[j];
   }
-  __shared__ float red[32][kD + 1];
+  __shared__ float red[kFull ? 32 * (kD + 1) : 256 * 9];   // rp rows of dcols + 1 floats
   __shared__ float red4[4][kD];
   __shared__ float qs[kD];
   __shared__ int s_last;
+  if (rl < rp) {
 #pragma unroll
-  for (int j = 0; j < 8; ++j) red[rl][cg * 8 + j] = acc[j];
+    for (int j = 0; j < 8; ++j) red[rl * (dcols + 1) + cg * 8 + j] = acc[j];
+  }
   __syncthreads();
   if (threadIdx.x < kD) {
     float s = 0.f;
+    if ((int)threadIdx.x < dcols) {
 #pragma unroll 8
-    for (int i = 0; i < 32; ++i) s += red[i][threadIdx.x];   // fixed order
+      for (int i = 0; i < rp; ++i) s += red[i * (dcols + 1) + threadIdx.x];   // fixed order
+    }
     qpart[((size_t)slab * gridDim.x + chunk) * kD + threadIdx.x] = s;
     __threadfence();
   }
@@ -155,7 +166,7 @@ __global__ void __launch_bounds__(256) k_qmean_gate(const T* __restrict__ Q, flo
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  slab_gate(qpart, gridDim.x, slab, H, n, L1, per_head, gate_w, gate_b, omega, qbar, sg, f, red4, qs);
+  slab_gate(qpart, gridDim.x, slab, H, n, L1, per_head, gate_w, gate_b, omega, qbar, sg, f, red4, qs, dcols);
   if (threadIdx.x == 0) slab_count[slab] = 0;
   if (per_head) return;
   __threadfence();
@@ -279,26 +290,31 @@ __global__ void __launch_bounds__(kD) k_gate_backward(
 // The launch shared by the workspace and the static-scratch variants.
 static cudaError_t launch_qmean_gate_impl(const Plan& p, const void* Q, float* qpart, const float* gate_w,
                                           const float* gate_b, const float* omega, float* qbar, float* sg, float* f,
-                                          int* counters, const void* W, __nv_bfloat16* Wt, cudaStream_t st) {
+                                          int* counters, const void* W, __nv_bfloat16* Wt, int cols,
+                                          cudaStream_t st) {
   dim3 grid(p.qchunks, p.slabs + (W != nullptr ? 1 : 0));
   int* slab_count = counters;
   int* batch_count = counters + p.slabs;
-  if (p.bf16)
-    k_qmean_gate<__nv_bfloat16><<<grid, 256, 0, st>>>(
-        (const __nv_bfloat16*)Q, qpart, p.cfg.seq_len, p.qchunk_rows, p.slabs, p.cfg.heads, p.L1, p.cfg.gate_per_head,
-        gate_w, gate_b, omega, qbar, sg, f, slab_count, batch_count, (const __nv_bfloat16*)W, Wt, p.cfg.features);
-  else
-    k_qmean_gate<float><<<grid, 256, 0, st>>>((const float*)Q, qpart, p.cfg.seq_len, p.qchunk_rows, p.slabs,
-                                              p.cfg.heads, p.L1, p.cfg.gate_per_head, gate_w, gate_b, omega, qbar, sg,
-                                              f, slab_count, batch_count, (const __nv_bfloat16*)W, Wt, p.cfg.features);
+  auto launch = [&](auto kernel, auto* q) {
+    kernel<<<grid, 256, 0, st>>>(q, qpart, p.cfg.seq_len, p.qchunk_rows, p.slabs, p.cfg.heads, p.L1,
+                                 p.cfg.gate_per_head, gate_w, gate_b, omega, qbar, sg, f, slab_count, batch_count,
+                                 (const __nv_bfloat16*)W, Wt, p.cfg.features, cols);
+  };
+  if (p.bf16) {
+    if (cols == kD) launch(k_qmean_gate<__nv_bfloat16, true>, (const __nv_bfloat16*)Q);
+    else launch(k_qmean_gate<__nv_bfloat16, false>, (const __nv_bfloat16*)Q);
+  } else {
+    if (cols == kD) launch(k_qmean_gate<float, true>, (const float*)Q);
+    else launch(k_qmean_gate<float, false>, (const float*)Q);
+  }
   return cudaGetLastError();
 }
 
 cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const float* gate_w,
-                              const float* gate_b, const float* omega, const void* W, cudaStream_t st,
+                              const float* gate_b, const float* omega, const void* W, int cols, cudaStream_t st,
                               int* launches) {
   *launches += 1;
-  return launch_qmean_gate_impl(p, Q, w.qpart, gate_w, gate_b, omega, w.qbar, w.sg, w.f, w.counters, W, w.Wt, st);
+  return launch_qmean_gate_impl(p, Q, w.qpart, gate_w, gate_b, omega, w.qbar, w.sg, w.f, w.counters, W, w.Wt, cols, st);
 }
 
 // Device address of the static scratch array on the current device, resolved once per device.
@@ -331,7 +347,7 @@ cudaError_t launch_qmean_gate_static(const Plan& p, float* scratch, const void* 
   int* counters = reinterpret_cast<int*>(scratch + (kStaticScratchFloats - kStaticCounterInts));
   cudaError_t err = cudaMemsetAsync(counters, 0, sizeof(int) * ((size_t)p.slabs + (size_t)p.cfg.batch), st);
   if (err != cudaSuccess) return err;
-  return launch_qmean_gate_impl(p, Q, qpart, gate_w, gate_b, omega, qbar, sg, f, counters, nullptr, nullptr, st);
+  return launch_qmean_gate_impl(p, Q, qpart, gate_w, gate_b, omega, qbar, sg, f, counters, nullptr, nullptr, kD, st);
 }
 
 size_t static_scratch_floats_needed(const Plan& p) {

@@ -40,15 +40,15 @@ __global__ void __launch_bounds__(256) k_unpad_cols(const T* __restrict__ src, T
   store8(dst + row * d + c0, v);
 }
 
-// O[tok][:] = sum_g Og[g][tok][:] * den[g][tok] / sum_g den[g][tok], groups in a fixed order.
-// One thread per 8 columns of a token; tokens = slabs * n.
+// O[tok][:] = sum_g Og[g][tok][:] * den[g][tok] / sum_g den[g][tok], groups in a fixed order.  Og is 64 wide,
+// O has `cols` columns.  One thread per 8 columns of a token; tokens = slabs * n.
 template <typename T>
 __global__ void __launch_bounds__(256) k_combine_groups(const T* __restrict__ Og, const float* __restrict__ den,
-                                                        T* __restrict__ O, size_t tokens, int groups) {
+                                                        T* __restrict__ O, size_t tokens, int groups, int cols) {
   const size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x;
   const size_t tok = idx >> 3;
   const int c0 = (int)(idx & 7) * 8;
-  if (tok >= tokens) return;
+  if (tok >= tokens || c0 >= cols) return;
   float acc[8], dsum = 0.f;
 #pragma unroll
   for (int j = 0; j < 8; ++j) acc[j] = 0.f;
@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(256) k_combine_groups(const T* __restrict__ Og
   const float inv = 1.f / dsum;
 #pragma unroll
   for (int j = 0; j < 8; ++j) acc[j] *= inv;
-  store8(O + tok * kD + c0, acc);
+  store8(O + tok * cols + c0, acc);
 }
 
 // Group-major S' and z' (as the kernels leave them: [group][slab][256][...]) -> slab-major [slab][m][...].
@@ -106,13 +106,14 @@ cudaError_t launch_unpad_cols(const void* src, void* dst, size_t rows, int d, in
   return cudaGetLastError();
 }
 
-cudaError_t launch_combine_groups(const void* Og, const float* den, void* O, size_t tokens, int groups, int kind,
-                                  cudaStream_t st, int* launches) {
+cudaError_t launch_combine_groups(const void* Og, const float* den, void* O, size_t tokens, int groups, int cols,
+                                  int kind, cudaStream_t st, int* launches) {
   if (kind == 1)
     k_combine_groups<__nv_bfloat16><<<blocks_for(tokens * 8), 256, 0, st>>>((const __nv_bfloat16*)Og, den,
-                                                                           (__nv_bfloat16*)O, tokens, groups);
+                                                                           (__nv_bfloat16*)O, tokens, groups, cols);
   else
-    k_combine_groups<float><<<blocks_for(tokens * 8), 256, 0, st>>>((const float*)Og, den, (float*)O, tokens, groups);
+    k_combine_groups<float><<<blocks_for(tokens * 8), 256, 0, st>>>((const float*)Og, den, (float*)O, tokens, groups,
+                                                                   cols);
   *launches += 1;
   return cudaGetLastError();
 }

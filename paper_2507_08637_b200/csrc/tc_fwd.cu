@@ -1144,11 +1144,13 @@ EncodeTiledFn encode_fn() {
 
 // (slabs x n x 64) bf16 row-major tensor, boxes of `box_rows` rows x 64 columns of one slab, 128-byte
 // swizzle.  Rows past the end of a slab read as zeros and are not written.
-cudaError_t make_tile_map(const void* base, int slabs, int n, int box_rows, CUtensorMap* out) {
+// Rows of `cols` bf16 values (a multiple of 8: row pitches are multiples of 16 bytes); the box is always 64
+// columns wide, so that a narrower tensor arrives zero-filled up to column 63 and is stored clipped.
+cudaError_t make_tile_map(const void* base, int slabs, int n, int box_rows, CUtensorMap* out, int cols = kD) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return cudaErrorNotSupported;
-  const cuuint64_t dims[3] = {kD, (cuuint64_t)n, (cuuint64_t)slabs};
-  const cuuint64_t strides[2] = {kD * 2, (cuuint64_t)n * kD * 2};
+  const cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)n, (cuuint64_t)slabs};
+  const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)n * cols * 2};
   const cuuint32_t box[3] = {kD, (cuuint32_t)box_rows, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
@@ -1159,8 +1161,8 @@ cudaError_t make_tile_map(const void* base, int slabs, int n, int box_rows, CUte
 
 }  // namespace
 
-// (the head dimension does not enter: narrower heads reach the kernels zero-padded to 64 columns, and
-// feature maps wider than 256 as groups of 256)
+// (the head dimension does not enter: the tensor maps zero-fill narrower heads up to 64 columns, and feature
+// maps wider than 256 run as groups of 256)
 bool tc_supported(const wersa_config& cfg) {
   return cfg.dtype == WERSA_BF16 &&
          (cfg.features == 128 || cfg.features == 256 ||
@@ -1189,8 +1191,8 @@ cudaError_t launch_tc_kside(const Plan& p, const Ws& w, const void* K, const voi
                             int* launches) {
   CUtensorMap map_k, map_v;
   cudaError_t err;
-  if ((err = make_tile_map(K, p.slabs, p.cfg.seq_len, kTile, &map_k)) != cudaSuccess) return err;
-  if ((err = make_tile_map(V, p.slabs, p.cfg.seq_len, kTile, &map_v)) != cudaSuccess) return err;
+  if ((err = make_tile_map(K, p.slabs, p.cfg.seq_len, kTile, &map_k, p.fwd_cols)) != cudaSuccess) return err;
+  if ((err = make_tile_map(V, p.slabs, p.cfg.seq_len, kTile, &map_v, p.fwd_cols)) != cudaSuccess) return err;
   CUtensorMap map_w;   // W^T (m x 64) as one slab of m rows
   if ((err = make_tile_map(w.Wt, 1, p.cfg.features, kTile, &map_w)) != cudaSuccess) return err;
   const int items = p.tchunks * p.slabs;   // (slab, chunk) pairs; one CTA per SM walks them
@@ -1222,8 +1224,10 @@ cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const flo
                             cudaStream_t st, int* launches) {
   CUtensorMap map_q, map_o;
   cudaError_t err;
-  if ((err = make_tile_map(Q, p.slabs, p.cfg.seq_len, kTile, &map_q)) != cudaSuccess) return err;
-  if ((err = make_tile_map(O, p.slabs, p.cfg.seq_len, kTile, &map_o)) != cudaSuccess) return err;
+  // (with feature groups O is a 64-wide buffer of the workspace, else the caller's tensor)
+  if ((err = make_tile_map(Q, p.slabs, p.cfg.seq_len, kTile, &map_q, p.fwd_cols)) != cudaSuccess) return err;
+  if ((err = make_tile_map(O, p.slabs, p.cfg.seq_len, kTile, &map_o, den != nullptr ? kD : p.fwd_cols)) != cudaSuccess)
+    return err;
   // (the query side may start while the reduction that produces S', z' is still running; it waits for
   // that kernel where it first needs its results)
   CUtensorMap map_w;
