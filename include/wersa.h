@@ -70,10 +70,9 @@ typedef struct wersa_config {
                             64-wide copies in the workspace, which leaves Eqs. 1-7 unchanged) */
   int32_t levels;        /* L, Haar levels, 1..8                                        */
   int32_t features;      /* m, random features: 64, 128 or 256; with dtype bf16 and without
-                            WERSA_FLAG_SIMT_ONLY also 512, 768 and 1024 (Sec. 3.3 uses 1024),
-                            forward only: the features run in groups of 256 whose outputs
-                            are combined by their denominators, wersa_backward then returns
-                            WERSA_ERR_UNSUPPORTED                                        */
+                            WERSA_FLAG_SIMT_ONLY also 512, 768 and 1024 (Sec. 3.3 uses 1024):
+                            the features then run in groups of 256 whose outputs are combined
+                            by their denominators (the cost grows with the number of groups) */
   int32_t dtype;         /* wersa_dtype of Q, K, V, W, O, dO; accumulation is fp32      */
   int32_t grad_dtype;    /* wersa_dtype of dQ, dK, dV                                   */
   float eps;             /* denominator epsilon of Eq. 7 (paper: "small constant")      */

@@ -41,7 +41,7 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   // head dimensions 8, 16, ... 64 (narrower ones run zero-padded to 64 columns)
   if (c.head_dim > kD || c.head_dim < 8 || c.head_dim % 8 != 0) return WERSA_ERR_UNSUPPORTED;
   if (c.levels > kMaxLevels) return WERSA_ERR_UNSUPPORTED;
-  // feature maps of 64, 128 or 256, and (bf16 tensor-core path, forward only) 512, 768, 1024 in groups of 256
+  // feature maps of 64, 128 or 256, and (bf16 tensor-core path) 512, 768, 1024 in groups of 256
   const bool grouped = c.features > kGroupFeatures;
   if (grouped) {
     if (c.features % kGroupFeatures != 0 || c.features > 4 * kGroupFeatures) return WERSA_ERR_UNSUPPORTED;
@@ -56,7 +56,7 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
   p->L1 = c.levels + 1;
   p->bf16 = c.dtype == WERSA_BF16;
   p->grad_bf16 = c.grad_dtype == WERSA_BF16;
-  p->with_backward = !(c.flags & WERSA_FLAG_FORWARD_ONLY) && !grouped;
+  p->with_backward = !(c.flags & WERSA_FLAG_FORWARD_ONLY);
   p->dpad = c.head_dim < kD;
   p->groups = grouped ? c.features / kGroupFeatures : 1;
   p->use_tc = p->bf16 && !(c.flags & WERSA_FLAG_SIMT_ONLY) && tc_supported(c);
@@ -153,7 +153,9 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
     p->off_dKp = take(p->dpad ? grad_bytes * slab_elems : 0);
     p->off_dVp = take(p->dpad ? grad_bytes * slab_elems : 0);
     p->off_dgwp = take(p->dpad ? sizeof(float) * (size_t)c.heads * kD * p->L1 : 0);
+    p->off_Dtot = take(grouped ? sizeof(float) * 2 * slabs * n : 0);
   } else {
+    p->off_Dtot = 0;
     p->off_dS = p->off_dz = p->off_sumdD = p->off_bands = p->off_dqbar = p->off_dQF = p->off_dKF = p->off_dSbf = p->off_KF3 = p->off_QF3 = p->off_Slo = 0;
     p->off_dOp = p->off_dQp = p->off_dKp = p->off_dVp = p->off_dgwp = 0;
   }
@@ -205,6 +207,7 @@ Ws resolve(const Plan& p, void* workspace) {
   w.den = reinterpret_cast<float*>(b + p.off_den);
   w.Sout = reinterpret_cast<float*>(b + p.off_Sout);
   w.zout = reinterpret_cast<float*>(b + p.off_zout);
+  w.Dtot = reinterpret_cast<float*>(b + p.off_Dtot);
   return w;
 }
 
@@ -282,12 +285,19 @@ Plan group_plan(const Plan& p) {
   pg.cfg.features = kGroupFeatures;
   return pg;
 }
-Ws group_view(const Plan& p, const Ws& w, int g) {
+// `chunks`: chunks per slab of the partial sums the view is used with (forward: p.tchunks, backward: p.bchunks).
+Ws group_view(const Plan& p, const Ws& w, int g, int chunks) {
   Ws v = w;
   const size_t slabs = (size_t)p.slabs, mg = kGroupFeatures;
   v.Wt = w.Wt + (size_t)g * mg * kD;
-  v.spart = w.spart + (size_t)g * slabs * p.tchunks * mg * kD;
-  v.zpart = w.zpart + (size_t)g * slabs * p.tchunks * mg;
+  v.spart = w.spart + (size_t)g * slabs * chunks * mg * kD;
+  v.zpart = w.zpart + (size_t)g * slabs * chunks * mg;
+  if (p.with_backward) {
+    v.dS = w.dS + (size_t)g * slabs * mg * kD;
+    v.dz = w.dz + (size_t)g * slabs * mg;
+    v.dSbf = w.dSbf + (size_t)g * slabs * mg * kD;
+    v.Slo = w.Slo + (size_t)g * slabs * mg * kD;
+  }
   v.S = w.S + (size_t)g * slabs * mg * kD;
   v.z = w.z + (size_t)g * slabs * mg;
   v.Sbf = w.Sbf + (size_t)g * slabs * mg * kD;
@@ -390,7 +400,7 @@ wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const v
     const Plan pg = group_plan(p);
     const size_t es = p.bf16 ? 2 : 4;
     for (int g = 0; g < p.groups; ++g) {
-      const Ws wg = group_view(p, w, g);
+      const Ws wg = group_view(p, w, g, p.tchunks);
       WERSA_STEP(0, "tc_kside", launch_tc_kside(pg, wg, K, V, st, &launches));
       if (p.tchunks > 1)
         WERSA_STEP(0, "reduce_partials",
@@ -488,21 +498,43 @@ wersa_status wersa_backward(wersa_ctx* ctx, const void* Q, const void* K, const 
     if (gate_w != nullptr) gate_w = w.gwp;
     if (dgate_w != nullptr) dgate_w = w.dgwp;
   }
-  if (p.use_tc) {
+  if (p.groups > 1) {
+    // Feature groups: the denominator and dD' of the whole map come from what the forward left (the groups'
+    // outputs and denominators); every group then runs both tensor-core kernels on its own rows of W^T, S', z',
+    // dS', dz', and dQ_F, dV, dK_F accumulate over the groups in launch order.
+    WERSA_STEP(1, "haar_filter_q", launch_haar_filter_split3(p, Q, kind, w.f, w.QF3, st, &launches));
+    WERSA_STEP(1, "haar_filter_k", launch_haar_filter_split3(p, K, kind, w.f, w.KF3, st, &launches));
+    WERSA_STEP(1, "group_bwd_prep",
+               launch_group_bwd_prep(w.Og, w.den, dO, w.f, p.cfg.seq_len, p.L1, rows, p.groups, kind, w.Dtot,
+                                     w.Dtot + rows, st, &launches));
+    const Plan pg = group_plan(p);
+    for (int g = 0; g < p.groups; ++g) {
+      const Ws wg = group_view(p, w, g, bwd_chunks);
+      WERSA_STEP(1, "tc_bwd_qside",
+                 launch_tc_bwd_qside(pg, wg, w.QF3, beta, dO, w.Dtot, w.Dtot + rows, g > 0, st, &launches));
+      WERSA_STEP(1, "reduce_partials",
+                 launch_reduce_partials(pg, wg.spart, wg.zpart, bwd_chunks, wg.dS, wg.dz, wg.dSbf, nullptr, st, &launches));
+      WERSA_STEP(1, "tc_bwd_kside", launch_tc_bwd_kside(pg, wg, w.KF3, V, dV, g > 0, st, &launches));
+    }
+  } else if (p.use_tc) {
     // the tensor-core forward keeps Q_F, K_F on chip: rebuild them, as three bf16 planes each
     WERSA_STEP(1, "haar_filter_q", launch_haar_filter_split3(p, Q, kind, w.f, w.QF3, st, &launches));
     WERSA_STEP(1, "haar_filter_k", launch_haar_filter_split3(p, K, kind, w.f, w.KF3, st, &launches));
-    WERSA_STEP(1, "tc_bwd_qside", launch_tc_bwd_qside(p, w, w.QF3, beta, dO, st, &launches));
+    WERSA_STEP(1, "tc_bwd_qside", launch_tc_bwd_qside(p, w, w.QF3, beta, dO, nullptr, nullptr, false, st, &launches));
   } else {
     WERSA_STEP(1, "simt_bwd_qside", launch_simt_bwd_qside(p, w, W, beta, dO, st, &launches));
   }
-  WERSA_STEP(1, "reduce_partials",
-             launch_reduce_partials(p, w.spart, w.zpart, bwd_chunks, w.dS, w.dz, p.use_tc ? w.dSbf : nullptr, nullptr, st,
-                                    &launches));
-  if (p.use_tc)
-    WERSA_STEP(1, "tc_bwd_kside", launch_tc_bwd_kside(p, w, w.KF3, V, dV, st, &launches));
-  else
+  if (p.groups == 1)
+    WERSA_STEP(1, "reduce_partials",
+               launch_reduce_partials(p, w.spart, w.zpart, bwd_chunks, w.dS, w.dz, p.use_tc ? w.dSbf : nullptr, nullptr,
+                                      st, &launches));
+  if (p.groups > 1) {
+    // (done group by group above)
+  } else if (p.use_tc) {
+    WERSA_STEP(1, "tc_bwd_kside", launch_tc_bwd_kside(p, w, w.KF3, V, dV, false, st, &launches));
+  } else {
     WERSA_STEP(1, "simt_bwd_kside", launch_simt_bwd_kside(p, w, V, W, dV, st, &launches));
+  }
   // With gate weights dQ has a second term, d(qbar) / n on every row (Eq. 1), which is known only after the
   // gate backward: the first pass over dQ_F then takes the band inner products alone, and dQ is written
   // once, by a filter pass that adds the row vector.

@@ -45,7 +45,7 @@ struct Plan {
   size_t off_status, off_counters, status_bytes, off_qpart, off_qbar, off_sg, off_f, off_spart, off_zpart, off_S, off_z,
       off_Sbf, off_Wt, off_dS, off_dz, off_sumdD, off_bands, off_dqbar, off_QF, off_KF, off_dQF,
       off_dKF, off_dSbf, off_KF3, off_QF3, off_Slo, off_Simg, off_Qp, off_Kp, off_Vp, off_Op, off_Wp, off_gwp,
-      off_dOp, off_dQp, off_dKp, off_dVp, off_dgwp, off_Og, off_den, off_Sout, off_zout, total;
+      off_dOp, off_dQp, off_dKp, off_dVp, off_dgwp, off_Og, off_den, off_Sout, off_zout, off_Dtot, total;
   int part_chunks;    // max(schunks, tchunks): leading extent of the partial buffers
 };
 
@@ -65,6 +65,7 @@ struct Ws {   // resolved workspace pointers
   // features > 256: per-group outputs and denominators, and the slab-major S', z' handed out by wersa_saved
   void* Og;
   float *den, *Sout, *zout;
+  float* Dtot;   // backward with feature groups: the whole map's denominator per token, then dD' per token
 };
 Ws resolve(const Plan& p, void* workspace);
 
@@ -135,10 +136,13 @@ cudaError_t launch_tc_qside(const Plan& p, const Ws& w, const void* Q, const flo
 // Query-side backward on the tensor cores: dQ_F, and the split-sequence partials of dS', dz' and
 // sum dD' (w.spart, w.zpart, w.sumdD; p.bchunks chunks per slab), from Q_F as three bf16 planes, dO,
 // the bf16 S' image (w.Sbf), z' (w.z) and the bf16 W^T image.
+// Feature groups (p.cfg.features == 256 as one group of a wider map): den_ext / dd_ext hold the whole map's
+// denominator and dD' per token (slabs x n floats each), `add` makes dQ_F (dV, dK_F) accumulate.
 cudaError_t launch_tc_bwd_qside(const Plan& p, const Ws& w, const void* QF3, const float* beta, const void* dO,
+                                const float* den_ext, const float* dd_ext, bool add, cudaStream_t st, int* launches);
+cudaError_t launch_tc_bwd_kside(const Plan& p, const Ws& w, const void* KF3, const void* V, void* dV, bool add,
                                 cudaStream_t st, int* launches);
-cudaError_t launch_tc_bwd_kside(const Plan& p, const Ws& w, const void* KF3, const void* V, void* dV,
-                                cudaStream_t st, int* launches);
+
 
 // ---- glue.cu -------------------------------------------------------------------------------
 // kind: 0 = float, 1 = bf16.  rows x d <-> rows x 64 (zero-filled); d is a multiple of 8.
@@ -148,6 +152,12 @@ cudaError_t launch_unpad_cols(const void* src, void* dst, size_t rows, int d, in
 // O has `cols` columns (the first `cols` of the 64 are written).
 cudaError_t launch_combine_groups(const void* Og, const float* den, void* O, size_t tokens, int groups, int cols,
                                   int kind, cudaStream_t st, int* launches);
+// Backward of the combination: per token the whole map's denominator D = sum_g den_g / r (r = the filter
+// stage's factor carried by the forward's denominators, from f) and dD' = -(dO . O) / D with
+// O = sum_g Og den_g / sum_g den_g.  dO and Og are 64 wide.
+cudaError_t launch_group_bwd_prep(const void* Og, const float* den, const void* dO, const float* f, int n, int L1,
+                                  size_t tokens, int groups, int kind, float* Dtot, float* dDtot, cudaStream_t st,
+                                  int* launches);
 // Group-major S', z' ([group][slab][mg][...]) -> slab-major ([slab][groups * mg][...]).
 cudaError_t launch_gather_groups(const float* Sg, const float* zg, float* S, float* z, int slabs, int groups, int mg,
                                  cudaStream_t st, int* launches);

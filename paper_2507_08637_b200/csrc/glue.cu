@@ -66,6 +66,49 @@ __global__ void __launch_bounds__(256) k_combine_groups(const T* __restrict__ Og
   store8(O + tok * cols + c0, acc);
 }
 
+// One token per 8 threads (8 columns each): O = sum_g Og den_g / sum_g den_g, D = sum_g den_g / r,
+// dD' = -(dO . O) / D.  The forward's denominators carry the factor r = bf16(f_0) / f_0 of its filter stage,
+// which the backward's filtered planes do not.
+template <typename T>
+__global__ void __launch_bounds__(256) k_group_bwd_prep(const T* __restrict__ Og, const float* __restrict__ den,
+                                                        const T* __restrict__ dO, const float* __restrict__ f, int n,
+                                                        int L1, size_t tokens, int groups, float* __restrict__ Dtot,
+                                                        float* __restrict__ dDtot) {
+  const size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x;
+  const size_t tok = idx >> 3;
+  const int c0 = (int)(idx & 7) * 8;
+  const bool live = tok < tokens;
+  float acc[8], dsum = 0.f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+  float dot = 0.f;
+  if (live) {
+    for (int g = 0; g < groups; ++g) {
+      const float dg = den[(size_t)g * tokens + tok];
+      float v[8];
+      load8(Og + ((size_t)g * tokens + tok) * kD + c0, v);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[j] = fmaf(v[j], dg, acc[j]);
+      dsum += dg;
+    }
+    float g8[8];
+    load8(dO + tok * kD + c0, g8);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) dot = fmaf(g8[j], acc[j], dot);
+  }
+#pragma unroll
+  for (int o = 4; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);   // the 8 threads of a token
+  if (live && c0 == 0) {
+    const float f0 = f[(tok / n) * L1];
+    const float f0b = __bfloat162float(__float2bfloat16_rn(f0));
+    const float r = f0 != 0.f ? f0b / f0 : 1.f;
+    const float D = dsum / r;
+    // dot = sum_c dO_c (sum_g Og_c den_g); O = that / dsum
+    Dtot[tok] = D;
+    dDtot[tok] = -(dot / dsum) / D;
+  }
+}
+
 // Group-major S' and z' (as the kernels leave them: [group][slab][256][...]) -> slab-major [slab][m][...].
 __global__ void __launch_bounds__(256) k_gather_groups(const float* __restrict__ Sg, const float* __restrict__ zg,
                                                        float* __restrict__ S, float* __restrict__ z, int slabs,
@@ -114,6 +157,19 @@ cudaError_t launch_combine_groups(const void* Og, const float* den, void* O, siz
   else
     k_combine_groups<float><<<blocks_for(tokens * 8), 256, 0, st>>>((const float*)Og, den, (float*)O, tokens, groups,
                                                                    cols);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_group_bwd_prep(const void* Og, const float* den, const void* dO, const float* f, int n, int L1,
+                                  size_t tokens, int groups, int kind, float* Dtot, float* dDtot, cudaStream_t st,
+                                  int* launches) {
+  if (kind == 1)
+    k_group_bwd_prep<__nv_bfloat16><<<blocks_for(tokens * 8), 256, 0, st>>>(
+        (const __nv_bfloat16*)Og, den, (const __nv_bfloat16*)dO, f, n, L1, tokens, groups, Dtot, dDtot);
+  else
+    k_group_bwd_prep<float><<<blocks_for(tokens * 8), 256, 0, st>>>((const float*)Og, den, (const float*)dO, f, n, L1,
+                                                                   tokens, groups, Dtot, dDtot);
   *launches += 1;
   return cudaGetLastError();
 }

@@ -121,10 +121,16 @@ __device__ __forceinline__ void stage_row32<__nv_bfloat16>(uint8_t* stage, int t
 }
 // Issued by one thread after the CTA barrier that follows the staging writes (each writer has fenced its
 // writes for the async proxy).  Rows past the end of the slab are clipped by the tensor map.
-template <typename TG>
+// kAdd: the tile is added to what the tensor holds (feature groups after the first accumulate their share).
+template <typename TG, bool kAdd = false>
 __device__ __forceinline__ void store_tile(const CUtensorMap* map, const uint8_t* stage, int row0, int slab) {
-  tma_store_3d(map, stage, 0, row0, slab);
-  if (sizeof(TG) == 4) tma_store_3d(map, stage + kTileBytes, 32, row0, slab);
+  if constexpr (kAdd) {
+    tma_reduce_add_3d(map, stage, 0, row0, slab);
+    if (sizeof(TG) == 4) tma_reduce_add_3d(map, stage + kTileBytes, 32, row0, slab);
+  } else {
+    tma_store_3d(map, stage, 0, row0, slab);
+    if (sizeof(TG) == 4) tma_store_3d(map, stage + kTileBytes, 32, row0, slab);
+  }
   bulk_commit_group();
 }
 
@@ -209,7 +215,7 @@ __device__ __forceinline__ void relu_grad_split(uint32_t trow, int wg, const uin
 
 // ---- key side -----------------------------------------------------------------------------------
 // grid (chunks, slabs), block 256.
-template <int NH, typename TG>
+template <int NH, typename TG, bool kAdd = false>
 __global__ void __launch_bounds__(256, 1)
 k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant__ CUtensorMap map_v,
                const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ dSbf,
@@ -357,7 +363,7 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
     __syncthreads();
     // ---- MMA3: G_h = V dS'_h^T
     if (threadIdx.x == 0) {
-      store_tile<TG>(&map_dv, out_stage, row0, slab);
+      store_tile<TG, kAdd>(&map_dv, out_stage, row0, slab);
       tc_fence_after_sync();
 #pragma unroll
       for (int h = 0; h < NH; ++h)
@@ -402,7 +408,7 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();   // the next tile's MMA1 overwrites what this tile read
-    if (threadIdx.x == 0) store_tile<float>(&map_dkf, out_stage + 2 * kTileBytes, row0, slab);
+    if (threadIdx.x == 0) store_tile<float, kAdd>(&map_dkf, out_stage + 2 * kTileBytes, row0, slab);
   }
   if (threadIdx.x == 0) {
     if (!ok)   // copies may still be in flight
@@ -436,7 +442,10 @@ template <int NH> struct BwdQSmem {
 // warpgroups contribute to (D', dD', and with m = 128 dz') meet in the 128-float array `dds`:
 // warpgroup 1 leaves its part there, warpgroup 0 adds its own (always in this order) and leaves the
 // total there for everybody, with the CTA barriers of the step sequence in between.
-template <int NH>
+// kGroup: the launch handles one group of 256 features of a wider feature map.  The denominator of Eq. 7 and
+// dD' then belong to the whole map and come from den_ext / dd_ext (one float per token), and with kAdd the
+// group's share of dQ_F is added to what the groups before it left.
+template <int NH, bool kGroup = false, bool kAdd = false>
 __global__ void __launch_bounds__(256, 1)
 k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant__ CUtensorMap map_do,
                const __grid_constant__ CUtensorMap map_slo, const __nv_bfloat16* __restrict__ Wt,
@@ -444,7 +453,7 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
                const float* __restrict__ zg, const float* __restrict__ beta, float eps, float bw_floor,
                const __grid_constant__ CUtensorMap map_dqf, float* __restrict__ dspart,
                float* __restrict__ dzpart, float* __restrict__ sumdD, int n, int chunk_tiles,
-               int* __restrict__ status) {
+               int* __restrict__ status, const float* __restrict__ den_ext, const float* __restrict__ dd_ext) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   using SL = BwdQSmem<NH>;
@@ -575,7 +584,8 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
     tc_fence_before_sync();
     __syncthreads();
     if (wg == 0) {
-      den = epsp + (den + dds[tl]);
+      if constexpr (kGroup) den = row < n ? den_ext[(size_t)slab * n + row] : 1.f;
+      else den = epsp + (den + dds[tl]);
       dds[tl] = den;
     }
     // ---- MMA2: N'
@@ -624,7 +634,8 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
     tc_fence_before_sync();
     __syncthreads();
     if (wg == 0) {
-      dd = -(dd + dds[tl]) * inv;
+      if constexpr (kGroup) dd = row < n ? dd_ext[(size_t)slab * n + row] : 0.f;
+      else dd = -(dd + dds[tl]) * inv;
       dds[tl] = dd;
       sum_dd += dd;
     }
@@ -711,7 +722,7 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
-    if (threadIdx.x == 0) store_tile<float>(&map_dqf, smem + SL::dn, row0, slab);
+    if (threadIdx.x == 0) store_tile<float, kAdd>(&map_dqf, smem + SL::dn, row0, slab);
   }
   // ---- partial dS', dz', sum dD' of this chunk (zeros if the chunk gave up)
   const size_t pidx = (size_t)slab * gridDim.x + chunk;
@@ -809,14 +820,14 @@ cudaError_t make_out_map(void* base, int slabs, int n, bool bf16, CUtensorMap* o
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-template <int NH, typename TG>
+template <int NH, typename TG, bool kAdd = false>
 cudaError_t launch_kside(const Plan& p, const Ws& w, const CUtensorMap& map_kf, const CUtensorMap& map_v, void* dV,
                          cudaStream_t st) {
   CUtensorMap map_dv, map_dkf;
   cudaError_t merr;
   if ((merr = make_out_map(dV, p.slabs, p.cfg.seq_len, sizeof(TG) == 2, &map_dv)) != cudaSuccess) return merr;
   if ((merr = make_out_map(w.dKF, p.slabs, p.cfg.seq_len, false, &map_dkf)) != cudaSuccess) return merr;
-  auto k = k_tc_bwd_kside<NH, TG>;
+  auto k = k_tc_bwd_kside<NH, TG, kAdd>;
   cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdKSmem<NH>::total);
   if (err != cudaSuccess) return err;
   const long long tiles_all = (long long)((p.cfg.seq_len + kTile - 1) / kTile) * p.slabs;
@@ -826,46 +837,58 @@ cudaError_t launch_kside(const Plan& p, const Ws& w, const CUtensorMap& map_kf, 
   return cudaGetLastError();
 }
 
-template <int NH>
+template <int NH, bool kGroup = false, bool kAdd = false>
 cudaError_t launch_qside(const Plan& p, const Ws& w, const CUtensorMap& map_qf, const CUtensorMap& map_do,
-                         const float* beta, cudaStream_t st) {
+                         const float* beta, cudaStream_t st, const float* den_ext = nullptr,
+                         const float* dd_ext = nullptr) {
   // low-order bf16 image of S' (rows = features of a slab), fetched tile by tile by the kernel
   const size_t count = (size_t)p.slabs * p.cfg.features * kD;
   k_split_lo<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(w.S, w.Sbf, w.Slo, count);
   CUtensorMap map_slo;
   cudaError_t merr;
   if ((merr = make_tile_map(w.Slo, p.slabs, p.cfg.features, &map_slo)) != cudaSuccess) return merr;
-  auto k = k_tc_bwd_qside<NH>;
+  auto k = k_tc_bwd_qside<NH, kGroup, kAdd>;
   cudaError_t err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdQSmem<NH>::total);
   if (err != cudaSuccess) return err;
   CUtensorMap map_dqf;
   if ((err = make_out_map(w.dQF, p.slabs, p.cfg.seq_len, false, &map_dqf)) != cudaSuccess) return err;
   dim3 grid(p.bchunks, p.slabs);
   k<<<grid, 256, BwdQSmem<NH>::total, st>>>(map_qf, map_do, map_slo, w.Wt, w.Sbf, w.z, beta, p.cfg.eps, p.cfg.bw_floor, map_dqf,
-                                            w.spart, w.zpart, w.sumdD, p.cfg.seq_len, p.bchunk_tiles, w.status);
+                                            w.spart, w.zpart, w.sumdD, p.cfg.seq_len, p.bchunk_tiles, w.status, den_ext,
+                                            dd_ext);
   return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_tc_bwd_qside(const Plan& p, const Ws& w, const void* QF3, const float* beta, const void* dO,
-                                cudaStream_t st, int* launches) {
+                                const float* den_ext, const float* dd_ext, bool add, cudaStream_t st, int* launches) {
   CUtensorMap map_qf, map_do;
   cudaError_t err;
   if ((err = make_tile_map(QF3, 3 * p.slabs, p.cfg.seq_len, &map_qf)) != cudaSuccess) return err;
   if ((err = make_tile_map(dO, p.slabs, p.cfg.seq_len, &map_do)) != cudaSuccess) return err;
   *launches += 2;   // the low-order image of S', then the kernel
+  if (den_ext != nullptr) {   // one group of 256 features of a wider map
+    if (p.cfg.features != 256 || dd_ext == nullptr) return cudaErrorInvalidValue;
+    return add ? launch_qside<2, true, true>(p, w, map_qf, map_do, beta, st, den_ext, dd_ext)
+               : launch_qside<2, true, false>(p, w, map_qf, map_do, beta, st, den_ext, dd_ext);
+  }
   return p.cfg.features == 256 ? launch_qside<2>(p, w, map_qf, map_do, beta, st)
                                : launch_qside<1>(p, w, map_qf, map_do, beta, st);
 }
 
-cudaError_t launch_tc_bwd_kside(const Plan& p, const Ws& w, const void* KF3, const void* V, void* dV, cudaStream_t st,
-                                int* launches) {
+cudaError_t launch_tc_bwd_kside(const Plan& p, const Ws& w, const void* KF3, const void* V, void* dV, bool add,
+                                cudaStream_t st, int* launches) {
   CUtensorMap map_kf, map_v;
   cudaError_t err;
   if ((err = make_tile_map(KF3, 3 * p.slabs, p.cfg.seq_len, &map_kf)) != cudaSuccess) return err;
   if ((err = make_tile_map(V, p.slabs, p.cfg.seq_len, &map_v)) != cudaSuccess) return err;
   *launches += 1;
+  if (add) {   // a feature group after the first: dV and dK_F accumulate
+    if (p.cfg.features != 256) return cudaErrorInvalidValue;
+    return p.grad_bf16 ? launch_kside<2, __nv_bfloat16, true>(p, w, map_kf, map_v, dV, st)
+                       : launch_kside<2, float, true>(p, w, map_kf, map_v, dV, st);
+  }
   if (p.cfg.features == 256)
     return p.grad_bf16 ? launch_kside<2, __nv_bfloat16>(p, w, map_kf, map_v, dV, st)
                        : launch_kside<2, float>(p, w, map_kf, map_v, dV, st);

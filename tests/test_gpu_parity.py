@@ -228,7 +228,6 @@ WIDE = [
 def test_forward_with_wide_feature_maps(case):
     """m = 512, 768, 1024 (groups of 256 features combined by their denominators) against the oracle on the
     whole feature map: the output and the saved S', z'; twice, bit-identical."""
-    import paper_2507_08637_b200 as wersa
     import torch
     cfg = dict(WIDE[case], dtype="bf16")
     inp = wi.make_inputs(**cfg, seed=1700 + case, w_seed=1800 + case, gate_std=0.3, gate_seed=1900 + case,
@@ -248,9 +247,39 @@ def test_forward_with_wide_feature_maps(case):
     errz = normalised_error(to_numpy64(ctx.saved("z")) * c, aux["z"])
     assert errS.max() < 2e-2 and errz.max() < 5e-3, (errS.max(), errz.max())
     _check(to_numpy64(O), ref, "bf16", "O")
-    with pytest.raises(wersa.WersaError) as e:   # no backward for grouped feature maps
-        ctx.backward(*args, torch.zeros_like(dev["Q"]))
-    assert e.value.status == 2
+
+
+WIDE_BWD = [
+    dict(B=1, H=2, n=1024, d=64, L=2, m=1024),
+    dict(B=2, H=1, n=1500, d=64, L=5, m=512),
+    dict(B=2, H=2, n=700, d=32, L=2, m=1024, gate_per_head=0),
+    dict(B=1, H=3, n=2304, d=64, L=6, m=768),
+]
+
+
+@pytest.mark.parametrize("grad_dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("case", range(len(WIDE_BWD)))
+def test_backward_with_wide_feature_maps(case, grad_dtype):
+    """Gradients with m = 512, 768, 1024: every group runs the tensor-core backward kernels with the whole map's
+    denominator and dD', and dQ_F, dV, dK_F accumulate over the groups."""
+    import torch
+    if grad_dtype == "bf16" and case not in (0, 2):
+        pytest.skip("bf16 gradients: two cases")
+    cfg = dict(WIDE_BWD[case], dtype="bf16", eps=1e-3)
+    inp = wi.make_inputs(**cfg, seed=2100 + case, w_seed=2200 + case, gate_std=0.3, gate_seed=2300 + case,
+                         mean_shift=0.25, scale=0.7, backward=True)
+    ctx = _ctx(cfg, grad_dtype=grad_dtype)
+    assert ctx.uses_tensor_cores()
+    dev = device_inputs(inp, "bf16")
+    args = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    ctx.forward(*args)
+    grads = ctx.backward(*args, dev["dO"])
+    grads2 = ctx.backward(*args, dev["dO"])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    for k in ("dQ", "dK", "dV"):
+        assert torch.equal(grads[k], grads2[k]), k   # accumulation in launch order: the same bits every time
+    _check_backward(cfg, inp, grads)
 
 
 def test_forward_is_bit_identical_run_to_run():
