@@ -171,6 +171,28 @@ wersa_status wersa_gate_static(const wersa_config* cfg, const void* Q, const flo
                                const float* gate_b, const float* omega, float* qbar, float* f,
                                void* cuda_stream);
 
+/* Sequence-sharded forward.  (The paper runs one GPU; Sec. 3.2's linear cost is what makes sequences longer
+ * than one device's memory worth having.)  The sequence of every slab is cut into contiguous shards, one per
+ * rank, every shard but the last a multiple of 2^levels tokens long, so that no wavelet block straddles two
+ * shards (all shards but the last must therefore also be at least 2^levels long).  Each rank creates its
+ * context with seq_len = its shard's length and calls, on one stream and in this order:
+ *   wersa_shard_pool    Q shard, W -> qsum (batch*heads, 64) floats: column sums of the shard's Q
+ *                       (columns >= head_dim zero).  The caller adds the qsum of all shards.
+ *   wersa_shard_gate    the added sums and the whole sequence's length n_total -> gate (Eqs. 1-3), kept in the
+ *                       context.
+ *   wersa_shard_keys    K, V shards -> this shard's S', z' (read them with wersa_saved, which = 2 and 3).  The
+ *                       caller adds the S' and the z' of all shards (Eq. 7's sums over the tokens).
+ *   wersa_shard_output  Q shard, the added S_total (batch*heads, features, 64) and z_total (batch*heads,
+ *                       features), beta -> O shard.
+ * The two additions are the only exchange between ranks (an all-reduce each; the library does not do them).
+ * bf16 tensor-core contexts with features <= 256 only, else WERSA_ERR_UNSUPPORTED; forward only. */
+wersa_status wersa_shard_pool(wersa_ctx* ctx, const void* Q, const void* W, float* qsum, void* cuda_stream);
+wersa_status wersa_shard_gate(wersa_ctx* ctx, const float* qsum_total, int64_t n_total, const float* gate_w,
+                              const float* gate_b, const float* omega, void* cuda_stream);
+wersa_status wersa_shard_keys(wersa_ctx* ctx, const void* K, const void* V, void* cuda_stream);
+wersa_status wersa_shard_output(wersa_ctx* ctx, const void* Q, const float* S_total, const float* z_total,
+                                const float* beta, void* O, void* cuda_stream);
+
 /* Device pointers into the workspace of quantities the last forward left there.
  * which: 0 = f (batch*heads, levels+1); 1 = qbar (batch*heads, 64);
  *        2 = S' (batch*heads, features, 64); 3 = z' (batch*heads, features),

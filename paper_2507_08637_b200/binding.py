@@ -72,6 +72,14 @@ def _lib():
     lib.wersa_launch_count.argtypes = [vp, ctypes.c_int]
     lib.wersa_gate_static.restype = ctypes.c_int
     lib.wersa_gate_static.argtypes = [ctypes.POINTER(wersa_config), vp, fp, fp, fp, fp, fp, vp]
+    lib.wersa_shard_pool.restype = ctypes.c_int
+    lib.wersa_shard_pool.argtypes = [vp, vp, vp, fp, vp]
+    lib.wersa_shard_gate.restype = ctypes.c_int
+    lib.wersa_shard_gate.argtypes = [vp, fp, ctypes.c_int64, fp, fp, fp, vp]
+    lib.wersa_shard_keys.restype = ctypes.c_int
+    lib.wersa_shard_keys.argtypes = [vp, vp, vp, vp]
+    lib.wersa_shard_output.restype = ctypes.c_int
+    lib.wersa_shard_output.argtypes = [vp, vp, fp, fp, fp, vp, vp]
     lib.wersa_selftest_wait_timeout.restype = ctypes.c_int
     lib.wersa_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint32, vp, vp]
     lib.wersa_uses_tensor_cores.restype = ctypes.c_int32
@@ -214,6 +222,51 @@ class WersaContext:
         if st != WERSA_OK:
             raise WersaError(st, "wersa_haar_filter")
         return out
+
+    # -- sequence-sharded forward: the four steps, the caller adds the sums of all shards in between --------
+    def shard_pool(self, Q, W, stream=None):
+        qsum = torch.empty((self.cfg.batch, self.cfg.heads, 64), dtype=torch.float32, device=self.device)
+        st = _lib().wersa_shard_pool(self._h, _ptr(Q, self.io_dtype, "Q"), _ptr(W, self.io_dtype, "W"), _ptr(qsum),
+                                     _stream_ptr(stream))
+        if st != WERSA_OK:
+            raise WersaError(st, "wersa_shard_pool")
+        return qsum
+
+    def shard_gate(self, qsum_total, n_total, gate_w, gate_b, omega, stream=None):
+        st = _lib().wersa_shard_gate(self._h, _ptr(qsum_total, torch.float32, "qsum_total"), int(n_total),
+                                     _ptr(gate_w, torch.float32, "gate_w", optional=True),
+                                     _ptr(gate_b, torch.float32, "gate_b", optional=True),
+                                     _ptr(omega, torch.float32, "omega"), _stream_ptr(stream))
+        if st != WERSA_OK:
+            raise WersaError(st, "wersa_shard_gate")
+
+    def shard_keys(self, K, V, stream=None):
+        """Returns views of this shard's S' (batch, heads, features, 64) and z' in the workspace."""
+        st = _lib().wersa_shard_keys(self._h, _ptr(K, self.io_dtype, "K"), _ptr(V, self.io_dtype, "V"),
+                                     _stream_ptr(stream))
+        if st != WERSA_OK:
+            raise WersaError(st, "wersa_shard_keys")
+        return self._saved_view(2), self._saved_view(3)
+
+    def shard_output(self, Q, S_total, z_total, beta, out=None, stream=None):
+        if out is None:
+            out = torch.empty_like(Q)
+        st = _lib().wersa_shard_output(self._h, _ptr(Q, self.io_dtype, "Q"), _ptr(S_total, torch.float32, "S_total"),
+                                       _ptr(z_total, torch.float32, "z_total"), _ptr(beta, torch.float32, "beta"),
+                                       _ptr(out, self.io_dtype, "O"), _stream_ptr(stream))
+        if st != WERSA_OK:
+            raise WersaError(st, "wersa_shard_output")
+        return out
+
+    def _saved_view(self, idx):
+        ptr, count = ctypes.c_void_p(), ctypes.c_size_t()
+        st = _lib().wersa_saved(self._h, idx, ctypes.byref(ptr), ctypes.byref(count))
+        if st != WERSA_OK:
+            raise WersaError(st, "wersa_saved")
+        off = ptr.value - self.workspace.data_ptr()
+        c = self.cfg
+        shape = {2: (c.batch, c.heads, c.features, 64), 3: (c.batch, c.heads, c.features)}[idx]
+        return self.workspace[off:off + 4 * count.value].view(torch.float32).view(shape)
 
     def saved(self, which):
         """Copy of a tensor the last forward left in the workspace: 'f', 'qbar', 'S', 'z'."""

@@ -433,6 +433,84 @@ wersa_status wersa_forward(wersa_ctx* ctx, const void* Q, const void* K, const v
   return WERSA_OK;
 }
 
+// ---- sequence-sharded forward ------------------------------------------------------------------------
+// The four steps of wersa_forward with the two places opened where shards of one sequence have to exchange
+// sums: after the mean pool (column sums of Q) and after the key side (S', z').  Tensor-core path, one feature
+// group; the context is created with the shard's own length.
+static bool shardable(const Plan& p) { return p.use_tc && p.groups == 1; }
+
+wersa_status wersa_shard_pool(wersa_ctx* ctx, const void* Q, const void* W, float* qsum, void* cuda_stream) {
+  if (ctx == nullptr || Q == nullptr || W == nullptr || qsum == nullptr) return WERSA_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(W)) return WERSA_ERR_INVALID_ARG;
+  const Plan& p = ctx->plan;
+  if (!shardable(p)) return WERSA_ERR_UNSUPPORTED;
+  const Ws& w = ctx->ws;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DeviceGuard guard(p.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  wersa_status s = clear_status_once(ctx, st);
+  if (s != WERSA_OK) return s;
+  int launches = 0;
+  // (the gate this launch also computes belongs to the shard alone and is replaced by wersa_shard_gate)
+  WERSA_CUDA(launch_qmean_gate(p, w, Q, nullptr, nullptr, nullptr, W, p.fwd_cols, st, &launches));
+  WERSA_CUDA(launch_shard_qsum(p, w, qsum, st, &launches));
+  ctx->launches_fwd = launches;
+  ctx->forward_done = false;
+  return WERSA_OK;
+}
+
+wersa_status wersa_shard_gate(wersa_ctx* ctx, const float* qsum_total, int64_t n_total, const float* gate_w,
+                              const float* gate_b, const float* omega, void* cuda_stream) {
+  if (ctx == nullptr || qsum_total == nullptr || omega == nullptr || n_total < 1 || n_total > 0x7fffffffLL)
+    return WERSA_ERR_INVALID_ARG;
+  const Plan& p = ctx->plan;
+  if (!shardable(p)) return WERSA_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DeviceGuard guard(p.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  int launches = 0;
+  WERSA_CUDA(launch_gate_from_sums(p, ctx->ws, qsum_total, n_total, gate_w, gate_b, omega, p.fwd_cols, st, &launches));
+  ctx->launches_fwd += launches;
+  return WERSA_OK;
+}
+
+wersa_status wersa_shard_keys(wersa_ctx* ctx, const void* K, const void* V, void* cuda_stream) {
+  if (ctx == nullptr || K == nullptr || V == nullptr) return WERSA_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V)) return WERSA_ERR_INVALID_ARG;
+  const Plan& p = ctx->plan;
+  if (!shardable(p)) return WERSA_ERR_UNSUPPORTED;
+  const Ws& w = ctx->ws;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DeviceGuard guard(p.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  int launches = 0;
+  WERSA_CUDA(launch_tc_kside(p, w, K, V, st, &launches));
+  if (p.tchunks > 1)
+    WERSA_CUDA(launch_reduce_partials(p, w.spart, w.zpart, p.tchunks, w.S, w.z, w.Sbf, w.Simg, st, &launches));
+  ctx->launches_fwd += launches;
+  ctx->forward_done = true;   // S', z' of this shard can be read with wersa_saved
+  return WERSA_OK;
+}
+
+wersa_status wersa_shard_output(wersa_ctx* ctx, const void* Q, const float* S_total, const float* z_total,
+                                const float* beta, void* O, void* cuda_stream) {
+  if (ctx == nullptr || Q == nullptr || S_total == nullptr || z_total == nullptr || beta == nullptr || O == nullptr)
+    return WERSA_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(O)) return WERSA_ERR_INVALID_ARG;
+  const Plan& p = ctx->plan;
+  if (!shardable(p)) return WERSA_ERR_UNSUPPORTED;
+  const Ws& w = ctx->ws;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DeviceGuard guard(p.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  int launches = 0;
+  // the totals take the place of a single partial: the reduction copies them and writes the operand images
+  WERSA_CUDA(launch_reduce_partials(p, S_total, z_total, 1, w.S, w.z, w.Sbf, w.Simg, st, &launches));
+  WERSA_CUDA(launch_tc_qside(p, w, Q, beta, O, nullptr, st, &launches));
+  ctx->launches_fwd += launches;
+  return WERSA_OK;
+}
+
 wersa_status wersa_forward_host(wersa_ctx* ctx, const void* hQ, const void* hK, const void* hV, void* dQ,
                                 void* dK, void* dV, const void* W, const float* beta, const float* gate_w,
                                 const float* gate_b, const float* omega, void* dO, void* hO, void* cuda_stream) {

@@ -77,6 +77,12 @@ Ws resolve(const Plan& p, void* workspace);
 cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const float* gate_w,
                               const float* gate_b, const float* omega, const void* W, int cols, cudaStream_t st,
                               int* launches);
+// Sequence shards: column sums of this shard's Q (q-bar times the shard's length), and the gate from the
+// sums of all shards and the whole sequence's length (writes w.qbar, w.sg, w.f).
+cudaError_t launch_shard_qsum(const Plan& p, const Ws& w, float* qsum, cudaStream_t st, int* launches);
+cudaError_t launch_gate_from_sums(const Plan& p, const Ws& w, const float* qsum, long long n_total,
+                                  const float* gate_w, const float* gate_b, const float* omega, int cols,
+                                  cudaStream_t st, int* launches);
 // Gate backward: band inner products -> df -> domega, dgate_b, dgate_w, dqbar; dbeta.
 cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, const float* gate_w,
                                  const float* omega, int n_sumdD, float* dbeta, float* dgate_w, float* dgate_b,

@@ -61,7 +61,7 @@ __device__ __forceinline__ void slab_gate(const float* __restrict__ qpart, int q
       if (gate_b != nullptr) u += gate_b[h * L1 + i];
       const float sgm = 1.f / (1.f + expf(-u));
       sg[(size_t)slab * L1 + i] = sgm;
-      f[(size_t)slab * L1 + i] = sgm * omega[i];
+      f[(size_t)slab * L1 + i] = sgm * (omega != nullptr ? omega[i] : 1.f);
     } else {
       f[(size_t)slab * L1 + i] = u;
     }
@@ -80,7 +80,7 @@ __device__ __forceinline__ void batch_gate(int b, int H, int L1, const float* __
   const float sgm = 1.f / (1.f + expf(-u));
   for (int h = 0; h < H; ++h) {
     sg[((size_t)b * H + h) * L1 + i] = sgm;
-    f[((size_t)b * H + h) * L1 + i] = sgm * omega[i];
+    f[((size_t)b * H + h) * L1 + i] = sgm * (omega != nullptr ? omega[i] : 1.f);
   }
 }
 
@@ -178,6 +178,30 @@ __global__ void __launch_bounds__(256) k_qmean_gate(const T* __restrict__ Q, flo
   __threadfence();
   batch_gate(b, H, L1, gate_b, omega, sg, f);
   if (threadIdx.x == 0) batch_count[b] = 0;
+}
+
+// Gate from column sums that are already complete (sequence shards: the sums of all shards were added by the
+// caller): one CTA of 256 threads per slab runs slab_gate on a single "partial" with the whole sequence's
+// length, then, for the batch-wide gate, a second launch runs batch_gate per batch element.
+// qbar_scale: q-bar of a shard times its length gives the shard's column sums back.
+__global__ void __launch_bounds__(256) k_scale_qbar(const float* __restrict__ qbar, float scale,
+                                                    float* __restrict__ qsum, int count) {
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i < count) qsum[i] = qbar[i] * scale;
+}
+__global__ void __launch_bounds__(256) k_gate_from_sums(const float* __restrict__ qsum, int H, int n_total, int L1,
+                                                        int per_head, const float* __restrict__ gate_w,
+                                                        const float* __restrict__ gate_b,
+                                                        const float* __restrict__ omega, float* __restrict__ qbar,
+                                                        float* __restrict__ sg, float* __restrict__ f, int dcols) {
+  __shared__ float red4[4][kD];
+  __shared__ float qs[kD];
+  slab_gate(qsum, 1, blockIdx.x, H, n_total, L1, per_head, gate_w, gate_b, omega, qbar, sg, f, red4, qs, dcols);
+}
+__global__ void __launch_bounds__(32) k_batch_gate(int H, int L1, const float* __restrict__ gate_b,
+                                                   const float* __restrict__ omega, float* __restrict__ sg,
+                                                   float* __restrict__ f) {
+  batch_gate(blockIdx.x, H, L1, gate_b, omega, sg, f);
 }
 
 // Sum the per-tile band inner products of both filtered tensors in tile order and turn them
@@ -315,6 +339,26 @@ cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const f
                               int* launches) {
   *launches += 1;
   return launch_qmean_gate_impl(p, Q, w.qpart, gate_w, gate_b, omega, w.qbar, w.sg, w.f, w.counters, W, w.Wt, cols, st);
+}
+
+cudaError_t launch_shard_qsum(const Plan& p, const Ws& w, float* qsum, cudaStream_t st, int* launches) {
+  const int count = p.slabs * kD;
+  k_scale_qbar<<<(count + 255) / 256, 256, 0, st>>>(w.qbar, (float)p.cfg.seq_len, qsum, count);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gate_from_sums(const Plan& p, const Ws& w, const float* qsum, long long n_total,
+                                  const float* gate_w, const float* gate_b, const float* omega, int cols,
+                                  cudaStream_t st, int* launches) {
+  k_gate_from_sums<<<p.slabs, 256, 0, st>>>(qsum, p.cfg.heads, (int)n_total, p.L1, p.cfg.gate_per_head, gate_w, gate_b,
+                                           omega, w.qbar, w.sg, w.f, cols);
+  *launches += 1;
+  if (!p.cfg.gate_per_head) {
+    k_batch_gate<<<p.cfg.batch, 32, 0, st>>>(p.cfg.heads, p.L1, gate_b, omega, w.sg, w.f);
+    *launches += 1;
+  }
+  return cudaGetLastError();
 }
 
 // Device address of the static scratch array on the current device, resolved once per device.

@@ -282,6 +282,50 @@ def test_backward_with_wide_feature_maps(case, grad_dtype):
     _check_backward(cfg, inp, grads)
 
 
+# ---------------------------------------------------------------- sequence shards (one GPU standing in for several)
+SHARDED = [
+    (dict(B=2, H=2, n=3000, d=64, L=5, m=256), [1024, 1024, 952]),
+    (dict(B=1, H=3, n=2304, d=32, L=8, m=128, gate_per_head=0), [1536, 768]),
+    (dict(B=1, H=1, n=70000, d=64, L=6, m=256), [32768, 37232]),       # several chunks per shard
+]
+
+
+@pytest.mark.parametrize("case", range(len(SHARDED)))
+def test_sequence_sharded_forward(case):
+    """The four shard steps on contexts of the shards' lengths, with the two sums between them taken here (on
+    several GPUs they are all-reduces): the shards' outputs put together meet the oracle's forward on the whole
+    sequence, and the whole-sequence context's forward to bf16 rounding."""
+    import torch
+    cfg, lens = SHARDED[case]
+    cfg = dict(cfg, dtype="bf16")
+    assert sum(lens) == cfg["n"] and all(l % (1 << cfg["L"]) == 0 for l in lens[:-1])
+    inp = wi.make_inputs(**cfg, seed=2500 + case, w_seed=2600 + case, gate_std=0.3, gate_seed=2700 + case,
+                         mean_shift=0.25, scale=0.7)
+    dev = device_inputs(inp, "bf16")
+    starts = np.concatenate([[0], np.cumsum(lens)]).astype(int)
+    shards = [{k: dev[k][:, :, a:b].contiguous() for k in ("Q", "K", "V")} for a, b in zip(starts[:-1], starts[1:])]
+    ctxs = [_ctx(dict(cfg, n=l)) for l in lens]
+    qsum = sum(c.shard_pool(s["Q"], dev["W"]) for c, s in zip(ctxs, shards))
+    S_total = z_total = None
+    for c, s in zip(ctxs, shards):
+        c.shard_gate(qsum, cfg["n"], dev["gate_w"], dev["gate_b"], dev["omega"])
+        S, z = c.shard_keys(s["K"], s["V"])
+        S_total = S.clone() if S_total is None else S_total + S
+        z_total = z.clone() if z_total is None else z_total + z
+    O = torch.cat([c.shard_output(s["Q"], S_total, z_total, dev["beta"]) for c, s in zip(ctxs, shards)], dim=2)
+    torch.cuda.synchronize()
+    assert all(c.query_status() == 0 for c in ctxs)
+    ref, aux = _oracle_forward(cfg, inp, want_aux=True)
+    _check(to_numpy64(O), ref, "bf16", "O")
+    f = to_numpy64(ctxs[0].saved("f"))
+    assert np.max(np.abs(f - aux["f"])) < 2e-6
+    whole = _ctx(cfg).forward(dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"],
+                              dev["omega"])
+    torch.cuda.synchronize()
+    diff = (whole.float() - O.float()).abs().max()
+    assert float(diff) <= 2.0 ** -6 * float(whole.float().abs().max())
+
+
 def test_forward_is_bit_identical_run_to_run():
     import paper_2507_08637_b200 as wersa
     import torch
