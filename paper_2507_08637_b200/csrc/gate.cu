@@ -87,7 +87,7 @@ __device__ __forceinline__ void batch_gate(int b, int H, int L1, const float* __
 // Mean pool and gate in one launch.  grid (qchunks, slabs [+ 1]), block 256.
 // Rows y < slabs: partial column sums of one row chunk of one slab of Q -- thread (cg = tid & 7,
 // rl = tid >> 3) owns 8 consecutive columns and every 32nd row, loads 16 bytes (bf16) / 32 bytes
-// (fp32) per row, four rows in flight.  The CTA that finds it is the last of its slab to finish
+// (fp32) per row, four rows in flight, with the streaming cache hint (Q is read once here).  The CTA that finds it is the last of its slab to finish
 // (a counter per slab) then runs slab_gate, and for the batch-wide gate the last slab of a batch
 // element (a counter per batch element) runs batch_gate; sums are taken in a fixed order, so the
 // result does not depend on which CTA comes last.  The counters start at zero and are left at zero.
@@ -130,16 +130,16 @@ __global__ void __launch_bounds__(256) k_qmean_gate(const T* __restrict__ Q, flo
   int r = rl < rp ? r0 + rl : r1;              // (256 need not be a multiple of cgs: the last threads idle)
   for (; r + 3 * rp < r1; r += 4 * rp) {
     float v0[8], v1[8], v2[8], v3[8];
-    load8(base + (size_t)r * dcols, v0);
-    load8(base + (size_t)(r + rp) * dcols, v1);
-    load8(base + (size_t)(r + 2 * rp) * dcols, v2);
-    load8(base + (size_t)(r + 3 * rp) * dcols, v3);
+    load8_stream(base + (size_t)r * dcols, v0);
+    load8_stream(base + (size_t)(r + rp) * dcols, v1);
+    load8_stream(base + (size_t)(r + 2 * rp) * dcols, v2);
+    load8_stream(base + (size_t)(r + 3 * rp) * dcols, v3);
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] += (v0[j] + v1[j]) + (v2[j] + v3[j]);
   }
   for (; r < r1; r += rp) {
     float v0[8];
-    load8(base + (size_t)r * dcols, v0);
+    load8_stream(base + (size_t)r * dcols, v0);
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] += v0[j];
   }
