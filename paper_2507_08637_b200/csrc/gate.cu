@@ -204,21 +204,35 @@ __global__ void __launch_bounds__(32) k_batch_gate(int H, int L1, const float* _
   batch_gate(blockIdx.x, H, L1, gate_b, omega, sg, f);
 }
 
-// Sum the per-tile band inner products of both filtered tensors in tile order and turn them
-// into df[slab][i]: i < L takes the detail-band product of level i+1, i = L the approximation
-// product of level L.  One CTA per slab, 32 threads.
-__global__ void __launch_bounds__(32) k_band_reduce(const float* __restrict__ bands, int slabs, int htiles,
-                                                    int L, float* __restrict__ df) {
-  const int slab = blockIdx.x, j = threadIdx.x;
-  if (j >= kBandVals) return;
+// Sum the per-tile band inner products of both filtered tensors and turn them into df[slab][i]: i < L takes
+// the detail-band product of level i+1, i = L the approximation product of level L.  One CTA of 256 threads
+// per slab: thread (j = tid & 15, part = tid >> 4) adds every 16th partial of band slot j in tile order
+// (four loads in flight), the 16 parts are added in a fixed order: the result repeats bit for bit.
+__global__ void __launch_bounds__(256) k_band_reduce(const float* __restrict__ bands, int slabs, int htiles,
+                                                     int L, float* __restrict__ df) {
+  __shared__ float part[16][kBandVals];
+  const int slab = blockIdx.x, j = threadIdx.x & (kBandVals - 1), pt = threadIdx.x >> 4;
   float s = 0.f;
   for (int which = 0; which < 2; ++which) {
-    const float* src = bands + (((size_t)which * slabs + slab) * htiles) * kBandVals;
-    for (int t = 0; t < htiles; ++t) s += src[(size_t)t * kBandVals + j];
+    const float* src = bands + (((size_t)which * slabs + slab) * htiles) * kBandVals + j;
+    int t = pt;
+    for (; t + 48 < htiles; t += 64) {
+      const float v0 = src[(size_t)t * kBandVals], v1 = src[(size_t)(t + 16) * kBandVals];
+      const float v2 = src[(size_t)(t + 32) * kBandVals], v3 = src[(size_t)(t + 48) * kBandVals];
+      s += (v0 + v1) + (v2 + v3);
+    }
+    for (; t < htiles; t += 16) s += src[(size_t)t * kBandVals];
   }
-  // slots 0..7: detail products of levels 1..8; slots 8..15: approximation products of levels 1..8
-  if (j < L) df[(size_t)slab * kBandVals + j] = s;
-  if (j == 8 + L - 1) df[(size_t)slab * kBandVals + L] = s;
+  part[pt][j] = s;
+  __syncthreads();
+  if (threadIdx.x < kBandVals) {
+    float tot = 0.f;
+#pragma unroll
+    for (int q = 0; q < 16; ++q) tot += part[q][j];
+    // slots 0..7: detail products of levels 1..8; slots 8..15: approximation products of levels 1..8
+    if (j < L) df[(size_t)slab * kBandVals + j] = tot;
+    if (j == 8 + L - 1) df[(size_t)slab * kBandVals + L] = tot;
+  }
 }
 
 // Chain rule through f = sigmoid(u) * omega, u = gate(qbar): domega, dgate_b, dgate_w, dqbar; and the
@@ -403,7 +417,7 @@ cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, 
                                  const float* omega, int n_sumdD, float* dbeta, float* dgate_w, float* dgate_b,
                                  float* domega, cudaStream_t st, int* launches) {
   float* df = w.dqbar + (size_t)p.slabs * kD;   // df lives behind dqbar in the same region
-  k_band_reduce<<<p.slabs, 32, 0, st>>>(w.bands, p.slabs, 2 * p.htiles, p.cfg.levels, df);   // two partials per tile
+  k_band_reduce<<<p.slabs, 256, 0, st>>>(w.bands, p.slabs, 2 * p.htiles, p.cfg.levels, df);   // two partials per tile
   k_gate_backward<<<p.cfg.heads + 2, kD, 0, st>>>(df, w.sg, w.qbar, gate_w, omega, w.sumdD, n_sumdD, beta,
                                     p.cfg.eps, p.cfg.bw_floor, p.cfg.features, p.cfg.batch, p.cfg.heads,
                                     p.L1, p.cfg.gate_per_head, dbeta, dgate_w, dgate_b, domega, w.dqbar);

@@ -346,15 +346,17 @@ __global__ void __launch_bounds__(256, 2) k_haar_filter_split3(const Tin* __rest
 //   slot 8+l-1:          sum over blocks of s_l(G) * s_l(X) / 2^l, the product of the level-l
 //                        approximation coefficients.
 // The transform acts on every column separately, so one CTA takes 256 rows x 32 columns (half of the
-// head dimension): 8 rows x 4 columns per thread, a small register tile (three CTAs per SM keep loads,
+// head dimension): 8 rows x 4 columns per thread, a small register tile (several CTAs per SM keep loads,
 // arithmetic and stores of different tiles overlapped).  G and X are loaded together.  Levels 1-3 live
 // in the register tiles; the 8-row sums go to a pyramid in shared memory (per tensor and column: 32
 // sums of level 3, then 16, 8, 4, 2, 1 of levels 4-8), from which one thread per column takes the level
 // 4-8 products and every thread the coarse part of its output rows.
 // grid (2 * htiles, slabs): blockIdx.x = 2 * tile + column half; one band partial per CTA.
-// kWrite = false leaves dX unwritten (only the band inner products are wanted).
+// kWrite = false leaves dX unwritten (only the band inner products are wanted).  Two CTAs per SM with the
+// output (at three the 85-register limit spilled the register tiles: 77 -> 69 us per pass on config 5), four
+// without it.
 template <typename Tin, typename Tout, bool kWrite>
-__global__ void __launch_bounds__(256, 3) k_haar_backward(const Tin* __restrict__ X, const float* __restrict__ G,
+__global__ void __launch_bounds__(256, kWrite ? 2 : 4) k_haar_backward(const Tin* __restrict__ X, const float* __restrict__ G,
                                                           const float* __restrict__ f, Tout* __restrict__ dX,
                                                           float* __restrict__ bands, int n, int L) {
   __shared__ float pyr[2][kPyr][kHalfD];   // [0] = G, [1] = X
