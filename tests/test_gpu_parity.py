@@ -342,12 +342,12 @@ def test_forward_is_bit_identical_run_to_run():
         assert torch.equal(a.view(torch.int16), b.view(torch.int16))
 
 
-@pytest.mark.parametrize("dtype", ["bf16", "f32"])
-def test_forward_host_matches_device_forward_and_oracle(dtype):
+@pytest.mark.parametrize("dtype,d", [("bf16", 64), ("f32", 64), ("bf16", 32)])
+def test_forward_host_matches_device_forward_and_oracle(dtype, d):
     """The end-to-end entry point (host tensors in, host tensor out) gives the device-resident forward's
     bits, page-locked or pageable, and meets the oracle at the same tolerance."""
     import torch
-    cfg = dict(B=2, H=3, n=1500, d=64, L=5, m=128, dtype=dtype)
+    cfg = dict(B=2, H=3, n=1500, d=d, L=5, m=128, dtype=dtype)
     inp = wi.make_inputs(**cfg, seed=41, w_seed=42, gate_std=0.2, gate_seed=43, mean_shift=0.2)
     ctx = _ctx(cfg)
     dev = device_inputs(inp, dtype)
