@@ -106,8 +106,10 @@ __global__ void __launch_bounds__(256) k_qmean_gate(const T* __restrict__ Q, flo
                                                     const __nv_bfloat16* __restrict__ W, __nv_bfloat16* __restrict__ Wt,
                                                     int m, int dcols_arg) {
   const int dcols = kFull ? kD : dcols_arg;
-  // the key-side kernel may be staged now (programmatic dependent launch; it waits for this grid
-  // before it reads W^T or the gate)
+  // This grid may have been placed while the work before it in the stream was still running: nothing is
+  // read or written before that work has completed.  After that the key-side kernel may be staged
+  // (programmatic dependent launch; it waits for this grid before it reads W^T or the gate).
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if ((int)blockIdx.y == slabs) {
     for (int i = blockIdx.x * 256 + threadIdx.x; i < m * kD; i += gridDim.x * 256) {
@@ -333,10 +335,23 @@ static cudaError_t launch_qmean_gate_impl(const Plan& p, const void* Q, float* q
   dim3 grid(p.qchunks, p.slabs + (W != nullptr ? 1 : 0));
   int* slab_count = counters;
   int* batch_count = counters + p.slabs;
+  cudaError_t launch_err = cudaSuccess;
   auto launch = [&](auto kernel, auto* q) {
-    kernel<<<grid, 256, 0, st>>>(q, qpart, p.cfg.seq_len, p.qchunk_rows, p.slabs, p.cfg.heads, p.L1,
-                                 p.cfg.gate_per_head, gate_w, gate_b, omega, qbar, sg, f, slab_count, batch_count,
-                                 (const __nv_bfloat16*)W, Wt, p.cfg.features, cols);
+    // Launched as a programmatic dependent of whatever precedes it in the stream: the kernel's first
+    // instruction waits for that work to complete, so ordering and visibility are those of a plain launch,
+    // but its CTAs are already placed when the wait ends (2 us per forward in a sequence of steps).
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid;
+    lc.blockDim = dim3(256);
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    launch_err = cudaLaunchKernelEx(&lc, kernel, q, qpart, p.cfg.seq_len, p.qchunk_rows, p.slabs, p.cfg.heads, p.L1,
+                                    p.cfg.gate_per_head, gate_w, gate_b, omega, qbar, sg, f, slab_count, batch_count,
+                                    (const __nv_bfloat16*)W, Wt, p.cfg.features, cols);
   };
   if (p.bf16) {
     if (cols == kD) launch(k_qmean_gate<__nv_bfloat16, true>, (const __nv_bfloat16*)Q);
@@ -345,7 +360,7 @@ static cudaError_t launch_qmean_gate_impl(const Plan& p, const void* Q, float* q
     if (cols == kD) launch(k_qmean_gate<float, true>, (const float*)Q);
     else launch(k_qmean_gate<float, false>, (const float*)Q);
   }
-  return cudaGetLastError();
+  return launch_err != cudaSuccess ? launch_err : cudaGetLastError();
 }
 
 cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const float* gate_w,
