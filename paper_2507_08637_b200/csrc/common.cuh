@@ -187,6 +187,26 @@ __device__ __forceinline__ size_t simg_offset(int f, int r) {
   return (size_t)(f >> 6) * kSimgBlockBytes + (size_t)r * 128 + (size_t)((((f & 63) >> 3) ^ (r & 7)) << 4) + (f & 7) * 2;
 }
 
+// Launch as a programmatic dependent of the work before it in the stream.  The kernel's first instruction
+// must be griddepcontrol.wait (nothing is read or written before that work has completed), so ordering and
+// visibility are those of a plain launch; only the placement of the CTAs overlaps the end of that work.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+__device__ __forceinline__ void wait_for_stream_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- device helpers ------------------------------------------------------------------------
 __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }

@@ -212,6 +212,7 @@ __global__ void __launch_bounds__(32) k_batch_gate(int H, int L1, const float* _
 // (four loads in flight), the 16 parts are added in a fixed order: the result repeats bit for bit.
 __global__ void __launch_bounds__(256) k_band_reduce(const float* __restrict__ bands, int slabs, int htiles,
                                                      int L, float* __restrict__ df) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   __shared__ float part[16][kBandVals];
   const int slab = blockIdx.x, j = threadIdx.x & (kBandVals - 1), pt = threadIdx.x >> 4;
   float s = 0.f;
@@ -247,6 +248,7 @@ __global__ void __launch_bounds__(kD) k_gate_backward(
     int n_sumdD, const float* __restrict__ beta, float eps, float bw_floor, int m, int B, int H, int L1,
     int per_head, float* __restrict__ dbeta, float* __restrict__ dgate_w, float* __restrict__ dgate_b,
     float* __restrict__ domega, float* __restrict__ dqbar) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   const int c = threadIdx.x;
   __shared__ float du[kMaxLevels + 1];
   __shared__ float part[kD];
@@ -432,8 +434,8 @@ cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, 
                                  const float* omega, int n_sumdD, float* dbeta, float* dgate_w, float* dgate_b,
                                  float* domega, cudaStream_t st, int* launches) {
   float* df = w.dqbar + (size_t)p.slabs * kD;   // df lives behind dqbar in the same region
-  k_band_reduce<<<p.slabs, 256, 0, st>>>(w.bands, p.slabs, 2 * p.htiles, p.cfg.levels, df);   // two partials per tile
-  k_gate_backward<<<p.cfg.heads + 2, kD, 0, st>>>(df, w.sg, w.qbar, gate_w, omega, w.sumdD, n_sumdD, beta,
+  launch_after(k_band_reduce, dim3(p.slabs), dim3(256), 0, st, w.bands, p.slabs, 2 * p.htiles, p.cfg.levels, df);   // two partials per tile
+  launch_after(k_gate_backward, dim3(p.cfg.heads + 2), dim3(kD), 0, st, df, w.sg, w.qbar, gate_w, omega, w.sumdD, n_sumdD, beta,
                                     p.cfg.eps, p.cfg.bw_floor, p.cfg.features, p.cfg.batch, p.cfg.heads,
                                     p.L1, p.cfg.gate_per_head, dbeta, dgate_w, dgate_b, domega, w.dqbar);
   *launches += 2;

@@ -85,6 +85,7 @@ template <typename Tin, typename Tout, bool kAddVec>
 __global__ void __launch_bounds__(256, 4) k_haar_filter(const Tin* __restrict__ X, const float* __restrict__ f,
                                                      Tout* __restrict__ XF, int n, int L,
                                                      const float* __restrict__ vec, float vec_scale) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   __shared__ float pyr[kPyr][kHalfD];
   __shared__ float hit[32][kHalfD];   // sum_{l=3..8} k_l * s_l(block of row group r), per column
   const int slab = blockIdx.y, half = blockIdx.x & 1;
@@ -158,6 +159,7 @@ template <typename Tout>
 __global__ void __launch_bounds__(256, 3) k_haar_filter_bf16(const __nv_bfloat16* __restrict__ X,
                                                              const float* __restrict__ f, Tout* __restrict__ XF,
                                                              int n, int L) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   __shared__ float pyr[kPyr][kD];
   __shared__ float hit[32][kD];   // sum_{l=3..8} k_l * s_l(block of row group r), per column
   const int slab = blockIdx.y;
@@ -271,6 +273,7 @@ template <typename Tin>
 __global__ void __launch_bounds__(256, 2) k_haar_filter_split3(const Tin* __restrict__ X, const float* __restrict__ f,
                                                             __nv_bfloat16* __restrict__ XF3, size_t plane, int n,
                                                             int L) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   // levels 4-8 through a pyramid of the 8-row sums in shared memory (per column: 32 sums of level 3,
   // then 16, 8, 4, 2, 1), as in k_haar_backward
   __shared__ float pyr[63][kD];
@@ -359,6 +362,7 @@ template <typename Tin, typename Tout, bool kWrite>
 __global__ void __launch_bounds__(256, kWrite ? 2 : 4) k_haar_backward(const Tin* __restrict__ X, const float* __restrict__ G,
                                                           const float* __restrict__ f, Tout* __restrict__ dX,
                                                           float* __restrict__ bands, int n, int L) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   __shared__ float pyr[2][kPyr][kHalfD];   // [0] = G, [1] = X
   __shared__ float hit[32][kHalfD];        // coarse part of the output of row group rg, per column
   __shared__ float red[8][kBandVals];
@@ -496,13 +500,13 @@ cudaError_t launch_haar_filter(const Plan& p, const void* X, int in_kind, const 
   dim3 grid_bf(p.htiles, p.slabs);
   const int n = p.cfg.seq_len, L = p.cfg.levels;
   if (in_kind == 1 && out_kind == 1)
-    k_haar_filter_bf16<__nv_bfloat16><<<grid_bf, 256, 0, st>>>((const __nv_bfloat16*)X, f, (__nv_bfloat16*)XF, n, L);
+    launch_after(k_haar_filter_bf16<__nv_bfloat16>, dim3(grid_bf), dim3(256), 0, st, (const __nv_bfloat16*)X, f, (__nv_bfloat16*)XF, n, L);
   else if (in_kind == 1 && out_kind == 0)
-    k_haar_filter_bf16<float><<<grid_bf, 256, 0, st>>>((const __nv_bfloat16*)X, f, (float*)XF, n, L);
+    launch_after(k_haar_filter_bf16<float>, dim3(grid_bf), dim3(256), 0, st, (const __nv_bfloat16*)X, f, (float*)XF, n, L);
   else if (in_kind == 0 && out_kind == 0)
-    k_haar_filter<float, float, false><<<grid, 256, 0, st>>>((const float*)X, f, (float*)XF, n, L, nullptr, 0.f);
+    launch_after(k_haar_filter<float, float, false>, dim3(grid), dim3(256), 0, st, (const float*)X, f, (float*)XF, n, L, nullptr, 0.f);
   else
-    k_haar_filter<float, __nv_bfloat16, false><<<grid, 256, 0, st>>>((const float*)X, f, (__nv_bfloat16*)XF, n, L,
+    launch_after(k_haar_filter<float, __nv_bfloat16, false>, dim3(grid), dim3(256), 0, st, (const float*)X, f, (__nv_bfloat16*)XF, n, L,
                                                                     nullptr, 0.f);
   *launches += 1;
   return cudaGetLastError();
@@ -513,9 +517,9 @@ cudaError_t launch_haar_filter_addvec(const Plan& p, const float* G, const float
   dim3 grid(2 * p.htiles, p.slabs);
   const int n = p.cfg.seq_len, L = p.cfg.levels;
   if (out_kind == 0)
-    k_haar_filter<float, float, true><<<grid, 256, 0, st>>>(G, f, (float*)dX, n, L, vec, vec_scale);
+    launch_after(k_haar_filter<float, float, true>, dim3(grid), dim3(256), 0, st, G, f, (float*)dX, n, L, vec, vec_scale);
   else
-    k_haar_filter<float, __nv_bfloat16, true><<<grid, 256, 0, st>>>(G, f, (__nv_bfloat16*)dX, n, L, vec, vec_scale);
+    launch_after(k_haar_filter<float, __nv_bfloat16, true>, dim3(grid), dim3(256), 0, st, G, f, (__nv_bfloat16*)dX, n, L, vec, vec_scale);
   *launches += 1;
   return cudaGetLastError();
 }
@@ -526,9 +530,9 @@ cudaError_t launch_haar_filter_split3(const Plan& p, const void* X, int in_kind,
   const int n = p.cfg.seq_len, L = p.cfg.levels;
   const size_t plane = (size_t)p.slabs * n * kD;
   if (in_kind == 1)
-    k_haar_filter_split3<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, f, XF3, plane, n, L);
+    launch_after(k_haar_filter_split3<__nv_bfloat16>, dim3(grid), dim3(256), 0, st, (const __nv_bfloat16*)X, f, XF3, plane, n, L);
   else
-    k_haar_filter_split3<float><<<grid, 256, 0, st>>>((const float*)X, f, XF3, plane, n, L);
+    launch_after(k_haar_filter_split3<float>, dim3(grid), dim3(256), 0, st, (const float*)X, f, XF3, plane, n, L);
   *launches += 1;
   return cudaGetLastError();
 }
@@ -540,20 +544,20 @@ cudaError_t launch_haar_backward(const Plan& p, const Ws& w, const void* X, int 
   float* bands = w.bands + (size_t)which * p.slabs * 2 * p.htiles * kBandVals;
   if (dX == nullptr) {   // band inner products only
     if (in_kind == 1)
-      k_haar_backward<__nv_bfloat16, float, false><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, G, w.f, nullptr,
+      launch_after(k_haar_backward<__nv_bfloat16, float, false>, dim3(grid), dim3(256), 0, st, (const __nv_bfloat16*)X, G, w.f, nullptr,
                                                                         bands, n, L);
     else
-      k_haar_backward<float, float, false><<<grid, 256, 0, st>>>((const float*)X, G, w.f, nullptr, bands, n, L);
+      launch_after(k_haar_backward<float, float, false>, dim3(grid), dim3(256), 0, st, (const float*)X, G, w.f, nullptr, bands, n, L);
   } else if (in_kind == 1 && out_kind == 1)
-    k_haar_backward<__nv_bfloat16, __nv_bfloat16, true><<<grid, 256, 0, st>>>(
+    launch_after(k_haar_backward<__nv_bfloat16, __nv_bfloat16, true>, dim3(grid), dim3(256), 0, st, 
         (const __nv_bfloat16*)X, G, w.f, (__nv_bfloat16*)dX, bands, n, L);
   else if (in_kind == 1 && out_kind == 0)
-    k_haar_backward<__nv_bfloat16, float, true><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, G, w.f, (float*)dX,
+    launch_after(k_haar_backward<__nv_bfloat16, float, true>, dim3(grid), dim3(256), 0, st, (const __nv_bfloat16*)X, G, w.f, (float*)dX,
                                                                      bands, n, L);
   else if (in_kind == 0 && out_kind == 0)
-    k_haar_backward<float, float, true><<<grid, 256, 0, st>>>((const float*)X, G, w.f, (float*)dX, bands, n, L);
+    launch_after(k_haar_backward<float, float, true>, dim3(grid), dim3(256), 0, st, (const float*)X, G, w.f, (float*)dX, bands, n, L);
   else
-    k_haar_backward<float, __nv_bfloat16, true><<<grid, 256, 0, st>>>((const float*)X, G, w.f, (__nv_bfloat16*)dX,
+    launch_after(k_haar_backward<float, __nv_bfloat16, true>, dim3(grid), dim3(256), 0, st, (const float*)X, G, w.f, (__nv_bfloat16*)dX,
                                                                      bands, n, L);
   *launches += 1;
   return cudaGetLastError();

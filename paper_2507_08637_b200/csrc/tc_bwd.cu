@@ -221,6 +221,7 @@ k_tc_bwd_kside(const __grid_constant__ CUtensorMap map_kf, const __grid_constant
                const __nv_bfloat16* __restrict__ Wt, const __nv_bfloat16* __restrict__ dSbf,
                const float* __restrict__ dzg, const __grid_constant__ CUtensorMap map_dv,
                const __grid_constant__ CUtensorMap map_dkf, int n, int slabs, int* __restrict__ status) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   using SL = BwdKSmem<NH>;
@@ -454,6 +455,7 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
                const __grid_constant__ CUtensorMap map_dqf, float* __restrict__ dspart,
                float* __restrict__ dzpart, float* __restrict__ sumdD, int n, int chunk_tiles,
                int* __restrict__ status, const float* __restrict__ den_ext, const float* __restrict__ dd_ext) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   using SL = BwdQSmem<NH>;
@@ -768,6 +770,7 @@ k_tc_bwd_qside(const __grid_constant__ CUtensorMap map_qf, const __grid_constant
 // lo = bf16(x - hi) for hi = bf16(x) as the forward left it: the second half of a hi + lo pair for S'.
 __global__ void __launch_bounds__(256) k_split_lo(const float* __restrict__ x, const __nv_bfloat16* __restrict__ hi_img,
                                                    __nv_bfloat16* __restrict__ lo_img, size_t count) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
   if (i < count) lo_img[i] = __float2bfloat16_rn(x[i] - __bfloat162float(hi_img[i]));
 }
@@ -832,7 +835,7 @@ cudaError_t launch_kside(const Plan& p, const Ws& w, const CUtensorMap& map_kf, 
   if (err != cudaSuccess) return err;
   const long long tiles_all = (long long)((p.cfg.seq_len + kTile - 1) / kTile) * p.slabs;
   const unsigned grid = (unsigned)(tiles_all < p.sms ? tiles_all : p.sms);   // one CTA per SM, one wave
-  k<<<grid, 256, BwdKSmem<NH>::total, st>>>(map_kf, map_v, w.Wt, w.dSbf, w.dz, map_dv, map_dkf, p.cfg.seq_len, p.slabs,
+  launch_after(k, dim3(grid), dim3(256), BwdKSmem<NH>::total, st, map_kf, map_v, w.Wt, w.dSbf, w.dz, map_dv, map_dkf, p.cfg.seq_len, p.slabs,
                                             w.status);
   return cudaGetLastError();
 }
@@ -843,7 +846,7 @@ cudaError_t launch_qside(const Plan& p, const Ws& w, const CUtensorMap& map_qf, 
                          const float* dd_ext = nullptr) {
   // low-order bf16 image of S' (rows = features of a slab), fetched tile by tile by the kernel
   const size_t count = (size_t)p.slabs * p.cfg.features * kD;
-  k_split_lo<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(w.S, w.Sbf, w.Slo, count);
+  launch_after(k_split_lo, dim3((unsigned)((count + 255) / 256)), dim3(256), 0, st, w.S, w.Sbf, w.Slo, count);
   CUtensorMap map_slo;
   cudaError_t merr;
   if ((merr = make_tile_map(w.Slo, p.slabs, p.cfg.features, &map_slo)) != cudaSuccess) return merr;
@@ -853,7 +856,7 @@ cudaError_t launch_qside(const Plan& p, const Ws& w, const CUtensorMap& map_qf, 
   CUtensorMap map_dqf;
   if ((err = make_out_map(w.dQF, p.slabs, p.cfg.seq_len, false, &map_dqf)) != cudaSuccess) return err;
   dim3 grid(p.bchunks, p.slabs);
-  k<<<grid, 256, BwdQSmem<NH>::total, st>>>(map_qf, map_do, map_slo, w.Wt, w.Sbf, w.z, beta, p.cfg.eps, p.cfg.bw_floor, map_dqf,
+  launch_after(k, dim3(grid), dim3(256), BwdQSmem<NH>::total, st, map_qf, map_do, map_slo, w.Wt, w.Sbf, w.z, beta, p.cfg.eps, p.cfg.bw_floor, map_dqf,
                                             w.spart, w.zpart, w.sumdD, p.cfg.seq_len, p.bchunk_tiles, w.status, den_ext,
                                             dd_ext);
   return cudaGetLastError();
