@@ -188,6 +188,7 @@ __global__ void __launch_bounds__(256) k_qmean_gate(const T* __restrict__ Q, flo
 // qbar_scale: q-bar of a shard times its length gives the shard's column sums back.
 __global__ void __launch_bounds__(256) k_scale_qbar(const float* __restrict__ qbar, float scale,
                                                     float* __restrict__ qsum, int count) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   const int i = blockIdx.x * 256 + threadIdx.x;
   if (i < count) qsum[i] = qbar[i] * scale;
 }
@@ -196,6 +197,7 @@ __global__ void __launch_bounds__(256) k_gate_from_sums(const float* __restrict_
                                                         const float* __restrict__ gate_b,
                                                         const float* __restrict__ omega, float* __restrict__ qbar,
                                                         float* __restrict__ sg, float* __restrict__ f, int dcols) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   __shared__ float red4[4][kD];
   __shared__ float qs[kD];
   slab_gate(qsum, 1, blockIdx.x, H, n_total, L1, per_head, gate_w, gate_b, omega, qbar, sg, f, red4, qs, dcols);
@@ -203,6 +205,7 @@ __global__ void __launch_bounds__(256) k_gate_from_sums(const float* __restrict_
 __global__ void __launch_bounds__(32) k_batch_gate(int H, int L1, const float* __restrict__ gate_b,
                                                    const float* __restrict__ omega, float* __restrict__ sg,
                                                    float* __restrict__ f) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   batch_gate(blockIdx.x, H, L1, gate_b, omega, sg, f);
 }
 
@@ -374,7 +377,7 @@ cudaError_t launch_qmean_gate(const Plan& p, const Ws& w, const void* Q, const f
 
 cudaError_t launch_shard_qsum(const Plan& p, const Ws& w, float* qsum, cudaStream_t st, int* launches) {
   const int count = p.slabs * kD;
-  k_scale_qbar<<<(count + 255) / 256, 256, 0, st>>>(w.qbar, (float)p.cfg.seq_len, qsum, count);
+  launch_after(k_scale_qbar, dim3((count + 255) / 256), dim3(256), 0, st, w.qbar, (float)p.cfg.seq_len, qsum, count);
   *launches += 1;
   return cudaGetLastError();
 }
@@ -382,11 +385,11 @@ cudaError_t launch_shard_qsum(const Plan& p, const Ws& w, float* qsum, cudaStrea
 cudaError_t launch_gate_from_sums(const Plan& p, const Ws& w, const float* qsum, long long n_total,
                                   const float* gate_w, const float* gate_b, const float* omega, int cols,
                                   cudaStream_t st, int* launches) {
-  k_gate_from_sums<<<p.slabs, 256, 0, st>>>(qsum, p.cfg.heads, (int)n_total, p.L1, p.cfg.gate_per_head, gate_w, gate_b,
+  launch_after(k_gate_from_sums, dim3(p.slabs), dim3(256), 0, st, qsum, p.cfg.heads, (int)n_total, p.L1, p.cfg.gate_per_head, gate_w, gate_b,
                                            omega, w.qbar, w.sg, w.f, cols);
   *launches += 1;
   if (!p.cfg.gate_per_head) {
-    k_batch_gate<<<p.cfg.batch, 32, 0, st>>>(p.cfg.heads, p.L1, gate_b, omega, w.sg, w.f);
+    launch_after(k_batch_gate, dim3(p.cfg.batch), dim3(32), 0, st, p.cfg.heads, p.L1, gate_b, omega, w.sg, w.f);
     *launches += 1;
   }
   return cudaGetLastError();

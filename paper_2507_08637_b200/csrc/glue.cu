@@ -14,6 +14,7 @@ namespace {
 // dst[row][0..63] = src[row][0..d) followed by zeros.  One thread per 8 elements of dst.
 template <typename T>
 __global__ void __launch_bounds__(256) k_pad_cols(const T* __restrict__ src, T* __restrict__ dst, size_t rows, int d) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   const size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x;
   const size_t row = idx >> 3;
   const int c0 = (int)(idx & 7) * 8;
@@ -31,6 +32,7 @@ __global__ void __launch_bounds__(256) k_pad_cols(const T* __restrict__ src, T* 
 // dst[row][0..d) = src[row][0..d) of a 64-wide source.
 template <typename T>
 __global__ void __launch_bounds__(256) k_unpad_cols(const T* __restrict__ src, T* __restrict__ dst, size_t rows, int d) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   const size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x;
   const size_t row = idx >> 3;
   const int c0 = (int)(idx & 7) * 8;
@@ -45,6 +47,7 @@ __global__ void __launch_bounds__(256) k_unpad_cols(const T* __restrict__ src, T
 template <typename T>
 __global__ void __launch_bounds__(256) k_combine_groups(const T* __restrict__ Og, const float* __restrict__ den,
                                                         T* __restrict__ O, size_t tokens, int groups, int cols) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   const size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x;
   const size_t tok = idx >> 3;
   const int c0 = (int)(idx & 7) * 8;
@@ -74,6 +77,7 @@ __global__ void __launch_bounds__(256) k_group_bwd_prep(const T* __restrict__ Og
                                                         const T* __restrict__ dO, const float* __restrict__ f, int n,
                                                         int L1, size_t tokens, int groups, float* __restrict__ Dtot,
                                                         float* __restrict__ dDtot) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   const size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x;
   const size_t tok = idx >> 3;
   const int c0 = (int)(idx & 7) * 8;
@@ -113,6 +117,7 @@ __global__ void __launch_bounds__(256) k_group_bwd_prep(const T* __restrict__ Og
 __global__ void __launch_bounds__(256) k_gather_groups(const float* __restrict__ Sg, const float* __restrict__ zg,
                                                        float* __restrict__ S, float* __restrict__ z, int slabs,
                                                        int groups, int mg) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   const size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x;   // one float4 of S
   const size_t total4 = (size_t)slabs * groups * mg * (kD / 4);
   if (idx >= total4) return;
@@ -131,9 +136,9 @@ unsigned blocks_for(size_t threads) { return (unsigned)((threads + 255) / 256); 
 
 cudaError_t launch_pad_cols(const void* src, void* dst, size_t rows, int d, int kind, cudaStream_t st, int* launches) {
   if (kind == 1)
-    k_pad_cols<__nv_bfloat16><<<blocks_for(rows * 8), 256, 0, st>>>((const __nv_bfloat16*)src, (__nv_bfloat16*)dst, rows, d);
+    launch_after(k_pad_cols<__nv_bfloat16>, dim3(blocks_for(rows * 8)), dim3(256), 0, st, (const __nv_bfloat16*)src, (__nv_bfloat16*)dst, rows, d);
   else
-    k_pad_cols<float><<<blocks_for(rows * 8), 256, 0, st>>>((const float*)src, (float*)dst, rows, d);
+    launch_after(k_pad_cols<float>, dim3(blocks_for(rows * 8)), dim3(256), 0, st, (const float*)src, (float*)dst, rows, d);
   *launches += 1;
   return cudaGetLastError();
 }
@@ -141,10 +146,10 @@ cudaError_t launch_pad_cols(const void* src, void* dst, size_t rows, int d, int 
 cudaError_t launch_unpad_cols(const void* src, void* dst, size_t rows, int d, int kind, cudaStream_t st,
                               int* launches) {
   if (kind == 1)
-    k_unpad_cols<__nv_bfloat16><<<blocks_for(rows * 8), 256, 0, st>>>((const __nv_bfloat16*)src, (__nv_bfloat16*)dst, rows,
+    launch_after(k_unpad_cols<__nv_bfloat16>, dim3(blocks_for(rows * 8)), dim3(256), 0, st, (const __nv_bfloat16*)src, (__nv_bfloat16*)dst, rows,
                                                                      d);
   else
-    k_unpad_cols<float><<<blocks_for(rows * 8), 256, 0, st>>>((const float*)src, (float*)dst, rows, d);
+    launch_after(k_unpad_cols<float>, dim3(blocks_for(rows * 8)), dim3(256), 0, st, (const float*)src, (float*)dst, rows, d);
   *launches += 1;
   return cudaGetLastError();
 }
@@ -152,10 +157,10 @@ cudaError_t launch_unpad_cols(const void* src, void* dst, size_t rows, int d, in
 cudaError_t launch_combine_groups(const void* Og, const float* den, void* O, size_t tokens, int groups, int cols,
                                   int kind, cudaStream_t st, int* launches) {
   if (kind == 1)
-    k_combine_groups<__nv_bfloat16><<<blocks_for(tokens * 8), 256, 0, st>>>((const __nv_bfloat16*)Og, den,
+    launch_after(k_combine_groups<__nv_bfloat16>, dim3(blocks_for(tokens * 8)), dim3(256), 0, st, (const __nv_bfloat16*)Og, den,
                                                                            (__nv_bfloat16*)O, tokens, groups, cols);
   else
-    k_combine_groups<float><<<blocks_for(tokens * 8), 256, 0, st>>>((const float*)Og, den, (float*)O, tokens, groups,
+    launch_after(k_combine_groups<float>, dim3(blocks_for(tokens * 8)), dim3(256), 0, st, (const float*)Og, den, (float*)O, tokens, groups,
                                                                    cols);
   *launches += 1;
   return cudaGetLastError();
@@ -165,10 +170,10 @@ cudaError_t launch_group_bwd_prep(const void* Og, const float* den, const void* 
                                   size_t tokens, int groups, int kind, float* Dtot, float* dDtot, cudaStream_t st,
                                   int* launches) {
   if (kind == 1)
-    k_group_bwd_prep<__nv_bfloat16><<<blocks_for(tokens * 8), 256, 0, st>>>(
+    launch_after(k_group_bwd_prep<__nv_bfloat16>, dim3(blocks_for(tokens * 8)), dim3(256), 0, st, 
         (const __nv_bfloat16*)Og, den, (const __nv_bfloat16*)dO, f, n, L1, tokens, groups, Dtot, dDtot);
   else
-    k_group_bwd_prep<float><<<blocks_for(tokens * 8), 256, 0, st>>>((const float*)Og, den, (const float*)dO, f, n, L1,
+    launch_after(k_group_bwd_prep<float>, dim3(blocks_for(tokens * 8)), dim3(256), 0, st, (const float*)Og, den, (const float*)dO, f, n, L1,
                                                                    tokens, groups, Dtot, dDtot);
   *launches += 1;
   return cudaGetLastError();
@@ -177,7 +182,7 @@ cudaError_t launch_group_bwd_prep(const void* Og, const float* den, const void* 
 cudaError_t launch_gather_groups(const float* Sg, const float* zg, float* S, float* z, int slabs, int groups, int mg,
                                  cudaStream_t st, int* launches) {
   const size_t total4 = (size_t)slabs * groups * mg * (kD / 4);
-  k_gather_groups<<<blocks_for(total4), 256, 0, st>>>(Sg, zg, S, z, slabs, groups, mg);
+  launch_after(k_gather_groups, dim3(blocks_for(total4)), dim3(256), 0, st, Sg, zg, S, z, slabs, groups, mg);
   *launches += 1;
   return cudaGetLastError();
 }

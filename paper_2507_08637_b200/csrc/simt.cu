@@ -219,6 +219,7 @@ template <int M, typename T>
 __global__ void __launch_bounds__(256) k_simt_kside(const float* __restrict__ KF, const T* __restrict__ V,
                                                     const T* __restrict__ W, float* __restrict__ spart,
                                                     float* __restrict__ zpart, int n, int chunk_tiles) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   extern __shared__ __align__(16) float sm[];
   using S = Smem<M>;
   float* WT = sm + S::wt;
@@ -258,6 +259,7 @@ __global__ void __launch_bounds__(256) k_simt_qside(const float* __restrict__ QF
                                                     const float* __restrict__ Sg, const float* __restrict__ zg,
                                                     const float* __restrict__ beta, float eps, float bw_floor,
                                                     T* __restrict__ O, int n, int chunk_tiles) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   extern __shared__ __align__(16) float sm[];
   using S = Smem<M>;
   float* WT = sm + S::wt;
@@ -301,6 +303,7 @@ __global__ void __launch_bounds__(256) k_simt_bwd_qside(
     const float* __restrict__ zg, const float* __restrict__ beta, float eps, float bw_floor,
     const T* __restrict__ dO, float* __restrict__ dQF, float* __restrict__ dspart, float* __restrict__ dzpart,
     float* __restrict__ sumdD, int n, int chunk_tiles) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   extern __shared__ __align__(16) float sm[];
   using S = Smem<M>;
   float* WT = sm + S::wt;
@@ -384,6 +387,7 @@ __global__ void __launch_bounds__(256) k_simt_bwd_kside(const float* __restrict_
                                                         const T* __restrict__ W, const float* __restrict__ dSg,
                                                         const float* __restrict__ dzg, TG* __restrict__ dV,
                                                         float* __restrict__ dKF, int n, int chunk_tiles) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
   extern __shared__ __align__(16) float sm[];
   using S = Smem<M>;
   float* WT = sm + S::wt;
@@ -505,12 +509,12 @@ cudaError_t launch_simt_kside(const Plan& p, const Ws& w, const void* V, const v
     if (p.bf16) {
       auto k = k_simt_kside<MM, __nv_bfloat16>;
       if ((err = set_smem(k, bytes)) != cudaSuccess) return err;
-      k<<<grid, 256, bytes, st>>>(w.KF, (const __nv_bfloat16*)V, (const __nv_bfloat16*)W, w.spart, w.zpart, n,
+      launch_after(k, dim3(grid), dim3(256), bytes, st, w.KF, (const __nv_bfloat16*)V, (const __nv_bfloat16*)W, w.spart, w.zpart, n,
                                   p.schunk_tiles);
     } else {
       auto k = k_simt_kside<MM, float>;
       if ((err = set_smem(k, bytes)) != cudaSuccess) return err;
-      k<<<grid, 256, bytes, st>>>(w.KF, (const float*)V, (const float*)W, w.spart, w.zpart, n, p.schunk_tiles);
+      launch_after(k, dim3(grid), dim3(256), bytes, st, w.KF, (const float*)V, (const float*)W, w.spart, w.zpart, n, p.schunk_tiles);
     }
   });
   *launches += 1;
@@ -545,12 +549,12 @@ cudaError_t launch_simt_qside(const Plan& p, const Ws& w, const void* W, const f
     if (p.bf16) {
       auto k = k_simt_qside<MM, __nv_bfloat16>;
       if ((err = set_smem(k, bytes)) != cudaSuccess) return err;
-      k<<<grid, 256, bytes, st>>>(w.QF, (const __nv_bfloat16*)W, w.S, w.z, beta, p.cfg.eps, p.cfg.bw_floor,
+      launch_after(k, dim3(grid), dim3(256), bytes, st, w.QF, (const __nv_bfloat16*)W, w.S, w.z, beta, p.cfg.eps, p.cfg.bw_floor,
                                   (__nv_bfloat16*)O, n, p.schunk_tiles);
     } else {
       auto k = k_simt_qside<MM, float>;
       if ((err = set_smem(k, bytes)) != cudaSuccess) return err;
-      k<<<grid, 256, bytes, st>>>(w.QF, (const float*)W, w.S, w.z, beta, p.cfg.eps, p.cfg.bw_floor, (float*)O, n,
+      launch_after(k, dim3(grid), dim3(256), bytes, st, w.QF, (const float*)W, w.S, w.z, beta, p.cfg.eps, p.cfg.bw_floor, (float*)O, n,
                                   p.schunk_tiles);
     }
   });
@@ -568,12 +572,12 @@ cudaError_t launch_simt_bwd_qside(const Plan& p, const Ws& w, const void* W, con
     if (p.bf16) {
       auto k = k_simt_bwd_qside<MM, __nv_bfloat16>;
       if ((err = set_smem(k, bytes)) != cudaSuccess) return err;
-      k<<<grid, 256, bytes, st>>>(w.QF, (const __nv_bfloat16*)W, w.S, w.z, beta, p.cfg.eps, p.cfg.bw_floor,
+      launch_after(k, dim3(grid), dim3(256), bytes, st, w.QF, (const __nv_bfloat16*)W, w.S, w.z, beta, p.cfg.eps, p.cfg.bw_floor,
                                   (const __nv_bfloat16*)dO, w.dQF, w.spart, w.zpart, w.sumdD, n, p.schunk_tiles);
     } else {
       auto k = k_simt_bwd_qside<MM, float>;
       if ((err = set_smem(k, bytes)) != cudaSuccess) return err;
-      k<<<grid, 256, bytes, st>>>(w.QF, (const float*)W, w.S, w.z, beta, p.cfg.eps, p.cfg.bw_floor,
+      launch_after(k, dim3(grid), dim3(256), bytes, st, w.QF, (const float*)W, w.S, w.z, beta, p.cfg.eps, p.cfg.bw_floor,
                                   (const float*)dO, w.dQF, w.spart, w.zpart, w.sumdD, n, p.schunk_tiles);
     }
   });
@@ -591,22 +595,22 @@ cudaError_t launch_simt_bwd_kside(const Plan& p, const Ws& w, const void* V, con
     if (p.bf16 && p.grad_bf16) {
       auto k = k_simt_bwd_kside<MM, __nv_bfloat16, __nv_bfloat16>;
       if ((err = set_smem(k, bytes)) != cudaSuccess) return err;
-      k<<<grid, 256, bytes, st>>>(w.KF, (const __nv_bfloat16*)V, (const __nv_bfloat16*)W, w.dS, w.dz,
+      launch_after(k, dim3(grid), dim3(256), bytes, st, w.KF, (const __nv_bfloat16*)V, (const __nv_bfloat16*)W, w.dS, w.dz,
                                   (__nv_bfloat16*)dV, w.dKF, n, p.schunk_tiles);
     } else if (p.bf16) {
       auto k = k_simt_bwd_kside<MM, __nv_bfloat16, float>;
       if ((err = set_smem(k, bytes)) != cudaSuccess) return err;
-      k<<<grid, 256, bytes, st>>>(w.KF, (const __nv_bfloat16*)V, (const __nv_bfloat16*)W, w.dS, w.dz, (float*)dV,
+      launch_after(k, dim3(grid), dim3(256), bytes, st, w.KF, (const __nv_bfloat16*)V, (const __nv_bfloat16*)W, w.dS, w.dz, (float*)dV,
                                   w.dKF, n, p.schunk_tiles);
     } else if (p.grad_bf16) {
       auto k = k_simt_bwd_kside<MM, float, __nv_bfloat16>;
       if ((err = set_smem(k, bytes)) != cudaSuccess) return err;
-      k<<<grid, 256, bytes, st>>>(w.KF, (const float*)V, (const float*)W, w.dS, w.dz, (__nv_bfloat16*)dV, w.dKF,
+      launch_after(k, dim3(grid), dim3(256), bytes, st, w.KF, (const float*)V, (const float*)W, w.dS, w.dz, (__nv_bfloat16*)dV, w.dKF,
                                   n, p.schunk_tiles);
     } else {
       auto k = k_simt_bwd_kside<MM, float, float>;
       if ((err = set_smem(k, bytes)) != cudaSuccess) return err;
-      k<<<grid, 256, bytes, st>>>(w.KF, (const float*)V, (const float*)W, w.dS, w.dz, (float*)dV, w.dKF, n,
+      launch_after(k, dim3(grid), dim3(256), bytes, st, w.KF, (const float*)V, (const float*)W, w.dS, w.dz, (float*)dV, w.dKF, n,
                                   p.schunk_tiles);
     }
   });
