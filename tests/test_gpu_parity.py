@@ -482,15 +482,29 @@ def _ambiguous_rows(cfg, inp, key):
     return out
 
 
-def _check_grad(got, ref, dtype, what, ambiguous=None):
+def _wavelet_block_mates(rows, block):
+    """Rows (last axis) that share an aligned block of `block` rows with a marked row."""
+    n = rows.shape[-1]
+    pad = (-n) % block
+    padded = np.concatenate([rows, np.zeros(rows.shape[:-1] + (pad,), dtype=bool)], axis=-1)
+    blocks = padded.reshape(rows.shape[:-1] + (-1, block)).any(axis=-1, keepdims=True)
+    return np.broadcast_to(blocks, padded.shape[:-1] + (padded.shape[-1] // block, block)).reshape(padded.shape)[..., :n]
+
+
+def _check_grad(got, ref, dtype, what, ambiguous=None, levels=0):
     """Element-by-element check of dQ / dK / dV.  Rows whose ReLU decision is ambiguous (see _ambiguous_rows)
-    are compared at a validity bound instead of the tolerance: one flipped feature moves the row by a
-    rank-one term, well below the row's own size."""
+    are compared at a validity bound instead of the tolerance: one flipped feature moves the row of dX_F by a
+    rank-one term, well below the row's own size.  dX = T_f(dX_F) spreads that term over the row's wavelet
+    block with the weights of the block means, 1/2 for the level-1 partner, 1/4 within the level-2 block, ...:
+    the rows that share a block of up to 16 rows (levels 1-4) with an ambiguous row are compared at the same
+    validity bound; beyond that the share (<= 1/32 of a term that is itself a fraction of the rms) is below
+    the tolerance."""
     err = normalised_error(got, ref)
     if ambiguous is not None and ambiguous.any():
         assert ambiguous.mean() <= 0.02, (what, "too many ambiguous rows", ambiguous.mean())
-        assert err[ambiguous].max() <= 1.0, (what, "ambiguous rows", err[ambiguous].max())
-        err = err[~ambiguous]
+        near = _wavelet_block_mates(ambiguous, 1 << min(levels, 4))
+        assert err[near].max() <= 1.0, (what, "ambiguous rows", err[near].max())
+        err = err[~near]
     if dtype == "f32":
         assert err.max() <= F32_MAX, (what, err.max())
     else:
@@ -504,8 +518,8 @@ def _check_backward(cfg, inp, grads, sub_slabs=None):
                        inp["gate_b"], inp["omega"], inp["dO"], cfg["L"], eps=cfg.get("eps", 1e-6),
                        gate_per_head=cfg.get("gate_per_head", 1))
     dtype = cfg["dtype"]
-    _check_grad(to_numpy64(grads["dQ"]), ref["dQ"], dtype, "dQ", _ambiguous_rows(cfg, inp, "Q"))
-    _check_grad(to_numpy64(grads["dK"]), ref["dK"], dtype, "dK", _ambiguous_rows(cfg, inp, "K"))
+    _check_grad(to_numpy64(grads["dQ"]), ref["dQ"], dtype, "dQ", _ambiguous_rows(cfg, inp, "Q"), cfg["L"])
+    _check_grad(to_numpy64(grads["dK"]), ref["dK"], dtype, "dK", _ambiguous_rows(cfg, inp, "K"), cfg["L"])
     _check_grad(to_numpy64(grads["dV"]), ref["dV"], dtype, "dV")
     tol = 1e-4 if dtype == "f32" else 2e-2
     for key in ("dgate_w", "dgate_b", "domega"):
@@ -601,7 +615,7 @@ def test_config5_training_step_bf16(flags):
     ref = _ORACLE_CACHE[name + "/bwd"]
     for key in ("dQ", "dK", "dV"):
         amb = _ambiguous_rows(cfg, inp, key[1]) if key != "dV" else None
-        err = _check_grad(to_numpy64(grads[key]), ref[key], "bf16", key, amb)
+        err = _check_grad(to_numpy64(grads[key]), ref[key], "bf16", key, amb, cfg["L"])
         print(f"cfg5 flags={flags} {key}: max {err.max():.3e} mean {err.mean():.3e} "
               f"(rows with an ambiguous ReLU decision: {0 if amb is None else int(amb.sum())} of {amb.size if amb is not None else 0})")
     for key in ("dgate_w", "dgate_b", "domega"):
