@@ -326,6 +326,24 @@ def test_sequence_sharded_forward(case):
     assert float(diff) <= 2.0 ** -6 * float(whole.float().abs().max())
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_forward_with_orthogonal_projection(dtype):
+    """The projection matrix is an input: an orthogonal R (Sec. 3.1, step 7 allows orthogonal or Gaussian),
+    drawn as orthonormal blocks of d columns, goes through the same kernels."""
+    import torch
+    cfg = dict(B=2, H=2, n=1500, d=64, L=4, m=256, dtype=dtype)
+    inp = wi.make_inputs(**cfg, seed=2800, w_seed=2801, gate_std=0.3, gate_seed=2802, mean_shift=0.25, scale=0.7,
+                         orthogonal_w=True)
+    W = inp["W"].astype(np.float64)
+    assert np.allclose(W[:, :64].T @ W[:, :64], 64.0 * np.eye(64), atol=1e-3 if dtype == "f32" else 0.5)   # (bf16: rounded entries)
+    ctx = _ctx(cfg)
+    dev = device_inputs(inp, dtype)
+    O = ctx.forward(dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    _check(to_numpy64(O), _oracle_forward(cfg, inp), dtype, "O")
+
+
 def test_forward_is_bit_identical_run_to_run():
     import paper_2507_08637_b200 as wersa
     import torch

@@ -43,7 +43,7 @@ def to_bf16_bits(x):
 
 
 def make_inputs(B, H, n, d, L, m, dtype="f32", scale=1.0, seed=0, w_seed=1, gate_std=None,
-                gate_seed=None, backward=False, beta=1.0, mean_shift=0.0, **_unused):
+                gate_seed=None, backward=False, beta=1.0, mean_shift=0.0, orthogonal_w=False, **_unused):
     """Draw one problem instance.  Returns a dict of float32 numpy arrays:
     Q, K, V (B,H,n,d), W (d,m), beta (1,), gate_w (H,d,L+1), gate_b (H,L+1), omega (L+1,),
     and dO (B,H,n,d) when backward=True.  `mean_shift` adds a constant to Q so that the
@@ -63,7 +63,14 @@ def make_inputs(B, H, n, d, L, m, dtype="f32", scale=1.0, seed=0, w_seed=1, gate
     out = dict(Q=Q, K=K, V=V)
     if backward:
         out["dO"] = rng.standard_normal(shape).astype(np.float32)
-    out["W"] = np.random.default_rng(w_seed).standard_normal((d, m)).astype(np.float32)
+    W = np.random.default_rng(w_seed).standard_normal((d, m))
+    if orthogonal_w:
+        # the paper allows an orthogonal R in place of the Gaussian one: blocks of d orthonormal columns (QR of
+        # the Gaussian draw, block by block), rescaled to the Gaussian columns' expected norm sqrt(d)
+        for c0 in range(0, m, d):
+            q, _ = np.linalg.qr(W[:, c0:c0 + d])
+            W[:, c0:c0 + q.shape[1]] = q[:, :min(d, m - c0)] * np.sqrt(d)
+    out["W"] = W.astype(np.float32)
     if gate_std is None:
         out["gate_w"] = np.zeros((H, d, L + 1), dtype=np.float32)
         out["gate_b"] = np.zeros((H, L + 1), dtype=np.float32)
