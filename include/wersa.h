@@ -66,8 +66,10 @@ typedef struct wersa_config {
   int32_t batch;         /* B >= 1                                                      */
   int32_t heads;         /* H >= 1                                                      */
   int32_t seq_len;       /* n >= 2; 2^levels must not exceed the next power of two >= n */
-  int32_t head_dim;      /* d: 8, 16, ... 64 (below 64 the tensors pass through zero-padded
-                            64-wide copies in the workspace, which leaves Eqs. 1-7 unchanged) */
+  int32_t head_dim;      /* d: 8, 16, ... 64.  Below 64 the problem runs as its zero-padded
+                            64-wide equivalent, which leaves Eqs. 1-7 unchanged: the bf16
+                            tensor-core forward reads and writes the narrow tensors directly,
+                            the fp32 path and the backward use padded copies in the workspace */
   int32_t levels;        /* L, Haar levels, 1..8                                        */
   int32_t features;      /* m, random features: 64, 128 or 256; with dtype bf16 and without
                             WERSA_FLAG_SIMT_ONLY also 512, 768 and 1024 (Sec. 3.3 uses 1024):
