@@ -187,7 +187,17 @@ wersa_status wersa_gate_static(const wersa_config* cfg, const void* Q, const flo
  *   wersa_shard_output  Q shard, the added S_total (batch*heads, features, 64) and z_total (batch*heads,
  *                       features), beta -> O shard.
  * The two additions are the only exchange between ranks (an all-reduce each; the library does not do them).
- * bf16 tensor-core contexts with features <= 256 only, else WERSA_ERR_UNSUPPORTED; forward only. */
+ * bf16 tensor-core contexts with features <= 256 only, else WERSA_ERR_UNSUPPORTED.
+ *
+ * Backward of the same (the chain rule through Eqs. 1-7, as wersa_backward; head_dim = 64 and a context created
+ * without WERSA_FLAG_FORWARD_ONLY), after the four forward steps, again on one stream and in this order:
+ *   wersa_shard_backward_queries  Q, dO shards -> this shard's dS' and dz' (wersa_saved, which = 4 and 5).  The
+ *                                 caller adds them over all shards.
+ *   wersa_shard_backward_keys     K, V shards and the added dS_total, dz_total -> dK, dV shards, and this shard's
+ *                                 band inner products df (batch*heads, 16) and sum of dD' (1 float) (wersa_saved,
+ *                                 which = 6 and 7).  The caller adds both over all shards.
+ *   wersa_shard_backward_gate     the added df_total, sumdD_total and n_total -> dbeta, dgate_w, dgate_b, domega
+ *                                 (the same on every rank; any may be NULL) and the dQ shard. */
 wersa_status wersa_shard_pool(wersa_ctx* ctx, const void* Q, const void* W, float* qsum, void* cuda_stream);
 wersa_status wersa_shard_gate(wersa_ctx* ctx, const float* qsum_total, int64_t n_total, const float* gate_w,
                               const float* gate_b, const float* omega, void* cuda_stream);
@@ -195,12 +205,22 @@ wersa_status wersa_shard_keys(wersa_ctx* ctx, const void* K, const void* V, void
 wersa_status wersa_shard_output(wersa_ctx* ctx, const void* Q, const float* S_total, const float* z_total,
                                 const float* beta, void* O, void* cuda_stream);
 
+wersa_status wersa_shard_backward_queries(wersa_ctx* ctx, const void* Q, const float* beta, const void* dO,
+                                          void* cuda_stream);
+wersa_status wersa_shard_backward_keys(wersa_ctx* ctx, const void* K, const void* V, const float* dS_total,
+                                       const float* dz_total, void* dK, void* dV, void* cuda_stream);
+wersa_status wersa_shard_backward_gate(wersa_ctx* ctx, const float* df_total, const float* sumdD_total,
+                                       int64_t n_total, const float* beta, const float* gate_w, const float* omega,
+                                       float* dbeta, float* dgate_w, float* dgate_b, float* domega, void* dQ,
+                                       void* cuda_stream);
+
 /* Device pointers into the workspace of quantities the last forward left there.
  * which: 0 = f (batch*heads, levels+1); 1 = qbar (batch*heads, 64);
  *        2 = S' (batch*heads, features, 64); 3 = z' (batch*heads, features),
  * the last axis of qbar and S' being the padded head dimension (columns >= head_dim are zero),
  * where S' = ReLU(K_F W)^T V and z' = ReLU(K_F W)^T 1 are the key summary and normaliser of
  * Eq. 7 without the 1/(bw sqrt(m)) factor of the feature map (S = S' / (bw sqrt(m))).
+ * which = 4 .. 7 are the sequence-sharded backward's exchange quantities (see wersa_shard_backward_*).
  * *count receives the number of floats. */
 wersa_status wersa_saved(wersa_ctx* ctx, int which, const float** device_ptr, size_t* count);
 

@@ -80,6 +80,12 @@ def _lib():
     lib.wersa_shard_keys.argtypes = [vp, vp, vp, vp]
     lib.wersa_shard_output.restype = ctypes.c_int
     lib.wersa_shard_output.argtypes = [vp, vp, fp, fp, fp, vp, vp]
+    lib.wersa_shard_backward_queries.restype = ctypes.c_int
+    lib.wersa_shard_backward_queries.argtypes = [vp, vp, fp, vp, vp]
+    lib.wersa_shard_backward_keys.restype = ctypes.c_int
+    lib.wersa_shard_backward_keys.argtypes = [vp, vp, vp, fp, fp, vp, vp, vp]
+    lib.wersa_shard_backward_gate.restype = ctypes.c_int
+    lib.wersa_shard_backward_gate.argtypes = [vp, fp, fp, ctypes.c_int64, fp, fp, fp, fp, fp, fp, fp, vp, vp]
     lib.wersa_selftest_wait_timeout.restype = ctypes.c_int
     lib.wersa_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint32, vp, vp]
     lib.wersa_uses_tensor_cores.restype = ctypes.c_int32
@@ -258,6 +264,45 @@ class WersaContext:
             raise WersaError(st, "wersa_shard_output")
         return out
 
+    def shard_backward_queries(self, Q, beta, dO, stream=None):
+        """Returns views of this shard's dS' and dz' in the workspace."""
+        st = _lib().wersa_shard_backward_queries(self._h, _ptr(Q, self.io_dtype, "Q"), _ptr(beta, torch.float32, "beta"),
+                                                 _ptr(dO, self.io_dtype, "dO"), _stream_ptr(stream))
+        if st != WERSA_OK:
+            raise WersaError(st, "wersa_shard_backward_queries")
+        return self._saved_view(4), self._saved_view(5)
+
+    def shard_backward_keys(self, K, V, dS_total, dz_total, stream=None):
+        """Returns dK, dV of this shard and views of its band inner products and its sum of dD'."""
+        dK = torch.empty(K.shape, dtype=self.grad_dtype, device=self.device)
+        dV = torch.empty(K.shape, dtype=self.grad_dtype, device=self.device)
+        st = _lib().wersa_shard_backward_keys(self._h, _ptr(K, self.io_dtype, "K"), _ptr(V, self.io_dtype, "V"),
+                                              _ptr(dS_total, torch.float32, "dS_total"),
+                                              _ptr(dz_total, torch.float32, "dz_total"), _ptr(dK), _ptr(dV),
+                                              _stream_ptr(stream))
+        if st != WERSA_OK:
+            raise WersaError(st, "wersa_shard_backward_keys")
+        return dK, dV, self._saved_view(6), self._saved_view(7)
+
+    def shard_backward_gate(self, Q, df_total, sumdD_total, n_total, beta, gate_w, omega, stream=None):
+        """Returns dict(dQ, dbeta, dgate_w, dgate_b, domega) for this shard (the parameter gradients are the
+        same on every rank)."""
+        c, dev = self.cfg, self.device
+        dQ = torch.empty(Q.shape, dtype=self.grad_dtype, device=dev)
+        dbeta = torch.empty(1, dtype=torch.float32, device=dev)
+        dgw = torch.empty((c.heads, c.head_dim, c.levels + 1), dtype=torch.float32, device=dev)
+        dgb = torch.empty((c.heads, c.levels + 1), dtype=torch.float32, device=dev)
+        dom = torch.empty(c.levels + 1, dtype=torch.float32, device=dev)
+        st = _lib().wersa_shard_backward_gate(self._h, _ptr(df_total, torch.float32, "df_total"),
+                                              _ptr(sumdD_total, torch.float32, "sumdD_total"), int(n_total),
+                                              _ptr(beta, torch.float32, "beta"),
+                                              _ptr(gate_w, torch.float32, "gate_w", optional=True),
+                                              _ptr(omega, torch.float32, "omega"), _ptr(dbeta), _ptr(dgw), _ptr(dgb),
+                                              _ptr(dom), _ptr(dQ), _stream_ptr(stream))
+        if st != WERSA_OK:
+            raise WersaError(st, "wersa_shard_backward_gate")
+        return dict(dQ=dQ, dbeta=dbeta, dgate_w=dgw, dgate_b=dgb, domega=dom)
+
     def _saved_view(self, idx):
         ptr, count = ctypes.c_void_p(), ctypes.c_size_t()
         st = _lib().wersa_saved(self._h, idx, ctypes.byref(ptr), ctypes.byref(count))
@@ -265,7 +310,9 @@ class WersaContext:
             raise WersaError(st, "wersa_saved")
         off = ptr.value - self.workspace.data_ptr()
         c = self.cfg
-        shape = {2: (c.batch, c.heads, c.features, 64), 3: (c.batch, c.heads, c.features)}[idx]
+        shape = {2: (c.batch, c.heads, c.features, 64), 3: (c.batch, c.heads, c.features),
+                 4: (c.batch, c.heads, c.features, 64), 5: (c.batch, c.heads, c.features),
+                 6: (c.batch, c.heads, 16), 7: (1,)}[idx]
         return self.workspace[off:off + 4 * count.value].view(torch.float32).view(shape)
 
     def saved(self, which):

@@ -154,8 +154,9 @@ wersa_status make_plan(const wersa_config& c, Plan* p) {
     p->off_dVp = take(p->dpad ? grad_bytes * slab_elems : 0);
     p->off_dgwp = take(p->dpad ? sizeof(float) * (size_t)c.heads * kD * p->L1 : 0);
     p->off_Dtot = take(grouped ? sizeof(float) * 2 * slabs * n : 0);
+    p->off_shardtot = take(256);
   } else {
-    p->off_Dtot = 0;
+    p->off_Dtot = p->off_shardtot = 0;
     p->off_dS = p->off_dz = p->off_sumdD = p->off_bands = p->off_dqbar = p->off_dQF = p->off_dKF = p->off_dSbf = p->off_KF3 = p->off_QF3 = p->off_Slo = 0;
     p->off_dOp = p->off_dQp = p->off_dKp = p->off_dVp = p->off_dgwp = 0;
   }
@@ -208,6 +209,7 @@ Ws resolve(const Plan& p, void* workspace) {
   w.Sout = reinterpret_cast<float*>(b + p.off_Sout);
   w.zout = reinterpret_cast<float*>(b + p.off_zout);
   w.Dtot = reinterpret_cast<float*>(b + p.off_Dtot);
+  w.shardtot = reinterpret_cast<float*>(b + p.off_shardtot);
   return w;
 }
 
@@ -511,6 +513,79 @@ wersa_status wersa_shard_output(wersa_ctx* ctx, const void* Q, const float* S_to
   return WERSA_OK;
 }
 
+// ---- sequence-sharded backward: three steps with the sums of dS', dz' and of (df, sum dD') taken by the caller
+static bool shardable_bwd(const Plan& p) { return shardable(p) && p.with_backward && !p.dpad; }
+
+wersa_status wersa_shard_backward_queries(wersa_ctx* ctx, const void* Q, const float* beta, const void* dO,
+                                          void* cuda_stream) {
+  if (ctx == nullptr || Q == nullptr || beta == nullptr || dO == nullptr) return WERSA_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(dO)) return WERSA_ERR_INVALID_ARG;
+  const Plan& p = ctx->plan;
+  if (!shardable_bwd(p)) return WERSA_ERR_UNSUPPORTED;
+  if (!ctx->forward_done) return WERSA_ERR_STATE;
+  const Ws& w = ctx->ws;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DeviceGuard guard(p.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  int launches = 0;
+  const int kind = 1, gkind = p.grad_bf16 ? 1 : 0;
+  WERSA_CUDA(launch_haar_filter_split3(p, Q, kind, w.f, w.QF3, st, &launches));
+  WERSA_CUDA(launch_tc_bwd_qside(p, w, w.QF3, beta, dO, nullptr, nullptr, false, st, &launches));
+  WERSA_CUDA(launch_reduce_partials(p, w.spart, w.zpart, p.bchunks, w.dS, w.dz, w.dSbf, nullptr, st, &launches));
+  WERSA_CUDA(launch_haar_backward(p, w, Q, kind, w.dQF, nullptr, gkind, 0, st, &launches));   // band inner products
+  ctx->launches_bwd = launches;
+  return WERSA_OK;
+}
+
+wersa_status wersa_shard_backward_keys(wersa_ctx* ctx, const void* K, const void* V, const float* dS_total,
+                                       const float* dz_total, void* dK, void* dV, void* cuda_stream) {
+  if (ctx == nullptr || K == nullptr || V == nullptr || dS_total == nullptr || dz_total == nullptr || dK == nullptr ||
+      dV == nullptr)
+    return WERSA_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(dK) || !aligned16(dV)) return WERSA_ERR_INVALID_ARG;
+  const Plan& p = ctx->plan;
+  if (!shardable_bwd(p)) return WERSA_ERR_UNSUPPORTED;
+  if (!ctx->forward_done) return WERSA_ERR_STATE;
+  const Ws& w = ctx->ws;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DeviceGuard guard(p.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  int launches = 0;
+  const int kind = 1, gkind = p.grad_bf16 ? 1 : 0;
+  // the totals take the place of a single partial: the reduction copies them and writes the bf16 image of dS'
+  WERSA_CUDA(launch_reduce_partials(p, dS_total, dz_total, 1, w.dS, w.dz, w.dSbf, nullptr, st, &launches));
+  WERSA_CUDA(launch_haar_filter_split3(p, K, kind, w.f, w.KF3, st, &launches));
+  WERSA_CUDA(launch_tc_bwd_kside(p, w, w.KF3, V, dV, false, st, &launches));
+  WERSA_CUDA(launch_haar_backward(p, w, K, kind, w.dKF, dK, gkind, 1, st, &launches));
+  float* df = w.dqbar + (size_t)p.slabs * kD;
+  WERSA_CUDA(launch_band_sums(p, w, p.slabs * p.bchunks, df, w.shardtot, st, &launches));
+  ctx->launches_bwd += launches;
+  return WERSA_OK;
+}
+
+wersa_status wersa_shard_backward_gate(wersa_ctx* ctx, const float* df_total, const float* sumdD_total, int64_t n_total,
+                                       const float* beta, const float* gate_w, const float* omega, float* dbeta,
+                                       float* dgate_w, float* dgate_b, float* domega, void* dQ, void* cuda_stream) {
+  if (ctx == nullptr || df_total == nullptr || sumdD_total == nullptr || beta == nullptr || omega == nullptr ||
+      dQ == nullptr || n_total < 1)
+    return WERSA_ERR_INVALID_ARG;
+  if (!aligned16(dQ)) return WERSA_ERR_INVALID_ARG;
+  const Plan& p = ctx->plan;
+  if (!shardable_bwd(p)) return WERSA_ERR_UNSUPPORTED;
+  if (!ctx->forward_done) return WERSA_ERR_STATE;
+  const Ws& w = ctx->ws;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DeviceGuard guard(p.cfg.device);
+  if (guard.err != cudaSuccess) return WERSA_ERR_CUDA;
+  int launches = 0;
+  WERSA_CUDA(launch_gate_backward_from(p, w, df_total, sumdD_total, beta, gate_w, omega, dbeta, dgate_w, dgate_b, domega,
+                                       st, &launches));
+  WERSA_CUDA(launch_haar_filter_addvec(p, w.dQF, w.f, w.dqbar, 1.f / (float)n_total, dQ, p.grad_bf16 ? 1 : 0, st,
+                                       &launches));
+  ctx->launches_bwd += launches;
+  return WERSA_OK;
+}
+
 wersa_status wersa_forward_host(wersa_ctx* ctx, const void* hQ, const void* hK, const void* hV, void* dQ,
                                 void* dK, void* dV, const void* W, const float* beta, const float* gate_w,
                                 const float* gate_b, const float* omega, void* dO, void* hO, void* cuda_stream) {
@@ -691,6 +766,11 @@ wersa_status wersa_saved(wersa_ctx* ctx, int which, const float** device_ptr, si
     case 1: *device_ptr = ctx->ws.qbar; *count = slabs * kD; break;
     case 2: *device_ptr = p.groups > 1 ? ctx->ws.Sout : ctx->ws.S; *count = slabs * p.cfg.features * kD; break;
     case 3: *device_ptr = p.groups > 1 ? ctx->ws.zout : ctx->ws.z; *count = slabs * p.cfg.features; break;
+    // sequence-sharded backward: this shard's dS', dz', band inner products and sum of dD'
+    case 4: if (!p.with_backward) return WERSA_ERR_UNSUPPORTED; *device_ptr = ctx->ws.dS; *count = slabs * p.cfg.features * kD; break;
+    case 5: if (!p.with_backward) return WERSA_ERR_UNSUPPORTED; *device_ptr = ctx->ws.dz; *count = slabs * p.cfg.features; break;
+    case 6: if (!p.with_backward) return WERSA_ERR_UNSUPPORTED; *device_ptr = ctx->ws.dqbar + slabs * kD; *count = slabs * kBandVals; break;
+    case 7: if (!p.with_backward) return WERSA_ERR_UNSUPPORTED; *device_ptr = ctx->ws.shardtot; *count = 1; break;
     default: return WERSA_ERR_INVALID_ARG;
   }
   return WERSA_OK;

@@ -45,7 +45,7 @@ struct Plan {
   size_t off_status, off_counters, status_bytes, off_qpart, off_qbar, off_sg, off_f, off_spart, off_zpart, off_S, off_z,
       off_Sbf, off_Wt, off_dS, off_dz, off_sumdD, off_bands, off_dqbar, off_QF, off_KF, off_dQF,
       off_dKF, off_dSbf, off_KF3, off_QF3, off_Slo, off_Simg, off_Qp, off_Kp, off_Vp, off_Op, off_Wp, off_gwp,
-      off_dOp, off_dQp, off_dKp, off_dVp, off_dgwp, off_Og, off_den, off_Sout, off_zout, off_Dtot, total;
+      off_dOp, off_dQp, off_dKp, off_dVp, off_dgwp, off_Og, off_den, off_Sout, off_zout, off_Dtot, off_shardtot, total;
   int part_chunks;    // max(schunks, tchunks): leading extent of the partial buffers
 };
 
@@ -65,6 +65,7 @@ struct Ws {   // resolved workspace pointers
   // features > 256: per-group outputs and denominators, and the slab-major S', z' handed out by wersa_saved
   void* Og;
   float *den, *Sout, *zout;
+  float* shardtot;   // sequence shards, backward: this shard's sum of dD' (one float)
   float* Dtot;   // backward with feature groups: the whole map's denominator per token, then dD' per token
 };
 Ws resolve(const Plan& p, void* workspace);
@@ -83,6 +84,11 @@ cudaError_t launch_shard_qsum(const Plan& p, const Ws& w, float* qsum, cudaStrea
 cudaError_t launch_gate_from_sums(const Plan& p, const Ws& w, const float* qsum, long long n_total,
                                   const float* gate_w, const float* gate_b, const float* omega, int cols,
                                   cudaStream_t st, int* launches);
+cudaError_t launch_band_sums(const Plan& p, const Ws& w, int n_sumdD, float* df, float* sumdD_total, cudaStream_t st,
+                             int* launches);
+cudaError_t launch_gate_backward_from(const Plan& p, const Ws& w, const float* df, const float* sumdD_total,
+                                      const float* beta, const float* gate_w, const float* omega, float* dbeta,
+                                      float* dgate_w, float* dgate_b, float* domega, cudaStream_t st, int* launches);
 // Gate backward: band inner products -> df -> domega, dgate_b, dgate_w, dqbar; dbeta.
 cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, const float* gate_w,
                                  const float* omega, int n_sumdD, float* dbeta, float* dgate_w, float* dgate_b,

@@ -241,6 +241,22 @@ __global__ void __launch_bounds__(256) k_band_reduce(const float* __restrict__ b
   }
 }
 
+// out[0] = sum of x[0..n) in a fixed order (64 threads, strided partial sums, then a tree).
+__global__ void __launch_bounds__(kD) k_sum_floats(const float* __restrict__ x, int n, float* __restrict__ out) {
+  wait_for_stream_predecessor();   // (launched as a programmatic dependent: see launch_after)
+  __shared__ float part[kD];
+  const int c = threadIdx.x;
+  float tot = 0.f;
+  for (int i = c; i < n; i += kD) tot += x[i];
+  part[c] = tot;
+  __syncthreads();
+  for (int o = kD / 2; o > 0; o >>= 1) {
+    if (c < o) part[c] += part[c + o];
+    __syncthreads();
+  }
+  if (c == 0) out[0] = part[0];
+}
+
 // Chain rule through f = sigmoid(u) * omega, u = gate(qbar): domega, dgate_b, dgate_w, dqbar; and the
 // bandwidth gradient dbeta = 2 eps m bw * sum_t dDh_t (ReLU is positively homogeneous, so beta only
 // acts through eps).  Grid H + 2, 64 threads: CTA h < H handles head h (thread c = column of q-bar,
@@ -432,6 +448,25 @@ size_t static_scratch_floats_needed(const Plan& p) {
   return (size_t)p.slabs * p.qchunks * kD + (size_t)p.slabs * p.L1;
 }
 size_t static_scratch_counters_needed(const Plan& p) { return (size_t)p.slabs + (size_t)p.cfg.batch; }
+
+// The two halves of launch_gate_backward, for sequence shards: this shard's band inner products (df, slabs x 16)
+// and its sum of dD'; then, from the sums over all shards, the parameter gradients and d(qbar).
+cudaError_t launch_band_sums(const Plan& p, const Ws& w, int n_sumdD, float* df, float* sumdD_total, cudaStream_t st,
+                             int* launches) {
+  launch_after(k_band_reduce, dim3(p.slabs), dim3(256), 0, st, w.bands, p.slabs, 2 * p.htiles, p.cfg.levels, df);
+  launch_after(k_sum_floats, dim3(1), dim3(kD), 0, st, w.sumdD, n_sumdD, sumdD_total);
+  *launches += 2;
+  return cudaGetLastError();
+}
+cudaError_t launch_gate_backward_from(const Plan& p, const Ws& w, const float* df, const float* sumdD_total,
+                                      const float* beta, const float* gate_w, const float* omega, float* dbeta,
+                                      float* dgate_w, float* dgate_b, float* domega, cudaStream_t st, int* launches) {
+  launch_after(k_gate_backward, dim3(p.cfg.heads + 2), dim3(kD), 0, st, df, w.sg, w.qbar, gate_w, omega, sumdD_total, 1,
+               beta, p.cfg.eps, p.cfg.bw_floor, p.cfg.features, p.cfg.batch, p.cfg.heads, p.L1, p.cfg.gate_per_head,
+               dbeta, dgate_w, dgate_b, domega, w.dqbar);
+  *launches += 1;
+  return cudaGetLastError();
+}
 
 cudaError_t launch_gate_backward(const Plan& p, const Ws& w, const float* beta, const float* gate_w,
                                  const float* omega, int n_sumdD, float* dbeta, float* dgate_w, float* dgate_b,

@@ -34,3 +34,21 @@ def forward_sharded(ctx, Q, K, V, W, beta, gate_w, gate_b, omega, out=None, grou
     S_total, z_total = S.clone(), z.clone()
     allreduce_sum_([S_total, z_total], group)
     return ctx.shard_output(Q, S_total, z_total, beta, out=out, stream=stream)
+
+
+def backward_sharded(ctx, Q, K, V, W, beta, gate_w, gate_b, omega, dO, group=None, n_total=None, stream=None):
+    """Backward of forward_sharded on the same context (call it after forward_sharded with the same shards).
+    Returns dict(dQ, dK, dV, dbeta, dgate_w, dgate_b, domega): dQ, dK, dV are this rank's shards, the parameter
+    gradients are those of the whole sequence (the same on every rank).  Three sums cross the ranks: dS' and dz',
+    then the band inner products together with the sum of dD'."""
+    if n_total is None:
+        n_total = total_length(ctx.cfg.seq_len, Q.device, group)
+    dS, dz = ctx.shard_backward_queries(Q, beta, dO, stream=stream)
+    dS_total, dz_total = dS.clone(), dz.clone()
+    allreduce_sum_([dS_total, dz_total], group)
+    dK, dV, df, sumdD = ctx.shard_backward_keys(K, V, dS_total, dz_total, stream=stream)
+    df_total, sumdD_total = df.clone(), sumdD.clone()
+    allreduce_sum_([df_total, sumdD_total], group)
+    grads = ctx.shard_backward_gate(Q, df_total, sumdD_total, n_total, beta, gate_w, omega, stream=stream)
+    grads.update(dK=dK, dV=dV)
+    return grads

@@ -344,6 +344,57 @@ def test_forward_with_orthogonal_projection(dtype):
     _check(to_numpy64(O), _oracle_forward(cfg, inp), dtype, "O")
 
 
+SHARDED_BWD = [
+    (dict(B=2, H=2, n=2000, d=64, L=5, m=256), [1024, 976]),
+    (dict(B=1, H=3, n=1536, d=64, L=8, m=128, gate_per_head=0), [768, 512, 256]),
+]
+
+
+@pytest.mark.parametrize("case", range(len(SHARDED_BWD)))
+def test_sequence_sharded_backward(case):
+    """Forward and backward shard steps on contexts of the shards' lengths, every sum between them taken here
+    (all-reduces on several GPUs): the shards' dQ, dK, dV put together and the parameter gradients meet the
+    oracle's backward on the whole sequence."""
+    import torch
+    cfg, lens = SHARDED_BWD[case]
+    cfg = dict(cfg, dtype="bf16", eps=1e-3)
+    assert sum(lens) == cfg["n"] and all(l % (1 << cfg["L"]) == 0 for l in lens[:-1])
+    inp = wi.make_inputs(**cfg, seed=2900 + case, w_seed=3000 + case, gate_std=0.3, gate_seed=3100 + case,
+                         mean_shift=0.25, scale=0.7, backward=True)
+    dev = device_inputs(inp, "bf16")
+    starts = np.concatenate([[0], np.cumsum(lens)]).astype(int)
+    shards = [{k: dev[k][:, :, a:b].contiguous() for k in ("Q", "K", "V", "dO")} for a, b in zip(starts[:-1], starts[1:])]
+    ctxs = [_ctx(dict(cfg, n=l)) for l in lens]
+    pairs = list(zip(ctxs, shards))
+    qsum = sum(c.shard_pool(s["Q"], dev["W"]) for c, s in pairs)
+    Ss, zs = [], []
+    for c, s in pairs:
+        c.shard_gate(qsum, cfg["n"], dev["gate_w"], dev["gate_b"], dev["omega"])
+        S, z = c.shard_keys(s["K"], s["V"])
+        Ss.append(S.clone()); zs.append(z.clone())
+    S_total, z_total = sum(Ss), sum(zs)
+    for c, s in pairs:
+        c.shard_output(s["Q"], S_total, z_total, dev["beta"])
+    parts = [c.shard_backward_queries(s["Q"], dev["beta"], s["dO"]) for c, s in pairs]
+    dS_total = sum(p[0].clone() for p in parts)
+    dz_total = sum(p[1].clone() for p in parts)
+    kv = [c.shard_backward_keys(s["K"], s["V"], dS_total, dz_total) for c, s in pairs]
+    df_total = sum(r[2].clone() for r in kv)
+    sumdD_total = sum(r[3].clone() for r in kv)
+    gates = [c.shard_backward_gate(s["Q"], df_total, sumdD_total, cfg["n"], dev["beta"], dev["gate_w"], dev["omega"])
+             for c, s in pairs]
+    torch.cuda.synchronize()
+    assert all(c.query_status() == 0 for c in ctxs)
+    grads = dict(gates[0])
+    grads["dQ"] = torch.cat([g["dQ"] for g in gates], dim=2)
+    grads["dK"] = torch.cat([r[0] for r in kv], dim=2)
+    grads["dV"] = torch.cat([r[1] for r in kv], dim=2)
+    for g in gates[1:]:   # the parameter gradients are the same on every shard
+        for k in ("dbeta", "dgate_w", "dgate_b", "domega"):
+            assert torch.equal(g[k], gates[0][k]), k
+    _check_backward(cfg, inp, grads)
+
+
 def test_forward_is_bit_identical_run_to_run():
     import paper_2507_08637_b200 as wersa
     import torch
