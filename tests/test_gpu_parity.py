@@ -395,6 +395,25 @@ def test_sequence_sharded_backward(case):
     _check_backward(cfg, inp, grads)
 
 
+def test_sharded_helpers_with_a_single_rank():
+    """paper_2507_08637_b200.sharded.forward_sharded / backward_sharded without a process group (one rank holds
+    the whole sequence, the all-reduces are no-ops): the same results as the oracle on that sequence."""
+    import torch
+    from paper_2507_08637_b200.sharded import backward_sharded, forward_sharded
+    cfg = dict(B=2, H=2, n=1300, d=64, L=4, m=256, dtype="bf16", eps=1e-3)
+    inp = wi.make_inputs(**cfg, seed=3200, w_seed=3201, gate_std=0.3, gate_seed=3202, mean_shift=0.25, scale=0.7,
+                         backward=True)
+    dev = device_inputs(inp, "bf16")
+    ctx = _ctx(cfg)
+    args = (dev["Q"], dev["K"], dev["V"], dev["W"], dev["beta"], dev["gate_w"], dev["gate_b"], dev["omega"])
+    O = forward_sharded(ctx, *args)
+    grads = backward_sharded(ctx, *args, dev["dO"])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    _check(to_numpy64(O), _oracle_forward(cfg, inp), "bf16", "O")
+    _check_backward(cfg, inp, grads)
+
+
 def test_forward_is_bit_identical_run_to_run():
     import paper_2507_08637_b200 as wersa
     import torch
