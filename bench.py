@@ -353,12 +353,15 @@ def main():
     tot = sum(avg.values())
     dom = max(avg, key=avg.get)
     # algorithmic work of each step per launch
-    unit_flops = TH * (4 * d * m + 2 * m)            # one projection + one (m x d) contraction per token-head
+    m_launch = min(m, 256)                           # feature maps wider than 256 run one launch per 256 features
+    unit_flops = TH * (4 * d * m_launch + 2 * m_launch)   # one projection + one (m x d) contraction per token-head
     flops = {"tc_kside": unit_flops, "tc_qside": unit_flops, "simt_kside": unit_flops, "simt_qside": unit_flops}
     bytes_ = {"qmean_gate": TH * d * s_bytes, "haar_filter_q": TH * d * (s_bytes + 4),
               "haar_filter_k": TH * d * (s_bytes + 4),
               "tc_kside": 2 * TH * d * s_bytes,      # K and V read once
-              "tc_qside": 2 * TH * d * s_bytes}      # Q read once, O written once
+              "tc_qside": 2 * TH * d * s_bytes,      # Q read once, O written once
+              # feature groups: G outputs of 64 columns and G denominators in, O out
+              "combine_groups": TH * ((m // 256) * (64 * s_bytes + 4) + d * s_bytes)}
     ncu_bytes_per_th, traffic_source = load_traffic()
     if dom in flops:
         if dom.startswith("tc_"):
@@ -369,7 +372,9 @@ def main():
     else:
         bound, peak, unit = "hbm", float(peaks["hbm_gbs"]), "GB/s"
         achieved = bytes_.get(dom, 0) / (avg[dom] * 1e-3) / 1e9
-    traffic = ncu_bytes_per_th[dom] * TH if (tensor_cores and dtype == "bf16" and dom in ncu_bytes_per_th) else None
+    # (the counters were taken with 64-column heads and one feature group: other shapes move other bytes)
+    traffic = ncu_bytes_per_th[dom] * TH if (tensor_cores and dtype == "bf16" and dom in ncu_bytes_per_th and d == 64
+                                             and m <= 256) else None
     roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
                 "frac": achieved / peak, "traffic": traffic, "traffic_source": traffic_source,
                 "peak_source": f"{peak_kind} ({regime})" if bound == "tensor" else

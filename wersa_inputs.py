@@ -1,6 +1,7 @@
 """Seeded synthetic inputs for the WERSA operator, shared by the tests, the smoke check and
 the benchmark.  This module holds none of the method's arithmetic: it only draws random
-tensors of the shapes and value distributions of the five benchmark configurations and
+tensors of the shapes and value distributions of the five benchmark configurations (and two
+shapes with the paper's own hyper-parameters) and
 rounds them to the storage type the configuration names.
 
 Recipe (every configuration): one numpy `default_rng(seed)`; Q, K, V and (where used) dO are
@@ -25,6 +26,12 @@ CONFIGS = {
                            seed=4, w_seed=1004, gate_std=None, gate_seed=None, backward=False),
     "cfg5_train_bf16": dict(B=4, H=8, n=16384, d=64, L=6, m=256, dtype="bf16", scale=1.0,
                             seed=5, w_seed=1005, gate_std=0.1, gate_seed=2005, backward=True),
+    # Shapes with the paper's own hyper-parameters (L = 2, m = 1024; heads of 32 and 16 dimensions), for
+    # `bench.py --workload`: a text-classification-sized batch and one 128k-token sequence.
+    "paper_text_bf16": dict(B=32, H=4, n=4096, d=32, L=2, m=1024, dtype="bf16", scale=1.0,
+                            seed=6, w_seed=1006, gate_std=0.1, gate_seed=2006, backward=True),
+    "paper_long_bf16": dict(B=1, H=4, n=131072, d=16, L=2, m=1024, dtype="bf16", scale=0.25,
+                            seed=7, w_seed=1007, gate_std=0.1, gate_seed=2007, backward=False),
 }
 
 
